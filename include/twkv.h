@@ -1,0 +1,183 @@
+/*
+ * libtwkv — token-wise adaptive low-rank KV-cache compression on one B200 (sm_100a).
+ *
+ * The method (Sec. 3 of the paper): a token's pre-RoPE key and value states are
+ * expressed in a spectral basis, x~ = x U (Eq. 1).  A learned gate decides per
+ * token, per layer and separately for K and V how many leading components to
+ * keep (Eq. 5, Eq. 6, Eq. 8); only those r components are persisted (Eq. 2).
+ * At decode time the states are rebuilt as x^[I] U^-1[I,:] (Eq. 3), keys are
+ * reshaped to heads and rotated (RoPE), and ordinary softmax attention runs
+ * over them.  The per-token "compression level" is the retained rank r.
+ *
+ * This library is the data-parallel hot path of that method:
+ *   twkv_compress     gate -> rank -> truncate -> pack into a rank-class-sorted paged cache
+ *   twkv_decode_attn  attention of one query per sequence over the mixed-rank cache
+ *
+ * Conventions
+ *   - Every pointer argument is a DEVICE pointer unless its comment says "host".
+ *   - The caller owns all device memory: inputs, outputs, layer parameters
+ *     (borrowed until the cache is destroyed or the parameters are replaced)
+ *     and the one `pool` buffer the cache lives in.  The library allocates no
+ *     device memory; it allocates small host structures only.
+ *   - Work is enqueued on `stream` (a cudaStream_t passed as void*; NULL = the
+ *     default stream) and is asynchronous unless stated otherwise.
+ *   - Errors are return codes, never aborts.  Argument errors that the host can
+ *     see are returned before anything is launched and leave the cache
+ *     unchanged.  Errors only the device can see (pool exhausted, a rank or
+ *     sequence id out of range) set a sticky status word; the offending piece
+ *     of work is skipped as a whole and the code is returned by the next
+ *     twkv_cache_status().
+ *   - Supported shapes: head_dim = 128, 1..8 KV heads (d_kv = n_kv_heads * 128,
+ *     at most 1024), n_q_heads / n_kv_heads in {1, 2, 4, 8}.
+ *
+ * Cache container (the paper only fixes WHAT is stored, the sentence after
+ * Eq. 2; the container is this library's):
+ *   - rank class c = ceil(r / 64); a stored row has 64 c 16-bit elements, the
+ *     elements r .. 64c-1 are +0, so reconstruction is exactly rank r;
+ *   - a tile = up to 128 tokens of one (layer, K|V, sequence, class); it owns c
+ *     consecutive 16 KiB blocks, block j = row-major panel [128 tokens x 64
+ *     elements] of elements 64j .. 64j+63; rows past the last token are zero;
+ *   - tokens of a (side, sequence, class) fill tiles in arrival order;
+ *   - K tiles are listed per class (decode walks classes from wide to narrow),
+ *     V tiles per sequence; every V slot links to the score slot of its token.
+ */
+#ifndef TWKV_H_
+#define TWKV_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  TWKV_OK = 0,
+  TWKV_ERR_INVALID_ARG = 1,   /* bad pointer, size, id or rank                                  */
+  TWKV_ERR_UNSUPPORTED = 2,   /* shape or mode outside the supported set                        */
+  TWKV_ERR_CAPACITY = 3,      /* pool, tile tables or per-sequence token limit exhausted        */
+  TWKV_ERR_CUDA = 4,          /* a CUDA runtime call failed                                     */
+  TWKV_ERR_DEVICE_CHECK = 5,  /* a device-side consistency check failed                         */
+  TWKV_ERR_TIMEOUT = 6        /* a bounded device-side wait ran out                             */
+} twkv_status;
+
+typedef enum { TWKV_F16 = 0, TWKV_BF16 = 1, TWKV_F32 = 2 } twkv_dtype;
+
+typedef enum {
+  TWKV_GATE_FORCED = 0,   /* levels[] is INPUT: the caller gives the ranks                          */
+  TWKV_GATE_LOGITS = 1,   /* scores[] is INPUT: gate logits z of Eq. 5; levels[] is OUTPUT          */
+  TWKV_GATE_COMPUTE = 2   /* z = x~ W + b is formed from the layer parameters; levels[] is OUTPUT   */
+} twkv_gate_mode;
+
+#define TWKV_TILE_TOKENS 128        /* tokens per tile                                               */
+#define TWKV_PANEL_ELEMS 64         /* elements per panel row = rank granule                         */
+#define TWKV_BLOCK_BYTES 16384      /* one panel: 128 rows x 64 elements x 2 bytes                   */
+#define TWKV_PIECE_TOKENS 65536     /* a compress call is processed in pieces of this many tokens    */
+#define TWKV_MAX_CLASSES 16
+
+typedef struct {
+  int32_t n_layers;
+  int32_t n_q_heads;
+  int32_t n_kv_heads;
+  int32_t head_dim;             /* must be 128                                                       */
+  int32_t dtype;                /* twkv_dtype of x~, U^-1, W and q: TWKV_F16 or TWKV_BF16            */
+  int32_t out_dtype;            /* twkv_dtype of `out` in twkv_decode_attn (any of the three)        */
+  int32_t max_seqs;             /* sequence ids are 0 .. max_seqs-1                                  */
+  int32_t max_tokens_per_seq;   /* per layer                                                         */
+  float tau;                    /* threshold of Eq. 8 (the paper's example value is 0.1)             */
+  float rope_base;              /* RoPE base; pairing (i, i + 64), angle pos * base^(-2i/128)        */
+  float sm_scale;               /* softmax scale, usually 1/sqrt(head_dim)                           */
+} twkv_config;
+
+typedef struct {
+  const void* Uinv_k;   /* [d_kv x d_kv] row-major, dtype; row j = spectral component j (Eq. 3)      */
+  const void* Uinv_v;
+  const void* W_k;      /* [d_kv x d_kv] row-major, dtype; gate weights of Eq. 5 (may be NULL)       */
+  const void* W_v;
+  const float* b_k;     /* [d_kv] fp32 gate bias of Eq. 5 (may be NULL = zero)                       */
+  const float* b_v;
+} twkv_layer_params;
+
+typedef struct {
+  uint64_t tokens;                  /* cached tokens in the layer(s)                                 */
+  uint64_t bytes_stored;            /* bytes of valid rows, class padding included                   */
+  uint64_t bytes_algorithmic;       /* 2 (r_K + r_V) summed over tokens                              */
+  uint64_t blocks_used, blocks_free;
+  double retain_rate_k;             /* Eq. 4 averaged over tokens                                    */
+  double retain_rate_v;
+  uint64_t tokens_per_class[2][TWKV_MAX_CLASSES];   /* [K|V][class - 1]                              */
+} twkv_stats;
+
+/* Byte offsets (from the start of `pool`) and strides of the cache's tables, for export,
+ * inspection and tests.  Per-layer tables are laid out [layer][...]; sides are K = 0, V = 1. */
+typedef struct {
+  uint64_t pool_bytes, n_blocks, blocks_off;         /* blocks_off: first 16 KiB block               */
+  uint64_t status_off;                               /* int32[8]: [0] sticky status, [1] next_block  */
+  uint64_t n_tiles_off;                              /* int32 [L][2]                                 */
+  uint64_t tile_desc_off;                            /* int32 [L][2][NT][4] = seq, class, n_valid, base block */
+  uint64_t tile_aux_off;                             /* int32 [L][2][NT][128]: K position / V score link      */
+  uint64_t tile_rank_off;                            /* uint16[L][2][NT][128]                        */
+  uint64_t fill_off;                                 /* int32 [L][2*S*NC] tokens per key             */
+  uint64_t kclass_count_off, kclass_tiles_off;       /* int32 [L][NC], int32 [L][NC][NT]             */
+  uint64_t seq_vcount_off, seq_vtiles_off;           /* int32 [L][S],  int32 [L][S][TPS]             */
+  uint64_t seq_tokens_off;                           /* int32 [L][S]                                 */
+  uint64_t max_tiles;                                /* NT: tile ids per (layer, side)               */
+  uint64_t tiles_per_seq;                            /* TPS                                          */
+  uint64_t n_classes;                                /* NC = d_kv / 64                               */
+} twkv_layout;
+
+typedef struct twkv_cache twkv_cache;   /* opaque, host memory */
+
+/* Pool size (bytes) that holds `payload_bytes` of packed rows plus worst-case partially
+ * filled tiles, all tables and the scratch the two calls use.  Returns 0 if cfg is unsupported. */
+size_t twkv_cache_required_bytes(const twkv_config* cfg /*host*/, size_t payload_bytes);
+
+/* Lays the cache out inside pool[0 .. pool_bytes) (256-byte aligned device memory), clears
+ * its tables and builds the RoPE tables on `stream`.  *out is host memory owned by the library. */
+twkv_status twkv_cache_create(const twkv_config* cfg /*host*/, void* pool, size_t pool_bytes,
+                              void* stream, twkv_cache** out /*host*/);
+twkv_status twkv_cache_destroy(twkv_cache* cache);
+/* Forgets every cached token of every layer (tables cleared, blocks reusable); layer
+ * parameters and a pending sticky status are kept / cleared respectively. */
+twkv_status twkv_cache_reset(twkv_cache* cache, void* stream);
+/* Borrows the layer's matrices (Eq. 3: U^-1; Eq. 5: W, b).  `params` itself is host memory. */
+twkv_status twkv_cache_set_layer_params(twkv_cache* cache, int layer, const twkv_layer_params* params /*host*/);
+
+/*
+ * Compress step (Eq. 5, 6, 8 for the rank; Eq. 2 for what is stored).
+ *   K, V      [n_tok x d_kv] spectral states x~ (pre-RoPE), dtype, row-major
+ *   seq_ids   [n_tok] int32, positions [n_tok] int32 (RoPE position of the token)
+ *   scores    [n_tok x 2 x d_kv] fp32 gate logits (K row then V row per token); LOGITS mode only, else NULL
+ *   levels    [n_tok x 2] uint16 (r_K, r_V): input in FORCED mode (1 <= r <= d_kv), output otherwise
+ * Tokens are appended in index order.  A piece of the call (TWKV_PIECE_TOKENS tokens) that does
+ * not fit, or that holds an invalid id or rank, is skipped whole and the sticky status is set.
+ */
+twkv_status twkv_compress(twkv_cache* cache, int layer, const void* K, const void* V,
+                          const int32_t* seq_ids, const int32_t* positions, int n_tok,
+                          const float* scores, uint16_t* levels, twkv_gate_mode mode, void* stream);
+
+/*
+ * Decode attention (Eq. 3, reshape to heads, RoPE on keys, softmax attention) of one query
+ * per listed sequence over all tokens cached for that sequence in `layer`.
+ *   q        [n_seq x n_q_heads x 128] dtype, already rotated at its own position
+ *   seq_ids  [n_seq] int32, distinct
+ *   out      [n_seq x n_q_heads x 128] out_dtype; a sequence with no cached token gets zeros
+ *   num_splits  V-side splits per sequence; 0 = choose automatically
+ */
+twkv_status twkv_decode_attn(twkv_cache* cache, int layer, const void* q, const int32_t* seq_ids,
+                             int n_seq, void* out, int num_splits, void* stream);
+
+/* Synchronises `stream`, returns the sticky device status and clears it. */
+twkv_status twkv_cache_status(twkv_cache* cache, void* stream);
+/* Synchronises `stream`; layer = -1 sums all layers.  `out` is host memory. */
+twkv_status twkv_cache_stats(twkv_cache* cache, int layer, void* stream, twkv_stats* out /*host*/);
+/* Where the tables live inside the pool (host call, no device work). */
+twkv_status twkv_cache_layout(const twkv_cache* cache, twkv_layout* out /*host*/);
+/* Number of kernels this library has launched so far in the process (host counter). */
+uint64_t twkv_launch_count(void);
+const char* twkv_status_string(twkv_status s);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* TWKV_H_ */

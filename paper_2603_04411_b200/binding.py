@@ -1,0 +1,174 @@
+"""Thin ctypes binding of libtwkv's C ABI (argument marshalling only).
+
+Every function has the name and the meaning of its C counterpart in
+include/twkv.h; tensors are torch CUDA tensors whose data pointers are handed
+through unchanged.  There is no fallback: if libtwkv.so is missing or cannot be
+loaded, importing this module raises.
+"""
+import ctypes
+import os
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libtwkv.so")
+
+TWKV_OK, TWKV_ERR_INVALID_ARG, TWKV_ERR_UNSUPPORTED, TWKV_ERR_CAPACITY = 0, 1, 2, 3
+TWKV_ERR_CUDA, TWKV_ERR_DEVICE_CHECK, TWKV_ERR_TIMEOUT = 4, 5, 6
+TWKV_F16, TWKV_BF16, TWKV_F32 = 0, 1, 2
+TWKV_GATE_FORCED, TWKV_GATE_LOGITS, TWKV_GATE_COMPUTE = 0, 1, 2
+TILE_TOKENS, PANEL_ELEMS, BLOCK_BYTES, PIECE_TOKENS, MAX_CLASSES = 128, 64, 16384, 65536, 16
+
+EXPORTS = ["twkv_cache_required_bytes", "twkv_cache_create", "twkv_cache_destroy", "twkv_cache_reset",
+           "twkv_cache_set_layer_params", "twkv_compress", "twkv_decode_attn", "twkv_cache_status",
+           "twkv_cache_stats", "twkv_cache_layout", "twkv_launch_count", "twkv_status_string"]
+
+
+class twkv_config(ctypes.Structure):
+    _fields_ = [("n_layers", ctypes.c_int32), ("n_q_heads", ctypes.c_int32), ("n_kv_heads", ctypes.c_int32),
+                ("head_dim", ctypes.c_int32), ("dtype", ctypes.c_int32), ("out_dtype", ctypes.c_int32),
+                ("max_seqs", ctypes.c_int32), ("max_tokens_per_seq", ctypes.c_int32),
+                ("tau", ctypes.c_float), ("rope_base", ctypes.c_float), ("sm_scale", ctypes.c_float)]
+
+
+class twkv_layer_params(ctypes.Structure):
+    _fields_ = [("Uinv_k", ctypes.c_void_p), ("Uinv_v", ctypes.c_void_p), ("W_k", ctypes.c_void_p),
+                ("W_v", ctypes.c_void_p), ("b_k", ctypes.c_void_p), ("b_v", ctypes.c_void_p)]
+
+
+class twkv_stats(ctypes.Structure):
+    _fields_ = [("tokens", ctypes.c_uint64), ("bytes_stored", ctypes.c_uint64), ("bytes_algorithmic", ctypes.c_uint64),
+                ("blocks_used", ctypes.c_uint64), ("blocks_free", ctypes.c_uint64),
+                ("retain_rate_k", ctypes.c_double), ("retain_rate_v", ctypes.c_double),
+                ("tokens_per_class", (ctypes.c_uint64 * MAX_CLASSES) * 2)]
+
+
+class twkv_layout(ctypes.Structure):
+    _fields_ = [(n, ctypes.c_uint64) for n in
+                ["pool_bytes", "n_blocks", "blocks_off", "status_off", "n_tiles_off", "tile_desc_off", "tile_aux_off",
+                 "tile_rank_off", "fill_off", "kclass_count_off", "kclass_tiles_off", "seq_vcount_off",
+                 "seq_vtiles_off", "seq_tokens_off", "max_tiles", "tiles_per_seq", "n_classes"]]
+
+
+def _load():
+    if not os.path.exists(LIB_PATH):
+        raise ImportError(f"{LIB_PATH} is missing: build it with `python -m paper_2603_04411_b200.build` "
+                          "(there is no CPU or PyTorch fallback)")
+    L = ctypes.CDLL(LIB_PATH)
+    vp, i32, sz = ctypes.c_void_p, ctypes.c_int, ctypes.c_size_t
+    L.twkv_cache_required_bytes.argtypes = [ctypes.POINTER(twkv_config), sz]
+    L.twkv_cache_required_bytes.restype = sz
+    L.twkv_cache_create.argtypes = [ctypes.POINTER(twkv_config), vp, sz, vp, ctypes.POINTER(vp)]
+    L.twkv_cache_destroy.argtypes = [vp]
+    L.twkv_cache_reset.argtypes = [vp, vp]
+    L.twkv_cache_set_layer_params.argtypes = [vp, i32, ctypes.POINTER(twkv_layer_params)]
+    L.twkv_compress.argtypes = [vp, i32, vp, vp, vp, vp, i32, vp, vp, i32, vp]
+    L.twkv_decode_attn.argtypes = [vp, i32, vp, vp, i32, vp, i32, vp]
+    L.twkv_cache_status.argtypes = [vp, vp]
+    L.twkv_cache_stats.argtypes = [vp, i32, vp, ctypes.POINTER(twkv_stats)]
+    L.twkv_cache_layout.argtypes = [vp, ctypes.POINTER(twkv_layout)]
+    L.twkv_launch_count.argtypes = []
+    L.twkv_launch_count.restype = ctypes.c_uint64
+    L.twkv_status_string.argtypes = [i32]
+    L.twkv_status_string.restype = ctypes.c_char_p
+    for name in ["twkv_cache_create", "twkv_cache_destroy", "twkv_cache_reset", "twkv_cache_set_layer_params",
+                 "twkv_compress", "twkv_decode_attn", "twkv_cache_status", "twkv_cache_stats", "twkv_cache_layout"]:
+        getattr(L, name).restype = i32
+    return L
+
+
+lib = _load()
+
+
+class TwkvError(RuntimeError):
+    def __init__(self, code, where):
+        self.code = code
+        super().__init__(f"{where}: {lib.twkv_status_string(code).decode()} ({code})")
+
+
+def _check(code, where):
+    if code != TWKV_OK:
+        raise TwkvError(code, where)
+
+
+def _ptr(t):
+    if t is None:
+        return None
+    assert t.is_cuda and t.is_contiguous(), "libtwkv takes contiguous CUDA tensors"
+    return ctypes.c_void_p(t.data_ptr())
+
+
+def _stream(stream=None):
+    s = torch.cuda.current_stream() if stream is None else stream
+    return ctypes.c_void_p(s.cuda_stream)
+
+
+def dtype_code(dt) -> int:
+    return {torch.float16: TWKV_F16, torch.bfloat16: TWKV_BF16, torch.float32: TWKV_F32}[dt]
+
+
+def make_config(*, n_layers, n_q_heads, n_kv_heads, head_dim=128, dtype=torch.float16, out_dtype=None,
+                max_seqs, max_tokens_per_seq, tau=0.1, rope_base=500000.0, sm_scale=None) -> twkv_config:
+    return twkv_config(n_layers, n_q_heads, n_kv_heads, head_dim, dtype_code(dtype),
+                       dtype_code(out_dtype if out_dtype is not None else dtype), max_seqs, max_tokens_per_seq,
+                       tau, rope_base, sm_scale if sm_scale is not None else head_dim ** -0.5)
+
+
+def twkv_cache_required_bytes(cfg: twkv_config, payload_bytes: int) -> int:
+    return int(lib.twkv_cache_required_bytes(ctypes.byref(cfg), payload_bytes))
+
+
+def twkv_cache_create(cfg: twkv_config, pool: torch.Tensor, stream=None):
+    """pool: 1-D uint8 CUDA tensor owned by the caller (kept alive by the caller)."""
+    h = ctypes.c_void_p()
+    _check(lib.twkv_cache_create(ctypes.byref(cfg), _ptr(pool), pool.numel() * pool.element_size(), _stream(stream),
+                                 ctypes.byref(h)), "twkv_cache_create")
+    return h
+
+
+def twkv_cache_destroy(cache):
+    _check(lib.twkv_cache_destroy(cache), "twkv_cache_destroy")
+
+
+def twkv_cache_reset(cache, stream=None):
+    _check(lib.twkv_cache_reset(cache, _stream(stream)), "twkv_cache_reset")
+
+
+def twkv_cache_set_layer_params(cache, layer, Uinv_k, Uinv_v, W_k=None, W_v=None, b_k=None, b_v=None):
+    p = twkv_layer_params(_ptr(Uinv_k), _ptr(Uinv_v), _ptr(W_k), _ptr(W_v), _ptr(b_k), _ptr(b_v))
+    _check(lib.twkv_cache_set_layer_params(cache, layer, ctypes.byref(p)), "twkv_cache_set_layer_params")
+
+
+def twkv_compress(cache, layer, K, V, seq_ids, positions, scores, levels, mode, stream=None, n_tok=None):
+    n = K.shape[0] if n_tok is None else n_tok
+    _check(lib.twkv_compress(cache, layer, _ptr(K), _ptr(V), _ptr(seq_ids), _ptr(positions), n, _ptr(scores),
+                             _ptr(levels), mode, _stream(stream)), "twkv_compress")
+
+
+def twkv_decode_attn(cache, layer, q, seq_ids, out, num_splits=0, stream=None):
+    _check(lib.twkv_decode_attn(cache, layer, _ptr(q), _ptr(seq_ids), seq_ids.numel(), _ptr(out), num_splits,
+                                _stream(stream)), "twkv_decode_attn")
+
+
+def twkv_cache_status(cache, stream=None) -> int:
+    return int(lib.twkv_cache_status(cache, _stream(stream)))
+
+
+def twkv_cache_stats(cache, layer=-1, stream=None) -> twkv_stats:
+    st = twkv_stats()
+    _check(lib.twkv_cache_stats(cache, layer, _stream(stream), ctypes.byref(st)), "twkv_cache_stats")
+    return st
+
+
+def twkv_cache_layout(cache) -> twkv_layout:
+    lay = twkv_layout()
+    _check(lib.twkv_cache_layout(cache, ctypes.byref(lay)), "twkv_cache_layout")
+    return lay
+
+
+def twkv_launch_count() -> int:
+    return int(lib.twkv_launch_count())
+
+
+def twkv_status_string(code: int) -> str:
+    return lib.twkv_status_string(code).decode()

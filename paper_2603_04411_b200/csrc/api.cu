@@ -1,0 +1,345 @@
+// C ABI of libtwkv: cache lifetime, argument checks, piece loop, launch bookkeeping.
+#include <atomic>
+#include <cstdio>
+#include <cstring>
+#include <new>
+#include <vector>
+
+#include "twkv_dev.h"
+
+namespace twkv {
+
+static std::atomic<unsigned long long> g_launches{0};
+void count_launch(int n) { g_launches.fetch_add((unsigned long long)n, std::memory_order_relaxed); }
+
+struct Region { size_t off, bytes; };
+
+struct Layout {
+  size_t total = 0;
+  size_t alloc(size_t bytes, size_t align = 256) {
+    total = (total + align - 1) / align * align;
+    const size_t off = total;
+    total += bytes;
+    return off;
+  }
+};
+
+constexpr int GATE_PIECE = 8192;       // tokens per COMPUTE-mode gate piece (logits scratch rows)
+
+struct Offsets {
+  size_t status, rope_lo, rope_hi, n_tiles, tile_desc, tile_aux, tile_rank, fill, key_last, kclass_count,
+      kclass_tiles, seq_vcount, seq_vtiles, seq_tokens, rank_sums, hist, key_cnt, key_old_fill, key_first_id,
+      key_first_base, key_old_last, scores, seqmax, qslot, part_acc, part_l, gate_scratch, stats_buf, tables_end,
+      blocks, end_fixed;
+};
+
+struct Dims { int d_kv, NC, NT, TPS, NK, rep, max_partials; };
+
+static bool config_ok(const twkv_config* c) {
+  if (!c) return false;
+  if (c->head_dim != HEAD_DIM) return false;
+  if (c->n_kv_heads < 1 || c->n_kv_heads > 8) return false;
+  if (c->n_q_heads % c->n_kv_heads) return false;
+  const int rep = c->n_q_heads / c->n_kv_heads;
+  if (!(rep == 1 || rep == 2 || rep == 4 || rep == 8)) return false;
+  if (c->dtype != TWKV_F16 && c->dtype != TWKV_BF16) return false;
+  if (c->out_dtype != TWKV_F16 && c->out_dtype != TWKV_BF16 && c->out_dtype != TWKV_F32) return false;
+  if (c->n_layers < 1 || c->max_seqs < 1 || c->max_tokens_per_seq < 1) return false;
+  if (c->max_seqs > 4096 || c->n_layers > 1024) return false;
+  if ((long long)c->max_tokens_per_seq > (long long)ROPE_LO * ROPE_HI) return false;
+  if (!(c->tau > 0.f && c->tau < 1.f)) return false;
+  return true;
+}
+
+static Dims dims_of(const twkv_config* c) {
+  Dims d;
+  d.d_kv = c->n_kv_heads * c->head_dim;
+  d.NC = d.d_kv / PANEL;
+  d.TPS = (c->max_tokens_per_seq + TILE - 1) / TILE + d.NC;
+  d.NT = c->max_seqs * d.TPS;
+  d.NK = 2 * c->max_seqs * d.NC;
+  d.rep = c->n_q_heads / c->n_kv_heads;
+  d.max_partials = c->max_seqs + MAX_PARTIALS_EXTRA;
+  return d;
+}
+
+static Offsets layout_of(const twkv_config* c, const Dims& d) {
+  Layout L;
+  Offsets o;
+  const size_t Ls = c->n_layers, S = c->max_seqs, NT = d.NT, NK = d.NK, Hq = c->n_q_heads;
+  o.status = L.alloc(8 * sizeof(int));
+  o.rope_lo = L.alloc((size_t)ROPE_LO * 64 * sizeof(float2));
+  o.rope_hi = L.alloc((size_t)ROPE_HI * 64 * sizeof(float2));
+  o.n_tiles = L.alloc(Ls * 2 * sizeof(int));
+  o.tile_desc = L.alloc(Ls * 2 * NT * sizeof(int4));
+  o.tile_aux = L.alloc(Ls * 2 * NT * TILE * sizeof(int));
+  o.tile_rank = L.alloc(Ls * 2 * NT * TILE * sizeof(unsigned short));
+  o.fill = L.alloc(Ls * NK * sizeof(int));
+  o.key_last = L.alloc(Ls * NK * sizeof(int));
+  o.kclass_count = L.alloc(Ls * d.NC * sizeof(int));
+  o.kclass_tiles = L.alloc(Ls * d.NC * NT * sizeof(int));
+  o.seq_vcount = L.alloc(Ls * S * sizeof(int));
+  o.seq_vtiles = L.alloc(Ls * S * d.TPS * sizeof(int));
+  o.seq_tokens = L.alloc(Ls * S * sizeof(int));
+  o.rank_sums = L.alloc(Ls * 2 * sizeof(unsigned long long));
+  o.tables_end = L.alloc(0);
+  o.hist = L.alloc((size_t)PIECE_CHUNKS * NK * sizeof(int));
+  o.key_cnt = L.alloc(NK * sizeof(int));
+  o.key_old_fill = L.alloc(NK * sizeof(int));
+  o.key_first_id = L.alloc(NK * sizeof(int));
+  o.key_first_base = L.alloc(NK * sizeof(int));
+  o.key_old_last = L.alloc(NK * sizeof(int));
+  o.scores = L.alloc(NT * TILE * Hq * sizeof(float));
+  o.seqmax = L.alloc(S * Hq * sizeof(unsigned));
+  o.qslot = L.alloc(S * sizeof(int));
+  o.part_acc = L.alloc((size_t)d.max_partials * Hq * d.d_kv * sizeof(float));
+  o.part_l = L.alloc((size_t)d.max_partials * Hq * sizeof(float));
+  o.gate_scratch = L.alloc((size_t)GATE_PIECE * 2 * d.d_kv * sizeof(float));
+  o.stats_buf = L.alloc(64 * sizeof(unsigned long long));
+  o.blocks = L.alloc(0, 1024);
+  o.end_fixed = o.blocks;
+  return o;
+}
+
+}  // namespace twkv
+
+using namespace twkv;
+
+struct twkv_cache {
+  twkv_config cfg;
+  Dims dims;
+  Offsets off;
+  DevView view;
+  unsigned char* pool;
+  size_t pool_bytes;
+  int device;
+  int sm_count;
+  std::vector<LayerParams> params;
+};
+
+struct DeviceGuard {
+  int prev = -1;
+  bool ok = true;
+  explicit DeviceGuard(int dev) {
+    if (cudaGetDevice(&prev) != cudaSuccess) { ok = false; return; }
+    if (prev != dev && cudaSetDevice(dev) != cudaSuccess) ok = false;
+    target = dev;
+  }
+  ~DeviceGuard() { if (prev >= 0 && prev != target) cudaSetDevice(prev); }
+  int target = -1;
+};
+
+extern "C" {
+
+const char* twkv_status_string(twkv_status s) {
+  switch (s) {
+    case TWKV_OK: return "ok";
+    case TWKV_ERR_INVALID_ARG: return "invalid argument";
+    case TWKV_ERR_UNSUPPORTED: return "unsupported configuration";
+    case TWKV_ERR_CAPACITY: return "cache capacity exhausted";
+    case TWKV_ERR_CUDA: return "CUDA runtime error";
+    case TWKV_ERR_DEVICE_CHECK: return "device-side check failed";
+    case TWKV_ERR_TIMEOUT: return "bounded device wait timed out";
+  }
+  return "unknown status";
+}
+
+uint64_t twkv_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
+
+size_t twkv_cache_required_bytes(const twkv_config* cfg, size_t payload_bytes) {
+  if (!config_ok(cfg)) return 0;
+  const Dims d = dims_of(cfg);
+  const Offsets o = layout_of(cfg, d);
+  // every (layer, sequence, side) may hold one partially filled tile of every class
+  const size_t slack_blocks = (size_t)cfg->n_layers * cfg->max_seqs * 2 * ((size_t)d.NC * (d.NC + 1) / 2);
+  const size_t payload_blocks = (payload_bytes + BLOCK_BYTES - 1) / BLOCK_BYTES;
+  return o.blocks + (payload_blocks + slack_blocks) * (size_t)BLOCK_BYTES;
+}
+
+static void fill_view(twkv_cache* c) {
+  DevView& v = c->view;
+  const twkv_config& cfg = c->cfg;
+  const Dims& d = c->dims;
+  const Offsets& o = c->off;
+  unsigned char* p = c->pool;
+  v.L = cfg.n_layers; v.Hq = cfg.n_q_heads; v.Hkv = cfg.n_kv_heads; v.rep = d.rep; v.d_kv = d.d_kv; v.NC = d.NC;
+  v.S = cfg.max_seqs; v.tmax = cfg.max_tokens_per_seq; v.NT = d.NT; v.TPS = d.TPS; v.dtype = cfg.dtype;
+  v.out_dtype = cfg.out_dtype; v.NK = d.NK; v.max_partials = d.max_partials; v.tau = cfg.tau; v.sm_scale = cfg.sm_scale;
+  const size_t nb = (c->pool_bytes - o.blocks) / BLOCK_BYTES;
+  v.n_blocks = (int)(nb > 0x7fffffffull ? 0x7fffffffull : nb);
+  v.status = (int*)(p + o.status);
+  v.rope_lo = (float2*)(p + o.rope_lo); v.rope_hi = (float2*)(p + o.rope_hi);
+  v.blocks = p + o.blocks;
+  v.n_tiles = (int*)(p + o.n_tiles); v.tile_desc = (int4*)(p + o.tile_desc); v.tile_aux = (int*)(p + o.tile_aux);
+  v.tile_rank = (unsigned short*)(p + o.tile_rank); v.fill = (int*)(p + o.fill); v.key_last = (int*)(p + o.key_last);
+  v.kclass_count = (int*)(p + o.kclass_count); v.kclass_tiles = (int*)(p + o.kclass_tiles);
+  v.seq_vcount = (int*)(p + o.seq_vcount); v.seq_vtiles = (int*)(p + o.seq_vtiles); v.seq_tokens = (int*)(p + o.seq_tokens);
+  v.rank_sums = (unsigned long long*)(p + o.rank_sums);
+  v.hist = (int*)(p + o.hist); v.key_cnt = (int*)(p + o.key_cnt); v.key_old_fill = (int*)(p + o.key_old_fill);
+  v.key_first_id = (int*)(p + o.key_first_id); v.key_first_base = (int*)(p + o.key_first_base);
+  v.key_old_last = (int*)(p + o.key_old_last);
+  v.scores = (float*)(p + o.scores); v.seqmax = (unsigned*)(p + o.seqmax); v.qslot = (int*)(p + o.qslot);
+  v.part_acc = (float*)(p + o.part_acc); v.part_l = (float*)(p + o.part_l);
+  v.gate_scratch = (float*)(p + o.gate_scratch);
+}
+
+twkv_status twkv_cache_reset(twkv_cache* c, void* stream) {
+  if (!c) return TWKV_ERR_INVALID_ARG;
+  DeviceGuard g(c->device);
+  if (!g.ok) return TWKV_ERR_CUDA;
+  cudaStream_t st = (cudaStream_t)stream;
+  // every table between the RoPE tables and the scratch starts from zero; key_last from -1
+  if (cudaMemsetAsync(c->pool + c->off.n_tiles, 0, c->off.tables_end - c->off.n_tiles, st) != cudaSuccess) return TWKV_ERR_CUDA;
+  if (cudaMemsetAsync(c->pool + c->off.key_last, 0xff, (size_t)c->cfg.n_layers * c->dims.NK * sizeof(int), st) != cudaSuccess)
+    return TWKV_ERR_CUDA;
+  if (cudaMemsetAsync(c->pool + c->off.status, 0, 8 * sizeof(int), st) != cudaSuccess) return TWKV_ERR_CUDA;
+  return TWKV_OK;
+}
+
+twkv_status twkv_cache_create(const twkv_config* cfg, void* pool, size_t pool_bytes, void* stream, twkv_cache** out) {
+  if (!cfg || !pool || !out) return TWKV_ERR_INVALID_ARG;
+  *out = nullptr;
+  if (!config_ok(cfg)) return TWKV_ERR_UNSUPPORTED;
+  if ((uintptr_t)pool % 256) return TWKV_ERR_INVALID_ARG;
+  cudaPointerAttributes attr;
+  if (cudaPointerGetAttributes(&attr, pool) != cudaSuccess) { cudaGetLastError(); return TWKV_ERR_CUDA; }
+  if (attr.type != cudaMemoryTypeDevice && attr.type != cudaMemoryTypeManaged) return TWKV_ERR_INVALID_ARG;
+  const Dims d = dims_of(cfg);
+  const Offsets o = layout_of(cfg, d);
+  if (pool_bytes < o.blocks + (size_t)BLOCK_BYTES) return TWKV_ERR_CAPACITY;
+  twkv_cache* c = new (std::nothrow) twkv_cache();
+  if (!c) return TWKV_ERR_INVALID_ARG;
+  c->cfg = *cfg; c->dims = d; c->off = o; c->pool = (unsigned char*)pool; c->pool_bytes = pool_bytes;
+  c->device = attr.device;
+  c->params.assign(cfg->n_layers, LayerParams{nullptr, nullptr, nullptr, nullptr, nullptr, nullptr});
+  DeviceGuard g(c->device);
+  if (!g.ok) { delete c; return TWKV_ERR_CUDA; }
+  if (cudaDeviceGetAttribute(&c->sm_count, cudaDevAttrMultiProcessorCount, c->device) != cudaSuccess) { delete c; return TWKV_ERR_CUDA; }
+  fill_view(c);
+  twkv_status s = twkv_cache_reset(c, stream);
+  if (s != TWKV_OK) { delete c; return s; }
+  if (launch_rope_tables(c->view, cfg->rope_base, (cudaStream_t)stream) != cudaSuccess) { delete c; return TWKV_ERR_CUDA; }
+  *out = c;
+  return TWKV_OK;
+}
+
+twkv_status twkv_cache_destroy(twkv_cache* c) {
+  if (!c) return TWKV_ERR_INVALID_ARG;
+  delete c;
+  return TWKV_OK;
+}
+
+twkv_status twkv_cache_set_layer_params(twkv_cache* c, int layer, const twkv_layer_params* p) {
+  if (!c || !p || layer < 0 || layer >= c->cfg.n_layers) return TWKV_ERR_INVALID_ARG;
+  if (!p->Uinv_k || !p->Uinv_v) return TWKV_ERR_INVALID_ARG;
+  if (((uintptr_t)p->Uinv_k | (uintptr_t)p->Uinv_v | (uintptr_t)p->W_k | (uintptr_t)p->W_v) % 16) return TWKV_ERR_INVALID_ARG;
+  c->params[layer] = LayerParams{p->Uinv_k, p->Uinv_v, p->W_k, p->W_v, p->b_k, p->b_v};
+  return TWKV_OK;
+}
+
+twkv_status twkv_compress(twkv_cache* c, int layer, const void* K, const void* V, const int32_t* seq_ids,
+                          const int32_t* positions, int n_tok, const float* scores, uint16_t* levels,
+                          twkv_gate_mode mode, void* stream) {
+  if (!c || layer < 0 || layer >= c->cfg.n_layers || n_tok < 0) return TWKV_ERR_INVALID_ARG;
+  if (n_tok == 0) return TWKV_OK;
+  if (!K || !V || !seq_ids || !positions || !levels) return TWKV_ERR_INVALID_ARG;
+  if (((uintptr_t)K | (uintptr_t)V) % 16 || (uintptr_t)levels % 4) return TWKV_ERR_INVALID_ARG;
+  if (mode == TWKV_GATE_LOGITS && (!scores || (uintptr_t)scores % 16)) return TWKV_ERR_INVALID_ARG;
+  if (mode == TWKV_GATE_COMPUTE && (!c->params[layer].W_k || !c->params[layer].W_v)) return TWKV_ERR_INVALID_ARG;
+  if (mode != TWKV_GATE_FORCED && mode != TWKV_GATE_LOGITS && mode != TWKV_GATE_COMPUTE) return TWKV_ERR_INVALID_ARG;
+  DeviceGuard g(c->device);
+  if (!g.ok) return TWKV_ERR_CUDA;
+  cudaStream_t st = (cudaStream_t)stream;
+  const DevView& v = c->view;
+  const size_t row = (size_t)v.d_kv * 2;
+  if (mode == TWKV_GATE_LOGITS) {
+    if (launch_gate_rank(v, scores, levels, n_tok, st) != cudaSuccess) return TWKV_ERR_CUDA;
+  } else if (mode == TWKV_GATE_COMPUTE) {
+    for (int lo = 0; lo < n_tok; lo += GATE_PIECE) {
+      const int n = n_tok - lo < GATE_PIECE ? n_tok - lo : GATE_PIECE;
+      if (launch_gate_logits(v, c->params[layer], (const unsigned char*)K + lo * row, (const unsigned char*)V + lo * row, n,
+                             v.gate_scratch, st) != cudaSuccess) return TWKV_ERR_CUDA;
+      if (launch_gate_rank(v, v.gate_scratch, levels + 2 * (size_t)lo, n, st) != cudaSuccess) return TWKV_ERR_CUDA;
+    }
+  }
+  for (int lo = 0; lo < n_tok; lo += TWKV_PIECE_TOKENS) {
+    const int n = n_tok - lo < TWKV_PIECE_TOKENS ? n_tok - lo : TWKV_PIECE_TOKENS;
+    if (launch_compress_piece(v, layer, (const unsigned char*)K + lo * row, (const unsigned char*)V + lo * row, seq_ids + lo,
+                              positions + lo, n, levels + 2 * (size_t)lo, st) != cudaSuccess) return TWKV_ERR_CUDA;
+  }
+  return TWKV_OK;
+}
+
+twkv_status twkv_decode_attn(twkv_cache* c, int layer, const void* q, const int32_t* seq_ids, int n_seq, void* out,
+                             int num_splits, void* stream) {
+  if (!c || layer < 0 || layer >= c->cfg.n_layers || n_seq < 0 || num_splits < 0) return TWKV_ERR_INVALID_ARG;
+  if (n_seq == 0) return TWKV_OK;
+  if (!q || !seq_ids || !out || n_seq > c->cfg.max_seqs) return TWKV_ERR_INVALID_ARG;
+  if (((uintptr_t)q | (uintptr_t)out) % 16) return TWKV_ERR_INVALID_ARG;
+  if (!c->params[layer].Uinv_k || !c->params[layer].Uinv_v) return TWKV_ERR_INVALID_ARG;
+  const int head_groups = (c->cfg.n_q_heads + 31) / 32;
+  if (num_splits == 0) {
+    num_splits = c->sm_count / (n_seq * head_groups);
+    if (num_splits < 1) num_splits = 1;
+    if (num_splits > 64) num_splits = 64;
+  }
+  if ((long long)n_seq * num_splits > c->dims.max_partials) return TWKV_ERR_INVALID_ARG;
+  DeviceGuard g(c->device);
+  if (!g.ok) return TWKV_ERR_CUDA;
+  if (launch_decode(c->view, layer, c->params[layer], q, seq_ids, n_seq, out, num_splits, c->sm_count,
+                    (cudaStream_t)stream) != cudaSuccess) return TWKV_ERR_CUDA;
+  return TWKV_OK;
+}
+
+twkv_status twkv_cache_status(twkv_cache* c, void* stream) {
+  if (!c) return TWKV_ERR_INVALID_ARG;
+  DeviceGuard g(c->device);
+  if (!g.ok) return TWKV_ERR_CUDA;
+  cudaStream_t st = (cudaStream_t)stream;
+  int code = 0;
+  if (cudaMemcpyAsync(&code, c->view.status, sizeof(int), cudaMemcpyDeviceToHost, st) != cudaSuccess) return TWKV_ERR_CUDA;
+  if (cudaStreamSynchronize(st) != cudaSuccess) return TWKV_ERR_CUDA;
+  if (code != 0) {
+    if (cudaMemsetAsync(c->view.status, 0, sizeof(int), st) != cudaSuccess) return TWKV_ERR_CUDA;
+    if (cudaStreamSynchronize(st) != cudaSuccess) return TWKV_ERR_CUDA;
+  }
+  return (twkv_status)code;
+}
+
+twkv_status twkv_cache_stats(twkv_cache* c, int layer, void* stream, twkv_stats* out) {
+  if (!c || !out || layer < -1 || layer >= c->cfg.n_layers) return TWKV_ERR_INVALID_ARG;
+  DeviceGuard g(c->device);
+  if (!g.ok) return TWKV_ERR_CUDA;
+  cudaStream_t st = (cudaStream_t)stream;
+  unsigned long long* dev = (unsigned long long*)(c->pool + c->off.stats_buf);
+  if (launch_stats(c->view, layer, dev, st) != cudaSuccess) return TWKV_ERR_CUDA;
+  unsigned long long h[5 + 2 * TWKV_MAX_CLASSES];
+  if (cudaMemcpyAsync(h, dev, sizeof(h), cudaMemcpyDeviceToHost, st) != cudaSuccess) return TWKV_ERR_CUDA;
+  if (cudaStreamSynchronize(st) != cudaSuccess) return TWKV_ERR_CUDA;
+  memset(out, 0, sizeof(*out));
+  out->tokens = h[0];
+  out->bytes_stored = h[1];
+  out->bytes_algorithmic = 2 * (h[2] + h[3]);
+  out->blocks_used = h[4];
+  out->blocks_free = (unsigned long long)c->view.n_blocks - h[4];
+  const double denom = (double)h[0] * c->dims.d_kv;
+  out->retain_rate_k = h[0] ? (double)h[2] / denom : 0.0;
+  out->retain_rate_v = h[0] ? (double)h[3] / denom : 0.0;
+  for (int s = 0; s < 2; ++s)
+    for (int k = 0; k < TWKV_MAX_CLASSES; ++k) out->tokens_per_class[s][k] = h[5 + s * TWKV_MAX_CLASSES + k];
+  return TWKV_OK;
+}
+
+twkv_status twkv_cache_layout(const twkv_cache* c, twkv_layout* out) {
+  if (!c || !out) return TWKV_ERR_INVALID_ARG;
+  const Offsets& o = c->off;
+  out->pool_bytes = c->pool_bytes; out->n_blocks = (uint64_t)c->view.n_blocks; out->blocks_off = o.blocks;
+  out->status_off = o.status; out->n_tiles_off = o.n_tiles; out->tile_desc_off = o.tile_desc; out->tile_aux_off = o.tile_aux;
+  out->tile_rank_off = o.tile_rank; out->fill_off = o.fill; out->kclass_count_off = o.kclass_count;
+  out->kclass_tiles_off = o.kclass_tiles; out->seq_vcount_off = o.seq_vcount; out->seq_vtiles_off = o.seq_vtiles;
+  out->seq_tokens_off = o.seq_tokens; out->max_tiles = (uint64_t)c->dims.NT; out->tiles_per_seq = (uint64_t)c->dims.TPS;
+  out->n_classes = (uint64_t)c->dims.NC;
+  return TWKV_OK;
+}
+
+}  // extern "C"

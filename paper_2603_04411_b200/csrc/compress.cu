@@ -1,0 +1,416 @@
+// Compress step: gate -> rank (Eq. 5, 6, 8), slot allocation, truncate + pack (Eq. 2).
+//
+// A compress piece (<= 65536 tokens) runs as: hist (per-chunk key counts) -> alloc (one CTA:
+// exclusive scans, capacity check, tile and block allocation in ascending key order) -> pack
+// (warp per token: 128-bit loads / stores of the retained prefix, +0 fill to the class width).
+// Slot assignment is a function of the token order only (no atomics decide placement), so the
+// packed bytes and tables are reproducible.
+#include "twkv_dev.h"
+
+namespace twkv {
+
+// ------------------------------------------------------------------------------------------
+// Gate: warp per (token, side).  Each lane owns d/32 consecutive logits, so the cumulative sum
+// of Eq. 6 is a lane-local running sum plus a warp scan of the lane totals.
+//   p = softmax(z) (Eq. 5), c_n = sum_{j<=n} p_j, m_i = c_{d+1-i} (Eq. 6),
+//   r = #{i : m_i > tau} = d - #{n : c_n <= tau} (Eq. 8).
+// The comparison c_n <= tau is done as S_n <= tau * S_d on the unnormalised sums.
+// ------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(256) gate_rank_kernel(const float* __restrict__ logits, unsigned short* __restrict__ levels,
+                                                        int n_rows, int d, float tau) {
+  const int warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+  const int lane = threadIdx.x & 31;
+  if (warp >= n_rows) return;
+  const int per = d >> 5;                       // 4 .. 32, multiple of 4
+  const float* z = logits + (size_t)warp * d + lane * per;
+  float v[32];
+  float mx = -INFINITY;
+#pragma unroll
+  for (int i = 0; i < 32; i += 4) {
+    if (i < per) {
+      float4 t = *reinterpret_cast<const float4*>(z + i);
+      v[i] = t.x; v[i + 1] = t.y; v[i + 2] = t.z; v[i + 3] = t.w;
+      mx = fmaxf(mx, fmaxf(fmaxf(t.x, t.y), fmaxf(t.z, t.w)));
+    }
+  }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
+  float run = 0.f;
+#pragma unroll
+  for (int i = 0; i < 32; ++i) {
+    if (i < per) { run += expf(v[i] - mx); v[i] = run; }
+  }
+  float incl = run;                             // inclusive scan of lane totals
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    float t = __shfl_up_sync(0xffffffffu, incl, o);
+    if (lane >= o) incl += t;
+  }
+  const float total = __shfl_sync(0xffffffffu, incl, 31);
+  const float offset = incl - run;
+  const float thr = tau * total;
+  int below = 0;
+#pragma unroll
+  for (int i = 0; i < 32; ++i) {
+    if (i < per) below += (offset + v[i] <= thr) ? 1 : 0;
+  }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) below += __shfl_xor_sync(0xffffffffu, below, o);
+  int r = d - below;
+  if (r < 1) r = 1;                             // only reachable with tau >= 1 or NaN logits
+  if (lane == 0) levels[warp] = (unsigned short)r;
+}
+
+cudaError_t launch_gate_rank(const DevView& v, const float* logits, unsigned short* levels, int n_tok, cudaStream_t st) {
+  const int rows = n_tok * 2;
+  if (rows == 0) return cudaSuccess;
+  const int blocks = (rows + 7) / 8;
+  gate_rank_kernel<<<blocks, 256, 0, st>>>(logits, levels, rows, v.d_kv, v.tau);
+  count_launch();
+  return cudaGetLastError();
+}
+
+// ------------------------------------------------------------------------------------------
+__device__ __forceinline__ int key_of(const DevView& v, int side, int seq, int cls) {
+  return (side * v.S + seq) * v.NC + (cls - 1);
+}
+
+__global__ void __launch_bounds__(CHUNK_TOKENS) hist_kernel(DevView v, const int* __restrict__ seq_ids, const int* __restrict__ positions,
+                                                            const unsigned short* __restrict__ levels, int n_tok) {
+  const int i = blockIdx.x * CHUNK_TOKENS + threadIdx.x;
+  if (i >= n_tok) return;
+  const int seq = seq_ids[i];
+  const int rk = levels[2 * i], rv = levels[2 * i + 1];
+  const int pos = positions[i];
+  if (seq < 0 || seq >= v.S || rk < 1 || rk > v.d_kv || rv < 1 || rv > v.d_kv || pos < 0 || pos >= ROPE_LO * ROPE_HI) {
+    atomicOr(&v.status[3], 1);
+    return;
+  }
+  int* row = v.hist + (size_t)blockIdx.x * v.NK;
+  atomicAdd(&row[key_of(v, 0, seq, (rk + PANEL - 1) / PANEL)], 1);
+  atomicAdd(&row[key_of(v, 1, seq, (rv + PANEL - 1) / PANEL)], 1);
+}
+
+__device__ __forceinline__ int ceil_div(int a, int b) { return (a + b - 1) / b; }
+
+// One CTA of 1024 threads.  Turns per-chunk counts into exclusive bases, checks capacity and,
+// if the whole piece fits, creates the new tiles in ascending key order.
+__global__ void __launch_bounds__(1024) alloc_kernel(DevView v, int layer, int n_chunks) {
+  __shared__ int s_scan[3][1024];
+  __shared__ int s_fail;
+  const int tid = threadIdx.x;
+  const int NK = v.NK;
+  int* fill = v.fill_l(layer);
+  int* key_last = v.key_last_l(layer);
+  if (tid == 0) s_fail = 0;
+  // phase 1: per key, exclusive scan over chunks
+  for (int k = tid; k < NK; k += 1024) {
+    int run = 0;
+    for (int ch = 0; ch < n_chunks; ++ch) {
+      int* p = v.hist + (size_t)ch * NK + k;
+      const int t = *p;
+      *p = run;
+      run += t;
+    }
+    v.key_cnt[k] = run;
+    v.key_old_fill[k] = fill[k];
+  }
+  __syncthreads();
+  // phase 2: new tiles / blocks per key, scanned in key order
+  const int KPT = ceil_div(NK, 1024);
+  const int k0 = tid * KPT, k1 = min(NK, k0 + KPT);
+  const int half = v.S * v.NC;                        // keys per side
+  int sum_tk = 0, sum_tv = 0, sum_b = 0;
+  for (int k = k0; k < k1; ++k) {
+    const int cnt = v.key_cnt[k], old = v.key_old_fill[k];
+    const int nnew = ceil_div(old + cnt, TILE) - ceil_div(old, TILE);
+    if (k < half) sum_tk += nnew; else sum_tv += nnew;
+    sum_b += nnew * (k % v.NC + 1);
+  }
+  s_scan[0][tid] = sum_tk; s_scan[1][tid] = sum_tv; s_scan[2][tid] = sum_b;
+  __syncthreads();
+  for (int o = 1; o < 1024; o <<= 1) {                 // inclusive Hillis-Steele scan
+    int a = 0, b = 0, c = 0;
+    if (tid >= o) { a = s_scan[0][tid - o]; b = s_scan[1][tid - o]; c = s_scan[2][tid - o]; }
+    __syncthreads();
+    s_scan[0][tid] += a; s_scan[1][tid] += b; s_scan[2][tid] += c;
+    __syncthreads();
+  }
+  const int tot_tk = s_scan[0][1023], tot_tv = s_scan[1][1023], tot_b = s_scan[2][1023];
+  const int next_block = v.status[1];
+  int* ntiles = v.ntiles(layer);
+  const int ntk = ntiles[0], ntv = ntiles[1];
+  // capacity: tokens per sequence
+  int* stok = v.stok(layer);
+  for (int s = tid; s < v.S; s += 1024) {
+    int add = 0;
+    for (int c = 0; c < v.NC; ++c) add += v.key_cnt[s * v.NC + c];
+    if (stok[s] + add > v.tmax) atomicOr(&s_fail, 1);
+  }
+  if (tid == 0) {
+    if (next_block + tot_b > v.n_blocks || ntk + tot_tk > v.NT || ntv + tot_tv > v.NT) atomicOr(&s_fail, 1);
+    if (v.status[3]) atomicOr(&s_fail, 2);
+  }
+  __syncthreads();
+  if (s_fail) {
+    if (tid == 0) {
+      v.status[2] = 0;
+      v.status[3] = 0;
+      set_status(v, (s_fail & 2) ? TWKV_ERR_INVALID_ARG : TWKV_ERR_CAPACITY);
+    }
+    return;
+  }
+  // commit
+  int off_tk = s_scan[0][tid] - sum_tk, off_tv = s_scan[1][tid] - sum_tv, off_b = s_scan[2][tid] - sum_b;
+  for (int k = k0; k < k1; ++k) {
+    const int cnt = v.key_cnt[k], old = v.key_old_fill[k];
+    const int side = k >= half ? 1 : 0;
+    const int cls = k % v.NC + 1;
+    const int seq = (k / v.NC) % v.S;
+    const int old_tiles = ceil_div(old, TILE);
+    const int nnew = ceil_div(old + cnt, TILE) - old_tiles;
+    const int first_id = (side ? ntv + off_tv : ntk + off_tk);
+    const int first_base = next_block + off_b;
+    v.key_first_id[k] = first_id;
+    v.key_first_base[k] = first_base;
+    v.key_old_last[k] = key_last[k];
+    if (cnt > 0) {
+      const int nf = old + cnt;
+      int4* desc = v.desc(layer, side);
+      if (old % TILE != 0) desc[key_last[k]].z = min(TILE, nf - (old_tiles - 1) * TILE);
+      for (int j = 0; j < nnew; ++j)
+        desc[first_id + j] = make_int4(seq, cls, min(TILE, nf - (old_tiles + j) * TILE), first_base + j * cls);
+      if (nnew > 0) key_last[k] = first_id + nnew - 1;
+      fill[k] = nf;
+    }
+    if (side) off_tv += nnew; else off_tk += nnew;
+    off_b += nnew * cls;
+  }
+  __syncthreads();
+  // tile lists: K per class (ascending sequence), V per sequence (ascending class)
+  if (tid < v.NC) {
+    int* cnt = v.kcc(layer);
+    int* list = v.kct(layer) + (size_t)tid * v.NT;
+    int run = cnt[tid];
+    for (int s = 0; s < v.S; ++s) {
+      const int k = s * v.NC + tid;
+      const int c = v.key_cnt[k], old = v.key_old_fill[k];
+      const int nnew = ceil_div(old + c, TILE) - ceil_div(old, TILE);
+      const int first = v.key_first_id[k];
+      for (int j = 0; j < nnew; ++j) list[run + j] = first + j;
+      run += nnew;
+    }
+    cnt[tid] = run;
+  }
+  for (int s = tid; s < v.S; s += 1024) {
+    int* list = v.svt(layer) + (size_t)s * v.TPS;
+    int run = v.svc(layer)[s];
+    int add = 0;
+    for (int c = 0; c < v.NC; ++c) {
+      const int k = half + s * v.NC + c;
+      const int cn = v.key_cnt[k], old = v.key_old_fill[k];
+      const int nnew = ceil_div(old + cn, TILE) - ceil_div(old, TILE);
+      const int first = v.key_first_id[k];
+      for (int j = 0; j < nnew; ++j) list[run + j] = first + j;
+      run += nnew;
+      add += v.key_cnt[s * v.NC + c];
+    }
+    v.svc(layer)[s] = run;
+    stok[s] += add;
+  }
+  if (tid == 0) {
+    v.status[1] = next_block + tot_b;
+    ntiles[0] = ntk + tot_tk;
+    ntiles[1] = ntv + tot_tv;
+    v.status[2] = 1;
+  }
+}
+
+// Copies the first r elements of a 16-bit row into the tile's panels, +0 beyond r.
+__device__ __forceinline__ void pack_row(const DevView& v, const uint4* __restrict__ src, int r, int cls, int base, int slot, int lane) {
+  const int nchunks = cls * 8;                            // 16-byte chunks of 8 elements
+  for (int ch = lane; ch < nchunks; ch += 32) {
+    const int e0 = ch * 8;
+    uint4 val = make_uint4(0u, 0u, 0u, 0u);
+    if (e0 < r) {
+      val = __ldg(src + ch);
+      const int keep = r - e0;                            // elements kept in this chunk (>= 1)
+      if (keep < 8) {
+        unsigned* w = reinterpret_cast<unsigned*>(&val);
+#pragma unroll
+        for (int p = 0; p < 4; ++p) {
+          const int left = keep - 2 * p;                  // elements kept in 32-bit word p
+          if (left <= 0) w[p] = 0u;
+          else if (left == 1) w[p] &= 0x0000ffffu;
+        }
+      }
+    }
+    unsigned char* dst = v.blocks + (size_t)(base + (ch >> 3)) * BLOCK_BYTES + slot * (PANEL * 2) + (ch & 7) * 16;
+    *reinterpret_cast<uint4*>(dst) = val;
+  }
+}
+
+__device__ __forceinline__ void zero_tail(const DevView& v, int cls, int base, int slot, int lane) {
+  const int rows = TILE - 1 - slot;
+  const int total = rows * cls * 8;
+  for (int i = lane; i < total; i += 32) {
+    const int panel = i / (rows * 8);
+    const int rem = i - panel * rows * 8;
+    unsigned char* dst = v.blocks + (size_t)(base + panel) * BLOCK_BYTES + (slot + 1) * (PANEL * 2) + rem * 16;
+    *reinterpret_cast<uint4*>(dst) = make_uint4(0u, 0u, 0u, 0u);
+  }
+}
+
+struct Place { int base, slot_cls_r, flags; };   // slot | cls << 8 | r << 16 ; flags bit0 = zero the tile's tail
+
+__global__ void __launch_bounds__(CHUNK_TOKENS) pack_kernel(DevView v, int layer, const void* __restrict__ K, const void* __restrict__ V,
+                                                            const int* __restrict__ seq_ids, const int* __restrict__ positions,
+                                                            const unsigned short* __restrict__ levels, int n_tok) {
+  if (v.status[2] == 0) return;                           // the piece was refused
+  __shared__ int s_key[2][CHUNK_TOKENS];
+  __shared__ Place s_place[2][CHUNK_TOKENS];
+  __shared__ unsigned long long s_sum[2];
+  const int tid = threadIdx.x;
+  const int i = blockIdx.x * CHUNK_TOKENS + tid;
+  const bool valid = i < n_tok;
+  int seq = 0, r[2] = {1, 1};
+  if (valid) { seq = seq_ids[i]; r[0] = levels[2 * i]; r[1] = levels[2 * i + 1]; }
+  int key[2];
+#pragma unroll
+  for (int side = 0; side < 2; ++side) {
+    key[side] = valid ? key_of(v, side, seq, (r[side] + PANEL - 1) / PANEL) : -1 - side;
+    s_key[side][tid] = key[side];
+  }
+  if (tid < 2) s_sum[tid] = 0ull;
+  __syncthreads();
+  int before[2] = {0, 0};
+  for (int j = 0; j < tid; ++j) {
+    before[0] += (s_key[0][j] == key[0]) ? 1 : 0;
+    before[1] += (s_key[1][j] == key[1]) ? 1 : 0;
+  }
+  if (valid) {
+    int kslot = 0;
+#pragma unroll
+    for (int side = 0; side < 2; ++side) {
+      const int k = key[side];
+      const int cls = k % v.NC + 1;
+      const int old = v.key_old_fill[k];
+      const int g = old + v.hist[(size_t)blockIdx.x * v.NK + k] + before[side];
+      const int ord = g / TILE, slot = g % TILE;
+      const int old_tiles = (old + TILE - 1) / TILE;
+      int tile, base;
+      const bool is_new = ord >= old_tiles;
+      if (is_new) {
+        tile = v.key_first_id[k] + (ord - old_tiles);
+        base = v.key_first_base[k] + (ord - old_tiles) * cls;
+      } else {
+        tile = v.key_old_last[k];
+        base = v.desc(layer, side)[tile].w;
+      }
+      const bool last_of_key = (g + 1 == old + v.key_cnt[k]);
+      s_place[side][tid].base = base;
+      s_place[side][tid].slot_cls_r = slot | (cls << 8) | (r[side] << 16);
+      s_place[side][tid].flags = (is_new && last_of_key && slot < TILE - 1) ? 1 : 0;
+      v.rank(layer, side)[(size_t)tile * TILE + slot] = (unsigned short)r[side];
+      if (side == 0) {
+        v.aux(layer, 0)[(size_t)tile * TILE + slot] = positions[i];
+        kslot = tile * TILE + slot;
+      } else {
+        v.aux(layer, 1)[(size_t)tile * TILE + slot] = kslot;
+      }
+    }
+    atomicAdd(&s_sum[0], (unsigned long long)r[0]);
+    atomicAdd(&s_sum[1], (unsigned long long)r[1]);
+  }
+  __syncthreads();
+  if (tid < 2 && s_sum[tid]) atomicAdd(&v.rank_sums[layer * 2 + tid], s_sum[tid]);
+  // warp per token: move the rows
+  const int warp = tid >> 5, lane = tid & 31;
+  const size_t row_bytes = (size_t)v.d_kv * 2;
+  for (int t = warp; t < CHUNK_TOKENS; t += CHUNK_TOKENS / 32) {
+    const int tok = blockIdx.x * CHUNK_TOKENS + t;
+    if (tok >= n_tok) break;
+#pragma unroll
+    for (int side = 0; side < 2; ++side) {
+      const Place p = s_place[side][t];
+      const int slot = p.slot_cls_r & 0xff, cls = (p.slot_cls_r >> 8) & 0xff, rr = p.slot_cls_r >> 16;
+      const unsigned char* src = reinterpret_cast<const unsigned char*>(side ? V : K) + (size_t)tok * row_bytes;
+      pack_row(v, reinterpret_cast<const uint4*>(src), rr, cls, p.base, slot, lane);
+      if (p.flags & 1) zero_tail(v, cls, p.base, slot, lane);
+    }
+  }
+}
+
+cudaError_t launch_compress_piece(const DevView& v, int layer, const void* K, const void* V, const int* seq_ids,
+                                  const int* positions, int n_tok, const unsigned short* levels, cudaStream_t st) {
+  if (n_tok <= 0) return cudaSuccess;
+  const int n_chunks = (n_tok + CHUNK_TOKENS - 1) / CHUNK_TOKENS;
+  cudaError_t e = cudaMemsetAsync(v.hist, 0, (size_t)n_chunks * v.NK * sizeof(int), st);
+  if (e != cudaSuccess) return e;
+  hist_kernel<<<n_chunks, CHUNK_TOKENS, 0, st>>>(v, seq_ids, positions, levels, n_tok);
+  alloc_kernel<<<1, 1024, 0, st>>>(v, layer, n_chunks);
+  pack_kernel<<<n_chunks, CHUNK_TOKENS, 0, st>>>(v, layer, K, V, seq_ids, positions, levels, n_tok);
+  count_launch(3);
+  return cudaGetLastError();
+}
+
+// ------------------------------------------------------------------------------------------
+// Two-level RoPE tables, built once per cache in fp64: angle(pos, i) = pos * base^(-2i/128),
+// pos = hi * 512 + lo.  cos/sin of the sum come from the angle-addition formulas at use.
+// ------------------------------------------------------------------------------------------
+__global__ void rope_tables_kernel(float2* lo, float2* hi, double base) {
+  const int i = threadIdx.x;                                   // frequency 0..63
+  const int row = blockIdx.x;
+  const double theta = pow(base, -2.0 * (double)i / (double)HEAD_DIM);
+  if (row < ROPE_LO) {
+    double s, c;
+    sincos((double)row * theta, &s, &c);
+    lo[row * 64 + i] = make_float2((float)c, (float)s);
+  }
+  if (row < ROPE_HI) {
+    double s, c;
+    sincos((double)row * (double)ROPE_LO * theta, &s, &c);
+    hi[row * 64 + i] = make_float2((float)c, (float)s);
+  }
+}
+
+cudaError_t launch_rope_tables(const DevView& v, float rope_base, cudaStream_t st) {
+  rope_tables_kernel<<<(ROPE_HI > ROPE_LO ? ROPE_HI : ROPE_LO), 64, 0, st>>>(v.rope_lo, v.rope_hi, (double)rope_base);
+  count_launch();
+  return cudaGetLastError();
+}
+
+// ------------------------------------------------------------------------------------------
+// Statistics: tokens per class from the fill table, rank sums, blocks in use.
+// out[0] tokens, [1] bytes_stored, [2] sum r_K, [3] sum r_V, [4] blocks used, [5 ..] tokens_per_class[2][16]
+// ------------------------------------------------------------------------------------------
+__global__ void stats_kernel(DevView v, int layer, unsigned long long* out) {
+  const int l0 = layer < 0 ? 0 : layer, l1 = layer < 0 ? v.L : layer + 1;
+  for (int i = threadIdx.x; i < 5 + 2 * TWKV_MAX_CLASSES; i += blockDim.x) out[i] = 0ull;
+  __syncthreads();
+  const int half = v.S * v.NC;
+  for (int l = l0; l < l1; ++l) {
+    const int* fill = v.fill_l(l);
+    for (int k = threadIdx.x; k < v.NK; k += blockDim.x) {
+      const unsigned long long f = (unsigned long long)fill[k];
+      if (!f) continue;
+      const int side = k >= half, cls = k % v.NC + 1;
+      atomicAdd(&out[5 + side * TWKV_MAX_CLASSES + cls - 1], f);
+      atomicAdd(&out[1], f * (unsigned long long)(cls * PANEL * 2));
+      if (!side) atomicAdd(&out[0], f);
+    }
+    if (threadIdx.x == 0) {
+      atomicAdd(&out[2], v.rank_sums[l * 2]);
+      atomicAdd(&out[3], v.rank_sums[l * 2 + 1]);
+    }
+  }
+  if (threadIdx.x == 0) out[4] = (unsigned long long)v.status[1];
+}
+
+cudaError_t launch_stats(const DevView& v, int layer, unsigned long long* out_dev, cudaStream_t st) {
+  stats_kernel<<<1, 256, 0, st>>>(v, layer, out_dev);
+  count_launch();
+  return cudaGetLastError();
+}
+
+}  // namespace twkv

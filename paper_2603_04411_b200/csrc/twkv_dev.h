@@ -1,0 +1,108 @@
+// Internal definitions shared by the libtwkv translation units (not part of the C ABI).
+#pragma once
+#include <cuda_runtime.h>
+#include <cuda_fp16.h>
+#include <cuda_bf16.h>
+#include <stdint.h>
+#include "twkv.h"
+
+namespace twkv {
+
+constexpr int TILE = TWKV_TILE_TOKENS;      // tokens per tile (the MMA M)
+constexpr int PANEL = TWKV_PANEL_ELEMS;     // elements per panel row
+constexpr int BLOCK_BYTES = TWKV_BLOCK_BYTES;
+constexpr int HEAD_DIM = 128;
+constexpr int CHUNK_TOKENS = 256;           // tokens per compress CTA
+constexpr int PIECE_CHUNKS = TWKV_PIECE_TOKENS / CHUNK_TOKENS;
+constexpr int ROPE_LO = 512;                // pos = hi * 512 + lo
+constexpr int ROPE_HI = 1024;               // positions up to 512 * 1024 - 1
+constexpr int MAX_PARTIALS_EXTRA = 320;     // V-side partial slots beyond max_seqs
+
+// Device view of a cache: plain pointers into the caller's pool.  Passed to kernels by value.
+struct DevView {
+  int L, Hq, Hkv, rep, d_kv, NC, S, tmax, NT, TPS, n_blocks, dtype, out_dtype, NK, max_partials;
+  float tau, sm_scale;
+  int* status;               // [8]: [0] sticky status, [1] next free block, [2] piece_ok, [3] piece flags
+  float2* rope_lo;           // [ROPE_LO][64] (cos, sin) of lo * theta_i
+  float2* rope_hi;           // [ROPE_HI][64] (cos, sin) of hi * 512 * theta_i
+  unsigned char* blocks;     // n_blocks x 16 KiB
+  // per-layer tables (index with the helpers below)
+  int* n_tiles;              // [L][2]
+  int4* tile_desc;           // [L][2][NT]  (seq, class, n_valid, base block)
+  int* tile_aux;             // [L][2][NT][128]
+  unsigned short* tile_rank; // [L][2][NT][128]
+  int* fill;                 // [L][NK]
+  int* key_last;             // [L][NK]  id of the key's newest tile, -1 if none
+  int* kclass_count;         // [L][NC]
+  int* kclass_tiles;         // [L][NC][NT]
+  int* seq_vcount;           // [L][S]
+  int* seq_vtiles;           // [L][S][TPS]
+  int* seq_tokens;           // [L][S]
+  unsigned long long* rank_sums;  // [L][2]  sum of r_K, r_V
+  // scratch shared by all layers
+  int* hist;                 // [PIECE_CHUNKS][NK]   per-chunk key counts -> exclusive bases
+  int* key_cnt;              // [NK]  tokens of the key in the current piece
+  int* key_old_fill;         // [NK]
+  int* key_first_id;         // [NK]  id of the key's first new tile
+  int* key_first_base;       // [NK]  base block of the key's first new tile
+  int* key_old_last;         // [NK]  the key's newest tile before the piece
+  float* scores;             // [NT*128][Hq]
+  unsigned* seqmax;          // [S][Hq]  order-preserving encoding of the running max
+  int* qslot;                // [S]   sequence id -> query index of the current decode call, -1
+  float* part_acc;           // [max_partials][Hq][d_kv]
+  float* part_l;             // [max_partials][Hq]
+  float* gate_scratch;       // COMPUTE mode logits [GATE_PIECE][2][d_kv]
+
+  __host__ __device__ int4* desc(int l, int side) const { return tile_desc + ((size_t)l * 2 + side) * NT; }
+  __host__ __device__ int* aux(int l, int side) const { return tile_aux + ((size_t)l * 2 + side) * NT * TILE; }
+  __host__ __device__ unsigned short* rank(int l, int side) const { return tile_rank + ((size_t)l * 2 + side) * NT * TILE; }
+  __host__ __device__ int* ntiles(int l) const { return n_tiles + l * 2; }
+  __host__ __device__ int* fill_l(int l) const { return fill + (size_t)l * NK; }
+  __host__ __device__ int* key_last_l(int l) const { return key_last + (size_t)l * NK; }
+  __host__ __device__ int* kcc(int l) const { return kclass_count + l * NC; }
+  __host__ __device__ int* kct(int l) const { return kclass_tiles + (size_t)l * NC * NT; }
+  __host__ __device__ int* svc(int l) const { return seq_vcount + l * S; }
+  __host__ __device__ int* svt(int l) const { return seq_vtiles + (size_t)l * S * TPS; }
+  __host__ __device__ int* stok(int l) const { return seq_tokens + l * S; }
+};
+
+struct LayerParams {
+  const void *Uinv_k, *Uinv_v, *W_k, *W_v;
+  const float *b_k, *b_v;
+};
+
+// Order-preserving float <-> unsigned encoding so that atomicMax on unsigned is a float max.
+// 0 encodes "nothing seen yet" (below every float, including -inf).
+__host__ __device__ inline unsigned enc_ordered(float f) {
+  unsigned b;
+#ifdef __CUDA_ARCH__
+  b = __float_as_uint(f);
+#else
+  union { float f; unsigned u; } c; c.f = f; b = c.u;
+#endif
+  return (b & 0x80000000u) ? ~b : (b | 0x80000000u);
+}
+__device__ inline float dec_ordered(unsigned u) {
+  if (u == 0u) return -INFINITY;
+  unsigned b = (u & 0x80000000u) ? (u & 0x7fffffffu) : ~u;
+  return __uint_as_float(b);
+}
+
+__device__ inline void set_status(const DevView& v, int code) { atomicCAS(v.status, 0, code); }
+
+// launch bookkeeping (host)
+void count_launch(int n = 1);
+
+// kernels' host launchers (defined in the .cu files)
+cudaError_t launch_rope_tables(const DevView& v, float rope_base, cudaStream_t st);
+cudaError_t launch_clear_tables(const DevView& v, cudaStream_t st);
+cudaError_t launch_gate_rank(const DevView& v, const float* logits, unsigned short* levels, int n_tok, cudaStream_t st);
+cudaError_t launch_compress_piece(const DevView& v, int layer, const void* K, const void* V, const int* seq_ids,
+                                  const int* positions, int n_tok, const unsigned short* levels, cudaStream_t st);
+cudaError_t launch_decode(const DevView& v, int layer, const LayerParams& lp, const void* q, const int* seq_ids,
+                          int n_seq, void* out, int num_splits, int sm_count, cudaStream_t st);
+cudaError_t launch_gate_logits(const DevView& v, const LayerParams& lp, const void* K, const void* V, int n_tok,
+                               float* logits, cudaStream_t st);
+cudaError_t launch_stats(const DevView& v, int layer, unsigned long long* out_dev, cudaStream_t st);
+
+}  // namespace twkv
