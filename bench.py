@@ -1,0 +1,350 @@
+#!/usr/bin/env python
+"""Benchmark of the libtwkv hot path on the Llama-3-8B-shaped 32k-context workload.
+
+One step = one pass of the whole hot path over one batch: reset the cache, compress all B*T
+tokens (gate logits GEMM -> rank -> truncate + pack) and run one decode-attention step over the
+mixed-rank cache.  The headline value is decode-attention KV tokens/s (B*T / decode time);
+compress tokens/s, HBM GB/s on the compressed bytes and the per-kernel times are reported
+beside it.  `--impl reference` times the fp64 CPU oracle on a bounded sample instead.
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+"""
+import argparse
+import json
+import os
+import subprocess
+import sys
+import tempfile
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+WORKLOAD = "llama3-8b-layer_B16_ctx32768_gqa4_fp16_gate-assigned-ranks"
+B_SEQ, CTX, HQ, HKV, DH = 16, 32768, 32, 8, 128
+D_KV = HKV * DH
+METRIC = "decode_attn_kv_tokens_per_s"
+UNIT = "KV tokens/s"
+NOMINAL_HBM_GBS = 8000.0
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            p = json.load(f)
+        return {"hbm_gbs": float(p["hbm_gbs"]), "tflops": float(p["bf16_tflops_sustained"]), "source": "measured"}
+    return {"hbm_gbs": 6650.0, "tflops": 1400.0, "source": "fallback"}
+
+
+class ClockSampler:
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, device_index):
+        self.f = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
+        self.p = None
+        try:
+            self.p = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits",
+                                       "-lms", "100", "-i", str(device_index)], stdout=self.f, stderr=subprocess.DEVNULL)
+        except OSError:
+            self.p = None
+
+    def stop(self):
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        if self.p is None:
+            return out
+        self.p.terminate()
+        try:
+            self.p.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.p.kill()
+        self.f.flush()
+        self.f.seek(0)
+        sm, mx, reasons, power = [], [], set(), []
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in self.f:
+            parts = [x.strip() for x in line.split(",")]
+            if len(parts) < 7:
+                continue
+            try:
+                sm.append(float(parts[0])); mx.append(float(parts[1])); power.append(float(parts[2]))
+            except ValueError:
+                continue
+            for n, v in zip(names, parts[3:7]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        self.f.close()
+        os.unlink(self.f.name)
+        if sm:
+            sm.sort()
+            out = {"sm_mhz": sm[len(sm) // 2], "sm_max_mhz": max(mx), "reasons": sorted(reasons),
+                   "samples": len(sm), "power_w_max": max(power)}
+        return out
+
+
+def oracle_sample_inputs(li, gate, n_tokens):
+    """Host copies of the first n_tokens of sequence 0 for the CPU oracle (fp64)."""
+    import numpy as np
+    import oracle
+    from tests.helpers import bits16
+    xk = oracle.widen16(bits16(li.xt_k[:n_tokens]), "f16")
+    xv = oracle.widen16(bits16(li.xt_v[:n_tokens]), "f16")
+    Wk, Wv, bk, bv = gate
+    return dict(xk=xk, xv=xv, pos=li.positions[:n_tokens].cpu().numpy(),
+                Uk=oracle.widen16(bits16(li.Uinv_k), "f16"), Uv=oracle.widen16(bits16(li.Uinv_v), "f16"),
+                Wk=oracle.widen16(bits16(Wk), "f16"), Wv=oracle.widen16(bits16(Wv), "f16"),
+                bk=bk.double().cpu().numpy(), bv=bv.double().cpu().numpy(),
+                q=oracle.widen16(bits16(li.q[0]), "f16"))
+
+
+def oracle_step(s, n):
+    """The oracle's pass over n tokens: gate (Eq. 5, 6, 8) then decode attention.  Returns (t_gate, t_decode)."""
+    import oracle
+    t0 = time.perf_counter()
+    rk, _ = oracle.gate_rank(oracle.gate_logits(s["xk"][:n], s["Wk"], s["bk"]), 0.1)
+    rv, _ = oracle.gate_rank(oracle.gate_logits(s["xv"][:n], s["Wv"], s["bv"]), 0.1)
+    t1 = time.perf_counter()
+    oracle.decode_attn(s["xk"][:n], s["xv"][:n], rk, rv, s["pos"][:n], s["Uk"], s["Uv"], s["q"], HKV, 500000.0, DH ** -0.5)
+    t2 = time.perf_counter()
+    return t1 - t0, t2 - t1
+
+
+def sized_oracle_sample(s, target_s, n_max):
+    """Pick a token count whose oracle pass takes about target_s seconds (calibrated on 512 tokens)."""
+    tg, td = oracle_step(s, 512)
+    per_tok = (tg + td) / 512
+    n = int(max(512, min(n_max, target_s / max(per_tok, 1e-9))))
+    return n // 128 * 128
+
+
+def build_workload(device):
+    import torch
+    from paper_2603_04411_b200 import workloads
+    li = workloads.build_layer(1, n_seq=B_SEQ, ctx=CTX, n_q_heads=HQ, n_kv_heads=HKV, dtype=torch.float16,
+                               device=device, outlier="pct:1", mode="forced", level_probs=None)
+    li.ranks = None
+    gate = workloads.gate_params(1, D_KV, torch.float16, device=device)
+    return li, gate
+
+
+def run_reference(args):
+    import torch
+    import oracle
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    from paper_2603_04411_b200 import workloads
+    n_max = 32768
+    li = workloads.build_layer(1, n_seq=1, ctx=n_max, n_q_heads=HQ, n_kv_heads=HKV, dtype=torch.float16,
+                               device="cpu", outlier="pct:1", mode="forced")
+    gate = workloads.gate_params(1, D_KV, torch.float16)
+    s = oracle_sample_inputs(li, gate, n_max)
+    n = sized_oracle_sample(s, 4.0, n_max)
+    for _ in range(args.warmup):
+        oracle_step(s, min(n, 512))
+    t_dec = []
+    t_all = []
+    for _ in range(args.steps):
+        tg, td = oracle_step(s, n)
+        t_dec.append(td); t_all.append(tg + td)
+    ms = 1e3 * sum(t_all) / len(t_all)
+    value = n / (sum(t_dec) / len(t_dec))
+    cores = oracle.num_threads()
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "f64", "data": "synthetic",
+            "config": {"workload": WORKLOAD, "sample": f"{n} tokens of one sequence, {HQ} query heads", "l2": "n/a (CPU)"},
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle",
+                             "sample": f"gate + decode attention over the first {n} tokens of one sequence, all {HQ} heads"},
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line), flush=True)
+
+
+def run_ours(args):
+    import numpy as np
+    import torch
+    import torch.distributed as dist
+
+    from paper_2603_04411_b200 import build as lib_build
+    lib_build.build()
+    from paper_2603_04411_b200 import binding as B
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    assert torch.cuda.is_available(), "bench.py needs a CUDA device; there is no CPU fallback"
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+
+    li, gate = build_workload(dev)
+    Wk, Wv, bk, bv = gate
+    n_tok = B_SEQ * CTX
+    cfg = B.make_config(n_layers=1, n_q_heads=HQ, n_kv_heads=HKV, dtype=torch.float16, out_dtype=torch.float16,
+                        max_seqs=B_SEQ, max_tokens_per_seq=CTX)
+    pool_bytes = B.twkv_cache_required_bytes(cfg, int(n_tok * 2 * 2 * 420))     # room for mean class width ~420
+    pool = torch.empty(pool_bytes, dtype=torch.uint8, device=dev)
+    cache = B.twkv_cache_create(cfg, pool)
+    B.twkv_cache_set_layer_params(cache, 0, li.Uinv_k, li.Uinv_v, Wk, Wv, bk, bv)
+    levels = torch.zeros(n_tok, 2, dtype=torch.int16, device=dev)
+    sid = torch.arange(B_SEQ, dtype=torch.int32, device=dev)
+    out = torch.empty(B_SEQ, HQ, DH, dtype=torch.float16, device=dev)
+    stream = torch.cuda.current_stream()
+
+    def step(ev=None):
+        B.twkv_cache_reset(cache)
+        if ev: ev[0].record(stream)
+        B.twkv_compress(cache, 0, li.xt_k, li.xt_v, li.seq_ids, li.positions, None, levels, B.TWKV_GATE_COMPUTE)
+        if ev: ev[1].record(stream)
+        B.twkv_decode_attn(cache, 0, li.q, sid, out)
+        if ev: ev[2].record(stream)
+
+    def barrier():
+        torch.cuda.synchronize()
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(max(args.warmup, 3)):
+        step()
+    torch.cuda.synchronize()
+    status = B.twkv_cache_status(cache)
+    assert status == B.TWKV_OK, B.twkv_status_string(status)
+    st = B.twkv_cache_stats(cache, 0)
+    assert st.tokens == n_tok
+
+    B.twkv_profile_enable(cache, True)
+    evs = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(args.steps)]
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    launches0 = B.twkv_launch_count()
+    sampler = ClockSampler(local) if rank == 0 else None
+    barrier()
+    e0.record(stream)
+    for i in range(args.steps):
+        step(evs[i])
+    e1.record(stream)
+    barrier()
+    clocks = sampler.stop() if sampler else None
+    launches = B.twkv_launch_count() - launches0
+    prof = B.twkv_profile_read(cache)
+    B.twkv_profile_enable(cache, False)
+    total_ms = e0.elapsed_time(e1)
+    comp_ms = sum(e[0].elapsed_time(e[1]) for e in evs) / args.steps
+    dec_ms = sum(e[1].elapsed_time(e[2]) for e in evs) / args.steps
+    t = torch.tensor([total_ms, comp_ms, dec_ms], dtype=torch.float64, device=dev)
+    if world > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    total_ms, comp_ms, dec_ms = [float(x) for x in t.tolist()]
+    ms_per_step = total_ms / args.steps
+
+    # end to end: host buffers in, host result out, through the same C ABI calls
+    e2e = None
+    n_e2e = min(args.steps, 3)
+    h_xk = torch.empty(li.xt_k.shape, dtype=torch.float16, pin_memory=True).copy_(li.xt_k)
+    h_xv = torch.empty(li.xt_v.shape, dtype=torch.float16, pin_memory=True).copy_(li.xt_v)
+    h_sid = li.seq_ids.cpu().pin_memory(); h_pos = li.positions.cpu().pin_memory(); h_q = li.q.cpu().pin_memory()
+    h_out = torch.empty(out.shape, dtype=out.dtype, pin_memory=True)
+    d_xk, d_xv = torch.empty_like(li.xt_k), torch.empty_like(li.xt_v)
+    d_sid, d_pos, d_q = torch.empty_like(li.seq_ids), torch.empty_like(li.positions), torch.empty_like(li.q)
+
+    def e2e_step():
+        d_xk.copy_(h_xk, non_blocking=True); d_xv.copy_(h_xv, non_blocking=True)
+        d_sid.copy_(h_sid, non_blocking=True); d_pos.copy_(h_pos, non_blocking=True); d_q.copy_(h_q, non_blocking=True)
+        B.twkv_cache_reset(cache)
+        B.twkv_compress(cache, 0, d_xk, d_xv, d_sid, d_pos, None, levels, B.TWKV_GATE_COMPUTE)
+        B.twkv_decode_attn(cache, 0, d_q, sid, out)
+        h_out.copy_(out, non_blocking=True)
+
+    e2e_step()
+    barrier()
+    g0, g1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    g0.record(stream)
+    for _ in range(n_e2e):
+        e2e_step()
+    g1.record(stream)
+    barrier()
+    t = torch.tensor([g0.elapsed_time(g1) / n_e2e], dtype=torch.float64, device=dev)
+    if world > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    e2e_ms = float(t.item())
+    h2d = sum(x.numel() * x.element_size() for x in (h_xk, h_xv, h_sid, h_pos, h_q))
+    d2h = h_out.numel() * h_out.element_size()
+    e2e = {"value": world * n_tok / (e2e_ms * 1e-3), "unit": "KV tokens/s through compress + decode, host buffers",
+           "ms_per_step": e2e_ms, "steps": n_e2e, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h}
+
+    if rank == 0:
+        peaks = measured_peaks()
+        sum_rk = st.retain_rate_k * n_tok * D_KV
+        ks_ms, ks_n = prof["kscore"]
+        flops_k = 2.0 * sum_rk * D_KV + n_tok * (3.0 * D_KV + 2.0 * HQ * DH)
+        ks_avg_ms = ks_ms / max(ks_n, 1)
+        achieved = flops_k / (ks_avg_ms * 1e-3) / 1e12
+        roofline = {"kernel": "kscore_kernel (K reconstruct + RoPE + q.K scores)", "bound": "tensor", "achieved": achieved,
+                    "peak": peaks["tflops"], "unit": "TFLOP/s", "frac": achieved / peaks["tflops"],
+                    "peak_source": f"{peaks['source']} bf16 sustained (fp16 has the same nominal rate)",
+                    "traffic": None, "flops_per_launch": flops_k, "avg_launch_ms": ks_avg_ms}
+        va_ms, va_n = prof["vacc"]
+        pk_ms, pk_n = prof["pack"]
+        gg_ms, gg_n = prof["gate_gemm"]
+        bytes_v = st.bytes_stored / 2.0
+        kernels = {k: {"ms_per_step": v[0] / args.steps, "launches_per_step": v[1] / args.steps} for k, v in prof.items() if v[1]}
+        dec_gbs = st.bytes_stored / (dec_ms * 1e-3) / 1e9
+        extra = {
+            "decode_ms": dec_ms, "compress_ms": comp_ms,
+            "compress_tokens_per_s": world * n_tok / (comp_ms * 1e-3),
+            "decode_hbm_gbs_on_stored_bytes": dec_gbs,
+            "decode_hbm_frac_of_8tbs": dec_gbs / NOMINAL_HBM_GBS,
+            "decode_hbm_frac_of_measured": dec_gbs / peaks["hbm_gbs"],
+            "binding_bound_ms": max(st.bytes_stored / peaks["hbm_gbs"] / 1e6,
+                                    (flops_k + 2.0 * HQ * (st.retain_rate_v * n_tok * D_KV)) / peaks["tflops"] / 1e9),
+            "vacc_gbs": (bytes_v + n_tok * HQ * 4.0) / (va_ms / max(va_n, 1) * 1e-3) / 1e9 if va_n else None,
+            "gate_gemm_tflops": (4.0 * n_tok * D_KV * D_KV) / (gg_ms / args.steps * 1e-3) / 1e12 if gg_n else None,
+            "pack_gbs": (n_tok * 2.0 * D_KV * 2 + st.bytes_stored) / (pk_ms / args.steps * 1e-3) / 1e9 if pk_n else None,
+            "retain_rate_k": st.retain_rate_k, "retain_rate_v": st.retain_rate_v,
+            "bytes_stored": st.bytes_stored, "bytes_algorithmic": st.bytes_algorithmic,
+            "kernels": kernels,
+        }
+        extra["frac_of_binding_bound"] = extra["binding_bound_ms"] / dec_ms
+        # CPU baseline: the oracle as it stands on a bounded sample of the same workload
+        s = oracle_sample_inputs(li, gate, CTX)
+        n_s = sized_oracle_sample(s, 12.0, CTX)
+        tg, td = oracle_step(s, n_s)
+        import oracle
+        cpu = {"value": n_s / td, "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle",
+               "sample": f"decode attention over the first {n_s} tokens of sequence 0, all {HQ} heads, {td:.2f} s "
+                         f"(its gate pass over the same tokens took {tg:.2f} s)"}
+        line = {"metric": METRIC, "value": world * n_tok / (dec_ms * 1e-3), "unit": UNIT, "n_gpus": world, "steps": args.steps,
+                "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
+                "vs_baseline": None, "dtype": "f16", "data": "synthetic",
+                "config": {"workload": WORKLOAD, "batch": B_SEQ, "context": CTX, "n_q_heads": HQ, "n_kv_heads": HKV,
+                           "head_dim": DH, "step": "cache reset + compress(COMPUTE gate) of B*T tokens + one decode-attention step",
+                           "l2": "inputs_exceed_l2 (cache %.0f MB, states 2.1 GB)" % (st.bytes_stored / 1e6),
+                           "sharding": "replica per GPU (independent sequences), no collective"},
+                "roofline": roofline, "cpu_baseline": cpu, "e2e": e2e, "gpu_launches": int(launches), "clocks": clocks}
+        line.update(extra)
+        print(json.dumps(line), flush=True)
+    B.twkv_cache_destroy(cache)
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

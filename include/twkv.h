@@ -173,6 +173,17 @@ twkv_status twkv_cache_status(twkv_cache* cache, void* stream);
 twkv_status twkv_cache_stats(twkv_cache* cache, int layer, void* stream, twkv_stats* out /*host*/);
 /* Where the tables live inside the pool (host call, no device work). */
 twkv_status twkv_cache_layout(const twkv_cache* cache, twkv_layout* out /*host*/);
+/* Per-kernel device timing.  While enabled, every kernel the library launches for this cache is
+ * bracketed by CUDA events on the launching stream (events are host-side resources; no device memory
+ * is allocated).  twkv_profile_read synchronises `stream`, adds the elapsed times of the launches
+ * recorded since the last read to ms[kind] / launches[kind] (host arrays of TWKV_N_KERNELS entries,
+ * overwritten) and forgets them.  At most 8192 launches are kept between reads; later ones are not timed. */
+typedef enum {
+  TWKV_K_GATE_GEMM = 0, TWKV_K_GATE_RANK = 1, TWKV_K_HIST = 2, TWKV_K_ALLOC = 3, TWKV_K_PACK = 4,
+  TWKV_K_PLAN = 5, TWKV_K_KSCORE = 6, TWKV_K_VACC = 7, TWKV_K_MERGE = 8, TWKV_K_OTHER = 9, TWKV_N_KERNELS = 10
+} twkv_kernel_kind;
+twkv_status twkv_profile_enable(twkv_cache* cache, int enable);
+twkv_status twkv_profile_read(twkv_cache* cache, void* stream, double* ms /*host*/, uint64_t* launches /*host*/);
 /* Number of kernels this library has launched so far in the process (host counter). */
 uint64_t twkv_launch_count(void);
 const char* twkv_status_string(twkv_status s);

@@ -21,7 +21,9 @@ TILE_TOKENS, PANEL_ELEMS, BLOCK_BYTES, PIECE_TOKENS, MAX_CLASSES = 128, 64, 1638
 
 EXPORTS = ["twkv_cache_required_bytes", "twkv_cache_create", "twkv_cache_destroy", "twkv_cache_reset",
            "twkv_cache_set_layer_params", "twkv_compress", "twkv_decode_attn", "twkv_cache_status",
-           "twkv_cache_stats", "twkv_cache_layout", "twkv_launch_count", "twkv_status_string"]
+           "twkv_cache_stats", "twkv_cache_layout", "twkv_launch_count", "twkv_status_string",
+           "twkv_profile_enable", "twkv_profile_read"]
+KERNEL_KINDS = ["gate_gemm", "gate_rank", "hist", "alloc", "pack", "plan", "kscore", "vacc", "merge", "other"]
 
 
 class twkv_config(ctypes.Structure):
@@ -67,12 +69,15 @@ def _load():
     L.twkv_cache_status.argtypes = [vp, vp]
     L.twkv_cache_stats.argtypes = [vp, i32, vp, ctypes.POINTER(twkv_stats)]
     L.twkv_cache_layout.argtypes = [vp, ctypes.POINTER(twkv_layout)]
+    L.twkv_profile_enable.argtypes = [vp, i32]
+    L.twkv_profile_read.argtypes = [vp, vp, ctypes.POINTER(ctypes.c_double), ctypes.POINTER(ctypes.c_uint64)]
     L.twkv_launch_count.argtypes = []
     L.twkv_launch_count.restype = ctypes.c_uint64
     L.twkv_status_string.argtypes = [i32]
     L.twkv_status_string.restype = ctypes.c_char_p
     for name in ["twkv_cache_create", "twkv_cache_destroy", "twkv_cache_reset", "twkv_cache_set_layer_params",
-                 "twkv_compress", "twkv_decode_attn", "twkv_cache_status", "twkv_cache_stats", "twkv_cache_layout"]:
+                 "twkv_compress", "twkv_decode_attn", "twkv_cache_status", "twkv_cache_stats", "twkv_cache_layout",
+                 "twkv_profile_enable", "twkv_profile_read"]:
         getattr(L, name).restype = i32
     return L
 
@@ -164,6 +169,19 @@ def twkv_cache_layout(cache) -> twkv_layout:
     lay = twkv_layout()
     _check(lib.twkv_cache_layout(cache, ctypes.byref(lay)), "twkv_cache_layout")
     return lay
+
+
+def twkv_profile_enable(cache, enable: bool):
+    _check(lib.twkv_profile_enable(cache, 1 if enable else 0), "twkv_profile_enable")
+
+
+def twkv_profile_read(cache, stream=None):
+    """-> {kernel name: (total ms, launches)} since the last read."""
+    n = len(KERNEL_KINDS)
+    ms = (ctypes.c_double * n)()
+    cnt = (ctypes.c_uint64 * n)()
+    _check(lib.twkv_profile_read(cache, _stream(stream), ms, cnt), "twkv_profile_read")
+    return {k: (ms[i], int(cnt[i])) for i, k in enumerate(KERNEL_KINDS)}
 
 
 def twkv_launch_count() -> int:

@@ -12,7 +12,31 @@ namespace twkv {
 static std::atomic<unsigned long long> g_launches{0};
 void count_launch(int n) { g_launches.fetch_add((unsigned long long)n, std::memory_order_relaxed); }
 
-struct Region { size_t off, bytes; };
+struct Prof {
+  bool on = false;
+  std::vector<cudaEvent_t> ev;      // pairs: 2 * i = start, 2 * i + 1 = stop
+  std::vector<int> kind;
+  size_t used = 0;
+  static constexpr size_t kMax = 8192;
+};
+static thread_local Prof* t_prof = nullptr;
+void prof_mark(int kind, cudaStream_t st, bool begin) {
+  Prof* p = t_prof;
+  if (!p || !p->on) return;
+  if (begin) {
+    if (p->used >= Prof::kMax) return;
+    p->kind[p->used] = kind;
+    cudaEventRecord(p->ev[2 * p->used], st);
+  } else {
+    if (p->used >= Prof::kMax) return;
+    cudaEventRecord(p->ev[2 * p->used + 1], st);
+    ++p->used;
+  }
+}
+struct ProfBind {
+  explicit ProfBind(Prof* p) { t_prof = p; }
+  ~ProfBind() { t_prof = nullptr; }
+};
 
 struct Layout {
   size_t total = 0;
@@ -115,6 +139,7 @@ struct twkv_cache {
   int device;
   int sm_count;
   std::vector<LayerParams> params;
+  Prof prof;
 };
 
 struct DeviceGuard {
@@ -223,8 +248,42 @@ twkv_status twkv_cache_create(const twkv_config* cfg, void* pool, size_t pool_by
   return TWKV_OK;
 }
 
+twkv_status twkv_profile_enable(twkv_cache* c, int enable) {
+  if (!c) return TWKV_ERR_INVALID_ARG;
+  DeviceGuard g(c->device);
+  if (!g.ok) return TWKV_ERR_CUDA;
+  Prof& p = c->prof;
+  if (enable && p.ev.empty()) {
+    p.ev.resize(2 * Prof::kMax);
+    p.kind.assign(Prof::kMax, 0);
+    for (auto& e : p.ev)
+      if (cudaEventCreate(&e) != cudaSuccess) return TWKV_ERR_CUDA;
+  }
+  p.on = enable != 0;
+  p.used = 0;
+  return TWKV_OK;
+}
+
+twkv_status twkv_profile_read(twkv_cache* c, void* stream, double* ms, uint64_t* launches) {
+  if (!c || !ms || !launches) return TWKV_ERR_INVALID_ARG;
+  DeviceGuard g(c->device);
+  if (!g.ok) return TWKV_ERR_CUDA;
+  if (cudaStreamSynchronize((cudaStream_t)stream) != cudaSuccess) return TWKV_ERR_CUDA;
+  for (int k = 0; k < TWKV_N_KERNELS; ++k) { ms[k] = 0.0; launches[k] = 0; }
+  Prof& p = c->prof;
+  for (size_t i = 0; i < p.used; ++i) {
+    float t = 0.f;
+    if (cudaEventElapsedTime(&t, p.ev[2 * i], p.ev[2 * i + 1]) != cudaSuccess) return TWKV_ERR_CUDA;
+    ms[p.kind[i]] += (double)t;
+    launches[p.kind[i]] += 1;
+  }
+  p.used = 0;
+  return TWKV_OK;
+}
+
 twkv_status twkv_cache_destroy(twkv_cache* c) {
   if (!c) return TWKV_ERR_INVALID_ARG;
+  for (auto& e : c->prof.ev) cudaEventDestroy(e);
   delete c;
   return TWKV_OK;
 }
@@ -249,6 +308,7 @@ twkv_status twkv_compress(twkv_cache* c, int layer, const void* K, const void* V
   if (mode != TWKV_GATE_FORCED && mode != TWKV_GATE_LOGITS && mode != TWKV_GATE_COMPUTE) return TWKV_ERR_INVALID_ARG;
   DeviceGuard g(c->device);
   if (!g.ok) return TWKV_ERR_CUDA;
+  ProfBind pb(&c->prof);
   cudaStream_t st = (cudaStream_t)stream;
   const DevView& v = c->view;
   const size_t row = (size_t)v.d_kv * 2;
@@ -286,6 +346,7 @@ twkv_status twkv_decode_attn(twkv_cache* c, int layer, const void* q, const int3
   if ((long long)n_seq * num_splits > c->dims.max_partials) return TWKV_ERR_INVALID_ARG;
   DeviceGuard g(c->device);
   if (!g.ok) return TWKV_ERR_CUDA;
+  ProfBind pb(&c->prof);
   if (launch_decode(c->view, layer, c->params[layer], q, seq_ids, n_seq, out, num_splits, c->sm_count,
                     (cudaStream_t)stream) != cudaSuccess) return TWKV_ERR_CUDA;
   return TWKV_OK;

@@ -65,7 +65,7 @@ cudaError_t launch_gate_rank(const DevView& v, const float* logits, unsigned sho
   const int rows = n_tok * 2;
   if (rows == 0) return cudaSuccess;
   const int blocks = (rows + 7) / 8;
-  gate_rank_kernel<<<blocks, 256, 0, st>>>(logits, levels, rows, v.d_kv, v.tau);
+  { ProfScope ps(TWKV_K_GATE_RANK, st); gate_rank_kernel<<<blocks, 256, 0, st>>>(logits, levels, rows, v.d_kv, v.tau); }
   count_launch();
   return cudaGetLastError();
 }
@@ -347,9 +347,9 @@ cudaError_t launch_compress_piece(const DevView& v, int layer, const void* K, co
   const int n_chunks = (n_tok + CHUNK_TOKENS - 1) / CHUNK_TOKENS;
   cudaError_t e = cudaMemsetAsync(v.hist, 0, (size_t)n_chunks * v.NK * sizeof(int), st);
   if (e != cudaSuccess) return e;
-  hist_kernel<<<n_chunks, CHUNK_TOKENS, 0, st>>>(v, seq_ids, positions, levels, n_tok);
-  alloc_kernel<<<1, 1024, 0, st>>>(v, layer, n_chunks);
-  pack_kernel<<<n_chunks, CHUNK_TOKENS, 0, st>>>(v, layer, K, V, seq_ids, positions, levels, n_tok);
+  { ProfScope ps(TWKV_K_HIST, st); hist_kernel<<<n_chunks, CHUNK_TOKENS, 0, st>>>(v, seq_ids, positions, levels, n_tok); }
+  { ProfScope ps(TWKV_K_ALLOC, st); alloc_kernel<<<1, 1024, 0, st>>>(v, layer, n_chunks); }
+  { ProfScope ps(TWKV_K_PACK, st); pack_kernel<<<n_chunks, CHUNK_TOKENS, 0, st>>>(v, layer, K, V, seq_ids, positions, levels, n_tok); }
   count_launch(3);
   return cudaGetLastError();
 }

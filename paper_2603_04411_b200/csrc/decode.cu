@@ -384,13 +384,14 @@ merge_kernel(DevView v, const unsigned short* __restrict__ Uinv_v, int n_splits,
 template <bool BF16>
 static cudaError_t launch_decode_t(const DevView& v, int layer, const LayerParams& lp, const void* q, const int* seq_ids,
                                    int n_seq, void* out, int n_splits, int sm_count, cudaStream_t st) {
-  plan_kernel<<<1, 256, 0, st>>>(v, seq_ids, n_seq);
+  { ProfScope ps(TWKV_K_PLAN, st); plan_kernel<<<1, 256, 0, st>>>(v, seq_ids, n_seq); }
   const size_t ks_smem = 2 * KS_STAGES * 16384 + (size_t)v.Hq * HEAD_DIM * 4 + (size_t)TILE * v.Hq * 4;
   const unsigned short* U = reinterpret_cast<const unsigned short*>(lp.Uinv_k);
   const unsigned short* qq = reinterpret_cast<const unsigned short*>(q);
 #define TWKV_KS(REP)                                                                                              \
   {                                                                                                               \
     cudaFuncSetAttribute(kscore_kernel<BF16, REP>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)ks_smem);    \
+    ProfScope ps(TWKV_K_KSCORE, st);                                                                              \
     kscore_kernel<BF16, REP><<<sm_count, KS_THREADS, ks_smem, st>>>(v, layer, U, qq);                             \
   }
   switch (v.rep) {
@@ -404,13 +405,18 @@ static cudaError_t launch_decode_t(const DevView& v, int layer, const LayerParam
   const dim3 vgrid(n_seq * n_splits, (v.Hq + 31) / 32);
   if (v.Hq <= 16) {
     cudaFuncSetAttribute(vacc_kernel<BF16, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)va_smem);
+    ProfScope ps(TWKV_K_VACC, st);
     vacc_kernel<BF16, 1><<<vgrid, VA_THREADS, va_smem, st>>>(v, layer, seq_ids, n_splits);
   } else {
     cudaFuncSetAttribute(vacc_kernel<BF16, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)va_smem);
+    ProfScope ps(TWKV_K_VACC, st);
     vacc_kernel<BF16, 2><<<vgrid, VA_THREADS, va_smem, st>>>(v, layer, seq_ids, n_splits);
   }
   const size_t mg_smem = (size_t)v.rep * v.d_kv * 4;
-  merge_kernel<BF16><<<dim3(n_seq, v.Hkv), 256, mg_smem, st>>>(v, reinterpret_cast<const unsigned short*>(lp.Uinv_v), n_splits, out);
+  {
+    ProfScope ps(TWKV_K_MERGE, st);
+    merge_kernel<BF16><<<dim3(n_seq, v.Hkv), 256, mg_smem, st>>>(v, reinterpret_cast<const unsigned short*>(lp.Uinv_v), n_splits, out);
+  }
   count_launch(4);
   return cudaGetLastError();
 }

@@ -87,6 +87,7 @@ cudaError_t launch_gate_logits(const DevView& v, const LayerParams& lp, const vo
   if (n_tok <= 0) return cudaSuccess;
   const size_t smem = 2 * GG_STAGES * 16384;
   const dim3 grid((n_tok + 127) / 128, v.d_kv / 128, 2);
+  ProfScope ps(TWKV_K_GATE_GEMM, st);
   auto X = [](const void* p) { return reinterpret_cast<const unsigned short*>(p); };
   if (v.dtype == TWKV_BF16) {
     cudaFuncSetAttribute(gate_gemm_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);

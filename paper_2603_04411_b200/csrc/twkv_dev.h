@@ -92,6 +92,13 @@ __device__ inline void set_status(const DevView& v, int code) { atomicCAS(v.stat
 
 // launch bookkeeping (host)
 void count_launch(int n = 1);
+// optional per-kernel event timing of the cache whose API call is running on this thread
+void prof_mark(int kind, cudaStream_t st, bool begin);
+struct ProfScope {
+  int kind; cudaStream_t st;
+  ProfScope(int k, cudaStream_t s) : kind(k), st(s) { prof_mark(kind, st, true); }
+  ~ProfScope() { prof_mark(kind, st, false); }
+};
 
 // kernels' host launchers (defined in the .cu files)
 cudaError_t launch_rope_tables(const DevView& v, float rope_base, cudaStream_t st);

@@ -245,3 +245,28 @@ def config(i: int, device="cpu", ctx=None, n_seq=None, keep_raw=False) -> LayerI
                            device=device, outlier="pct:1", mode="forced", level_probs=tuple(mix),
                            keep_raw=keep_raw)
     raise ValueError(i)
+
+
+def gate_params(seed: int, d_kv: int, dtype, device="cpu", n_bumps: int = 64, first_dim: int = 64,
+                gain: float = 8.0, r_min: int = 7):
+    """Synthetic gate parameters (W, b) of the linear layer in front of the softmax.
+
+    Row first_dim + k of W carries a narrow bump centred on truncation index d + 1 - r_k, with
+    r_k geometric between r_min and d, so the largest of n_bumps spectral components of a
+    token decides which bump wins the softmax.  The resulting ranks are spread over
+    r_min .. d with a mean near d / 4, like the paper's ~25 % Retain Rate operating point.
+    Returns (W_k, W_v, b_k, b_v): W [d, d] in `dtype`, b [d] fp32."""
+    g = _gen(seed + 49979687, "cpu")
+    j = torch.arange(1, d_kv + 1, dtype=torch.float64)
+    out = []
+    for side in range(2):
+        W = torch.zeros(d_kv, d_kv, dtype=torch.float64)
+        rk = r_min * (d_kv / r_min) ** (torch.arange(n_bumps, dtype=torch.float64) / (n_bumps - 1))
+        rk = rk.round().clamp(1, d_kv)
+        perm = torch.randperm(n_bumps, generator=g)
+        for k in range(n_bumps):
+            centre = d_kv + 1 - rk[perm[k]]
+            W[first_dim + k] = gain * torch.exp(-(j - centre).abs() / 2.0)
+        out.append(W.to(dtype).to(device))
+    b = [(0.1 * torch.randn(d_kv, generator=g)).to(torch.float32).to(device) for _ in range(2)]
+    return out[0], out[1], b[0], b[1]
