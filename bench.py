@@ -48,7 +48,7 @@ class ClockSampler:
         self.p = None
         try:
             self.p = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits",
-                                       "-lms", "100", "-i", str(device_index)], stdout=self.f, stderr=subprocess.DEVNULL)
+                                       "-lms", "20", "-i", str(device_index)], stdout=self.f, stderr=subprocess.DEVNULL)
         except OSError:
             self.p = None
 
@@ -311,13 +311,16 @@ def run_ours(args):
         }
         extra["frac_of_binding_bound"] = extra["binding_bound_ms"] / dec_ms
         # CPU baseline: the oracle as it stands on a bounded sample of the same workload
-        s = oracle_sample_inputs(li, gate, CTX)
-        n_s = sized_oracle_sample(s, 12.0, CTX)
-        tg, td = oracle_step(s, n_s)
         import oracle
-        cpu = {"value": n_s / td, "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle",
-               "sample": f"decode attention over the first {n_s} tokens of sequence 0, all {HQ} heads, {td:.2f} s "
-                         f"(its gate pass over the same tokens took {tg:.2f} s)"}
+        s = oracle_sample_inputs(li, gate, CTX)
+        n_s = sized_oracle_sample(s, 6.0, CTX)
+        reps, tg, td = 0, 0.0, 0.0
+        while reps < 16 and tg + td < 12.0:                    # repeat the sample until ~12 s of CPU work
+            a, b = oracle_step(s, n_s)
+            tg, td, reps = tg + a, td + b, reps + 1
+        cpu = {"value": reps * n_s / td, "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle",
+               "sample": f"{reps} x decode attention over the first {n_s} tokens of sequence 0, all {HQ} heads, "
+                         f"{td:.2f} s in total (the gate passes over the same tokens took {tg:.2f} s)"}
         line = {"metric": METRIC, "value": world * n_tok / (dec_ms * 1e-3), "unit": UNIT, "n_gpus": world, "steps": args.steps,
                 "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
                 "vs_baseline": None, "dtype": "f16", "data": "synthetic",
@@ -336,7 +339,7 @@ def run_ours(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--steps", type=int, default=40)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     args = ap.parse_args()
