@@ -244,38 +244,39 @@ def run_ours(args):
 
     # end to end: host buffers in, host result out, through the same C ABI calls
     e2e = None
-    n_e2e = min(args.steps, 3)
-    h_xk = torch.empty(li.xt_k.shape, dtype=torch.float16, pin_memory=True).copy_(li.xt_k)
-    h_xv = torch.empty(li.xt_v.shape, dtype=torch.float16, pin_memory=True).copy_(li.xt_v)
-    h_sid = li.seq_ids.cpu().pin_memory(); h_pos = li.positions.cpu().pin_memory(); h_q = li.q.cpu().pin_memory()
-    h_out = torch.empty(out.shape, dtype=out.dtype, pin_memory=True)
-    d_xk, d_xv = torch.empty_like(li.xt_k), torch.empty_like(li.xt_v)
-    d_sid, d_pos, d_q = torch.empty_like(li.seq_ids), torch.empty_like(li.positions), torch.empty_like(li.q)
+    n_e2e = 0 if args.skip_e2e else min(args.steps, 3)
+    if n_e2e:
+        h_xk = torch.empty(li.xt_k.shape, dtype=torch.float16, pin_memory=True).copy_(li.xt_k)
+        h_xv = torch.empty(li.xt_v.shape, dtype=torch.float16, pin_memory=True).copy_(li.xt_v)
+        h_sid = li.seq_ids.cpu().pin_memory(); h_pos = li.positions.cpu().pin_memory(); h_q = li.q.cpu().pin_memory()
+        h_out = torch.empty(out.shape, dtype=out.dtype, pin_memory=True)
+        d_xk, d_xv = torch.empty_like(li.xt_k), torch.empty_like(li.xt_v)
+        d_sid, d_pos, d_q = torch.empty_like(li.seq_ids), torch.empty_like(li.positions), torch.empty_like(li.q)
 
-    def e2e_step():
-        d_xk.copy_(h_xk, non_blocking=True); d_xv.copy_(h_xv, non_blocking=True)
-        d_sid.copy_(h_sid, non_blocking=True); d_pos.copy_(h_pos, non_blocking=True); d_q.copy_(h_q, non_blocking=True)
-        B.twkv_cache_reset(cache)
-        B.twkv_compress(cache, 0, d_xk, d_xv, d_sid, d_pos, None, levels, B.TWKV_GATE_COMPUTE)
-        B.twkv_decode_attn(cache, 0, d_q, sid, out)
-        h_out.copy_(out, non_blocking=True)
+        def e2e_step():
+            d_xk.copy_(h_xk, non_blocking=True); d_xv.copy_(h_xv, non_blocking=True)
+            d_sid.copy_(h_sid, non_blocking=True); d_pos.copy_(h_pos, non_blocking=True); d_q.copy_(h_q, non_blocking=True)
+            B.twkv_cache_reset(cache)
+            B.twkv_compress(cache, 0, d_xk, d_xv, d_sid, d_pos, None, levels, B.TWKV_GATE_COMPUTE)
+            B.twkv_decode_attn(cache, 0, d_q, sid, out)
+            h_out.copy_(out, non_blocking=True)
 
-    e2e_step()
-    barrier()
-    g0, g1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    g0.record(stream)
-    for _ in range(n_e2e):
         e2e_step()
-    g1.record(stream)
-    barrier()
-    t = torch.tensor([g0.elapsed_time(g1) / n_e2e], dtype=torch.float64, device=dev)
-    if world > 1:
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-    e2e_ms = float(t.item())
-    h2d = sum(x.numel() * x.element_size() for x in (h_xk, h_xv, h_sid, h_pos, h_q))
-    d2h = h_out.numel() * h_out.element_size()
-    e2e = {"value": world * n_tok / (e2e_ms * 1e-3), "unit": "KV tokens/s through compress + decode, host buffers",
-           "ms_per_step": e2e_ms, "steps": n_e2e, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h}
+        barrier()
+        g0, g1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        g0.record(stream)
+        for _ in range(n_e2e):
+            e2e_step()
+        g1.record(stream)
+        barrier()
+        t = torch.tensor([g0.elapsed_time(g1) / n_e2e], dtype=torch.float64, device=dev)
+        if world > 1:
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        e2e_ms = float(t.item())
+        h2d = sum(x.numel() * x.element_size() for x in (h_xk, h_xv, h_sid, h_pos, h_q))
+        d2h = h_out.numel() * h_out.element_size()
+        e2e = {"value": world * n_tok / (e2e_ms * 1e-3), "unit": "KV tokens/s through compress + decode, host buffers",
+               "ms_per_step": e2e_ms, "steps": n_e2e, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h}
 
     if rank == 0:
         peaks = measured_peaks()
@@ -312,13 +313,15 @@ def run_ours(args):
         extra["frac_of_binding_bound"] = extra["binding_bound_ms"] / dec_ms
         # CPU baseline: the oracle as it stands on a bounded sample of the same workload
         import oracle
-        s = oracle_sample_inputs(li, gate, CTX)
-        n_s = sized_oracle_sample(s, 6.0, CTX)
+        cpu = None
+        s = None if args.skip_cpu_baseline else oracle_sample_inputs(li, gate, CTX)
+        n_s = sized_oracle_sample(s, 6.0, CTX) if s else 0
         reps, tg, td = 0, 0.0, 0.0
-        while reps < 16 and tg + td < 12.0:                    # repeat the sample until ~12 s of CPU work
+        while s and reps < 16 and tg + td < 12.0:              # repeat the sample until ~12 s of CPU work
             a, b = oracle_step(s, n_s)
             tg, td, reps = tg + a, td + b, reps + 1
-        cpu = {"value": reps * n_s / td, "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle",
+        if s:
+          cpu = {"value": reps * n_s / td, "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle",
                "sample": f"{reps} x decode attention over the first {n_s} tokens of sequence 0, all {HQ} heads, "
                          f"{td:.2f} s in total (the gate passes over the same tokens took {tg:.2f} s)"}
         line = {"metric": METRIC, "value": world * n_tok / (dec_ms * 1e-3), "unit": UNIT, "n_gpus": world, "steps": args.steps,
@@ -337,12 +340,20 @@ def run_ours(args):
 
 
 def main():
+    global B_SEQ, CTX, WORKLOAD
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=40)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--batch", type=int, default=B_SEQ, help="sequences (default: the benchmark workload's 16)")
+    ap.add_argument("--ctx", type=int, default=CTX, help="context length (default: the benchmark workload's 32768)")
+    ap.add_argument("--skip-e2e", action="store_true", help="profiling runs: leave the host-buffer leg out")
+    ap.add_argument("--skip-cpu-baseline", action="store_true", help="profiling runs: leave the oracle leg out")
     args = ap.parse_args()
+    if (args.batch, args.ctx) != (B_SEQ, CTX):
+        B_SEQ, CTX = args.batch, args.ctx
+        WORKLOAD = f"reduced-for-profiling_B{B_SEQ}_ctx{CTX}_gqa4_fp16_gate-assigned-ranks"
     if args.impl == "reference":
         run_reference(args)
     else:

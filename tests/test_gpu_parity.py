@@ -284,3 +284,39 @@ def test_two_layers_share_one_pool(B):
     B.twkv_cache_reset(gc.h)
     assert gc.tables()["fill"].sum() == 0 and B.twkv_cache_stats(gc.h, -1).tokens == 0
     gc.close()
+
+
+def test_compute_mode_gate_levels_bit_exact(B):
+    # the library forms z = x~ W + b itself (tensor cores, fp32 accumulation of 16-bit products);
+    # tokens whose cumulative softmax comes within 1e-2 (relative) of tau in the oracle are left
+    # out, because their integer rank may legitimately depend on the accumulation order
+    li = workloads.config(2, ctx=700, n_seq=2)
+    Wk, Wv, bk, bv = workloads.gate_params(7, li.d_kv, torch.float16)
+    zk = oracle.gate_logits(oracle.widen16(bits16(li.xt_k), "f16"), oracle.widen16(bits16(Wk), "f16"), bk.double().numpy())
+    zv = oracle.gate_logits(oracle.widen16(bits16(li.xt_v), "f16"), oracle.widen16(bits16(Wv), "f16"), bv.double().numpy())
+    rk, mk = oracle.gate_rank(zk, 0.1)
+    rv, mv = oracle.gate_rank(zv, 0.1)
+    keep = np.nonzero((mk >= 1e-2) & (mv >= 1e-2))[0]
+    assert len(keep) > 0.9 * len(rk)
+    sel = torch.from_numpy(keep)
+    for name in ["xt_k", "xt_v", "seq_ids", "positions"]:
+        setattr(li, name, getattr(li, name)[sel].contiguous())
+    ranks = np.stack([rk[keep], rv[keep]], axis=1).astype(np.int64)
+    li = to_cuda(li)
+    n = len(keep)
+    gc = GpuCache(B, n_layers=1, n_q_heads=32, n_kv_heads=8, dtype=torch.float16, out_dtype=torch.float32,
+                  max_seqs=2, max_tokens_per_seq=700, payload_bytes=int((-(-ranks // 64) * 128).sum()))
+    gate = [t.cuda().contiguous() for t in (Wk, Wv, bk, bv)]       # borrowed by the cache: keep them alive
+    B.twkv_cache_set_layer_params(gc.h, 0, li.Uinv_k, li.Uinv_v, *gate)
+    levels = torch.zeros(n, 2, dtype=torch.int16, device="cuda")
+    B.twkv_compress(gc.h, 0, li.xt_k, li.xt_v, li.seq_ids, li.positions, None, levels, B.TWKV_GATE_COMPUTE)
+    assert B.twkv_cache_status(gc.h) == B.TWKV_OK
+    np.testing.assert_array_equal(levels.cpu().numpy().view(np.uint16).astype(np.int64), ranks)
+    img = CacheImage(1, li.d_kv, 2, 700, int(gc.lay.n_blocks))
+    assert img.append(0, bits16(li.xt_k), bits16(li.xt_v), li.seq_ids.cpu().numpy(), li.positions.cpu().numpy(), ranks)
+    compare_cache_with_image(gc, img)
+    out = torch.empty(2, 32, 128, device="cuda")
+    B.twkv_decode_attn(gc.h, 0, li.q, torch.tensor([0, 1], dtype=torch.int32, device="cuda"), out)
+    max_abs, rel_l2 = attn_errors(out.cpu().numpy(), oracle_decode(li, ranks, [0, 1]))
+    assert max_abs < MAX_ABS and rel_l2 < REL_L2, (max_abs, rel_l2)
+    gc.close()
