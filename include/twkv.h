@@ -173,6 +173,28 @@ twkv_status twkv_cache_status(twkv_cache* cache, void* stream);
 twkv_status twkv_cache_stats(twkv_cache* cache, int layer, void* stream, twkv_stats* out /*host*/);
 /* Where the tables live inside the pool (host call, no device work). */
 twkv_status twkv_cache_layout(const twkv_cache* cache, twkv_layout* out /*host*/);
+/*
+ * Gate ranks without any caller-provided scratch (the paper has no counterpart; this is a
+ * convenience of the library).  Computes, for n_tok tokens, the same (r_K, r_V) that twkv_compress
+ * produces in TWKV_GATE_COMPUTE mode (Eq. 5, 6, 8), but needs no cache and allocates nothing: the
+ * fp32 logits are staged in a 4 MiB array that is part of the library image and is resident on
+ * every GPU that loads the library, until the process exits.  It is meant for callers that cannot
+ * obtain device memory at the point of the call, for instance a scheduler that sizes cache blocks
+ * from predicted ranks before a pool exists, or a serving loop whose framework owns all device
+ * memory and forbids allocations (which may also synchronise the whole device).
+ *   K, V      [n_tok x d_kv] spectral states, `dtype` (TWKV_F16 / TWKV_BF16); W_k, W_v [d_kv x d_kv] `dtype`;
+ *   b_k, b_v  [d_kv] fp32 or NULL; levels [n_tok x 2] uint16 OUTPUT; d_kv a multiple of 128, at most 1024
+ * Limit: n_tok * 2 * d_kv <= TWKV_STATIC_GATE_MAX_ROWS * 1024 (512 tokens at d_kv = 1024); more returns
+ * TWKV_ERR_CAPACITY and launches nothing.  The first call on a device looks the array's address up
+ * (a host-side set-up step), so make that first call before any stream capture begins.  All calls on a
+ * device share the array: calls that overlap on the GPU (other streams or threads) race; calls queued
+ * on one stream are safe.  Nothing has to be cleared between calls.
+ */
+#define TWKV_STATIC_GATE_MAX_ROWS 1024
+twkv_status twkv_gate_ranks_static(const void* K, const void* V, const void* W_k, const void* W_v,
+                                   const float* b_k, const float* b_v, int n_tok, int d_kv, int dtype,
+                                   float tau, uint16_t* levels, void* stream);
+
 /* Per-kernel device timing.  While enabled, every kernel the library launches for this cache is
  * bracketed by CUDA events on the launching stream (events are host-side resources; no device memory
  * is allocated).  twkv_profile_read synchronises `stream`, adds the elapsed times of the launches

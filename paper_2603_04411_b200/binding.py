@@ -22,7 +22,8 @@ TILE_TOKENS, PANEL_ELEMS, BLOCK_BYTES, PIECE_TOKENS, MAX_CLASSES = 128, 64, 1638
 EXPORTS = ["twkv_cache_required_bytes", "twkv_cache_create", "twkv_cache_destroy", "twkv_cache_reset",
            "twkv_cache_set_layer_params", "twkv_compress", "twkv_decode_attn", "twkv_cache_status",
            "twkv_cache_stats", "twkv_cache_layout", "twkv_launch_count", "twkv_status_string",
-           "twkv_profile_enable", "twkv_profile_read"]
+           "twkv_profile_enable", "twkv_profile_read", "twkv_gate_ranks_static"]
+STATIC_GATE_MAX_ROWS = 1024
 KERNEL_KINDS = ["gate_gemm", "gate_rank", "hist", "alloc", "pack", "plan", "kscore", "vacc", "merge", "other"]
 
 
@@ -71,6 +72,8 @@ def _load():
     L.twkv_cache_layout.argtypes = [vp, ctypes.POINTER(twkv_layout)]
     L.twkv_profile_enable.argtypes = [vp, i32]
     L.twkv_profile_read.argtypes = [vp, vp, ctypes.POINTER(ctypes.c_double), ctypes.POINTER(ctypes.c_uint64)]
+    L.twkv_gate_ranks_static.argtypes = [vp, vp, vp, vp, vp, vp, i32, i32, i32, ctypes.c_float, vp, vp]
+    L.twkv_gate_ranks_static.restype = i32
     L.twkv_launch_count.argtypes = []
     L.twkv_launch_count.restype = ctypes.c_uint64
     L.twkv_status_string.argtypes = [i32]
@@ -182,6 +185,16 @@ def twkv_profile_read(cache, stream=None):
     cnt = (ctypes.c_uint64 * n)()
     _check(lib.twkv_profile_read(cache, _stream(stream), ms, cnt), "twkv_profile_read")
     return {k: (ms[i], int(cnt[i])) for i, k in enumerate(KERNEL_KINDS)}
+
+
+def twkv_gate_ranks_static(K, V, W_k, W_v, b_k, b_v, levels, tau=0.1, stream=None, n_tok=None):
+    """Gate ranks for a few tokens with the logits staged in the library's own fixed 4 MiB device
+    array: no cache, no pool, no allocation.  For callers that cannot get device memory when they
+    need the ranks (see include/twkv.h).  At most 512 tokens at d_kv = 1024; calls that overlap on
+    the GPU share that array and race, calls on one stream do not."""
+    n = K.shape[0] if n_tok is None else n_tok
+    _check(lib.twkv_gate_ranks_static(_ptr(K), _ptr(V), _ptr(W_k), _ptr(W_v), _ptr(b_k), _ptr(b_v), n, K.shape[1],
+                                      dtype_code(K.dtype), tau, _ptr(levels), _stream(stream)), "twkv_gate_ranks_static")
 
 
 def twkv_launch_count() -> int:
