@@ -5,7 +5,11 @@
 #include <new>
 #include <vector>
 
+#include <cstdlib>
+#include <cudaTypedefs.h>
+
 #include "twkv_dev.h"
+#include "tc_util.cuh"
 
 namespace twkv {
 
@@ -38,6 +42,27 @@ struct ProfBind {
   ~ProfBind() { t_prof = nullptr; }
 };
 
+// cuTensorMapEncodeTiled through the runtime's driver entry point (no link against libcuda).
+bool make_tmap_2d(CUtensorMap* out, const void* base, uint64_t rows, uint64_t cols, uint64_t row_stride_bytes, uint32_t box_rows) {
+  static PFN_cuTensorMapEncodeTiled_v12000 encode = nullptr;
+  if (!encode) {
+    void* fn = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) != cudaSuccess || !fn) {
+      cudaGetLastError();
+      return false;
+    }
+    encode = reinterpret_cast<PFN_cuTensorMapEncodeTiled_v12000>(fn);
+  }
+  const cuuint64_t dims[2] = {cols, rows};
+  const cuuint64_t strides[1] = {row_stride_bytes};
+  const cuuint32_t box[2] = {(cuuint32_t)PANEL, box_rows};
+  const cuuint32_t estr[2] = {1, 1};
+  return encode(out, CU_TENSOR_MAP_DATA_TYPE_UINT16, 2, const_cast<void*>(base), dims, strides, box, estr,
+                CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
 struct Layout {
   size_t total = 0;
   size_t alloc(size_t bytes, size_t align = 256) {
@@ -53,7 +78,7 @@ constexpr int GATE_PIECE = 8192;       // tokens per COMPUTE-mode gate piece (lo
 struct Offsets {
   size_t status, rope_lo, rope_hi, n_tiles, tile_desc, tile_aux, tile_rank, fill, key_last, kclass_count,
       kclass_tiles, seq_vcount, seq_vtiles, seq_tokens, rank_sums, hist, key_cnt, key_old_fill, key_first_id,
-      key_first_base, key_old_last, scores, seqmax, qslot, part_acc, part_l, gate_scratch, stats_buf, tables_end,
+      key_first_base, key_old_last, scores, seqmax, qslot, part_acc, part_l, gate_scratch, stats_buf, tables_end, prep_uinvT,
       blocks, end_fixed;
 };
 
@@ -120,6 +145,7 @@ static Offsets layout_of(const twkv_config* c, const Dims& d) {
   o.part_l = L.alloc((size_t)d.max_partials * Hq * sizeof(float));
   o.gate_scratch = L.alloc((size_t)GATE_PIECE * 2 * d.d_kv * sizeof(float));
   o.stats_buf = L.alloc(64 * sizeof(unsigned long long));
+  o.prep_uinvT = L.alloc(Ls * (size_t)d.d_kv * d.d_kv * 2, 1024);
   o.blocks = L.alloc(0, 1024);
   o.end_fixed = o.blocks;
   return o;
@@ -140,6 +166,10 @@ struct twkv_cache {
   int sm_count;
   std::vector<LayerParams> params;
   Prof prof;
+  bool use_tc = false;                 // tcgen05 / TMA kernels (tensor maps could be built)
+  CUtensorMap map_blocks;
+  std::vector<CUtensorMap> map_uinvT;  // per layer, over the transposed copy of U_K^-1 inside the pool
+  std::vector<char> prepared;          // per layer: transposed copy and its map are current
 };
 
 struct DeviceGuard {
@@ -241,6 +271,11 @@ twkv_status twkv_cache_create(const twkv_config* cfg, void* pool, size_t pool_by
   if (!g.ok) { delete c; return TWKV_ERR_CUDA; }
   if (cudaDeviceGetAttribute(&c->sm_count, cudaDevAttrMultiProcessorCount, c->device) != cudaSuccess) { delete c; return TWKV_ERR_CUDA; }
   fill_view(c);
+  c->map_uinvT.resize(cfg->n_layers);
+  c->prepared.assign(cfg->n_layers, 0);
+  const char* legacy = getenv("TWKV_LEGACY_MMA");
+  c->use_tc = !(legacy && legacy[0] == '1') &&
+              make_tmap_2d(&c->map_blocks, c->view.blocks, (uint64_t)c->view.n_blocks * TILE, PANEL, PANEL * 2, TILE);
   twkv_status s = twkv_cache_reset(c, stream);
   if (s != TWKV_OK) { delete c; return s; }
   if (launch_rope_tables(c->view, cfg->rope_base, (cudaStream_t)stream) != cudaSuccess) { delete c; return TWKV_ERR_CUDA; }
@@ -293,6 +328,7 @@ twkv_status twkv_cache_set_layer_params(twkv_cache* c, int layer, const twkv_lay
   if (!p->Uinv_k || !p->Uinv_v) return TWKV_ERR_INVALID_ARG;
   if (((uintptr_t)p->Uinv_k | (uintptr_t)p->Uinv_v | (uintptr_t)p->W_k | (uintptr_t)p->W_v) % 16) return TWKV_ERR_INVALID_ARG;
   c->params[layer] = LayerParams{p->Uinv_k, p->Uinv_v, p->W_k, p->W_v, p->b_k, p->b_v};
+  c->prepared[layer] = 0;
   return TWKV_OK;
 }
 
@@ -347,7 +383,21 @@ twkv_status twkv_decode_attn(twkv_cache* c, int layer, const void* q, const int3
   DeviceGuard g(c->device);
   if (!g.ok) return TWKV_ERR_CUDA;
   ProfBind pb(&c->prof);
-  if (launch_decode(c->view, layer, c->params[layer], q, seq_ids, n_seq, out, num_splits, c->sm_count,
+  TcMaps maps;
+  const TcMaps* pm = nullptr;
+  if (c->use_tc) {
+    if (!c->prepared[layer]) {
+      // first decode after the parameters were (re)set: K-major copy of U_K^-1 for the tensor cores
+      unsigned char* dst = c->pool + c->off.prep_uinvT + (size_t)layer * c->dims.d_kv * c->dims.d_kv * 2;
+      if (launch_transpose16(c->params[layer].Uinv_k, dst, c->dims.d_kv, (cudaStream_t)stream) != cudaSuccess) return TWKV_ERR_CUDA;
+      if (!make_tmap_2d(&c->map_uinvT[layer], dst, c->dims.d_kv, c->dims.d_kv, (uint64_t)c->dims.d_kv * 2, HEAD_DIM)) return TWKV_ERR_CUDA;
+      c->prepared[layer] = 1;
+    }
+    maps.blocks = c->map_blocks;
+    maps.uinvT_k = c->map_uinvT[layer];
+    pm = &maps;
+  }
+  if (launch_decode(c->view, layer, c->params[layer], q, seq_ids, n_seq, out, num_splits, c->sm_count, pm,
                     (cudaStream_t)stream) != cudaSuccess) return TWKV_ERR_CUDA;
   return TWKV_OK;
 }

@@ -12,6 +12,7 @@
 #include <type_traits>
 #include "twkv_dev.h"
 #include "mma_util.cuh"
+#include "tc_util.cuh"
 
 namespace twkv {
 
@@ -381,10 +382,17 @@ merge_kernel(DevView v, const unsigned short* __restrict__ Uinv_v, int n_splits,
 }
 
 // ------------------------------------------------------------------------- host side
+cudaError_t launch_kscore_tc(const DevView& v, int layer, const CUtensorMap& map_blocks, const CUtensorMap& map_uinvT,
+                             const void* q, int sm_count, cudaStream_t st);
+
 template <bool BF16>
 static cudaError_t launch_decode_t(const DevView& v, int layer, const LayerParams& lp, const void* q, const int* seq_ids,
-                                   int n_seq, void* out, int n_splits, int sm_count, cudaStream_t st) {
+                                   int n_seq, void* out, int n_splits, int sm_count, const TcMaps* maps, cudaStream_t st) {
   { ProfScope ps(TWKV_K_PLAN, st); plan_kernel<<<1, 256, 0, st>>>(v, seq_ids, n_seq); }
+  if (maps) {
+    cudaError_t e = launch_kscore_tc(v, layer, maps->blocks, maps->uinvT_k, q, sm_count, st);
+    if (e != cudaSuccess) return e;
+  } else {
   const size_t ks_smem = 2 * KS_STAGES * 16384 + (size_t)v.Hq * HEAD_DIM * 4 + (size_t)TILE * v.Hq * 4;
   const unsigned short* U = reinterpret_cast<const unsigned short*>(lp.Uinv_k);
   const unsigned short* qq = reinterpret_cast<const unsigned short*>(q);
@@ -401,6 +409,7 @@ static cudaError_t launch_decode_t(const DevView& v, int layer, const LayerParam
     default: TWKV_KS(8) break;
   }
 #undef TWKV_KS
+  }
   const size_t va_smem = VA_STAGES * 16384 + 2 * 8192 + 32 * 4;
   const dim3 vgrid(n_seq * n_splits, (v.Hq + 31) / 32);
   if (v.Hq <= 16) {
@@ -422,10 +431,10 @@ static cudaError_t launch_decode_t(const DevView& v, int layer, const LayerParam
 }
 
 cudaError_t launch_decode(const DevView& v, int layer, const LayerParams& lp, const void* q, const int* seq_ids,
-                          int n_seq, void* out, int num_splits, int sm_count, cudaStream_t st) {
+                          int n_seq, void* out, int num_splits, int sm_count, const TcMaps* maps, cudaStream_t st) {
   if (n_seq <= 0) return cudaSuccess;
-  return v.dtype == TWKV_BF16 ? launch_decode_t<true>(v, layer, lp, q, seq_ids, n_seq, out, num_splits, sm_count, st)
-                              : launch_decode_t<false>(v, layer, lp, q, seq_ids, n_seq, out, num_splits, sm_count, st);
+  return v.dtype == TWKV_BF16 ? launch_decode_t<true>(v, layer, lp, q, seq_ids, n_seq, out, num_splits, sm_count, maps, st)
+                              : launch_decode_t<false>(v, layer, lp, q, seq_ids, n_seq, out, num_splits, sm_count, maps, st);
 }
 
 }  // namespace twkv

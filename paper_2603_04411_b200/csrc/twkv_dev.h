@@ -106,8 +106,10 @@ cudaError_t launch_clear_tables(const DevView& v, cudaStream_t st);
 cudaError_t launch_gate_rank(const DevView& v, const float* logits, unsigned short* levels, int n_tok, cudaStream_t st);
 cudaError_t launch_compress_piece(const DevView& v, int layer, const void* K, const void* V, const int* seq_ids,
                                   const int* positions, int n_tok, const unsigned short* levels, cudaStream_t st);
+struct TcMaps;   // tensor maps of the tcgen05 path (api.cu); null = legacy warp-MMA kernels
 cudaError_t launch_decode(const DevView& v, int layer, const LayerParams& lp, const void* q, const int* seq_ids,
-                          int n_seq, void* out, int num_splits, int sm_count, cudaStream_t st);
+                          int n_seq, void* out, int num_splits, int sm_count, const TcMaps* maps, cudaStream_t st);
+cudaError_t launch_transpose16(const void* in, void* out, int n, cudaStream_t st);
 cudaError_t launch_gate_logits(const DevView& v, const LayerParams& lp, const void* K, const void* V, int n_tok,
                                float* logits, cudaStream_t st);
 cudaError_t launch_stats(const DevView& v, int layer, unsigned long long* out_dev, cudaStream_t st);
