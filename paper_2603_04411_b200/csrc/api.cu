@@ -5,7 +5,6 @@
 #include <new>
 #include <vector>
 
-#include <cstdlib>
 #include <cudaTypedefs.h>
 
 #include "twkv_dev.h"
@@ -78,7 +77,7 @@ constexpr int GATE_PIECE = 8192;       // tokens per COMPUTE-mode gate piece (lo
 struct Offsets {
   size_t status, rope_lo, rope_hi, n_tiles, tile_desc, tile_aux, tile_rank, fill, key_last, kclass_count,
       kclass_tiles, seq_vcount, seq_vtiles, seq_tokens, rank_sums, hist, key_cnt, key_old_fill, key_first_id,
-      key_first_base, key_old_last, scores, seqmax, qslot, part_acc, part_l, gate_scratch, stats_buf, tables_end, prep_uinvT,
+      key_first_base, key_old_last, scores, seqmax, qslot, klist, klist_count, part_acc, part_l, gate_scratch, stats_buf, tables_end, prep_uinvT,
       blocks, end_fixed;
 };
 
@@ -141,6 +140,8 @@ static Offsets layout_of(const twkv_config* c, const Dims& d) {
   o.scores = L.alloc(NT * TILE * Hq * sizeof(float));
   o.seqmax = L.alloc(S * Hq * sizeof(unsigned));
   o.qslot = L.alloc(S * sizeof(int));
+  o.klist = L.alloc(NT * sizeof(int4));
+  o.klist_count = L.alloc(sizeof(int));
   o.part_acc = L.alloc((size_t)d.max_partials * Hq * d.d_kv * sizeof(float));
   o.part_l = L.alloc((size_t)d.max_partials * Hq * sizeof(float));
   o.gate_scratch = L.alloc((size_t)GATE_PIECE * 2 * d.d_kv * sizeof(float));
@@ -166,7 +167,6 @@ struct twkv_cache {
   int sm_count;
   std::vector<LayerParams> params;
   Prof prof;
-  bool use_tc = false;                 // tcgen05 / TMA kernels (tensor maps could be built)
   CUtensorMap map_blocks;
   std::vector<CUtensorMap> map_uinvT;  // per layer, over the transposed copy of U_K^-1 inside the pool
   std::vector<char> prepared;          // per layer: transposed copy and its map are current
@@ -234,6 +234,7 @@ static void fill_view(twkv_cache* c) {
   v.key_first_id = (int*)(p + o.key_first_id); v.key_first_base = (int*)(p + o.key_first_base);
   v.key_old_last = (int*)(p + o.key_old_last);
   v.scores = (float*)(p + o.scores); v.seqmax = (unsigned*)(p + o.seqmax); v.qslot = (int*)(p + o.qslot);
+  v.klist = (int4*)(p + o.klist); v.klist_count = (int*)(p + o.klist_count);
   v.part_acc = (float*)(p + o.part_acc); v.part_l = (float*)(p + o.part_l);
   v.gate_scratch = (float*)(p + o.gate_scratch);
 }
@@ -273,9 +274,7 @@ twkv_status twkv_cache_create(const twkv_config* cfg, void* pool, size_t pool_by
   fill_view(c);
   c->map_uinvT.resize(cfg->n_layers);
   c->prepared.assign(cfg->n_layers, 0);
-  const char* legacy = getenv("TWKV_LEGACY_MMA");
-  c->use_tc = !(legacy && legacy[0] == '1') &&
-              make_tmap_2d(&c->map_blocks, c->view.blocks, (uint64_t)c->view.n_blocks * TILE, PANEL, PANEL * 2, TILE);
+  if (!make_tmap_2d(&c->map_blocks, c->view.blocks, (uint64_t)c->view.n_blocks * TILE, PANEL, PANEL * 2, TILE)) { delete c; return TWKV_ERR_CUDA; }
   twkv_status s = twkv_cache_reset(c, stream);
   if (s != TWKV_OK) { delete c; return s; }
   if (launch_rope_tables(c->view, cfg->rope_base, (cudaStream_t)stream) != cudaSuccess) { delete c; return TWKV_ERR_CUDA; }
@@ -383,21 +382,17 @@ twkv_status twkv_decode_attn(twkv_cache* c, int layer, const void* q, const int3
   DeviceGuard g(c->device);
   if (!g.ok) return TWKV_ERR_CUDA;
   ProfBind pb(&c->prof);
-  TcMaps maps;
-  const TcMaps* pm = nullptr;
-  if (c->use_tc) {
-    if (!c->prepared[layer]) {
-      // first decode after the parameters were (re)set: K-major copy of U_K^-1 for the tensor cores
-      unsigned char* dst = c->pool + c->off.prep_uinvT + (size_t)layer * c->dims.d_kv * c->dims.d_kv * 2;
-      if (launch_transpose16(c->params[layer].Uinv_k, dst, c->dims.d_kv, (cudaStream_t)stream) != cudaSuccess) return TWKV_ERR_CUDA;
-      if (!make_tmap_2d(&c->map_uinvT[layer], dst, c->dims.d_kv, c->dims.d_kv, (uint64_t)c->dims.d_kv * 2, HEAD_DIM)) return TWKV_ERR_CUDA;
-      c->prepared[layer] = 1;
-    }
-    maps.blocks = c->map_blocks;
-    maps.uinvT_k = c->map_uinvT[layer];
-    pm = &maps;
+  if (!c->prepared[layer]) {
+    // first decode after the parameters were (re)set: K-major copy of U_K^-1 for the tensor cores
+    unsigned char* dst = c->pool + c->off.prep_uinvT + (size_t)layer * c->dims.d_kv * c->dims.d_kv * 2;
+    if (launch_transpose16(c->params[layer].Uinv_k, dst, c->dims.d_kv, (cudaStream_t)stream) != cudaSuccess) return TWKV_ERR_CUDA;
+    if (!make_tmap_2d(&c->map_uinvT[layer], dst, c->dims.d_kv, c->dims.d_kv, (uint64_t)c->dims.d_kv * 2, HEAD_DIM)) return TWKV_ERR_CUDA;
+    c->prepared[layer] = 1;
   }
-  if (launch_decode(c->view, layer, c->params[layer], q, seq_ids, n_seq, out, num_splits, c->sm_count, pm,
+  TcMaps maps;
+  maps.blocks = c->map_blocks;
+  maps.uinvT_k = c->map_uinvT[layer];
+  if (launch_decode(c->view, layer, c->params[layer], q, seq_ids, n_seq, out, num_splits, c->sm_count, &maps,
                     (cudaStream_t)stream) != cudaSuccess) return TWKV_ERR_CUDA;
   return TWKV_OK;
 }

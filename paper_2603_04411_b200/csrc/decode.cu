@@ -1,7 +1,7 @@
 // Decode attention over the mixed-rank cache (Eq. 3, reshape to heads, RoPE, softmax attention).
 //
-//   plan_kernel    sequence id -> query slot map, running-max reset
-//   kscore_kernel  per K tile: Kbar = X^_K U_K^-1 (tensor cores), RoPE by stored position,
+//   plan_kernel    sequence id -> query slot map, running-max reset, K-tile work list
+//   kscore_tc_kernel (kscore_tc.cu)  per K tile: Kbar = X^_K U_K^-1, RoPE by stored position,
 //                  s = q . Kbar * scale for the GQA group, scores to scratch, per-sequence max
 //   vacc_kernel    per (sequence, split): p = exp(s - max), acc += p^T X^_V in spectral space
 //                  (tensor cores), l = sum p
@@ -17,173 +17,56 @@
 namespace twkv {
 
 // ------------------------------------------------------------------------------ plan
-__global__ void plan_kernel(DevView v, const int* __restrict__ seq_ids, int n_seq) {
-  for (int s = threadIdx.x; s < v.S; s += blockDim.x) v.qslot[s] = -1;
+// One CTA: sequence id -> query slot map, running-max reset, and the K-score work list: the K tiles
+// of the listed sequences in class order (widest first, inside a class in table order), compacted
+// with a block-wide scan so the order does not depend on thread timing.
+__global__ void __launch_bounds__(1024) plan_kernel(DevView v, int layer, const int* __restrict__ seq_ids, int n_seq) {
+  __shared__ int s_scan[1024];
+  __shared__ int s_base;
+  const int tid = threadIdx.x;
+  for (int s = tid; s < v.S; s += blockDim.x) v.qslot[s] = -1;
   __syncthreads();
-  for (int i = threadIdx.x; i < n_seq; i += blockDim.x) {
+  for (int i = tid; i < n_seq; i += blockDim.x) {
     const int s = seq_ids[i];
     if (s < 0 || s >= v.S) set_status(v, TWKV_ERR_INVALID_ARG);
     else v.qslot[s] = i;
   }
-  for (int i = threadIdx.x; i < n_seq * v.Hq; i += blockDim.x) v.seqmax[i] = 0u;
+  for (int i = tid; i < n_seq * v.Hq; i += blockDim.x) v.seqmax[i] = 0u;
+  if (tid == 0) s_base = 0;
   __syncthreads();
-  for (int i = threadIdx.x; i < n_seq; i += blockDim.x) {
+  for (int i = tid; i < n_seq; i += blockDim.x) {
     const int s = seq_ids[i];
     if (s >= 0 && s < v.S && v.qslot[s] != i) set_status(v, TWKV_ERR_INVALID_ARG);   // duplicate id
   }
-}
-
-// ---------------------------------------------------------------------------- K scores
-constexpr int KS_STAGES = 3;
-constexpr int KS_THREADS = 256;
-
-template <bool BF16, int REP>
-__global__ void __launch_bounds__(KS_THREADS, 1)
-kscore_kernel(DevView v, int layer, const unsigned short* __restrict__ Uinv, const unsigned short* __restrict__ q) {
-  extern __shared__ __align__(128) unsigned char smem[];
-  unsigned char* sA = smem;                                   // [STAGES][128 rows][128 B]
-  unsigned char* sB = smem + KS_STAGES * 16384;               // [STAGES][64 k][256 B]
-  float* sQ = reinterpret_cast<float*>(smem + 2 * KS_STAGES * 16384);   // [Hq][128], pre-scaled
-  float* sS = sQ + v.Hq * HEAD_DIM;                           // [128][Hq]
-  __shared__ int s_cls_cnt[TWKV_MAX_CLASSES];
-
-  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  const int Hq = v.Hq, d_kv = v.d_kv, Hkv = v.Hkv;
-  const int* kcc = v.kcc(layer);
-  if (tid < TWKV_MAX_CLASSES) s_cls_cnt[tid] = tid < v.NC ? kcc[tid] : 0;
-  __syncthreads();
-  int total = 0;
-  for (int c = 0; c < v.NC; ++c) total += s_cls_cnt[c];
   const int4* desc = v.desc(layer, 0);
-  const int* aux = v.aux(layer, 0);
+  const int* kcc = v.kcc(layer);
   const int* kct = v.kct(layer);
-
-  for (int w = blockIdx.x; w < total; w += gridDim.x) {
-    // work items are ordered from the widest class to the narrowest
-    int cls = v.NC, idx = w;
-    while (idx >= s_cls_cnt[cls - 1]) { idx -= s_cls_cnt[cls - 1]; --cls; }
-    const int tile = kct[(size_t)(cls - 1) * v.NT + idx];
-    const int4 dsc = desc[tile];
-    const int qs = v.qslot[dsc.x];
-    if (qs < 0) continue;
-    const int n_valid = dsc.z, base = dsc.w;
-    __syncthreads();                                          // previous tile's smem is free
-    for (int i = tid; i < Hq * HEAD_DIM; i += KS_THREADS)
-      sQ[i] = to_f32<BF16>(q[(size_t)qs * Hq * HEAD_DIM + i]) * v.sm_scale;
-
-    // cos / sin of this thread's two rows and sixteen frequencies
-    const int row0 = warp * 16 + (lane >> 2), row1 = row0 + 8;
-    float cs0[16], sn0[16], cs1[16], sn1[16];
-    {
-      const int p0 = aux[(size_t)tile * TILE + row0], p1 = aux[(size_t)tile * TILE + row1];
-      const float2* h0 = v.rope_hi + (size_t)((p0 >> 9) & (ROPE_HI - 1)) * 64;
-      const float2* l0 = v.rope_lo + (size_t)(p0 & (ROPE_LO - 1)) * 64;
-      const float2* h1 = v.rope_hi + (size_t)((p1 >> 9) & (ROPE_HI - 1)) * 64;
-      const float2* l1 = v.rope_lo + (size_t)(p1 & (ROPE_LO - 1)) * 64;
-#pragma unroll
-      for (int f = 0; f < 16; ++f) {
-        const int fi = (f >> 1) * 8 + (lane & 3) * 2 + (f & 1);
-        float2 a = h0[fi], b = l0[fi];
-        cs0[f] = a.x * b.x - a.y * b.y; sn0[f] = a.y * b.x + a.x * b.y;
-        a = h1[fi]; b = l1[fi];
-        cs1[f] = a.x * b.x - a.y * b.y; sn1[f] = a.y * b.x + a.x * b.y;
+  for (int cls = v.NC; cls >= 1; --cls) {
+    const int cnt = kcc[cls - 1];
+    for (int i0 = 0; i0 < cnt; i0 += 1024) {
+      const int i = i0 + tid;
+      int4 e = make_int4(0, 0, 0, -1);
+      if (i < cnt) {
+        const int tile = kct[(size_t)(cls - 1) * v.NT + i];
+        const int4 d = desc[tile];
+        e = make_int4(tile, d.y | (d.z << 8), d.w, v.qslot[d.x]);
       }
-    }
-
-    const int iters = Hkv * cls;
-    auto issue = [&](int it) {
-      if (it < iters) {
-        const int g = it / cls, j = it - g * cls, st = it % KS_STAGES;
-        const unsigned char* srcA = v.blocks + (size_t)(base + j) * BLOCK_BYTES;
-        const unsigned dA = smem_u32(sA + st * 16384);
-#pragma unroll
-        for (int i = 0; i < 4; ++i) {
-          const int c = tid + i * KS_THREADS, row = c >> 3, ch = c & 7;
-          cp_async16(dA + row * 128 + ((ch ^ (row & 7)) << 4), srcA + row * 128 + ch * 16);
-        }
-        const unsigned char* srcB = reinterpret_cast<const unsigned char*>(Uinv) + ((size_t)(j * PANEL) * d_kv + g * HEAD_DIM) * 2;
-        const unsigned dB = smem_u32(sB + st * 16384);
-#pragma unroll
-        for (int i = 0; i < 4; ++i) {
-          const int c = tid + i * KS_THREADS, kr = c >> 4, ch = c & 15;
-          cp_async16(dB + kr * 256 + ((ch ^ (kr & 7)) << 4), srcB + (size_t)kr * d_kv * 2 + ch * 16);
-        }
-      }
-      cp_async_commit();
-    };
-    for (int it = 0; it < KS_STAGES - 1; ++it) issue(it);
-
-    float acc[16][4];
-    for (int it = 0; it < iters; ++it) {
-      const int g = it / cls, j = it - g * cls, st = it % KS_STAGES;
-      if (j == 0) {
-#pragma unroll
-        for (int n = 0; n < 16; ++n) { acc[n][0] = acc[n][1] = acc[n][2] = acc[n][3] = 0.f; }
-      }
-      cp_async_wait<KS_STAGES - 2>();
+      const int keep = e.w >= 0 ? 1 : 0;
+      s_scan[tid] = keep;
       __syncthreads();
-      issue(it + KS_STAGES - 1);
-      const unsigned aBase = smem_u32(sA + st * 16384), bBase = smem_u32(sB + st * 16384);
-      const int mat = lane >> 3, rin = lane & 7;
-#pragma unroll
-      for (int ks = 0; ks < 4; ++ks) {
-        unsigned a[4];
-        {
-          const int row = warp * 16 + rin + (mat & 1) * 8, kc = ks * 2 + (mat >> 1);
-          ldsm_x4(a, aBase + row * 128 + ((kc ^ (row & 7)) << 4));
-        }
-#pragma unroll
-        for (int np = 0; np < 8; ++np) {
-          unsigned b[4];
-          const int kr = ks * 16 + rin + (mat & 1) * 8, nc = np * 2 + (mat >> 1);
-          ldsm_x4_t(b, bBase + kr * 256 + ((nc ^ (kr & 7)) << 4));
-          mma16816<BF16>(acc[np * 2], a, b[0], b[1]);
-          mma16816<BF16>(acc[np * 2 + 1], a, b[2], b[3]);
-        }
+      for (int o = 1; o < 1024; o <<= 1) {                  // inclusive Hillis-Steele scan
+        const int a = tid >= o ? s_scan[tid - o] : 0;
+        __syncthreads();
+        s_scan[tid] += a;
+        __syncthreads();
       }
-      if (j == cls - 1) {
-        // slab g is complete: RoPE pairs (i, i + 64) live in n-tiles (n, n + 8) of the same thread
-        float s0[REP], s1[REP];
-#pragma unroll
-        for (int h = 0; h < REP; ++h) { s0[h] = 0.f; s1[h] = 0.f; }
-#pragma unroll
-        for (int n = 0; n < 8; ++n) {
-#pragma unroll
-          for (int e = 0; e < 2; ++e) {
-            const int f = n * 2 + e, dim = n * 8 + (lane & 3) * 2 + e;
-            const float x1 = acc[n][e], x2 = acc[n + 8][e];
-            const float y1 = x1 * cs0[f] - x2 * sn0[f], y2 = x2 * cs0[f] + x1 * sn0[f];
-            const float u1 = acc[n][2 + e], u2 = acc[n + 8][2 + e];
-            const float z1 = u1 * cs1[f] - u2 * sn1[f], z2 = u2 * cs1[f] + u1 * sn1[f];
-#pragma unroll
-            for (int h = 0; h < REP; ++h) {
-              const float qa = sQ[(g * REP + h) * HEAD_DIM + dim], qb = sQ[(g * REP + h) * HEAD_DIM + dim + 64];
-              s0[h] += y1 * qa + y2 * qb;
-              s1[h] += z1 * qa + z2 * qb;
-            }
-          }
-        }
-#pragma unroll
-        for (int h = 0; h < REP; ++h) {
-          s0[h] += __shfl_xor_sync(0xffffffffu, s0[h], 1); s0[h] += __shfl_xor_sync(0xffffffffu, s0[h], 2);
-          s1[h] += __shfl_xor_sync(0xffffffffu, s1[h], 1); s1[h] += __shfl_xor_sync(0xffffffffu, s1[h], 2);
-          if ((lane & 3) == 0) {
-            sS[row0 * Hq + g * REP + h] = s0[h];
-            sS[row1 * Hq + g * REP + h] = s1[h];
-          }
-        }
-      }
-    }
-    cp_async_wait<0>();
-    __syncthreads();
-    float* out = v.scores + (size_t)tile * TILE * Hq;
-    for (int i = tid; i < TILE * Hq; i += KS_THREADS) out[i] = (i / Hq < n_valid) ? sS[i] : -INFINITY;
-    if (tid < Hq) {
-      float m = -INFINITY;
-      for (int r = 0; r < n_valid; ++r) m = fmaxf(m, sS[r * Hq + tid]);
-      atomicMax(&v.seqmax[qs * Hq + tid], enc_ordered(m));
+      if (keep) v.klist[s_base + s_scan[tid] - 1] = e;
+      __syncthreads();
+      if (tid == 1023) s_base += s_scan[1023];
+      __syncthreads();
     }
   }
+  if (tid == 0) *v.klist_count = s_base;
 }
 
 // ------------------------------------------------------------------------ V accumulate
@@ -388,27 +271,10 @@ cudaError_t launch_kscore_tc(const DevView& v, int layer, const CUtensorMap& map
 template <bool BF16>
 static cudaError_t launch_decode_t(const DevView& v, int layer, const LayerParams& lp, const void* q, const int* seq_ids,
                                    int n_seq, void* out, int n_splits, int sm_count, const TcMaps* maps, cudaStream_t st) {
-  { ProfScope ps(TWKV_K_PLAN, st); plan_kernel<<<1, 256, 0, st>>>(v, seq_ids, n_seq); }
-  if (maps) {
+  { ProfScope ps(TWKV_K_PLAN, st); plan_kernel<<<1, 1024, 0, st>>>(v, layer, seq_ids, n_seq); }
+  {
     cudaError_t e = launch_kscore_tc(v, layer, maps->blocks, maps->uinvT_k, q, sm_count, st);
     if (e != cudaSuccess) return e;
-  } else {
-  const size_t ks_smem = 2 * KS_STAGES * 16384 + (size_t)v.Hq * HEAD_DIM * 4 + (size_t)TILE * v.Hq * 4;
-  const unsigned short* U = reinterpret_cast<const unsigned short*>(lp.Uinv_k);
-  const unsigned short* qq = reinterpret_cast<const unsigned short*>(q);
-#define TWKV_KS(REP)                                                                                              \
-  {                                                                                                               \
-    cudaFuncSetAttribute(kscore_kernel<BF16, REP>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)ks_smem);    \
-    ProfScope ps(TWKV_K_KSCORE, st);                                                                              \
-    kscore_kernel<BF16, REP><<<sm_count, KS_THREADS, ks_smem, st>>>(v, layer, U, qq);                             \
-  }
-  switch (v.rep) {
-    case 1: TWKV_KS(1) break;
-    case 2: TWKV_KS(2) break;
-    case 4: TWKV_KS(4) break;
-    default: TWKV_KS(8) break;
-  }
-#undef TWKV_KS
   }
   const size_t va_smem = VA_STAGES * 16384 + 2 * 8192 + 32 * 4;
   const dim3 vgrid(n_seq * n_splits, (v.Hq + 31) / 32);

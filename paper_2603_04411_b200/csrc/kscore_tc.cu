@@ -37,6 +37,7 @@ constexpr uint32_t TM_SLAB = 0, TM_KR = 256, TM_S = 384;      // column offsets 
 constexpr uint32_t PANEL_BYTES = 16384;
 constexpr int KT_Q_ROWS = 72;                                 // 8 rows per KV head + 8 rows of padding
 constexpr uint32_t KT_Q_PANEL_BYTES = KT_Q_ROWS * 128;        // one 64-wide K panel of the query operand
+constexpr uint32_t KT_ROPE_STAGE_BYTES = 8 * 32 * 8 * 8;      // per epilogue warp: 32 rows x 8 frequencies x (cos, sin)
 
 template <bool BF16> __device__ __forceinline__ float kt_to_f32(unsigned short bits) {
   if constexpr (BF16) return __uint_as_float((unsigned)bits << 16);
@@ -66,14 +67,14 @@ kscore_tc_kernel(const __grid_constant__ CUtensorMap map_blocks, const __grid_co
   const uint32_t sB = sA + KT_A_SLOTS * PANEL_BYTES;
   const uint32_t sQ = sB + nb * PANEL_BYTES;
   unsigned char* sQ_ptr = smem_raw + (KT_A_SLOTS + nb) * PANEL_BYTES;
-  unsigned char* tail = sQ_ptr + 2 * KT_Q_PANEL_BYTES;
+  float2* sRope = reinterpret_cast<float2*>(sQ_ptr + 2 * KT_Q_PANEL_BYTES);   // [8 epilogue warps][32 rows][8 frequencies]
+  unsigned char* tail = sQ_ptr + 2 * KT_Q_PANEL_BYTES + KT_ROPE_STAGE_BYTES;
   const uint32_t bars = smem_addr(tail);
   // barrier map (8 bytes each)
   const uint32_t a_full = bars, a_empty = a_full + 8 * KT_A_SLOTS, b_full = a_empty + 8 * KT_A_SLOTS;
   const uint32_t b_empty = b_full + 8 * nb, slab_full = b_empty + 8 * nb, slab_empty = slab_full + 16;
   const uint32_t kr_full = slab_empty + 16, kr_empty = kr_full + 16, s_full = kr_empty + 16;
-  int* s_cls_cnt = reinterpret_cast<int*>(tail + 8 * (2 * KT_A_SLOTS + 2 * nb + 9));
-  uint32_t* s_tmem_base = reinterpret_cast<uint32_t*>(s_cls_cnt + TWKV_MAX_CLASSES);
+  uint32_t* s_tmem_base = reinterpret_cast<uint32_t*>(tail + 8 * (2 * KT_A_SLOTS + 2 * nb + 9));
   volatile int* abort_flag = reinterpret_cast<int*>(s_tmem_base + 1);
 
   if (tid == 0) {
@@ -87,7 +88,6 @@ kscore_tc_kernel(const __grid_constant__ CUtensorMap map_blocks, const __grid_co
     *abort_flag = 0;
     mbar_init_fence();
   }
-  if (tid < TWKV_MAX_CLASSES) s_cls_cnt[tid] = tid < v.NC ? v.kcc(layer)[tid] : 0;
   if (warp == 1) tmem_alloc(smem_addr(s_tmem_base), KT_TMEM_COLS);
   for (int i = tid; i < 2 * (int)KT_Q_PANEL_BYTES / 16; i += KT_THREADS)        // padding rows of the query operand stay zero
     reinterpret_cast<uint4*>(sQ_ptr)[i] = make_uint4(0u, 0u, 0u, 0u);
@@ -97,144 +97,138 @@ kscore_tc_kernel(const __grid_constant__ CUtensorMap map_blocks, const __grid_co
   fence_after_sync();
   const uint32_t tmem_base = *s_tmem_base;
 
-  int total = 0;
-  for (int c = 0; c < v.NC; ++c) total += s_cls_cnt[c];
-  const int4* desc = v.desc(layer, 0);
-  const int* kct = v.kct(layer);
-
-  // tile w of the class-sorted list (widest class first) -> (tile id, descriptor); false if not decoded now
-  auto tile_of = [&](int w, int& tile, int4& dsc, int& qs) {
-    int cls = v.NC, idx = w;
-    while (idx >= s_cls_cnt[cls - 1]) { idx -= s_cls_cnt[cls - 1]; --cls; }
-    tile = kct[(size_t)(cls - 1) * v.NT + idx];
-    dsc = desc[tile];
-    qs = v.qslot[dsc.x];
-    return qs >= 0;
-  };
+  // work list written by plan_kernel: the K tiles of the sequences being decoded, widest class first
+  const int total = *v.klist_count;
+  const int4* klist = v.klist;
+  const int4 kt_none = make_int4(0, 0, 0, -1);
+  const int w0 = blockIdx.x, wstep = gridDim.x;
 
   if (warp == 10) {
-    // ------------------------------------------------------------- TMA producer: X^_K panels
-    if (lane == 0) tma_prefetch_desc(&map_blocks);
-    uint32_t ak = 0;                                            // panels loaded so far; slot = ak % 8
-    bool ok = true;
-    for (int w = blockIdx.x; w < total && ok; w += gridDim.x) {
-      int tile, qs; int4 dsc;
-      if (!tile_of(w, tile, dsc, qs)) continue;
-      const int cls = dsc.y, blk = dsc.w;
-      for (int j = 0; j < cls && ok; ++j, ++ak) {
-        const uint32_t slot = ak % KT_A_SLOTS, ph = (ak / KT_A_SLOTS) & 1u;
-        ok = __all_sync(0xffffffffu, mbar_wait(a_empty + 8 * slot, ph ^ 1u, abort_flag));
-        if (!ok) break;
-        if (lane == 0) {
+    // ------------------------------------------------------------- TMA producer: X^_K panels (one elected lane)
+    if (elect_one()) {
+      tma_prefetch_desc(&map_blocks);
+      uint32_t ak = 0;                                          // panels loaded so far; slot = ak % 8
+      bool ok = true;
+      int4 e = w0 < total ? klist[w0] : kt_none;
+      for (int w = w0; w < total && ok; w += wstep) {
+        const int4 nxt = w + wstep < total ? klist[w + wstep] : kt_none;
+        const int cls = e.y & 0xff, blk = e.z;
+        for (int j = 0; j < cls; ++j, ++ak) {
+          const uint32_t slot = ak % KT_A_SLOTS, ph = (ak / KT_A_SLOTS) & 1u;
+          if (!(ok = mbar_wait(a_empty + 8 * slot, ph ^ 1u, abort_flag))) break;
           mbar_expect_tx(a_full + 8 * slot, PANEL_BYTES);
           tma_load_2d(sA + slot * PANEL_BYTES, &map_blocks, a_full + 8 * slot, 0, (blk + j) * TILE);
         }
+        e = nxt;
       }
+      if (!ok)                                                  // let copies in flight land before the CTA goes away
+        for (uint32_t i = 0; i < (uint32_t)KT_A_SLOTS && i < ak; ++i) {
+          const uint32_t n = ak - 1 - i;
+          mbar_wait_drain(a_full + 8 * (n % KT_A_SLOTS), (n / KT_A_SLOTS) & 1u);
+        }
     }
-    if (!ok)                                                    // let copies in flight land before the CTA goes away
-      for (uint32_t i = 0; i < (uint32_t)KT_A_SLOTS && i < ak; ++i) {
-        const uint32_t n = ak - 1 - i;
-        mbar_wait_drain(a_full + 8 * (n % KT_A_SLOTS), (n / KT_A_SLOTS) & 1u);
-      }
+    __syncwarp();
   } else if (warp == 0) {
-    // ------------------------------------------------------------- TMA producer: U_K^-1 panels
-    if (lane == 0) tma_prefetch_desc(&map_uinvT);
-    uint32_t bk = 0;
-    bool ok = true;
-    for (int w = blockIdx.x; w < total && ok; w += gridDim.x) {
-      int tile, qs; int4 dsc;
-      if (!tile_of(w, tile, dsc, qs)) continue;
-      const int cls = dsc.y;
-      for (int p0 = 0; p0 < cls && ok; p0 += KT_A_SLOTS) {
-        const int np = min(KT_A_SLOTS, cls - p0);
-        for (int g = 0; g < Hkv && ok; ++g) {
-          for (int j = 0; j < np && ok; ++j, ++bk) {
-            const uint32_t st = bk % nb, ph = (bk / nb) & 1u;
-            ok = __all_sync(0xffffffffu, mbar_wait(b_empty + 8 * st, ph ^ 1u, abort_flag));
-            if (!ok) break;
-            if (lane == 0) {
+    // ------------------------------------------------------------- TMA producer: U_K^-1 panels (one elected lane)
+    if (elect_one()) {
+      tma_prefetch_desc(&map_uinvT);
+      uint32_t bk = 0;
+      bool ok = true;
+      int4 e = w0 < total ? klist[w0] : kt_none;
+      for (int w = w0; w < total && ok; w += wstep) {
+        const int4 nxt = w + wstep < total ? klist[w + wstep] : kt_none;
+        const int cls = e.y & 0xff;
+        for (int p0 = 0; p0 < cls && ok; p0 += KT_A_SLOTS) {
+          const int np = min(KT_A_SLOTS, cls - p0);
+          for (int g = 0; g < Hkv && ok; ++g) {
+            for (int j = 0; j < np; ++j, ++bk) {
+              const uint32_t st = bk % nb, ph = (bk / nb) & 1u;
+              if (!(ok = mbar_wait(b_empty + 8 * st, ph ^ 1u, abort_flag))) break;
               mbar_expect_tx(b_full + 8 * st, PANEL_BYTES);
               tma_load_2d(sB + st * PANEL_BYTES, &map_uinvT, b_full + 8 * st, (p0 + j) * PANEL, g * HEAD_DIM);
             }
           }
         }
+        e = nxt;
       }
-    }
-    if (!ok)
-      for (uint32_t i = 0; i < (uint32_t)nb && i < bk; ++i) {
-        const uint32_t n = bk - 1 - i;
-        mbar_wait_drain(b_full + 8 * (n % nb), (n / nb) & 1u);
-      }
-  } else if (warp == 1) {
-    // ------------------------------------------------------------- MMA issuer
-    const uint32_t idesc_main = idesc_f16(BF16 ? 1 : 0, 128, 128);
-    const uint32_t idesc_s = idesc_f16(0, 128, 16);
-    uint32_t bk = 0, ak = 0, sc = 0;
-    bool ok = true;
-    // the score product of slab n is issued after the main product of slab n + 1, so the tensor
-    // pipe has work while the epilogue warps rotate slab n
-    bool pend = false, pend_acc = false, pend_last = false;
-    uint32_t pend_sc = 0; int pend_g = 0;
-    auto issue_scores = [&]() {
-      const uint32_t kb = pend_sc & 1u;
-      if (!__all_sync(0xffffffffu, mbar_wait(kr_full + 8 * kb, (pend_sc >> 1) & 1u, abort_flag))) return false;
-      fence_after_sync();
-      if (lane == 0) {
-#pragma unroll
-        for (int ks = 0; ks < 8; ++ks) {
-          const uint64_t qdesc = kmajor_sw128_desc(sQ + (ks >> 2) * KT_Q_PANEL_BYTES + pend_g * 1024) + 2 * (ks & 3);
-          mma_f16_ts(tmem_base + TM_S + 16 * pend_g, tmem_base + TM_KR + 64 * kb + 8 * ks, qdesc, idesc_s,
-                     (pend_acc || ks > 0) ? 1u : 0u);
+      if (!ok)
+        for (uint32_t i = 0; i < (uint32_t)nb && i < bk; ++i) {
+          const uint32_t n = bk - 1 - i;
+          mbar_wait_drain(b_full + 8 * (n % nb), (n / nb) & 1u);
         }
-        mma_commit(kr_empty + 8 * kb);
-        if (pend_last) mma_commit(s_full);
-      }
-      __syncwarp();
-      pend = false;
-      return true;
-    };
-    for (int w = blockIdx.x; w < total && ok; w += gridDim.x) {
-      int tile, qs; int4 dsc;
-      if (!tile_of(w, tile, dsc, qs)) continue;
-      const int cls = dsc.y;
-      for (int p0 = 0; p0 < cls && ok; p0 += KT_A_SLOTS) {
-        const int np = min(KT_A_SLOTS, cls - p0);
-        for (int g = 0; g < Hkv && ok; ++g) {
-          const uint32_t buf = sc & 1u;
-          ok = __all_sync(0xffffffffu, mbar_wait(slab_empty + 8 * buf, ((sc >> 1) & 1u) ^ 1u, abort_flag));
-          if (!ok) break;
-          fence_after_sync();
-          for (int j = 0; j < np && ok; ++j, ++bk) {
-            const uint32_t an = ak + j, slot = an % KT_A_SLOTS;
-            if (g == 0) {
-              ok = __all_sync(0xffffffffu, mbar_wait(a_full + 8 * slot, (an / KT_A_SLOTS) & 1u, abort_flag));
-              if (!ok) break;
-            }
-            const uint32_t st = bk % nb, ph = (bk / nb) & 1u;
-            ok = __all_sync(0xffffffffu, mbar_wait(b_full + 8 * st, ph, abort_flag));
-            if (!ok) break;
-            fence_after_sync();
-            if (lane == 0) {
-              const uint64_t adesc = kmajor_sw128_desc(sA + slot * PANEL_BYTES);
-              const uint64_t bdesc = kmajor_sw128_desc(sB + st * PANEL_BYTES);
+    }
+    __syncwarp();
+  } else if (warp == 1) {
+    // ------------------------------------------------------------- MMA issuer (one elected lane runs the whole role)
+    if (elect_one()) {
+      const uint32_t idesc_main = idesc_f16(BF16 ? 1 : 0, 128, 128);
+      const uint32_t idesc_s = idesc_f16(0, 128, 16);
+      const uint64_t adesc0 = kmajor_sw128_desc(sA), bdesc0 = kmajor_sw128_desc(sB), qdesc0 = kmajor_sw128_desc(sQ);
+      uint32_t bk = 0, ak = 0, sc = 0;
+      bool ok = true;
+      // The score product of slab n is issued after the main product of slab n + 2: the tensor pipe
+      // then always has a slab queued while the epilogue warps rotate an earlier one.
+      // A pending entry packs: slab counter << 8 | g << 2 | accumulate << 1 | last slab of its tile.
+      uint32_t pq0 = 0, pq1 = 0;
+      int npend = 0;
+      auto issue_scores = [&](uint32_t pe) {
+        const uint32_t psc = pe >> 8, kb = psc & 1u, pg = (pe >> 2) & 63u, pacc = (pe >> 1) & 1u;
+        if (!mbar_wait(kr_full + 8 * kb, (psc >> 1) & 1u, abort_flag)) return false;
+        fence_after_sync();
+        const uint64_t qd = qdesc0 + (uint64_t)(pg * (1024 >> 4));
+        const uint32_t d = tmem_base + TM_S + 16 * pg, a = tmem_base + TM_KR + 64 * kb;
+        mma_f16_ts(d, a, qd, idesc_s, pacc);
 #pragma unroll
-              for (int ks = 0; ks < 4; ++ks)
-                mma_f16_ss(tmem_base + TM_SLAB + buf * 128, adesc + 2 * ks, bdesc + 2 * ks, idesc_main, (j > 0 || ks > 0) ? 1u : 0u);
+        for (int ks = 1; ks < 8; ++ks)
+          mma_f16_ts(d, a + 8 * ks, qd + (ks >> 2) * (KT_Q_PANEL_BYTES >> 4) + 2 * (ks & 3), idesc_s, 1u);
+        mma_commit(kr_empty + 8 * kb);
+        if (pe & 1u) mma_commit(s_full);
+        return true;
+      };
+      int4 e = w0 < total ? klist[w0] : kt_none;
+      for (int w = w0; w < total && ok; w += wstep) {
+        const int4 nxt = w + wstep < total ? klist[w + wstep] : kt_none;
+        const int cls = e.y & 0xff;
+        for (int p0 = 0; p0 < cls && ok; p0 += KT_A_SLOTS) {
+          const int np = min(KT_A_SLOTS, cls - p0);
+          for (int g = 0; g < Hkv && ok; ++g) {
+            const uint32_t buf = sc & 1u;
+            if (!(ok = mbar_wait(slab_empty + 8 * buf, ((sc >> 1) & 1u) ^ 1u, abort_flag))) break;
+            const uint32_t d = tmem_base + TM_SLAB + buf * 128;
+            for (int j = 0; j < np; ++j, ++bk) {
+              const uint32_t an = ak + j, slot = an % KT_A_SLOTS;
+              if (g == 0 && !(ok = mbar_wait(a_full + 8 * slot, (an / KT_A_SLOTS) & 1u, abort_flag))) break;
+              const uint32_t st = bk % nb, ph = (bk / nb) & 1u;
+              if (!(ok = mbar_wait(b_full + 8 * st, ph, abort_flag))) break;
+              fence_after_sync();
+              const uint64_t adesc = adesc0 + (uint64_t)(slot * (PANEL_BYTES >> 4));
+              const uint64_t bdesc = bdesc0 + (uint64_t)(st * (PANEL_BYTES >> 4));
+              mma_f16_ss(d, adesc, bdesc, idesc_main, j > 0 ? 1u : 0u);
+#pragma unroll
+              for (int ks = 1; ks < 4; ++ks) mma_f16_ss(d, adesc + 2 * ks, bdesc + 2 * ks, idesc_main, 1u);
               mma_commit(b_empty + 8 * st);                             // ring stage reusable when these MMAs retire
               if (g == Hkv - 1) mma_commit(a_empty + 8 * slot);         // last slab of the pass: the X^_K panel is done
-              if (j == np - 1) mma_commit(slab_full + 8 * buf);         // slab accumulator complete
             }
-            __syncwarp();
+            if (!ok) break;
+            mma_commit(slab_full + 8 * buf);                            // slab accumulator complete
+            if (npend == 2) {
+              if (!(ok = issue_scores(pq0))) break;
+              pq0 = pq1;
+              npend = 1;
+            }
+            const uint32_t pe = (sc << 8) | ((uint32_t)g << 2) | (p0 > 0 ? 2u : 0u) | ((p0 + np >= cls && g == Hkv - 1) ? 1u : 0u);
+            if (npend == 0) pq0 = pe; else pq1 = pe;
+            ++npend;
+            ++sc;
           }
-          if (!ok) break;
-          if (pend && !(ok = issue_scores())) break;
-          pend = true; pend_sc = sc; pend_g = g; pend_acc = p0 > 0; pend_last = (p0 + np >= cls) && (g == Hkv - 1);
-          ++sc;
+          ak += np;
         }
-        ak += np;
+        e = nxt;
       }
+      if (ok && npend >= 1) ok = issue_scores(pq0);
+      if (ok && npend == 2) issue_scores(pq1);
     }
-    if (ok && pend) issue_scores();
+    __syncwarp();
   } else {
     // ------------------------------------------------------------- epilogue
     const int et = tid - 64;
@@ -242,80 +236,97 @@ kscore_tc_kernel(const __grid_constant__ CUtensorMap map_blocks, const __grid_co
     const int row = quarter * 32 + lane;
     const uint32_t lane_addr = tmem_base + ((uint32_t)(quarter * 32) << 16);
     const int g_lo = hf ? (Hkv + 1) / 2 : 0, g_hi = hf ? Hkv : (Hkv + 1) / 2;
+    const float sm_scale = v.sm_scale;
+    const int* kpos = v.aux(layer, 0);
     uint32_t sc = 0, tcount = 0;
-    int prev_qs = -1;
     bool ok = true;
-    for (int w = blockIdx.x; w < total && ok; w += gridDim.x) {
-      int tile, qs; int4 dsc;
-      if (!tile_of(w, tile, dsc, qs)) continue;
-      const int cls = dsc.y, n_valid = dsc.z;
-      if (qs != prev_qs) {
-        // the group's queries as the K-major, 128-byte-swizzled B operand: row 8 g + h, two 64-wide panels.
-        // The previous tile's score products have retired (s_full was waited for), so the rows are free.
-        for (int i = et; i < Hq * 16; i += KT_EPI) {
-          const int head = i >> 4, ch = i & 15;                               // 8 dims per chunk
-          const uint4 raw = *reinterpret_cast<const uint4*>(q + ((size_t)qs * Hq + head) * HEAD_DIM + ch * 8);
-          uint4 val = raw;
-          if constexpr (BF16) {
-            const unsigned short* e = reinterpret_cast<const unsigned short*>(&raw);
-            val.x = pack_f16x2_sat(kt_to_f32<true>(e[0]), kt_to_f32<true>(e[1]));
-            val.y = pack_f16x2_sat(kt_to_f32<true>(e[2]), kt_to_f32<true>(e[3]));
-            val.z = pack_f16x2_sat(kt_to_f32<true>(e[4]), kt_to_f32<true>(e[5]));
-            val.w = pack_f16x2_sat(kt_to_f32<true>(e[6]), kt_to_f32<true>(e[7]));
-          }
-          const int qrow = (head / REP) * 8 + head % REP, c8 = ch & 7;
-          *reinterpret_cast<uint4*>(sQ_ptr + (ch >> 3) * KT_Q_PANEL_BYTES + qrow * 128 + ((c8 ^ (qrow & 7)) << 4)) = val;
-        }
-        fence_proxy_async_smem();
-        prev_qs = qs;
-      }
-      float cs[32], sn[32];
-      {
-        const int pos = v.aux(layer, 0)[(size_t)tile * TILE + row];
-        const float2* th = v.rope_hi + (size_t)((pos >> 9) & (ROPE_HI - 1)) * 64 + hf * 32;
-        const float2* tl = v.rope_lo + (size_t)(pos & (ROPE_LO - 1)) * 64 + hf * 32;
+    float cs[32], sn[32];
+
+    // cos / sin of (row, frequency): pos = hi * 512 + lo, the two table rows combine by the angle-addition
+    // formulas.  Table rows are read coalesced (8 lanes per row) and handed to the row's lane through a
+    // per-warp staging buffer, 8 frequencies at a time.
+    auto rope_setup = [&](int tile) {
+      const int pos = kpos[(size_t)tile * TILE + row];
+      float2* stage = sRope + (warp - 2) * 256;
+      const int rs = lane >> 3, t8 = lane & 7;
 #pragma unroll
-        for (int t = 0; t < 32; ++t) {
-          const float2 a = th[t], b = tl[t];
-          cs[t] = a.x * b.x - a.y * b.y;
-          sn[t] = a.y * b.x + a.x * b.y;
+      for (int k = 0; k < 4; ++k) {
+        const int f = hf * 32 + k * 8 + t8;
+#pragma unroll
+        for (int it = 0; it < 8; ++it) {
+          const int r = it * 4 + rs;
+          const int p = __shfl_sync(0xffffffffu, pos, r);
+          const float2 a = v.rope_hi[(size_t)((p >> 9) & (ROPE_HI - 1)) * 64 + f];
+          const float2 b = v.rope_lo[(size_t)(p & (ROPE_LO - 1)) * 64 + f];
+          stage[r * 8 + (t8 ^ (r & 7))] = make_float2(a.x * b.x - a.y * b.y, a.y * b.x + a.x * b.y);
         }
+        __syncwarp();
+#pragma unroll
+        for (int t = 0; t < 8; ++t) {
+          const float2 c = stage[lane * 8 + (t ^ (lane & 7))];
+          cs[k * 8 + t] = c.x;
+          sn[k * 8 + t] = c.y;
+        }
+        __syncwarp();
       }
+    };
+    // The group's queries as the K-major, 128-byte-swizzled B operand: row 8 g + h, two 64-wide panels.
+    // Only called when no score product that reads the rows can still be in flight.
+    auto write_q = [&](int qs) {
+      for (int i = et; i < Hq * 16; i += KT_EPI) {
+        const int head = i >> 4, ch = i & 15;                               // 8 dims per chunk
+        const uint4 raw = *reinterpret_cast<const uint4*>(q + ((size_t)qs * Hq + head) * HEAD_DIM + ch * 8);
+        uint4 val = raw;
+        if constexpr (BF16) {
+          const unsigned short* e = reinterpret_cast<const unsigned short*>(&raw);
+          val.x = pack_f16x2_sat(kt_to_f32<true>(e[0]), kt_to_f32<true>(e[1]));
+          val.y = pack_f16x2_sat(kt_to_f32<true>(e[2]), kt_to_f32<true>(e[3]));
+          val.z = pack_f16x2_sat(kt_to_f32<true>(e[4]), kt_to_f32<true>(e[5]));
+          val.w = pack_f16x2_sat(kt_to_f32<true>(e[6]), kt_to_f32<true>(e[7]));
+        }
+        const int qrow = (head / REP) * 8 + head % REP, c8 = ch & 7;
+        *reinterpret_cast<uint4*>(sQ_ptr + (ch >> 3) * KT_Q_PANEL_BYTES + qrow * 128 + ((c8 ^ (qrow & 7)) << 4)) = val;
+      }
+      fence_proxy_async_smem();
+    };
+
+    int4 e = w0 < total ? klist[w0] : kt_none;
+    if (w0 < total) { write_q(e.w); rope_setup(e.x); }
+    for (int w = w0; w < total && ok; w += wstep) {
+      const int4 nxt = w + wstep < total ? klist[w + wstep] : kt_none;
+      const int tile = e.x, cls = e.y & 0xff, n_valid = e.y >> 8, qs = e.w;
       const int n_slabs = ((cls + KT_A_SLOTS - 1) / KT_A_SLOTS) * Hkv;
       for (int sl = 0; sl < n_slabs; ++sl, ++sc) {
         const uint32_t buf = sc & 1u, par = (sc >> 1) & 1u;
         if (!(ok = __all_sync(0xffffffffu, mbar_wait(slab_full + 8 * buf, par, abort_flag)))) break;
-        if (!(ok = __all_sync(0xffffffffu, mbar_wait(kr_empty + 8 * buf, par ^ 1u, abort_flag)))) break;
         fence_after_sync();
         const uint32_t slab = lane_addr + TM_SLAB + buf * 128 + hf * 32;
         const uint32_t kr = lane_addr + TM_KR + buf * 64 + hf * 16;
+        float lo[32], hi[32];
+        tmem_ld32(slab, reinterpret_cast<uint32_t*>(lo));
+        tmem_ld32(slab + 64, reinterpret_cast<uint32_t*>(hi));
+        tmem_ld_wait();
+        fence_before_sync();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(slab_empty + 8 * buf);                    // the slab accumulator is free for slab n + 2
+        uint32_t p1[16], p2[16];
 #pragma unroll
-        for (int half = 0; half < 2; ++half) {
-          float lo[16], hi[16];
-          tmem_ld16(slab + half * 16, reinterpret_cast<uint32_t*>(lo));
-          tmem_ld16(slab + 64 + half * 16, reinterpret_cast<uint32_t*>(hi));
-          tmem_ld_wait();
-          if (half == 1) {                                                  // the slab accumulator is free for slab n + 2
-            fence_before_sync();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(slab_empty + 8 * buf);
-          }
-          uint32_t p1[8], p2[8];
-#pragma unroll
-          for (int t = 0; t < 16; t += 2) {
-            const float c0 = cs[half * 16 + t], s0 = sn[half * 16 + t], c1 = cs[half * 16 + t + 1], s1 = sn[half * 16 + t + 1];
-            p1[t >> 1] = pack_f16x2_sat(lo[t] * c0 - hi[t] * s0, lo[t + 1] * c1 - hi[t + 1] * s1);
-            p2[t >> 1] = pack_f16x2_sat(hi[t] * c0 + lo[t] * s0, hi[t + 1] * c1 + lo[t + 1] * s1);
-          }
-          tmem_st8(kr + half * 8, p1);                                      // dims d -> column d / 2
-          tmem_st8(kr + 32 + half * 8, p2);                                 // dims 64 + d
+        for (int t = 0; t < 32; t += 2) {
+          p1[t >> 1] = pack_f16x2_sat(lo[t] * cs[t] - hi[t] * sn[t], lo[t + 1] * cs[t + 1] - hi[t + 1] * sn[t + 1]);
+          p2[t >> 1] = pack_f16x2_sat(hi[t] * cs[t] + lo[t] * sn[t], hi[t + 1] * cs[t + 1] + lo[t + 1] * sn[t + 1]);
         }
+        if (!(ok = __all_sync(0xffffffffu, mbar_wait(kr_empty + 8 * buf, par ^ 1u, abort_flag)))) break;
+        fence_after_sync();
+        tmem_st16(kr, p1);                                                  // dims d -> column d / 2
+        tmem_st16(kr + 32, p2);                                             // dims 64 + d
         tmem_st_wait();
         fence_before_sync();
         __syncwarp();
         if (lane == 0) mbar_arrive(kr_full + 8 * buf);
       }
       if (!ok) break;
+      // the next tile's rotation factors are fetched while this tile's last score products drain
+      if (nxt.w >= 0) rope_setup(nxt.x);
       // all score products of the tile have retired: scale, mask the rows past the last token, store
       if (!(ok = __all_sync(0xffffffffu, mbar_wait(s_full, tcount & 1u, abort_flag)))) break;
       ++tcount;
@@ -326,7 +337,7 @@ kscore_tc_kernel(const __grid_constant__ CUtensorMap map_blocks, const __grid_co
         tmem_ldN<REP>(lane_addr + TM_S + 16 * g, reinterpret_cast<uint32_t*>(s));
         tmem_ld_wait();
 #pragma unroll
-        for (int h = 0; h < REP; ++h) s[h] = row < n_valid ? s[h] * v.sm_scale : -INFINITY;
+        for (int h = 0; h < REP; ++h) s[h] = row < n_valid ? s[h] * sm_scale : -INFINITY;
         if constexpr (REP == 1) out[g] = s[0];
         else if constexpr (REP == 2) *reinterpret_cast<float2*>(out + g * 2) = make_float2(s[0], s[1]);
         else {
@@ -341,6 +352,8 @@ kscore_tc_kernel(const __grid_constant__ CUtensorMap map_blocks, const __grid_co
           if (lane == 0) atomicMax(&v.seqmax[qs * Hq + g * REP + h], enc_ordered(m));
         }
       }
+      if (nxt.w >= 0 && nxt.w != qs) write_q(nxt.w);
+      e = nxt;
     }
   }
 
@@ -371,8 +384,8 @@ cudaError_t launch_transpose16(const void* in, void* out, int n, cudaStream_t st
 }
 
 size_t kscore_tc_smem_bytes(int nb) {
-  return (size_t)(KT_A_SLOTS + nb) * PANEL_BYTES + 2 * KT_Q_PANEL_BYTES + 8 * (2 * KT_A_SLOTS + 2 * nb + 9) +
-         (TWKV_MAX_CLASSES + 2) * sizeof(int);
+  return (size_t)(KT_A_SLOTS + nb) * PANEL_BYTES + 2 * KT_Q_PANEL_BYTES + KT_ROPE_STAGE_BYTES + 8 * (2 * KT_A_SLOTS + 2 * nb + 9) +
+         2 * sizeof(int);
 }
 
 template <bool BF16>

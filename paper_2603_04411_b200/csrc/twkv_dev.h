@@ -49,6 +49,8 @@ struct DevView {
   float* scores;             // [NT*128][Hq]
   unsigned* seqmax;          // [S][Hq]  order-preserving encoding of the running max
   int* qslot;                // [S]   sequence id -> query index of the current decode call, -1
+  int4* klist;               // [NT]  K tiles of the current decode call, widest class first: (tile, class | n_valid << 8, base block, query slot)
+  int* klist_count;          // [1]
   float* part_acc;           // [max_partials][Hq][d_kv]
   float* part_l;             // [max_partials][Hq]
   float* gate_scratch;       // COMPUTE mode logits [GATE_PIECE][2][d_kv]
@@ -106,7 +108,7 @@ cudaError_t launch_clear_tables(const DevView& v, cudaStream_t st);
 cudaError_t launch_gate_rank(const DevView& v, const float* logits, unsigned short* levels, int n_tok, cudaStream_t st);
 cudaError_t launch_compress_piece(const DevView& v, int layer, const void* K, const void* V, const int* seq_ids,
                                   const int* positions, int n_tok, const unsigned short* levels, cudaStream_t st);
-struct TcMaps;   // tensor maps of the tcgen05 path (api.cu); null = legacy warp-MMA kernels
+struct TcMaps;   // tensor maps of the K-score kernel (api.cu)
 cudaError_t launch_decode(const DevView& v, int layer, const LayerParams& lp, const void* q, const int* seq_ids,
                           int n_seq, void* out, int num_splits, int sm_count, const TcMaps* maps, cudaStream_t st);
 cudaError_t launch_transpose16(const void* in, void* out, int n, cudaStream_t st);
