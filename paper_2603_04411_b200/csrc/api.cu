@@ -77,7 +77,7 @@ constexpr int GATE_PIECE = 8192;       // tokens per COMPUTE-mode gate piece (lo
 struct Offsets {
   size_t status, rope_lo, rope_hi, n_tiles, tile_desc, tile_aux, tile_rank, fill, key_last, kclass_count,
       kclass_tiles, seq_vcount, seq_vtiles, seq_tokens, rank_sums, hist, key_cnt, key_old_fill, key_first_id,
-      key_first_base, key_old_last, scores, seqmax, qslot, klist, klist_count, part_acc, part_l, gate_scratch, stats_buf, tables_end, prep_uinvT,
+      key_first_base, key_old_last, scores, seqmax, qslot, klist, klist_count, klist_cost, cta_start, part_acc, part_l, gate_scratch, stats_buf, tables_end, prep_uinvT,
       blocks, end_fixed;
 };
 
@@ -142,6 +142,8 @@ static Offsets layout_of(const twkv_config* c, const Dims& d) {
   o.qslot = L.alloc(S * sizeof(int));
   o.klist = L.alloc(NT * sizeof(int4));
   o.klist_count = L.alloc(sizeof(int));
+  o.klist_cost = L.alloc(NT * sizeof(unsigned));
+  o.cta_start = L.alloc((MAX_PLAN_CTAS + 1) * sizeof(int));
   o.part_acc = L.alloc((size_t)d.max_partials * Hq * d.d_kv * sizeof(float));
   o.part_l = L.alloc((size_t)d.max_partials * Hq * sizeof(float));
   o.gate_scratch = L.alloc((size_t)GATE_PIECE * 2 * d.d_kv * sizeof(float));
@@ -235,6 +237,7 @@ static void fill_view(twkv_cache* c) {
   v.key_old_last = (int*)(p + o.key_old_last);
   v.scores = (float*)(p + o.scores); v.seqmax = (unsigned*)(p + o.seqmax); v.qslot = (int*)(p + o.qslot);
   v.klist = (int4*)(p + o.klist); v.klist_count = (int*)(p + o.klist_count);
+  v.klist_cost = (unsigned*)(p + o.klist_cost); v.cta_start = (int*)(p + o.cta_start);
   v.part_acc = (float*)(p + o.part_acc); v.part_l = (float*)(p + o.part_l);
   v.gate_scratch = (float*)(p + o.gate_scratch);
 }
@@ -271,6 +274,7 @@ twkv_status twkv_cache_create(const twkv_config* cfg, void* pool, size_t pool_by
   DeviceGuard g(c->device);
   if (!g.ok) { delete c; return TWKV_ERR_CUDA; }
   if (cudaDeviceGetAttribute(&c->sm_count, cudaDevAttrMultiProcessorCount, c->device) != cudaSuccess) { delete c; return TWKV_ERR_CUDA; }
+  if (c->sm_count > MAX_PLAN_CTAS) c->sm_count = MAX_PLAN_CTAS;
   fill_view(c);
   c->map_uinvT.resize(cfg->n_layers);
   c->prepared.assign(cfg->n_layers, 0);

@@ -19,12 +19,29 @@ namespace twkv {
 // ------------------------------------------------------------------------------ plan
 // One CTA: sequence id -> query slot map, running-max reset, and the K-score work list: the K tiles
 // of the listed sequences in class order (widest first, inside a class in table order), compacted
-// with a block-wide scan so the order does not depend on thread timing.
-__global__ void __launch_bounds__(1024) plan_kernel(DevView v, int layer, const int* __restrict__ seq_ids, int n_seq) {
-  __shared__ int s_scan[1024];
-  __shared__ int s_base;
-  const int tid = threadIdx.x;
+// with block-wide scans so the order does not depend on thread timing.  The list is then cut into
+// n_cta contiguous pieces of about equal estimated cost, so a CTA of the K-score kernel mostly
+// stays inside one (class, sequence) run.
+__device__ __forceinline__ unsigned ktile_cost(int cls) {
+  // cycles, roughly: per slab max(epilogue, panels * MMA time) + score product; per tile a fixed part
+  const int passes = (cls + 7) / 8, np = (cls + passes - 1) / passes;
+  const int slab = max(700, np * 280 + 250);
+  return 3000u + (unsigned)(passes * 8 * slab);
+}
+
+__global__ void __launch_bounds__(1024) plan_kernel(DevView v, int layer, const int* __restrict__ seq_ids, int n_seq, int n_cta) {
+  __shared__ int s_cls_off[TWKV_MAX_CLASSES + 1];
+  __shared__ unsigned s_wsum[32][2];
+  __shared__ unsigned s_base[2];                                  // entries kept so far, their cost
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   for (int s = tid; s < v.S; s += blockDim.x) v.qslot[s] = -1;
+  if (tid == 0) {
+    const int* kcc = v.kcc(layer);
+    int run = 0;
+    for (int c = v.NC; c >= 1; --c) { s_cls_off[v.NC - c] = run; run += kcc[c - 1]; }    // widest class first
+    s_cls_off[v.NC] = run;
+    s_base[0] = 0u; s_base[1] = 0u;
+  }
   __syncthreads();
   for (int i = tid; i < n_seq; i += blockDim.x) {
     const int s = seq_ids[i];
@@ -32,41 +49,69 @@ __global__ void __launch_bounds__(1024) plan_kernel(DevView v, int layer, const 
     else v.qslot[s] = i;
   }
   for (int i = tid; i < n_seq * v.Hq; i += blockDim.x) v.seqmax[i] = 0u;
-  if (tid == 0) s_base = 0;
   __syncthreads();
   for (int i = tid; i < n_seq; i += blockDim.x) {
     const int s = seq_ids[i];
     if (s >= 0 && s < v.S && v.qslot[s] != i) set_status(v, TWKV_ERR_INVALID_ARG);   // duplicate id
   }
   const int4* desc = v.desc(layer, 0);
-  const int* kcc = v.kcc(layer);
   const int* kct = v.kct(layer);
-  for (int cls = v.NC; cls >= 1; --cls) {
-    const int cnt = kcc[cls - 1];
-    for (int i0 = 0; i0 < cnt; i0 += 1024) {
-      const int i = i0 + tid;
-      int4 e = make_int4(0, 0, 0, -1);
-      if (i < cnt) {
-        const int tile = kct[(size_t)(cls - 1) * v.NT + i];
-        const int4 d = desc[tile];
-        e = make_int4(tile, d.y | (d.z << 8), d.w, v.qslot[d.x]);
-      }
-      const int keep = e.w >= 0 ? 1 : 0;
-      s_scan[tid] = keep;
-      __syncthreads();
-      for (int o = 1; o < 1024; o <<= 1) {                  // inclusive Hillis-Steele scan
-        const int a = tid >= o ? s_scan[tid - o] : 0;
-        __syncthreads();
-        s_scan[tid] += a;
-        __syncthreads();
-      }
-      if (keep) v.klist[s_base + s_scan[tid] - 1] = e;
-      __syncthreads();
-      if (tid == 1023) s_base += s_scan[1023];
-      __syncthreads();
+  const int n_all = s_cls_off[v.NC];
+  for (int f0 = 0; f0 < n_all; f0 += 1024) {
+    const int f = f0 + tid;
+    int4 e = make_int4(0, 0, 0, -1);
+    if (f < n_all) {
+      int k = 0;
+      while (f >= s_cls_off[k + 1]) ++k;
+      const int cls = v.NC - k;
+      const int tile = kct[(size_t)(cls - 1) * v.NT + (f - s_cls_off[k])];
+      const int4 d = desc[tile];
+      e = make_int4(tile, d.y | (d.z << 8), d.w, v.qslot[d.x]);
     }
+    const unsigned keep = e.w >= 0 ? 1u : 0u;
+    const unsigned cost = keep ? ktile_cost(e.y & 0xff) : 0u;
+    unsigned ik = keep, ic = cost;                              // inclusive scans inside the warp
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const unsigned a = __shfl_up_sync(0xffffffffu, ik, o), b = __shfl_up_sync(0xffffffffu, ic, o);
+      if (lane >= o) { ik += a; ic += b; }
+    }
+    if (lane == 31) { s_wsum[warp][0] = ik; s_wsum[warp][1] = ic; }
+    __syncthreads();
+    if (warp == 0) {
+      unsigned wk = s_wsum[lane][0], wc = s_wsum[lane][1];
+#pragma unroll
+      for (int o = 1; o < 32; o <<= 1) {
+        const unsigned a = __shfl_up_sync(0xffffffffu, wk, o), b = __shfl_up_sync(0xffffffffu, wc, o);
+        if (lane >= o) { wk += a; wc += b; }
+      }
+      s_wsum[lane][0] = wk; s_wsum[lane][1] = wc;               // inclusive over warps
+    }
+    __syncthreads();
+    const unsigned pk = s_base[0] + (warp ? s_wsum[warp - 1][0] : 0u) + ik - keep;      // exclusive position
+    const unsigned pc = s_base[1] + (warp ? s_wsum[warp - 1][1] : 0u) + ic - cost;      // exclusive cost prefix
+    if (keep) { v.klist[pk] = e; v.klist_cost[pk] = pc; }
+    __syncthreads();
+    if (tid == 0) { s_base[0] += s_wsum[31][0]; s_base[1] += s_wsum[31][1]; }
+    __syncthreads();
   }
-  if (tid == 0) *v.klist_count = s_base;
+  // cut points: piece b starts at the first entry whose cost prefix reaches b / n_cta of the total
+  const unsigned n_keep = s_base[0];
+  const unsigned long long total = s_base[1];
+  if (tid == 0) { *v.klist_count = (int)n_keep; v.cta_start[n_cta] = (int)n_keep; }
+  if (n_keep == 0 || total == 0ull) {
+    for (int b = tid; b < n_cta; b += blockDim.x) v.cta_start[b] = 0;
+    return;
+  }
+  for (unsigned i = tid; i < n_keep; i += blockDim.x) {
+    const unsigned long long lo = v.klist_cost[i];
+    const unsigned long long hi = i + 1 < n_keep ? v.klist_cost[i + 1] : total;
+    // pieces b with lo <= b * total / n_cta < hi, i.e. b in [ceil(lo n / T), ceil(hi n / T) - 1]
+    const int b0 = (int)((lo * n_cta + total - 1) / total);
+    int b1 = (int)((hi * n_cta + total - 1) / total) - 1;
+    if (b1 > n_cta - 1) b1 = n_cta - 1;
+    for (int b = b0; b <= b1; ++b) v.cta_start[b] = (int)i;
+  }
 }
 
 // ------------------------------------------------------------------------ V accumulate
@@ -271,7 +316,7 @@ cudaError_t launch_kscore_tc(const DevView& v, int layer, const CUtensorMap& map
 template <bool BF16>
 static cudaError_t launch_decode_t(const DevView& v, int layer, const LayerParams& lp, const void* q, const int* seq_ids,
                                    int n_seq, void* out, int n_splits, int sm_count, const TcMaps* maps, cudaStream_t st) {
-  { ProfScope ps(TWKV_K_PLAN, st); plan_kernel<<<1, 1024, 0, st>>>(v, layer, seq_ids, n_seq); }
+  { ProfScope ps(TWKV_K_PLAN, st); plan_kernel<<<1, 1024, 0, st>>>(v, layer, seq_ids, n_seq, sm_count); }
   {
     cudaError_t e = launch_kscore_tc(v, layer, maps->blocks, maps->uinvT_k, q, sm_count, st);
     if (e != cudaSuccess) return e;

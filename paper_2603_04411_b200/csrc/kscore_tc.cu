@@ -14,11 +14,11 @@
 // over its panels that accumulate into the same S.
 //
 // Tensor memory (512 columns): slab accumulators 2 x 128 | rotated keys 2 x 64 | S 8 x 16.
-// Warp roles (352 threads, one persistent CTA per SM, tiles taken widest class first):
-//   warp 0      TMA producer of U_K^-1 panels (ring)
+// Warp roles (352 threads, one persistent CTA per SM working through a contiguous, cost-balanced piece of the tile list):
+//   warp 0      TMA producer of U_K^-1 panels (ring, one lane per stage)
 //   warp 1      MMA issuer (one lane issues; owns the TMEM allocation)
 //   warps 2-9   epilogue (thread = one token row x one half of the RoPE frequencies)
-//   warp 10     TMA producer of X^_K panels (ring of 8 slots, runs ahead into the next tile)
+//   warp 10     TMA producer of X^_K panels (ring of 8 slots served by four lanes, runs ahead into the next tile)
 // All waits are bounded (tc_util.cuh); a wait that runs out ends the kernel with TWKV_ERR_TIMEOUT.
 //
 // Precision: X^_K, U_K^-1 keep the cache dtype with fp32 accumulation; rotated keys and queries enter
@@ -42,13 +42,6 @@ constexpr uint32_t KT_ROPE_STAGE_BYTES = 8 * 32 * 8 * 8;      // per epilogue wa
 template <bool BF16> __device__ __forceinline__ float kt_to_f32(unsigned short bits) {
   if constexpr (BF16) return __uint_as_float((unsigned)bits << 16);
   else return __half2float(__ushort_as_half(bits));
-}
-
-template <int N> __device__ __forceinline__ void tmem_ldN(uint32_t taddr, uint32_t* r) {
-  if constexpr (N == 1) tmem_ld1(taddr, r);
-  else if constexpr (N == 2) tmem_ld2(taddr, r);
-  else if constexpr (N == 4) tmem_ld4(taddr, r);
-  else tmem_ld8(taddr, r);
 }
 
 template <bool BF16, int REP>
@@ -98,16 +91,21 @@ kscore_tc_kernel(const __grid_constant__ CUtensorMap map_blocks, const __grid_co
   const uint32_t tmem_base = *s_tmem_base;
 
   // work list written by plan_kernel: the K tiles of the sequences being decoded, widest class first
-  const int total = *v.klist_count;
+  // this CTA's contiguous piece [w0, total) of the list (cut by estimated cost)
+  const int w0 = v.cta_start[blockIdx.x], total = v.cta_start[blockIdx.x + 1];
   const int4* klist = v.klist;
   const int4 kt_none = make_int4(0, 0, 0, -1);
-  const int w0 = blockIdx.x, wstep = gridDim.x;
+  constexpr int wstep = 1;
+  // CTAs walk the KV heads in rotated order, so that at any moment they read different panels of U_K^-1 from L2
+  const int g_rot = blockIdx.x % Hkv;
 
   if (warp == 10) {
-    // ------------------------------------------------------------- TMA producer: X^_K panels (one elected lane)
-    if (elect_one()) {
-      tma_prefetch_desc(&map_blocks);
-      uint32_t ak = 0;                                          // panels loaded so far; slot = ak % 8
+    // ------------------------------------------------------------- TMA producer: X^_K panels
+    // A thread's TMA copies complete one after the other, so the ring is served by four lanes
+    // (lane L owns slots L and L + 4) that each keep their own copy in flight.
+    if (lane < 4) {
+      if (lane == 0) tma_prefetch_desc(&map_blocks);
+      uint32_t ak = 0;                                          // panels so far; slot = ak % 8
       bool ok = true;
       int4 e = w0 < total ? klist[w0] : kt_none;
       for (int w = w0; w < total && ok; w += wstep) {
@@ -115,6 +113,7 @@ kscore_tc_kernel(const __grid_constant__ CUtensorMap map_blocks, const __grid_co
         const int cls = e.y & 0xff, blk = e.z;
         for (int j = 0; j < cls; ++j, ++ak) {
           const uint32_t slot = ak % KT_A_SLOTS, ph = (ak / KT_A_SLOTS) & 1u;
+          if ((slot & 3u) != (uint32_t)lane) continue;
           if (!(ok = mbar_wait(a_empty + 8 * slot, ph ^ 1u, abort_flag))) break;
           mbar_expect_tx(a_full + 8 * slot, PANEL_BYTES);
           tma_load_2d(sA + slot * PANEL_BYTES, &map_blocks, a_full + 8 * slot, 0, (blk + j) * TILE);
@@ -124,15 +123,16 @@ kscore_tc_kernel(const __grid_constant__ CUtensorMap map_blocks, const __grid_co
       if (!ok)                                                  // let copies in flight land before the CTA goes away
         for (uint32_t i = 0; i < (uint32_t)KT_A_SLOTS && i < ak; ++i) {
           const uint32_t n = ak - 1 - i;
-          mbar_wait_drain(a_full + 8 * (n % KT_A_SLOTS), (n / KT_A_SLOTS) & 1u);
+          if (((n % KT_A_SLOTS) & 3u) == (uint32_t)lane) mbar_wait_drain(a_full + 8 * (n % KT_A_SLOTS), (n / KT_A_SLOTS) & 1u);
         }
     }
     __syncwarp();
   } else if (warp == 0) {
-    // ------------------------------------------------------------- TMA producer: U_K^-1 panels (one elected lane)
-    if (elect_one()) {
-      tma_prefetch_desc(&map_uinvT);
-      uint32_t bk = 0;
+    // ------------------------------------------------------------- TMA producer: U_K^-1 panels
+    // one lane per ring stage, for the same reason
+    if (lane < nb) {
+      if (lane == 0) tma_prefetch_desc(&map_uinvT);
+      uint32_t bk = 0, bst = 0, bph = 0;                        // panels so far; ring stage and its phase
       bool ok = true;
       int4 e = w0 < total ? klist[w0] : kt_none;
       for (int w = w0; w < total && ok; w += wstep) {
@@ -140,9 +140,12 @@ kscore_tc_kernel(const __grid_constant__ CUtensorMap map_blocks, const __grid_co
         const int cls = e.y & 0xff;
         for (int p0 = 0; p0 < cls && ok; p0 += KT_A_SLOTS) {
           const int np = min(KT_A_SLOTS, cls - p0);
-          for (int g = 0; g < Hkv && ok; ++g) {
+          for (int sl = 0; sl < Hkv && ok; ++sl) {
+            const int g = sl + g_rot < Hkv ? sl + g_rot : sl + g_rot - Hkv;
             for (int j = 0; j < np; ++j, ++bk) {
-              const uint32_t st = bk % nb, ph = (bk / nb) & 1u;
+              const uint32_t st = bst, ph = bph;
+              if (++bst == (uint32_t)nb) { bst = 0; bph ^= 1u; }
+              if (st != (uint32_t)lane) continue;
               if (!(ok = mbar_wait(b_empty + 8 * st, ph ^ 1u, abort_flag))) break;
               mbar_expect_tx(b_full + 8 * st, PANEL_BYTES);
               tma_load_2d(sB + st * PANEL_BYTES, &map_uinvT, b_full + 8 * st, (p0 + j) * PANEL, g * HEAD_DIM);
@@ -154,7 +157,7 @@ kscore_tc_kernel(const __grid_constant__ CUtensorMap map_blocks, const __grid_co
       if (!ok)
         for (uint32_t i = 0; i < (uint32_t)nb && i < bk; ++i) {
           const uint32_t n = bk - 1 - i;
-          mbar_wait_drain(b_full + 8 * (n % nb), (n / nb) & 1u);
+          if (n % nb == (uint32_t)lane) mbar_wait_drain(b_full + 8 * (n % nb), (n / nb) & 1u);
         }
     }
     __syncwarp();
@@ -164,7 +167,7 @@ kscore_tc_kernel(const __grid_constant__ CUtensorMap map_blocks, const __grid_co
       const uint32_t idesc_main = idesc_f16(BF16 ? 1 : 0, 128, 128);
       const uint32_t idesc_s = idesc_f16(0, 128, 16);
       const uint64_t adesc0 = kmajor_sw128_desc(sA), bdesc0 = kmajor_sw128_desc(sB), qdesc0 = kmajor_sw128_desc(sQ);
-      uint32_t bk = 0, ak = 0, sc = 0;
+      uint32_t bst = 0, bph = 0, ak = 0, sc = 0;
       bool ok = true;
       // The score product of slab n is issued after the main product of slab n + 2: the tensor pipe
       // then always has a slab queued while the epilogue warps rotate an earlier one.
@@ -191,14 +194,16 @@ kscore_tc_kernel(const __grid_constant__ CUtensorMap map_blocks, const __grid_co
         const int cls = e.y & 0xff;
         for (int p0 = 0; p0 < cls && ok; p0 += KT_A_SLOTS) {
           const int np = min(KT_A_SLOTS, cls - p0);
-          for (int g = 0; g < Hkv && ok; ++g) {
+          for (int sl = 0; sl < Hkv && ok; ++sl) {
+            const int g = sl + g_rot < Hkv ? sl + g_rot : sl + g_rot - Hkv;
             const uint32_t buf = sc & 1u;
             if (!(ok = mbar_wait(slab_empty + 8 * buf, ((sc >> 1) & 1u) ^ 1u, abort_flag))) break;
             const uint32_t d = tmem_base + TM_SLAB + buf * 128;
-            for (int j = 0; j < np; ++j, ++bk) {
+            for (int j = 0; j < np; ++j) {
               const uint32_t an = ak + j, slot = an % KT_A_SLOTS;
-              if (g == 0 && !(ok = mbar_wait(a_full + 8 * slot, (an / KT_A_SLOTS) & 1u, abort_flag))) break;
-              const uint32_t st = bk % nb, ph = (bk / nb) & 1u;
+              if (sl == 0 && !(ok = mbar_wait(a_full + 8 * slot, (an / KT_A_SLOTS) & 1u, abort_flag))) break;
+              const uint32_t st = bst, ph = bph;
+              if (++bst == (uint32_t)nb) { bst = 0; bph ^= 1u; }
               if (!(ok = mbar_wait(b_full + 8 * st, ph, abort_flag))) break;
               fence_after_sync();
               const uint64_t adesc = adesc0 + (uint64_t)(slot * (PANEL_BYTES >> 4));
@@ -207,7 +212,7 @@ kscore_tc_kernel(const __grid_constant__ CUtensorMap map_blocks, const __grid_co
 #pragma unroll
               for (int ks = 1; ks < 4; ++ks) mma_f16_ss(d, adesc + 2 * ks, bdesc + 2 * ks, idesc_main, 1u);
               mma_commit(b_empty + 8 * st);                             // ring stage reusable when these MMAs retire
-              if (g == Hkv - 1) mma_commit(a_empty + 8 * slot);         // last slab of the pass: the X^_K panel is done
+              if (sl == Hkv - 1) mma_commit(a_empty + 8 * slot);        // last slab of the pass: the X^_K panel is done
             }
             if (!ok) break;
             mma_commit(slab_full + 8 * buf);                            // slab accumulator complete
@@ -216,7 +221,7 @@ kscore_tc_kernel(const __grid_constant__ CUtensorMap map_blocks, const __grid_co
               pq0 = pq1;
               npend = 1;
             }
-            const uint32_t pe = (sc << 8) | ((uint32_t)g << 2) | (p0 > 0 ? 2u : 0u) | ((p0 + np >= cls && g == Hkv - 1) ? 1u : 0u);
+            const uint32_t pe = (sc << 8) | ((uint32_t)g << 2) | (p0 > 0 ? 2u : 0u) | ((p0 + np >= cls && sl == Hkv - 1) ? 1u : 0u);
             if (npend == 0) pq0 = pe; else pq1 = pe;
             ++npend;
             ++sc;
@@ -235,12 +240,17 @@ kscore_tc_kernel(const __grid_constant__ CUtensorMap map_blocks, const __grid_co
     const int quarter = warp & 3, hf = (warp - 2) >> 2;
     const int row = quarter * 32 + lane;
     const uint32_t lane_addr = tmem_base + ((uint32_t)(quarter * 32) << 16);
-    const int g_lo = hf ? (Hkv + 1) / 2 : 0, g_hi = hf ? Hkv : (Hkv + 1) / 2;
+    const int g_lo = hf ? (Hkv + 1) / 2 : 0, g_hi = hf ? Hkv : (Hkv + 1) / 2;      // this thread's KV-head groups (at most 4)
     const float sm_scale = v.sm_scale;
     const int* kpos = v.aux(layer, 0);
+    const float2* __restrict__ rope_hi = v.rope_hi;
+    const float2* __restrict__ rope_lo = v.rope_lo;
     uint32_t sc = 0, tcount = 0;
     bool ok = true;
     float cs[32], sn[32];
+    float tmax[4 * REP];                                            // running maxima of this thread's heads for the current query slot
+#pragma unroll
+    for (int i = 0; i < 4 * REP; ++i) tmax[i] = -INFINITY;
 
     // cos / sin of (row, frequency): pos = hi * 512 + lo, the two table rows combine by the angle-addition
     // formulas.  Table rows are read coalesced (8 lanes per row) and handed to the row's lane through a
@@ -249,25 +259,41 @@ kscore_tc_kernel(const __grid_constant__ CUtensorMap map_blocks, const __grid_co
       const int pos = kpos[(size_t)tile * TILE + row];
       float2* stage = sRope + (warp - 2) * 256;
       const int rs = lane >> 3, t8 = lane & 7;
+      int off_hi[8], off_lo[8];
 #pragma unroll
-      for (int k = 0; k < 4; ++k) {
-        const int f = hf * 32 + k * 8 + t8;
+      for (int it = 0; it < 8; ++it) {
+        const int p = __shfl_sync(0xffffffffu, pos, it * 4 + rs);
+        off_hi[it] = ((p >> 9) & (ROPE_HI - 1)) * 64 + hf * 32 + t8;
+        off_lo[it] = (p & (ROPE_LO - 1)) * 64 + hf * 32 + t8;
+      }
 #pragma unroll
-        for (int it = 0; it < 8; ++it) {
-          const int r = it * 4 + rs;
-          const int p = __shfl_sync(0xffffffffu, pos, r);
-          const float2 a = v.rope_hi[(size_t)((p >> 9) & (ROPE_HI - 1)) * 64 + f];
-          const float2 b = v.rope_lo[(size_t)(p & (ROPE_LO - 1)) * 64 + f];
-          stage[r * 8 + (t8 ^ (r & 7))] = make_float2(a.x * b.x - a.y * b.y, a.y * b.x + a.x * b.y);
+      for (int k2 = 0; k2 < 2; ++k2) {
+        float2 a[2][8], b[2][8];
+#pragma unroll
+        for (int kk = 0; kk < 2; ++kk)
+#pragma unroll
+          for (int it = 0; it < 8; ++it) {
+            a[kk][it] = __ldg(rope_hi + off_hi[it] + (k2 * 2 + kk) * 8);
+            b[kk][it] = __ldg(rope_lo + off_lo[it] + (k2 * 2 + kk) * 8);
+          }
+#pragma unroll
+        for (int kk = 0; kk < 2; ++kk) {
+          const int k = k2 * 2 + kk;
+#pragma unroll
+          for (int it = 0; it < 8; ++it) {
+            const int r = it * 4 + rs;
+            stage[r * 8 + (t8 ^ (r & 7))] = make_float2(a[kk][it].x * b[kk][it].x - a[kk][it].y * b[kk][it].y,
+                                                        a[kk][it].y * b[kk][it].x + a[kk][it].x * b[kk][it].y);
+          }
+          __syncwarp();
+#pragma unroll
+          for (int t = 0; t < 8; ++t) {
+            const float2 c = stage[lane * 8 + (t ^ (lane & 7))];
+            cs[k * 8 + t] = c.x;
+            sn[k * 8 + t] = c.y;
+          }
+          __syncwarp();
         }
-        __syncwarp();
-#pragma unroll
-        for (int t = 0; t < 8; ++t) {
-          const float2 c = stage[lane * 8 + (t ^ (lane & 7))];
-          cs[k * 8 + t] = c.x;
-          sn[k * 8 + t] = c.y;
-        }
-        __syncwarp();
       }
     };
     // The group's queries as the K-major, 128-byte-swizzled B operand: row 8 g + h, two 64-wide panels.
@@ -331,25 +357,45 @@ kscore_tc_kernel(const __grid_constant__ CUtensorMap map_blocks, const __grid_co
       if (!(ok = __all_sync(0xffffffffu, mbar_wait(s_full, tcount & 1u, abort_flag)))) break;
       ++tcount;
       fence_after_sync();
-      float* out = v.scores + ((size_t)tile * TILE + row) * Hq;
-      for (int g = g_lo; g < g_hi; ++g) {
-        float s[REP];
-        tmem_ldN<REP>(lane_addr + TM_S + 16 * g, reinterpret_cast<uint32_t*>(s));
+      {
+        // this thread's groups g_lo .. g_hi - 1: REP columns of each group's 16-column region, all loads in flight at once
+        float sv[4 * REP];
+#pragma unroll
+        for (int gi = 0; gi < 4; ++gi)
+          if (g_lo + gi < g_hi) {
+            uint32_t* dst = reinterpret_cast<uint32_t*>(sv + gi * REP);
+            const uint32_t src = lane_addr + TM_S + 16 * (g_lo + gi);
+            if constexpr (REP == 1) tmem_ld1(src, dst);
+            else if constexpr (REP == 2) tmem_ld2(src, dst);
+            else if constexpr (REP == 4) tmem_ld4(src, dst);
+            else tmem_ld8(src, dst);
+          }
         tmem_ld_wait();
+        const int h0 = g_lo * REP, nh = (g_hi - g_lo) * REP;
+        float* out = v.scores + ((size_t)tile * TILE + row) * Hq + h0;
+        const bool live = row < n_valid;
 #pragma unroll
-        for (int h = 0; h < REP; ++h) s[h] = row < n_valid ? s[h] * sm_scale : -INFINITY;
-        if constexpr (REP == 1) out[g] = s[0];
-        else if constexpr (REP == 2) *reinterpret_cast<float2*>(out + g * 2) = make_float2(s[0], s[1]);
-        else {
+        for (int i = 0; i < 4 * REP; ++i) sv[i] = (live && i < nh) ? sv[i] * sm_scale : -INFINITY;
+        if constexpr (REP >= 4) {
 #pragma unroll
-          for (int h = 0; h < REP; h += 4) *reinterpret_cast<float4*>(out + g * REP + h) = make_float4(s[h], s[h + 1], s[h + 2], s[h + 3]);
+          for (int i = 0; i < 4 * REP; i += 4)
+            if (i < nh) *reinterpret_cast<float4*>(out + i) = make_float4(sv[i], sv[i + 1], sv[i + 2], sv[i + 3]);
+        } else {
+#pragma unroll
+          for (int i = 0; i < 4 * REP; ++i) if (i < nh) out[i] = sv[i];
         }
 #pragma unroll
-        for (int h = 0; h < REP; ++h) {
-          float m = s[h];
+        for (int i = 0; i < 4 * REP; ++i) tmax[i] = fmaxf(tmax[i], sv[i]);
+        if (nxt.w != qs) {
+          // last tile of this query slot in the piece: maximum over the warp's rows, one atomic per head
 #pragma unroll
-          for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
-          if (lane == 0) atomicMax(&v.seqmax[qs * Hq + g * REP + h], enc_ordered(m));
+          for (int i = 0; i < 4 * REP; ++i) {
+            float m = tmax[i];
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
+            if (lane == i && i < nh) atomicMax(&v.seqmax[qs * Hq + h0 + i], enc_ordered(m));
+            tmax[i] = -INFINITY;
+          }
         }
       }
       if (nxt.w >= 0 && nxt.w != qs) write_q(nxt.w);

@@ -17,6 +17,7 @@ constexpr int PIECE_CHUNKS = TWKV_PIECE_TOKENS / CHUNK_TOKENS;
 constexpr int ROPE_LO = 512;                // pos = hi * 512 + lo
 constexpr int ROPE_HI = 1024;               // positions up to 512 * 1024 - 1
 constexpr int MAX_PARTIALS_EXTRA = 320;     // V-side partial slots beyond max_seqs
+constexpr int MAX_PLAN_CTAS = 1024;         // upper bound on the K-score kernel's grid
 
 // Device view of a cache: plain pointers into the caller's pool.  Passed to kernels by value.
 struct DevView {
@@ -51,6 +52,8 @@ struct DevView {
   int* qslot;                // [S]   sequence id -> query index of the current decode call, -1
   int4* klist;               // [NT]  K tiles of the current decode call, widest class first: (tile, class | n_valid << 8, base block, query slot)
   int* klist_count;          // [1]
+  unsigned* klist_cost;      // [NT]  exclusive prefix of the estimated cost of the listed tiles
+  int* cta_start;            // [MAX_PLAN_CTAS + 1]  first list entry of every K-score CTA
   float* part_acc;           // [max_partials][Hq][d_kv]
   float* part_l;             // [max_partials][Hq]
   float* gate_scratch;       // COMPUTE mode logits [GATE_PIECE][2][d_kv]
