@@ -285,7 +285,7 @@ def run_ours(args):
         flops_k = 2.0 * sum_rk * D_KV + n_tok * (3.0 * D_KV + 2.0 * HQ * DH)
         ks_avg_ms = ks_ms / max(ks_n, 1)
         achieved = flops_k / (ks_avg_ms * 1e-3) / 1e12
-        roofline = {"kernel": "kscore_kernel (K reconstruct + RoPE + q.K scores)", "bound": "tensor", "achieved": achieved,
+        roofline = {"kernel": "kscore_tc_kernel (tcgen05: K reconstruct + RoPE + q.K scores)", "bound": "tensor", "achieved": achieved,
                     "peak": peaks["tflops"], "unit": "TFLOP/s", "frac": achieved / peaks["tflops"],
                     "peak_source": f"{peaks['source']} bf16 sustained (fp16 has the same nominal rate)",
                     "traffic": None, "flops_per_launch": flops_k, "avg_launch_ms": ks_avg_ms}
