@@ -73,11 +73,12 @@ struct Layout {
 };
 
 constexpr int GATE_PIECE = 8192;       // tokens per COMPUTE-mode gate piece (logits scratch rows)
+constexpr int GATE_TC_MIN_TOKENS = 1024;   // calls at least this large run the fused tcgen05 gate kernel
 
 struct Offsets {
   size_t status, rope_lo, rope_hi, n_tiles, tile_desc, tile_aux, tile_rank, fill, key_last, kclass_count,
       kclass_tiles, seq_vcount, seq_vtiles, seq_tokens, rank_sums, hist, key_cnt, key_old_fill, key_first_id,
-      key_first_base, key_old_last, scores, seqmax, qslot, klist, klist_count, klist_cost, cta_start, part_acc, part_l, gate_scratch, stats_buf, tables_end, prep_uinvT,
+      key_first_base, key_old_last, scores, seqmax, qslot, klist, klist_count, klist_cost, cta_start, part_acc, part_l, gate_scratch, stats_buf, tables_end, prep_uinvT, prep_wT,
       blocks, end_fixed;
 };
 
@@ -146,9 +147,13 @@ static Offsets layout_of(const twkv_config* c, const Dims& d) {
   o.cta_start = L.alloc((MAX_PLAN_CTAS + 1) * sizeof(int));
   o.part_acc = L.alloc((size_t)d.max_partials * Hq * d.d_kv * sizeof(float));
   o.part_l = L.alloc((size_t)d.max_partials * Hq * sizeof(float));
-  o.gate_scratch = L.alloc((size_t)GATE_PIECE * 2 * d.d_kv * sizeof(float));
+  {
+    const size_t small = (size_t)GATE_PIECE * 2 * d.d_kv * sizeof(float), fused = gate_tc_stage_bytes(MAX_PLAN_CTAS < 160 ? MAX_PLAN_CTAS : 160, d.d_kv);
+    o.gate_scratch = L.alloc(small > fused ? small : fused);
+  }
   o.stats_buf = L.alloc(64 * sizeof(unsigned long long));
   o.prep_uinvT = L.alloc(Ls * (size_t)d.d_kv * d.d_kv * 2, 1024);
+  o.prep_wT = L.alloc(Ls * 2 * (size_t)d.d_kv * d.d_kv * 2, 1024);
   o.blocks = L.alloc(0, 1024);
   o.end_fixed = o.blocks;
   return o;
@@ -172,6 +177,8 @@ struct twkv_cache {
   CUtensorMap map_blocks;
   std::vector<CUtensorMap> map_uinvT;  // per layer, over the transposed copy of U_K^-1 inside the pool
   std::vector<char> prepared;          // per layer: transposed copy and its map are current
+  std::vector<CUtensorMap> map_wT;     // per layer x side, over the transposed copies of the gate weights
+  std::vector<char> prepared_w;        // per layer: those copies and maps are current
 };
 
 struct DeviceGuard {
@@ -278,6 +285,8 @@ twkv_status twkv_cache_create(const twkv_config* cfg, void* pool, size_t pool_by
   fill_view(c);
   c->map_uinvT.resize(cfg->n_layers);
   c->prepared.assign(cfg->n_layers, 0);
+  c->map_wT.resize(2 * (size_t)cfg->n_layers);
+  c->prepared_w.assign(cfg->n_layers, 0);
   if (!make_tmap_2d(&c->map_blocks, c->view.blocks, (uint64_t)c->view.n_blocks * TILE, PANEL, PANEL * 2, TILE)) { delete c; return TWKV_ERR_CUDA; }
   twkv_status s = twkv_cache_reset(c, stream);
   if (s != TWKV_OK) { delete c; return s; }
@@ -329,9 +338,10 @@ twkv_status twkv_cache_destroy(twkv_cache* c) {
 twkv_status twkv_cache_set_layer_params(twkv_cache* c, int layer, const twkv_layer_params* p) {
   if (!c || !p || layer < 0 || layer >= c->cfg.n_layers) return TWKV_ERR_INVALID_ARG;
   if (!p->Uinv_k || !p->Uinv_v) return TWKV_ERR_INVALID_ARG;
-  if (((uintptr_t)p->Uinv_k | (uintptr_t)p->Uinv_v | (uintptr_t)p->W_k | (uintptr_t)p->W_v) % 16) return TWKV_ERR_INVALID_ARG;
+  if (((uintptr_t)p->Uinv_k | (uintptr_t)p->Uinv_v | (uintptr_t)p->W_k | (uintptr_t)p->W_v | (uintptr_t)p->b_k | (uintptr_t)p->b_v) % 16) return TWKV_ERR_INVALID_ARG;
   c->params[layer] = LayerParams{p->Uinv_k, p->Uinv_v, p->W_k, p->W_v, p->b_k, p->b_v};
   c->prepared[layer] = 0;
+  c->prepared_w[layer] = 0;
   return TWKV_OK;
 }
 
@@ -353,6 +363,25 @@ twkv_status twkv_compress(twkv_cache* c, int layer, const void* K, const void* V
   const size_t row = (size_t)v.d_kv * 2;
   if (mode == TWKV_GATE_LOGITS) {
     if (launch_gate_rank(v, scores, levels, n_tok, st) != cudaSuccess) return TWKV_ERR_CUDA;
+  } else if (mode == TWKV_GATE_COMPUTE && n_tok >= GATE_TC_MIN_TOKENS && c->sm_count <= 160) {
+    // fused tcgen05 kernel: logits and ranks in one launch, the logits never leave the CTA's staging block
+    const int d = c->dims.d_kv;
+    if (!c->prepared_w[layer]) {
+      // first COMPUTE call after the parameters were (re)set: K-major copies of W_k, W_v for the tensor cores
+      const int ns = (d % 256 == 0) ? 256 : 128;
+      for (int side = 0; side < 2; ++side) {
+        unsigned char* dst = c->pool + c->off.prep_wT + ((size_t)layer * 2 + side) * d * d * 2;
+        if (launch_transpose16(side ? c->params[layer].W_v : c->params[layer].W_k, dst, d, st) != cudaSuccess) return TWKV_ERR_CUDA;
+        if (!make_tmap_2d(&c->map_wT[2 * (size_t)layer + side], dst, d, d, (uint64_t)d * 2, ns)) return TWKV_ERR_CUDA;
+      }
+      c->prepared_w[layer] = 1;
+    }
+    GateMaps maps;
+    maps.wk = c->map_wT[2 * (size_t)layer];
+    maps.wv = c->map_wT[2 * (size_t)layer + 1];
+    if (!make_tmap_2d(&maps.xk, K, (uint64_t)n_tok, d, (uint64_t)d * 2, TILE) ||
+        !make_tmap_2d(&maps.xv, V, (uint64_t)n_tok, d, (uint64_t)d * 2, TILE)) return TWKV_ERR_CUDA;
+    if (launch_gate_ranks_tc(v, maps, c->params[layer], n_tok, levels, c->sm_count, st) != cudaSuccess) return TWKV_ERR_CUDA;
   } else if (mode == TWKV_GATE_COMPUTE) {
     for (int lo = 0; lo < n_tok; lo += GATE_PIECE) {
       const int n = n_tok - lo < GATE_PIECE ? n_tok - lo : GATE_PIECE;

@@ -56,7 +56,7 @@ struct DevView {
   int* cta_start;            // [MAX_PLAN_CTAS + 1]  first list entry of every K-score CTA
   float* part_acc;           // [max_partials][Hq][d_kv]
   float* part_l;             // [max_partials][Hq]
-  float* gate_scratch;       // COMPUTE mode logits [GATE_PIECE][2][d_kv]
+  float* gate_scratch;       // COMPUTE mode logits: [GATE_PIECE][2][d_kv] (small calls) or one [128][d_kv] block per CTA (fused kernel)
 
   __host__ __device__ int4* desc(int l, int side) const { return tile_desc + ((size_t)l * 2 + side) * NT; }
   __host__ __device__ int* aux(int l, int side) const { return tile_aux + ((size_t)l * 2 + side) * NT * TILE; }
@@ -114,6 +114,10 @@ cudaError_t launch_compress_piece(const DevView& v, int layer, const void* K, co
 struct TcMaps;   // tensor maps of the K-score kernel (api.cu)
 cudaError_t launch_decode(const DevView& v, int layer, const LayerParams& lp, const void* q, const int* seq_ids,
                           int n_seq, void* out, int num_splits, int sm_count, const TcMaps* maps, cudaStream_t st);
+struct GateMaps;   // tensor maps of the fused gate kernel (api.cu)
+cudaError_t launch_gate_ranks_tc(const DevView& v, const GateMaps& maps, const LayerParams& lp, int n_tok, unsigned short* levels,
+                                 int sm_count, cudaStream_t st);
+size_t gate_tc_stage_bytes(int n_cta, int d);
 cudaError_t launch_transpose16(const void* in, void* out, int n, cudaStream_t st);
 cudaError_t launch_gate_logits(const DevView& v, const LayerParams& lp, const void* K, const void* V, int n_tok,
                                float* logits, cudaStream_t st);
