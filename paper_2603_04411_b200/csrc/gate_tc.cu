@@ -10,10 +10,12 @@
 // the 128-byte swizzle; a token tile of d = 1024 is 256 KB and cannot stay resident, it is re-read
 // from L2 once per slab.  CTAs walk the slabs in rotated order so that they do not all ask L2 for
 // the same panel of W at the same time.
-// Epilogue warps add the bias and spill each finished slab to a 128 x d fp32 staging area owned
-// by the CTA (rewritten for every item, so it lives in L2); once the item's last slab is out, the
-// same warps run the softmax / prefix-sum / threshold count one row per warp from that staging
-// area while the tensor cores already work on the next item.
+// Epilogue warps (thread = one token row x half a slab) add the bias, reduce every block of 32 logits
+// to (maximum, sum of exp(z - maximum)) in shared memory, and spill the logits to a 128 x d fp32
+// staging area owned by the CTA.  Once the item's last slab is out, one thread per row combines the
+// block summaries into the softmax denominator, finds the block in which the cumulative sum crosses
+// tau and finishes the count inside that block from its 32 staged logits: only 128 bytes per row are
+// read back, and the tensor cores already work on the next item meanwhile.
 //
 // Warp roles (320 threads, one persistent CTA per SM):
 //   warp 0      TMA producer: lanes 0-3 the W^T panel of ring stage L, lanes 4-7 the X~ panel of stage L - 4
@@ -32,6 +34,7 @@ constexpr int GT_EPI = 256;
 constexpr int GT_STAGES = 4;
 constexpr uint32_t GT_TMEM_COLS = 512;
 constexpr uint32_t GT_PANEL_BYTES = 16384;
+constexpr int GT_BLK_STRIDE = 33;                              // row stride of the block summaries (32 blocks + 1 against bank conflicts)
 
 __global__ void __launch_bounds__(GT_THREADS, 1)
 gate_tc_kernel(const __grid_constant__ CUtensorMap map_xk, const __grid_constant__ CUtensorMap map_xv,
@@ -50,7 +53,8 @@ gate_tc_kernel(const __grid_constant__ CUtensorMap map_xk, const __grid_constant
     return;
   }
   const uint32_t stage_bytes = GT_PANEL_BYTES + b_stage_bytes;           // [X~ panel | W^T panel]
-  unsigned char* tail = smem_raw + GT_STAGES * stage_bytes;
+  float2* sBlk = reinterpret_cast<float2*>(smem_raw + GT_STAGES * stage_bytes);   // [128 rows][33]: (max, sum of exp) per block of 32 logits
+  unsigned char* tail = smem_raw + GT_STAGES * stage_bytes + TILE * GT_BLK_STRIDE * sizeof(float2);
   const uint32_t bars = smem_addr(tail);
   // barrier map (8 bytes each)
   const uint32_t full = bars, empty = full + 8 * GT_STAGES, acc_full = empty + 8 * GT_STAGES, acc_empty = acc_full + 16;
@@ -173,66 +177,63 @@ gate_tc_kernel(const __grid_constant__ CUtensorMap map_xk, const __grid_constant
             __syncwarp();
             if (lane == 0) mbar_arrive(acc_empty + 8 * buf);
           }
+          float bm = -INFINITY;
 #pragma unroll
           for (int u = 0; u < 32; u += 4) {
-            float4 o = make_float4(z[u], z[u + 1], z[u + 2], z[u + 3]);
             if (bias) {
               const float4 bb = __ldg(reinterpret_cast<const float4*>(bias + col0 + c + u));
-              o.x += bb.x; o.y += bb.y; o.z += bb.z; o.w += bb.w;
+              z[u] += bb.x; z[u + 1] += bb.y; z[u + 2] += bb.z; z[u + 3] += bb.w;
             }
-            __stcg(reinterpret_cast<float4*>(dst + c + u), o);
+            __stcg(reinterpret_cast<float4*>(dst + c + u), make_float4(z[u], z[u + 1], z[u + 2], z[u + 3]));
+            bm = fmaxf(bm, fmaxf(fmaxf(z[u], z[u + 1]), fmaxf(z[u + 2], z[u + 3])));
           }
+          // block of 32 logits: its maximum and the sum of exp(z - maximum)
+          float bs = 0.f;
+#pragma unroll
+          for (int u = 0; u < 32; ++u) bs += __expf(z[u] - bm);
+          sBlk[row * GT_BLK_STRIDE + ((col0 + c) >> 5)] = make_float2(bm, bs);
         }
       }
       if (!ok) break;
-      if (!(ok = epi_sync())) break;                           // the whole 128 x d block of logits is in the staging area
-      // rank: one row per warp at a time.  Lane L holds the logits i * 128 + 4 L .. + 3 of the row for i = 0 .. d/128 - 1
-      // (coalesced 512-byte reads); prefix sums run over that order with one warp scan per group of 128.
-      const int groups = d >> 7;
-      for (int rr = ew; rr < TILE; rr += GT_EPI / 32) {
-        if (m0 + rr >= n_tok) break;                           // rows past the last token (rr ascends)
-        const float* zrow = stage + (size_t)rr * d;
-        float v[32];
-        float mx = -INFINITY;
-#pragma unroll
-        for (int i = 0; i < 8; ++i) {
-          if (i < groups) {
-            const float4 t = __ldcg(reinterpret_cast<const float4*>(zrow + i * 128 + lane * 4));
-            v[4 * i] = t.x; v[4 * i + 1] = t.y; v[4 * i + 2] = t.z; v[4 * i + 3] = t.w;
-            mx = fmaxf(mx, fmaxf(fmaxf(t.x, t.y), fmaxf(t.z, t.w)));
+      if (!(ok = epi_sync())) break;                           // every block summary and every staged logit of the item is out
+      // rank (Eq. 6, Eq. 8), one thread per row: combine the block summaries into the row total S_d, walk the blocks to
+      // the one where the running sum crosses tau * S_d, and finish inside that block from its 32 staged logits
+      if (ew < 4) {
+        const int rr = ew * 32 + lane;
+        if (m0 + rr < n_tok) {
+          const float2* blk = sBlk + rr * GT_BLK_STRIDE;
+          const int nblk = d >> 5;
+          float M = -INFINITY;
+          for (int b = 0; b < nblk; ++b) M = fmaxf(M, blk[b].x);
+          float total = 0.f;
+          for (int b = 0; b < nblk; ++b) total += blk[b].y * __expf(blk[b].x - M);
+          const float thr = tau * total;                        // c_n <= tau  <=>  S_n <= tau * S_d
+          float run = 0.f, base = 0.f;
+          int bstar = -1;
+          for (int b = 0; b < nblk; ++b) {
+            const float t = blk[b].y * __expf(blk[b].x - M);
+            if (bstar < 0 && run + t > thr) { bstar = b; base = run; }
+            run += t;
           }
-        }
+          int below = d;                                        // NaN logits: nothing crosses, r clamps to 1
+          if (bstar >= 0) {
+            const float4* zb = reinterpret_cast<const float4*>(stage + (size_t)rr * d + bstar * 32);
+            float sn = base;
+            int cnt = 0;
 #pragma unroll
-        for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, o));
-        float carry = 0.f;                                      // sum of all earlier groups
-#pragma unroll
-        for (int i = 0; i < 8; ++i) {
-          if (i < groups) {
-            float run = 0.f;
-#pragma unroll
-            for (int u = 0; u < 4; ++u) { run += expf(v[4 * i + u] - mx); v[4 * i + u] = run; }
-            float incl = run;
-#pragma unroll
-            for (int o = 1; o < 32; o <<= 1) {
-              const float t = __shfl_up_sync(0xffffffffu, incl, o);
-              if (lane >= o) incl += t;
+            for (int u = 0; u < 8; ++u) {
+              const float4 t = __ldcg(zb + u);
+              sn += __expf(t.x - M); cnt += sn <= thr ? 1 : 0;
+              sn += __expf(t.y - M); cnt += sn <= thr ? 1 : 0;
+              sn += __expf(t.z - M); cnt += sn <= thr ? 1 : 0;
+              sn += __expf(t.w - M); cnt += sn <= thr ? 1 : 0;
             }
-            const float off = carry + incl - run;
-#pragma unroll
-            for (int u = 0; u < 4; ++u) v[4 * i + u] += off;
-            carry += __shfl_sync(0xffffffffu, incl, 31);
+            below = bstar * 32 + cnt;
           }
+          int r = d - below;
+          if (r < 1) r = 1;
+          levels[(size_t)(m0 + rr) * 2 + side] = (unsigned short)r;
         }
-        const float thr = tau * carry;                          // c_n <= tau  <=>  S_n <= tau * S_d
-        int below = 0;
-#pragma unroll
-        for (int i = 0; i < 32; ++i)
-          if (i < 4 * groups) below += (v[i] <= thr) ? 1 : 0;
-#pragma unroll
-        for (int o = 16; o > 0; o >>= 1) below += __shfl_xor_sync(0xffffffffu, below, o);
-        int r = d - below;
-        if (r < 1) r = 1;                                       // only reachable with NaN logits
-        if (lane == 0) levels[(size_t)(m0 + rr) * 2 + side] = (unsigned short)r;
       }
       if (!(ok = epi_sync())) break;                           // the staging area may be overwritten by the next item
     }
@@ -252,7 +253,7 @@ cudaError_t launch_gate_ranks_tc(const DevView& v, const GateMaps& maps, const L
   if (n_tok <= 0) return cudaSuccess;
   const int d = v.d_kv;
   const int NS = (d % 256 == 0) ? 256 : 128;
-  const size_t smem = (size_t)GT_STAGES * (GT_PANEL_BYTES + (size_t)NS * 128) + 8 * (2 * GT_STAGES + 5) + 16;
+  const size_t smem = (size_t)GT_STAGES * (GT_PANEL_BYTES + (size_t)NS * 128) + TILE * GT_BLK_STRIDE * sizeof(float2) + 8 * (2 * GT_STAGES + 5) + 16;
   cudaError_t e = cudaFuncSetAttribute(gate_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (e != cudaSuccess) return e;
   const int n_items = 2 * ((n_tok + TILE - 1) / TILE);
