@@ -266,42 +266,65 @@ vacc_kernel(DevView v, int layer, const int* __restrict__ seq_ids, int n_splits)
 
 // -------------------------------------------------------------- merge + V projection
 // One CTA per (query slot, KV head g): sums the splits, normalises, and projects the REP heads
-// of the group through U_V^-1[:, g*128 .. g*128+127].
+// of the group through U_V^-1[:, g*128 .. g*128+127].  512 threads: thread = (pair of output
+// columns, one eighth of the spectral index range), several rows of U_V^-1 in flight per thread.
+constexpr int MG_THREADS = 512;
+constexpr int MG_JGROUPS = MG_THREADS / 64;
+
 template <bool BF16>
-__global__ void __launch_bounds__(256)
+__global__ void __launch_bounds__(MG_THREADS)
 merge_kernel(DevView v, const unsigned short* __restrict__ Uinv_v, int n_splits, void* __restrict__ out) {
-  extern __shared__ float sAcc[];                    // [REP][d_kv] normalised spectral accumulators, then [2][REP][128]
+  extern __shared__ float sAcc[];                    // [REP][d_kv] normalised spectral accumulators, then [MG_JGROUPS][REP][128]
+  __shared__ float sInvL[8];
   const int qs = blockIdx.x, g = blockIdx.y, tid = threadIdx.x;
   const int Hq = v.Hq, d_kv = v.d_kv, REP = v.rep;
-  for (int i = tid; i < REP * d_kv; i += 256) {
-    const int h = g * REP + i / d_kv, j = i % d_kv;
-    float a = 0.f, l = 0.f;
-    for (int s = 0; s < n_splits; ++s) {
-      const size_t pidx = (size_t)qs * n_splits + s;
-      a += v.part_acc[(pidx * Hq + h) * d_kv + j];
-      l += v.part_l[pidx * Hq + h];
+  if (tid < REP) {
+    float l = 0.f;
+    for (int s = 0; s < n_splits; ++s) l += v.part_l[((size_t)qs * n_splits + s) * Hq + g * REP + tid];
+    sInvL[tid] = l > 0.f ? 1.f / l : 0.f;
+  }
+  __syncthreads();
+  for (int i = tid; i < REP * d_kv; i += MG_THREADS) {
+    const int hh = i / d_kv, j = i - hh * d_kv;
+    const float* p = v.part_acc + (((size_t)qs * n_splits) * Hq + g * REP + hh) * d_kv + j;
+    float a = 0.f;
+    for (int s = 0; s < n_splits; ++s) a += p[(size_t)s * Hq * d_kv];
+    sAcc[i] = a * sInvL[hh];
+  }
+  __syncthreads();
+  const int dp = tid & 63, jg = tid >> 6;
+  const int jn = d_kv / MG_JGROUPS, j0 = jg * jn;
+  float o[8][2];
+#pragma unroll
+  for (int h = 0; h < 8; ++h) { o[h][0] = 0.f; o[h][1] = 0.f; }
+  const unsigned* ucol = reinterpret_cast<const unsigned*>(Uinv_v + g * HEAD_DIM) + dp;    // two 16-bit columns per load
+  for (int jb = 0; jb < jn; jb += 8) {
+    unsigned u[8];
+#pragma unroll
+    for (int t = 0; t < 8; ++t) u[t] = __ldg(ucol + (size_t)(j0 + jb + t) * (d_kv / 2));
+#pragma unroll
+    for (int t = 0; t < 8; ++t) {
+      const float u0 = to_f32<BF16>((unsigned short)(u[t] & 0xffffu)), u1 = to_f32<BF16>((unsigned short)(u[t] >> 16));
+#pragma unroll
+      for (int h = 0; h < 8; ++h)
+        if (h < REP) {
+          const float a = sAcc[h * d_kv + j0 + jb + t];
+          o[h][0] += a * u0;
+          o[h][1] += a * u1;
+        }
     }
-    sAcc[i] = l > 0.f ? a / l : 0.f;
   }
   __syncthreads();
-  const int dcol = tid & 127, jh = tid >> 7;         // two threads per output column, half of j each
-  float o[8];
+  float* red = sAcc;                                 // reuse: [MG_JGROUPS][REP][128]
 #pragma unroll
-  for (int h = 0; h < 8; ++h) o[h] = 0.f;
-  const int j0 = jh * (d_kv / 2), j1 = j0 + d_kv / 2;
-  for (int j = j0; j < j1; ++j) {
-    const float u = to_f32<BF16>(Uinv_v[(size_t)j * d_kv + g * HEAD_DIM + dcol]);
+  for (int h = 0; h < 8; ++h)
+    if (h < REP) *reinterpret_cast<float2*>(red + (jg * REP + h) * 128 + 2 * dp) = make_float2(o[h][0], o[h][1]);
+  __syncthreads();
+  for (int i = tid; i < REP * 128; i += MG_THREADS) {
+    float val = 0.f;
 #pragma unroll
-    for (int h = 0; h < 8; ++h)
-      if (h < REP) o[h] += sAcc[h * d_kv + j] * u;
-  }
-  __syncthreads();
-  float* red = sAcc;                                 // reuse: [2][REP][128]
-  for (int h = 0; h < REP; ++h) red[(jh * REP + h) * 128 + dcol] = o[h];
-  __syncthreads();
-  for (int i = tid; i < REP * 128; i += 256) {
+    for (int k = 0; k < MG_JGROUPS; ++k) val += red[k * REP * 128 + i];        // fixed order
     const int h = i >> 7, dc = i & 127;
-    const float val = red[i] + red[REP * 128 + i];
     const size_t oi = ((size_t)qs * Hq + g * REP + h) * HEAD_DIM + dc;
     if (v.out_dtype == TWKV_F32) reinterpret_cast<float*>(out)[oi] = val;
     else if (v.out_dtype == TWKV_BF16) reinterpret_cast<unsigned short*>(out)[oi] = from_f32<true>(val);
@@ -332,10 +355,11 @@ static cudaError_t launch_decode_t(const DevView& v, int layer, const LayerParam
     ProfScope ps(TWKV_K_VACC, st);
     vacc_kernel<BF16, 2><<<vgrid, VA_THREADS, va_smem, st>>>(v, layer, seq_ids, n_splits);
   }
-  const size_t mg_smem = (size_t)v.rep * v.d_kv * 4;
+  const size_t mg_a = (size_t)v.rep * v.d_kv * 4, mg_b = (size_t)MG_JGROUPS * v.rep * 128 * 4;
+  const size_t mg_smem = mg_a > mg_b ? mg_a : mg_b;
   {
     ProfScope ps(TWKV_K_MERGE, st);
-    merge_kernel<BF16><<<dim3(n_seq, v.Hkv), 256, mg_smem, st>>>(v, reinterpret_cast<const unsigned short*>(lp.Uinv_v), n_splits, out);
+    merge_kernel<BF16><<<dim3(n_seq, v.Hkv), MG_THREADS, mg_smem, st>>>(v, reinterpret_cast<const unsigned short*>(lp.Uinv_v), n_splits, out);
   }
   count_launch(4);
   return cudaGetLastError();
