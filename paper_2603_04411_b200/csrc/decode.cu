@@ -141,6 +141,25 @@ vacc_kernel(DevView v, int layer, const int* __restrict__ seq_ids, int n_splits)
 
   for (int i = tid; i < 2 * 8192 / 4; i += VA_THREADS) reinterpret_cast<unsigned*>(sP)[i] = 0u;
   if (tid < 32) sM[tid] = tid < nh ? dec_ordered(v.seqmax[qs * Hq + h0 + tid]) : 0.f;
+  // Descriptors of this split's tiles (the k-th is list[split + k * n_splits]) are kept in a ring of 64 in
+  // shared memory, refilled 16 at a time well ahead of both cursors, so neither the copy cursor nor the
+  // consumer waits for the two dependent global reads list -> descriptor.
+  __shared__ int4 s_desc[64];
+  __shared__ int s_tile[64];
+  const int n_mine = n_tiles > split ? (n_tiles - split + n_splits - 1) / n_splits : 0;
+  auto refill = [&](int k_lo) {                                    // entries k_lo .. k_lo + 15, one thread each
+    if (tid < 16 && k_lo + tid < n_mine) {
+      const int t = list[split + (k_lo + tid) * n_splits];
+      s_tile[(k_lo + tid) & 63] = t;
+      s_desc[(k_lo + tid) & 63] = desc[t];
+    }
+  };
+  if (tid < 48 && tid < n_mine) {                                  // initial fill: entries 0 .. 47
+    const int t = list[split + tid * n_splits];
+    s_tile[tid] = t;
+    s_desc[tid] = desc[t];
+  }
+  __syncthreads();
 
   float acc[TWKV_MAX_CLASSES][MTW][4];
   float accl[MTW][4];
@@ -152,13 +171,13 @@ vacc_kernel(DevView v, int layer, const int* __restrict__ seq_ids, int n_splits)
   for (int m = 0; m < MTW; ++m) { accl[m][0] = accl[m][1] = accl[m][2] = accl[m][3] = 0.f; }
 
   // producer cursor over (tile, panel) jobs of this split
-  int p_ti = split, p_j = 0, p_cls = 0, p_base = 0, p_n = 0;
+  int p_k = 0, p_j = 0, p_cls = 0, p_base = 0, p_n = 0;
   auto p_load_desc = [&]() {
-    if (p_ti < n_tiles) { const int4 d = desc[list[p_ti]]; p_cls = d.y; p_base = d.w; }
+    if (p_k < n_mine) { const int4 d = s_desc[p_k & 63]; p_cls = d.y; p_base = d.w; }
   };
   p_load_desc();
   auto issue = [&]() {
-    if (p_ti < n_tiles) {
+    if (p_k < n_mine) {
       const unsigned char* src = v.blocks + (size_t)(p_base + p_j) * BLOCK_BYTES;
       const unsigned dst = smem_u32(sV + (p_n % VA_STAGES) * 16384);
 #pragma unroll
@@ -167,7 +186,7 @@ vacc_kernel(DevView v, int layer, const int* __restrict__ seq_ids, int n_splits)
         cp_async16(dst + row * 128 + ((ch ^ (row & 7)) << 4), src + row * 128 + ch * 16);
       }
       ++p_n;
-      if (++p_j == p_cls) { p_j = 0; p_ti += n_splits; p_load_desc(); }
+      if (++p_j == p_cls) { p_j = 0; ++p_k; p_load_desc(); }
     }
     cp_async_commit();
   };
@@ -175,28 +194,47 @@ vacc_kernel(DevView v, int layer, const int* __restrict__ seq_ids, int n_splits)
 
   const unsigned ones = BF16 ? 0x3f803f80u : 0x3c003c00u;
   int c_n = 0, pbuf = 0;
-  for (int ti = split; ti < n_tiles; ti += n_splits) {
-    const int tile = list[ti];
-    const int4 dsc = desc[tile];
-    const int cls = dsc.y, n_valid = dsc.z;
+  // Scores of a tile are fetched one tile ahead (the V slot's link to its score row two tiles ahead),
+  // so the gather's latency hides behind the previous tile's panels.
+  const int slot = tid >> 1, part = tid & 1;                       // two threads per token, 16 heads each
+  float sc_next[16];
+  int link_next = -1;                                              // score row of this thread's token in the tile after next (-1: none)
+  auto fetch_link = [&](int k) {
+    link_next = -1;
+    if (k < n_mine && slot < s_desc[k & 63].z) link_next = aux[(size_t)s_tile[k & 63] * TILE + slot];
+  };
+  auto fetch_scores = [&]() {                                      // uses link_next
+    if (link_next >= 0) {
+      const float* srow = v.scores + (size_t)link_next * Hq + h0 + part * 16;
+#pragma unroll
+      for (int hh = 0; hh < 16; ++hh) sc_next[hh] = (part * 16 + hh < nh) ? __ldg(srow + hh) : -INFINITY;
+    } else {
+#pragma unroll
+      for (int hh = 0; hh < 16; ++hh) sc_next[hh] = -INFINITY;
+    }
+  };
+  fetch_link(0);
+  fetch_scores();
+  fetch_link(1);
+  for (int k = 0; k < n_mine; ++k) {
+    if ((k & 15) == 0) refill(k + 48);                             // used from tile k + 16 on; many barriers in between
+    const int cls = s_desc[k & 63].y;
     // probabilities of this tile's tokens: p = exp(s - max), rounded to the storage type
     __syncthreads();
     {
       unsigned char* P = sP + pbuf * 8192;
-      const int slot = tid >> 1, part = tid & 1;                   // two threads per token, 16 heads each
-      const bool ok = slot < n_valid;
-      const int link = ok ? aux[(size_t)tile * TILE + slot] : 0;
-      const float* srow = v.scores + (size_t)link * Hq + h0;
 #pragma unroll
       for (int hh = 0; hh < 16; ++hh) {
         const int h = part * 16 + hh;
         if (h < nh) {
-          const float pv = ok ? __expf(srow[h] - sM[h]) : 0.f;
+          const float pv = __expf(sc_next[hh] - sM[h]);             // -inf for rows past the last token: weight 0
           const int chunk = slot >> 3;
           *reinterpret_cast<unsigned short*>(P + h * 256 + ((chunk ^ (h & 7)) << 4) + (slot & 7) * 2) = from_f32<BF16>(pv);
         }
       }
     }
+    fetch_scores();                                                // next tile's scores (link fetched one tile ago)
+    fetch_link(k + 2);
     for (int j = 0; j < cls; ++j) {
       cp_async_wait<VA_STAGES - 2>();
       __syncthreads();
