@@ -206,8 +206,20 @@ vacc_kernel(DevView v, int layer, const int* __restrict__ seq_ids, int n_splits)
   auto fetch_scores = [&]() {                                      // uses link_next
     if (link_next >= 0) {
       const float* srow = v.scores + (size_t)link_next * Hq + h0 + part * 16;
+      if ((Hq & 3) == 0) {                                         // rows are 16-byte aligned: four heads per load
 #pragma unroll
-      for (int hh = 0; hh < 16; ++hh) sc_next[hh] = (part * 16 + hh < nh) ? __ldg(srow + hh) : -INFINITY;
+        for (int hh = 0; hh < 16; hh += 4) {
+          if (part * 16 + hh < nh) {
+            const float4 t = __ldg(reinterpret_cast<const float4*>(srow + hh));
+            sc_next[hh] = t.x; sc_next[hh + 1] = t.y; sc_next[hh + 2] = t.z; sc_next[hh + 3] = t.w;
+          } else {
+            sc_next[hh] = sc_next[hh + 1] = sc_next[hh + 2] = sc_next[hh + 3] = -INFINITY;
+          }
+        }
+      } else {
+#pragma unroll
+        for (int hh = 0; hh < 16; ++hh) sc_next[hh] = (part * 16 + hh < nh) ? __ldg(srow + hh) : -INFINITY;
+      }
     } else {
 #pragma unroll
       for (int hh = 0; hh < 16; ++hh) sc_next[hh] = -INFINITY;
