@@ -148,7 +148,8 @@ gate_tc_kernel(const __grid_constant__ CUtensorMap map_xk, const __grid_constant
     const int quarter = warp & 3, chalf = ew >> 2;
     const int row = quarter * 32 + lane;
     const uint32_t lane_addr = tmem_base + ((uint32_t)(quarter * 32) << 16);
-    float* stage = stage_all + (size_t)blockIdx.x * TILE * d;  // this CTA's 128 x d staging area
+    // this CTA's staging area, layout [d / 4][128 rows][4 floats]: the 32 rows of a warp store 512 contiguous bytes per instruction
+    float* stage = stage_all + (size_t)blockIdx.x * TILE * d;
     const int cols_per_thread = NS / 2;                        // each row of a slab is split between two threads
     uint32_t ac = 0, epar = 0;
     bool ok = true;
@@ -167,7 +168,7 @@ gate_tc_kernel(const __grid_constant__ CUtensorMap map_xk, const __grid_constant
         if (!(ok = __all_sync(0xffffffffu, mbar_wait(acc_full + 8 * buf, (ac >> 1) & 1u, abort_flag)))) break;
         fence_after_sync();
         const int col0 = ns * NS + chalf * cols_per_thread;
-        float* dst = stage + (size_t)row * d + col0;
+        float* dst = stage + (size_t)(col0 >> 2) * (TILE * 4) + row * 4;
         for (int c = 0; c < cols_per_thread; c += 32) {
           float z[32];
           tmem_ld32(lane_addr + buf * 256 + chalf * cols_per_thread + c, reinterpret_cast<uint32_t*>(z));
@@ -184,7 +185,7 @@ gate_tc_kernel(const __grid_constant__ CUtensorMap map_xk, const __grid_constant
               const float4 bb = __ldg(reinterpret_cast<const float4*>(bias + col0 + c + u));
               z[u] += bb.x; z[u + 1] += bb.y; z[u + 2] += bb.z; z[u + 3] += bb.w;
             }
-            __stcg(reinterpret_cast<float4*>(dst + c + u), make_float4(z[u], z[u + 1], z[u + 2], z[u + 3]));
+            __stcg(reinterpret_cast<float4*>(dst + (size_t)((c + u) >> 2) * (TILE * 4)), make_float4(z[u], z[u + 1], z[u + 2], z[u + 3]));
             bm = fmaxf(bm, fmaxf(fmaxf(z[u], z[u + 1]), fmaxf(z[u + 2], z[u + 3])));
           }
           // block of 32 logits: its maximum and the sum of exp(z - maximum)
@@ -217,12 +218,12 @@ gate_tc_kernel(const __grid_constant__ CUtensorMap map_xk, const __grid_constant
           }
           int below = d;                                        // NaN logits: nothing crosses, r clamps to 1
           if (bstar >= 0) {
-            const float4* zb = reinterpret_cast<const float4*>(stage + (size_t)rr * d + bstar * 32);
+            const float* zb = stage + (size_t)(bstar * 8) * (TILE * 4) + rr * 4;
             float sn = base;
             int cnt = 0;
 #pragma unroll
             for (int u = 0; u < 8; ++u) {
-              const float4 t = __ldcg(zb + u);
+              const float4 t = __ldcg(reinterpret_cast<const float4*>(zb + (size_t)u * (TILE * 4)));
               sn += __expf(t.x - M); cnt += sn <= thr ? 1 : 0;
               sn += __expf(t.y - M); cnt += sn <= thr ? 1 : 0;
               sn += __expf(t.z - M); cnt += sn <= thr ? 1 : 0;
