@@ -86,9 +86,35 @@ __global__ void __launch_bounds__(CHUNK_TOKENS) hist_kernel(DevView v, const int
     atomicOr(&v.status[3], 1);
     return;
   }
-  int* row = v.hist + (size_t)blockIdx.x * v.NK;
-  atomicAdd(&row[key_of(v, 0, seq, (rk + PANEL - 1) / PANEL)], 1);
-  atomicAdd(&row[key_of(v, 1, seq, (rv + PANEL - 1) / PANEL)], 1);
+  atomicAdd(&v.hist[(size_t)key_of(v, 0, seq, (rk + PANEL - 1) / PANEL) * PIECE_CHUNKS + blockIdx.x], 1);
+  atomicAdd(&v.hist[(size_t)key_of(v, 1, seq, (rv + PANEL - 1) / PANEL) * PIECE_CHUNKS + blockIdx.x], 1);
+}
+
+// Warp per key: the key's per-chunk counts (contiguous, [key][chunk]) become exclusive bases, their sum the key's count.
+__global__ void __launch_bounds__(256) scan_kernel(DevView v, int layer, int n_chunks) {
+  const int key = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, lane = threadIdx.x & 31;
+  if (key >= v.NK) return;
+  int* h = v.hist + (size_t)key * PIECE_CHUNKS;
+  int carry = 0;
+  for (int c0 = 0; c0 < n_chunks; c0 += 128) {
+    const int c = c0 + lane * 4;
+    int4 t = make_int4(0, 0, 0, 0);
+    if (c < n_chunks) t = *reinterpret_cast<const int4*>(h + c);          // chunks past n_chunks were cleared
+    const int sum = t.x + t.y + t.z + t.w;
+    int incl = sum;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const int u = __shfl_up_sync(0xffffffffu, incl, o);
+      if (lane >= o) incl += u;
+    }
+    const int base = carry + incl - sum;
+    if (c < n_chunks) *reinterpret_cast<int4*>(h + c) = make_int4(base, base + t.x, base + t.x + t.y, base + t.x + t.y + t.z);
+    carry += __shfl_sync(0xffffffffu, incl, 31);
+  }
+  if (lane == 0) {
+    v.key_cnt[key] = carry;
+    v.key_old_fill[key] = v.fill_l(layer)[key];
+  }
 }
 
 __device__ __forceinline__ int ceil_div(int a, int b) { return (a + b - 1) / b; }
@@ -103,20 +129,8 @@ __global__ void __launch_bounds__(1024) alloc_kernel(DevView v, int layer, int n
   int* fill = v.fill_l(layer);
   int* key_last = v.key_last_l(layer);
   if (tid == 0) s_fail = 0;
-  // phase 1: per key, exclusive scan over chunks
-  for (int k = tid; k < NK; k += 1024) {
-    int run = 0;
-    for (int ch = 0; ch < n_chunks; ++ch) {
-      int* p = v.hist + (size_t)ch * NK + k;
-      const int t = *p;
-      *p = run;
-      run += t;
-    }
-    v.key_cnt[k] = run;
-    v.key_old_fill[k] = fill[k];
-  }
   __syncthreads();
-  // phase 2: new tiles / blocks per key, scanned in key order
+  // (per-key counts and per-chunk bases come from scan_kernel)  new tiles / blocks per key, scanned in key order
   const int KPT = ceil_div(NK, 1024);
   const int k0 = tid * KPT, k1 = min(NK, k0 + KPT);
   const int half = v.S * v.NC;                        // keys per side
@@ -227,9 +241,9 @@ __global__ void __launch_bounds__(1024) alloc_kernel(DevView v, int layer, int n
 }
 
 // Copies the first r elements of a 16-bit row into the tile's panels, +0 beyond r.
-__device__ __forceinline__ void pack_row(const DevView& v, const uint4* __restrict__ src, int r, int cls, int base, int slot, int lane) {
+__device__ __forceinline__ void pack_row(const DevView& v, const uint4* __restrict__ src, int r, int cls, int base, int slot, int lane, int first_chunk) {
   const int nchunks = cls * 8;                            // 16-byte chunks of 8 elements
-  for (int ch = lane; ch < nchunks; ch += 32) {
+  for (int ch = first_chunk + lane; ch < nchunks; ch += 32) {
     const int e0 = ch * 8;
     uint4 val = make_uint4(0u, 0u, 0u, 0u);
     if (e0 < r) {
@@ -295,7 +309,7 @@ __global__ void __launch_bounds__(CHUNK_TOKENS) pack_kernel(DevView v, int layer
       const int k = key[side];
       const int cls = k % v.NC + 1;
       const int old = v.key_old_fill[k];
-      const int g = old + v.hist[(size_t)blockIdx.x * v.NK + k] + before[side];
+      const int g = old + v.hist[(size_t)k * PIECE_CHUNKS + blockIdx.x] + before[side];
       const int ord = g / TILE, slot = g % TILE;
       const int old_tiles = (old + TILE - 1) / TILE;
       int tile, base;
@@ -324,19 +338,53 @@ __global__ void __launch_bounds__(CHUNK_TOKENS) pack_kernel(DevView v, int layer
   }
   __syncthreads();
   if (tid < 2 && s_sum[tid]) atomicAdd(&v.rank_sums[layer * 2 + tid], s_sum[tid]);
-  // warp per token: move the rows
+  // warp per token: move the rows.  The first 32 chunks (256 elements) of four rows are loaded before any is stored,
+  // so a warp keeps four independent copies in flight; wider rows finish in pack_row.
   const int warp = tid >> 5, lane = tid & 31;
   const size_t row_bytes = (size_t)v.d_kv * 2;
-  for (int t = warp; t < CHUNK_TOKENS; t += CHUNK_TOKENS / 32) {
-    const int tok = blockIdx.x * CHUNK_TOKENS + t;
-    if (tok >= n_tok) break;
+  constexpr int WARPS = CHUNK_TOKENS / 32;
+  for (int t0 = warp * 2; t0 < CHUNK_TOKENS; t0 += WARPS * 2) {          // two tokens x two sides per round
+    uint4 val[4];
+    int meta[4], base[4];
+    bool live[4];
 #pragma unroll
-    for (int side = 0; side < 2; ++side) {
-      const Place p = s_place[side][t];
-      const int slot = p.slot_cls_r & 0xff, cls = (p.slot_cls_r >> 8) & 0xff, rr = p.slot_cls_r >> 16;
-      const unsigned char* src = reinterpret_cast<const unsigned char*>(side ? V : K) + (size_t)tok * row_bytes;
-      pack_row(v, reinterpret_cast<const uint4*>(src), rr, cls, p.base, slot, lane);
-      if (p.flags & 1) zero_tail(v, cls, p.base, slot, lane);
+    for (int q = 0; q < 4; ++q) {
+      const int t = t0 + (q >> 1), side = q & 1, tok = blockIdx.x * CHUNK_TOKENS + t;
+      live[q] = tok < n_tok;
+      val[q] = make_uint4(0u, 0u, 0u, 0u);
+      meta[q] = 0; base[q] = 0;
+      if (live[q]) {
+        const Place p = s_place[side][t];
+        meta[q] = p.slot_cls_r; base[q] = p.base;
+        const int cls = (p.slot_cls_r >> 8) & 0xff, rr = p.slot_cls_r >> 16;
+        if (lane < cls * 8 && lane * 8 < rr)
+          val[q] = __ldg(reinterpret_cast<const uint4*>(reinterpret_cast<const unsigned char*>(side ? V : K) + (size_t)tok * row_bytes) + lane);
+      }
+    }
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {
+      if (!live[q]) continue;
+      const int t = t0 + (q >> 1), side = q & 1, tok = blockIdx.x * CHUNK_TOKENS + t;
+      const int slot = meta[q] & 0xff, cls = (meta[q] >> 8) & 0xff, rr = meta[q] >> 16;
+      if (lane < cls * 8) {
+        uint4 o = val[q];
+        const int keep = rr - lane * 8;                       // elements kept in this chunk
+        if (keep < 8) {
+          unsigned* w = reinterpret_cast<unsigned*>(&o);
+#pragma unroll
+          for (int p = 0; p < 4; ++p) {
+            const int left = keep - 2 * p;
+            if (left <= 0) w[p] = 0u;
+            else if (left == 1) w[p] &= 0x0000ffffu;
+          }
+        }
+        *reinterpret_cast<uint4*>(v.blocks + (size_t)(base[q] + (lane >> 3)) * BLOCK_BYTES + slot * (PANEL * 2) + (lane & 7) * 16) = o;
+      }
+      if (cls > 4) {
+        const unsigned char* src = reinterpret_cast<const unsigned char*>(side ? V : K) + (size_t)tok * row_bytes;
+        pack_row(v, reinterpret_cast<const uint4*>(src), rr, cls, base[q], slot, lane, 32);
+      }
+      if (s_place[side][t].flags & 1) zero_tail(v, cls, base[q], slot, lane);
     }
   }
 }
@@ -345,12 +393,17 @@ cudaError_t launch_compress_piece(const DevView& v, int layer, const void* K, co
                                   const int* positions, int n_tok, const unsigned short* levels, cudaStream_t st) {
   if (n_tok <= 0) return cudaSuccess;
   const int n_chunks = (n_tok + CHUNK_TOKENS - 1) / CHUNK_TOKENS;
-  cudaError_t e = cudaMemsetAsync(v.hist, 0, (size_t)n_chunks * v.NK * sizeof(int), st);
+  const int n_cols = (n_chunks + 3) & ~3;                  // scan_kernel reads the counts four at a time
+  cudaError_t e = cudaMemset2DAsync(v.hist, (size_t)PIECE_CHUNKS * sizeof(int), 0, (size_t)n_cols * sizeof(int), (size_t)v.NK, st);
   if (e != cudaSuccess) return e;
   { ProfScope ps(TWKV_K_HIST, st); hist_kernel<<<n_chunks, CHUNK_TOKENS, 0, st>>>(v, seq_ids, positions, levels, n_tok); }
-  { ProfScope ps(TWKV_K_ALLOC, st); alloc_kernel<<<1, 1024, 0, st>>>(v, layer, n_chunks); }
+  {
+    ProfScope ps(TWKV_K_ALLOC, st);
+    scan_kernel<<<(v.NK + 7) / 8, 256, 0, st>>>(v, layer, n_chunks);
+    alloc_kernel<<<1, 1024, 0, st>>>(v, layer, n_chunks);
+  }
   { ProfScope ps(TWKV_K_PACK, st); pack_kernel<<<n_chunks, CHUNK_TOKENS, 0, st>>>(v, layer, K, V, seq_ids, positions, levels, n_tok); }
-  count_launch(3);
+  count_launch(4);
   return cudaGetLastError();
 }
 
