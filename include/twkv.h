@@ -72,7 +72,7 @@ typedef enum {
 #define TWKV_TILE_TOKENS 128        /* tokens per tile                                               */
 #define TWKV_PANEL_ELEMS 64         /* elements per panel row = rank granule                         */
 #define TWKV_BLOCK_BYTES 16384      /* one panel: 128 rows x 64 elements x 2 bytes                   */
-#define TWKV_PIECE_TOKENS 65536     /* a compress call is processed in pieces of this many tokens    */
+#define TWKV_PIECE_TOKENS 131072    /* a compress call is processed in pieces of this many tokens    */
 #define TWKV_MAX_CLASSES 16
 
 typedef struct {

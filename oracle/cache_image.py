@@ -33,7 +33,7 @@ import numpy as np
 TILE = 128
 PANEL = 64
 BLOCK_ELEMS = TILE * PANEL
-PIECE_TOKENS = 65536
+PIECE_TOKENS = 131072
 
 
 class CacheImage:

@@ -17,7 +17,7 @@ TWKV_OK, TWKV_ERR_INVALID_ARG, TWKV_ERR_UNSUPPORTED, TWKV_ERR_CAPACITY = 0, 1, 2
 TWKV_ERR_CUDA, TWKV_ERR_DEVICE_CHECK, TWKV_ERR_TIMEOUT = 4, 5, 6
 TWKV_F16, TWKV_BF16, TWKV_F32 = 0, 1, 2
 TWKV_GATE_FORCED, TWKV_GATE_LOGITS, TWKV_GATE_COMPUTE = 0, 1, 2
-TILE_TOKENS, PANEL_ELEMS, BLOCK_BYTES, PIECE_TOKENS, MAX_CLASSES = 128, 64, 16384, 65536, 16
+TILE_TOKENS, PANEL_ELEMS, BLOCK_BYTES, PIECE_TOKENS, MAX_CLASSES = 128, 64, 16384, 131072, 16
 
 EXPORTS = ["twkv_cache_required_bytes", "twkv_cache_create", "twkv_cache_destroy", "twkv_cache_reset",
            "twkv_cache_set_layer_params", "twkv_compress", "twkv_decode_attn", "twkv_cache_status",

@@ -12,7 +12,7 @@ constexpr int TILE = TWKV_TILE_TOKENS;      // tokens per tile (the MMA M)
 constexpr int PANEL = TWKV_PANEL_ELEMS;     // elements per panel row
 constexpr int BLOCK_BYTES = TWKV_BLOCK_BYTES;
 constexpr int HEAD_DIM = 128;
-constexpr int CHUNK_TOKENS = 256;           // tokens per compress CTA
+constexpr int CHUNK_TOKENS = 128;           // tokens per compress CTA
 constexpr int PIECE_CHUNKS = TWKV_PIECE_TOKENS / CHUNK_TOKENS;
 constexpr int ROPE_LO = 512;                // pos = hi * 512 + lo
 constexpr int ROPE_HI = 1024;               // positions up to 512 * 1024 - 1
@@ -41,7 +41,7 @@ struct DevView {
   int* seq_tokens;           // [L][S]
   unsigned long long* rank_sums;  // [L][2]  sum of r_K, r_V
   // scratch shared by all layers
-  int* hist;                 // [PIECE_CHUNKS][NK]   per-chunk key counts -> exclusive bases
+  int* hist;                 // [NK][PIECE_CHUNKS]   per-chunk key counts -> exclusive bases
   int* key_cnt;              // [NK]  tokens of the key in the current piece
   int* key_old_fill;         // [NK]
   int* key_first_id;         // [NK]  id of the key's first new tile
