@@ -320,3 +320,85 @@ def test_compute_mode_gate_levels_bit_exact(B):
     max_abs, rel_l2 = attn_errors(out.cpu().numpy(), oracle_decode(li, ranks, [0, 1]))
     assert max_abs < MAX_ABS and rel_l2 < REL_L2, (max_abs, rel_l2)
     gc.close()
+
+
+def _compute_mode_case(B, *, n_kv_heads, n_q_heads, dtype, ctx, n_seq, seed, min_keep=0.85):
+    """COMPUTE-mode compress (fused tcgen05 gate for calls of 1024 tokens or more) + decode against the oracle;
+    tokens whose cumulative softmax comes within 1e-2 (relative) of tau in the oracle are left out."""
+    dn = "f16" if dtype == torch.float16 else "bf16"
+    li = workloads.build_layer(seed, n_seq=n_seq, ctx=ctx, n_q_heads=n_q_heads, n_kv_heads=n_kv_heads, dtype=dtype,
+                               outlier="pct:1", mode="forced")
+    d = li.d_kv
+    Wk, Wv, bk, bv = workloads.gate_params(seed + 1, d, dtype, n_bumps=min(64, d // 4), first_dim=min(64, d // 4))
+    zk = oracle.gate_logits(oracle.widen16(bits16(li.xt_k), dn), oracle.widen16(bits16(Wk), dn), bk.double().numpy())
+    zv = oracle.gate_logits(oracle.widen16(bits16(li.xt_v), dn), oracle.widen16(bits16(Wv), dn), bv.double().numpy())
+    rk, mk = oracle.gate_rank(zk, 0.1)
+    rv, mv = oracle.gate_rank(zv, 0.1)
+    keep = np.nonzero((mk >= 1e-2) & (mv >= 1e-2))[0]
+    assert len(keep) > min_keep * len(rk) and len(keep) >= 1024
+    sel = torch.from_numpy(keep)
+    for name in ["xt_k", "xt_v", "seq_ids", "positions"]:
+        setattr(li, name, getattr(li, name)[sel].contiguous())
+    ranks = np.stack([rk[keep], rv[keep]], axis=1).astype(np.int64)
+    li = to_cuda(li)
+    n = len(keep)
+    gc = GpuCache(B, n_layers=1, n_q_heads=n_q_heads, n_kv_heads=n_kv_heads, dtype=dtype, out_dtype=torch.float32,
+                  max_seqs=n_seq, max_tokens_per_seq=ctx, payload_bytes=int((-(-ranks // 64) * 128).sum()))
+    gate = [t.cuda().contiguous() for t in (Wk, Wv, bk, bv)]
+    B.twkv_cache_set_layer_params(gc.h, 0, li.Uinv_k, li.Uinv_v, *gate)
+    levels = torch.zeros(n, 2, dtype=torch.int16, device="cuda")
+    B.twkv_compress(gc.h, 0, li.xt_k, li.xt_v, li.seq_ids, li.positions, None, levels, B.TWKV_GATE_COMPUTE)
+    assert B.twkv_cache_status(gc.h) == B.TWKV_OK
+    np.testing.assert_array_equal(levels.cpu().numpy().view(np.uint16).astype(np.int64), ranks)
+    img = CacheImage(1, d, n_seq, ctx, int(gc.lay.n_blocks))
+    assert img.append(0, bits16(li.xt_k), bits16(li.xt_v), li.seq_ids.cpu().numpy(), li.positions.cpu().numpy(), ranks)
+    compare_cache_with_image(gc, img)
+    seqs = list(range(n_seq))
+    out = torch.empty(n_seq, n_q_heads, 128, device="cuda")
+    B.twkv_decode_attn(gc.h, 0, li.q, torch.tensor(seqs, dtype=torch.int32, device="cuda"), out)
+    assert B.twkv_cache_status(gc.h) == B.TWKV_OK
+    errs = attn_errors(out.cpu().numpy(), oracle_decode(li, ranks, seqs))
+    gc.close()
+    return errs, ranks
+
+
+def test_compute_mode_bf16_four_kv_heads(B):
+    # d_kv = 512 (two 256-wide logit slabs), bf16, GQA 8, a ragged 1300-token call
+    (max_abs, rel_l2), ranks = _compute_mode_case(B, n_kv_heads=4, n_q_heads=32, dtype=torch.bfloat16, ctx=650, n_seq=2, seed=71)
+    assert max_abs < MAX_ABS and rel_l2 < REL_L2, (max_abs, rel_l2)
+    assert ranks.min() >= 1 and ranks.max() <= 512
+
+
+def test_compute_mode_three_kv_heads(B):
+    # d_kv = 384: 128-wide logit slabs in the gate, an odd number of KV-head slabs in the K-score kernel, GQA 2
+    (max_abs, rel_l2), _ = _compute_mode_case(B, n_kv_heads=3, n_q_heads=6, dtype=torch.float16, ctx=600, n_seq=2, seed=73)
+    assert max_abs < MAX_ABS and rel_l2 < REL_L2, (max_abs, rel_l2)
+
+
+def test_compress_spanning_two_pieces(B):
+    # one call of 131072 + 300 tokens is processed as two pieces; levels, tables and packed bytes must still match
+    # the oracle's image (small ranks keep the case light), and decode must agree on one of the sequences
+    n_seq, ctx = 4, 32843
+    li = workloads.build_layer(81, n_seq=n_seq, ctx=ctx, n_q_heads=8, mode="forced", level_probs=(0.0, 0.0, 0.02, 0.98),
+                               n_calib=2048)
+    assert li.xt_k.shape[0] > B.PIECE_TOKENS
+    li = to_cuda(li)
+    ranks = li.ranks.cpu().numpy().astype(np.int64)
+    gc = GpuCache(B, n_layers=1, n_q_heads=8, n_kv_heads=8, dtype=torch.float16, out_dtype=torch.float32,
+                  max_seqs=n_seq, max_tokens_per_seq=ctx, payload_bytes=int((-(-ranks // 64) * 128).sum()))
+    B.twkv_cache_set_layer_params(gc.h, 0, li.Uinv_k, li.Uinv_v)
+    B.twkv_compress(gc.h, 0, li.xt_k, li.xt_v, li.seq_ids, li.positions, None, levels_tensor(ranks), B.TWKV_GATE_FORCED)
+    assert B.twkv_cache_status(gc.h) == B.TWKV_OK
+    img = CacheImage(1, li.d_kv, n_seq, ctx, int(gc.lay.n_blocks))
+    assert img.append(0, bits16(li.xt_k), bits16(li.xt_v), li.seq_ids.cpu().numpy(), li.positions.cpu().numpy(), ranks)
+    compare_cache_with_image(gc, img)
+    out = torch.empty(1, 8, 128, device="cuda")
+    B.twkv_decode_attn(gc.h, 0, li.q[3:4].contiguous(), torch.tensor([3], dtype=torch.int32, device="cuda"), out)
+    assert B.twkv_cache_status(gc.h) == B.TWKV_OK
+    li_q = li.q
+    li.q = li.q[3:4]
+    want = oracle_decode(li, ranks, [3])
+    li.q = li_q
+    max_abs, rel_l2 = attn_errors(out.cpu().numpy(), want)
+    assert max_abs < MAX_ABS and rel_l2 < REL_L2, (max_abs, rel_l2)
+    gc.close()
