@@ -402,3 +402,45 @@ def test_compress_spanning_two_pieces(B):
     max_abs, rel_l2 = attn_errors(out.cpu().numpy(), want)
     assert max_abs < MAX_ABS and rel_l2 < REL_L2, (max_abs, rel_l2)
     gc.close()
+
+
+def test_benchmark_workload_full_size_sampled(B):
+    # the workload and launch configuration bench.py times (B = 16, T = 32768, GQA 4, fp16, COMPUTE gate), checked
+    # on what the oracle can afford: the ranks of every token of one sequence, and that sequence's attention output
+    import bench
+    dev = torch.device("cuda", 0)
+    li, gate = bench.build_workload(dev)
+    Wk, Wv, bk, bv = gate
+    n_seq, ctx, Hq = bench.B_SEQ, bench.CTX, bench.HQ
+    n_tok = n_seq * ctx
+    cfg = B.make_config(n_layers=1, n_q_heads=Hq, n_kv_heads=bench.HKV, dtype=torch.float16, out_dtype=torch.float32,
+                        max_seqs=n_seq, max_tokens_per_seq=ctx)
+    pool = torch.empty(B.twkv_cache_required_bytes(cfg, int(n_tok * 2 * 2 * 420)), dtype=torch.uint8, device=dev)
+    cache = B.twkv_cache_create(cfg, pool)
+    B.twkv_cache_set_layer_params(cache, 0, li.Uinv_k, li.Uinv_v, Wk, Wv, bk, bv)
+    levels = torch.zeros(n_tok, 2, dtype=torch.int16, device=dev)
+    B.twkv_compress(cache, 0, li.xt_k, li.xt_v, li.seq_ids, li.positions, None, levels, B.TWKV_GATE_COMPUTE)
+    out = torch.empty(n_seq, Hq, 128, dtype=torch.float32, device=dev)
+    B.twkv_decode_attn(cache, 0, li.q, torch.arange(n_seq, dtype=torch.int32, device=dev), out)
+    assert B.twkv_cache_status(cache) == B.TWKV_OK
+    st = B.twkv_cache_stats(cache, 0)
+    got = levels.cpu().numpy().view(np.uint16).astype(np.int64)
+    assert st.tokens == n_tok and st.bytes_algorithmic == int(2 * got.sum())
+    s = 5                                                                 # the sampled sequence
+    lo, hi = s * ctx, (s + 1) * ctx
+    xk = oracle.widen16(bits16(li.xt_k[lo:hi]), "f16")
+    xv = oracle.widen16(bits16(li.xt_v[lo:hi]), "f16")
+    rk, mk = oracle.gate_rank(oracle.gate_logits(xk, oracle.widen16(bits16(Wk), "f16"), bk.double().cpu().numpy()), 0.1)
+    rv, mv = oracle.gate_rank(oracle.gate_logits(xv, oracle.widen16(bits16(Wv), "f16"), bv.double().cpu().numpy()), 0.1)
+    safe_k, safe_v = mk >= 1e-2, mv >= 1e-2
+    assert safe_k.mean() > 0.9 and safe_v.mean() > 0.9
+    np.testing.assert_array_equal(got[lo:hi, 0][safe_k], rk[safe_k])
+    np.testing.assert_array_equal(got[lo:hi, 1][safe_v], rv[safe_v])
+    # attention of the sampled sequence, with the ranks the library assigned (they equal the oracle's wherever the
+    # oracle's decision does not hinge on rounding)
+    want = oracle.decode_attn(xk, xv, got[lo:hi, 0], got[lo:hi, 1], li.positions[lo:hi].cpu().numpy(),
+                              oracle.widen16(bits16(li.Uinv_k), "f16"), oracle.widen16(bits16(li.Uinv_v), "f16"),
+                              oracle.widen16(bits16(li.q[s]), "f16"), bench.HKV, 500000.0, 128 ** -0.5)
+    max_abs, rel_l2 = attn_errors(out[s].cpu().numpy(), want)
+    assert max_abs < MAX_ABS and rel_l2 < REL_L2, (max_abs, rel_l2)
+    B.twkv_cache_destroy(cache)
