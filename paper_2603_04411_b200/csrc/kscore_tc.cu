@@ -255,8 +255,7 @@ kscore_tc_kernel(const __grid_constant__ CUtensorMap map_blocks, const __grid_co
     // cos / sin of (row, frequency): pos = hi * 512 + lo, the two table rows combine by the angle-addition
     // formulas.  Table rows are read coalesced (8 lanes per row) and handed to the row's lane through a
     // per-warp staging buffer, 8 frequencies at a time.
-    auto rope_setup = [&](int tile) {
-      const int pos = kpos[(size_t)tile * TILE + row];
+    auto rope_setup = [&](int pos) {
       float2* stage = sRope + (warp - 2) * 256;
       const int rs = lane >> 3, t8 = lane & 7;
       int off_hi[8], off_lo[8];
@@ -317,11 +316,12 @@ kscore_tc_kernel(const __grid_constant__ CUtensorMap map_blocks, const __grid_co
     };
 
     int4 e = w0 < total ? klist[w0] : kt_none;
-    if (w0 < total) { write_q(e.w); rope_setup(e.x); }
+    if (w0 < total) { write_q(e.w); rope_setup(kpos[(size_t)e.x * TILE + row]); }
     for (int w = w0; w < total && ok; w += wstep) {
       const int4 nxt = w + wstep < total ? klist[w + wstep] : kt_none;
       const int tile = e.x, cls = e.y & 0xff, n_valid = e.y >> 8, qs = e.w;
       const int n_slabs = ((cls + KT_A_SLOTS - 1) / KT_A_SLOTS) * Hkv;
+      const int pos_next = nxt.w >= 0 ? kpos[(size_t)nxt.x * TILE + row] : 0;      // fetched now, used after the tile's slabs
       for (int sl = 0; sl < n_slabs; ++sl, ++sc) {
         const uint32_t buf = sc & 1u, par = (sc >> 1) & 1u;
         if (!(ok = __all_sync(0xffffffffu, mbar_wait(slab_full + 8 * buf, par, abort_flag)))) break;
@@ -352,7 +352,7 @@ kscore_tc_kernel(const __grid_constant__ CUtensorMap map_blocks, const __grid_co
       }
       if (!ok) break;
       // the next tile's rotation factors are fetched while this tile's last score products drain
-      if (nxt.w >= 0) rope_setup(nxt.x);
+      if (nxt.w >= 0) rope_setup(pos_next);
       // all score products of the tile have retired: scale, mask the rows past the last token, store
       if (!(ok = __all_sync(0xffffffffu, mbar_wait(s_full, tcount & 1u, abort_flag)))) break;
       ++tcount;
