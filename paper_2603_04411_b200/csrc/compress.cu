@@ -333,8 +333,12 @@ __global__ void __launch_bounds__(CHUNK_TOKENS) pack_kernel(DevView v, int layer
         v.aux(layer, 1)[(size_t)tile * TILE + slot] = kslot;
       }
     }
-    atomicAdd(&s_sum[0], (unsigned long long)r[0]);
-    atomicAdd(&s_sum[1], (unsigned long long)r[1]);
+  }
+  {
+    unsigned rk = valid ? (unsigned)r[0] : 0u, rv = valid ? (unsigned)r[1] : 0u;          // <= 32 * 1024 per warp
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) { rk += __shfl_xor_sync(0xffffffffu, rk, o); rv += __shfl_xor_sync(0xffffffffu, rv, o); }
+    if ((tid & 31) == 0) { atomicAdd(&s_sum[0], (unsigned long long)rk); atomicAdd(&s_sum[1], (unsigned long long)rv); }
   }
   __syncthreads();
   if (tid < 2 && s_sum[tid]) atomicAdd(&v.rank_sums[layer * 2 + tid], s_sum[tid]);
@@ -343,12 +347,13 @@ __global__ void __launch_bounds__(CHUNK_TOKENS) pack_kernel(DevView v, int layer
   const int warp = tid >> 5, lane = tid & 31;
   const size_t row_bytes = (size_t)v.d_kv * 2;
   constexpr int WARPS = CHUNK_TOKENS / 32;
-  for (int t0 = warp * 2; t0 < CHUNK_TOKENS; t0 += WARPS * 2) {          // two tokens x two sides per round
-    uint4 val[4];
-    int meta[4], base[4];
-    bool live[4];
+  constexpr int NQ = 4;                                                  // two tokens x two sides per round
+  for (int t0 = warp * (NQ / 2); t0 < CHUNK_TOKENS; t0 += WARPS * (NQ / 2)) {
+    uint4 val[NQ];
+    int meta[NQ], base[NQ];
+    bool live[NQ];
 #pragma unroll
-    for (int q = 0; q < 4; ++q) {
+    for (int q = 0; q < NQ; ++q) {
       const int t = t0 + (q >> 1), side = q & 1, tok = blockIdx.x * CHUNK_TOKENS + t;
       live[q] = tok < n_tok;
       val[q] = make_uint4(0u, 0u, 0u, 0u);
@@ -362,7 +367,7 @@ __global__ void __launch_bounds__(CHUNK_TOKENS) pack_kernel(DevView v, int layer
       }
     }
 #pragma unroll
-    for (int q = 0; q < 4; ++q) {
+    for (int q = 0; q < NQ; ++q) {
       if (!live[q]) continue;
       const int t = t0 + (q >> 1), side = q & 1, tok = blockIdx.x * CHUNK_TOKENS + t;
       const int slot = meta[q] & 0xff, cls = (meta[q] >> 8) & 0xff, rr = meta[q] >> 16;
