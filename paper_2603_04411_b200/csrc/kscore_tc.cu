@@ -31,7 +31,7 @@ using namespace tc;
 
 constexpr int KT_THREADS = 352;
 constexpr int KT_EPI = 256;
-constexpr int KT_A_SLOTS = 8;
+constexpr int KT_A_SLOTS = 8;                                  // power of two (slot = panel count & 7, phase = bit 3)
 constexpr uint32_t KT_TMEM_COLS = 512;
 constexpr uint32_t TM_SLAB = 0, TM_KR = 256, TM_S = 384;      // column offsets inside the allocation
 constexpr uint32_t PANEL_BYTES = 16384;
@@ -164,9 +164,12 @@ kscore_tc_kernel(const __grid_constant__ CUtensorMap map_blocks, const __grid_co
   } else if (warp == 1) {
     // ------------------------------------------------------------- MMA issuer (one elected lane runs the whole role)
     if (elect_one()) {
+      // This role is one thread issuing asynchronous work; what it costs is its own instruction stream (a 64-cycle MMA
+      // per few instructions), so descriptors are stepped with 32-bit adds, a panel's four MMAs are one asm block, and
+      // every wait tries once inline before it falls into the bounded loop.
       const uint32_t idesc_main = idesc_f16(BF16 ? 1 : 0, 128, 128);
       const uint32_t idesc_s = idesc_f16(0, 128, 16);
-      const uint64_t adesc0 = kmajor_sw128_desc(sA), bdesc0 = kmajor_sw128_desc(sB), qdesc0 = kmajor_sw128_desc(sQ);
+      const uint32_t a_lo0 = kmajor_sw128_desc_lo(sA), b_lo0 = kmajor_sw128_desc_lo(sB), q_lo0 = kmajor_sw128_desc_lo(sQ);
       uint32_t bst = 0, bph = 0, ak = 0, sc = 0;
       bool ok = true;
       // The score product of slab n is issued after the main product of slab n + 2: the tensor pipe
@@ -175,15 +178,11 @@ kscore_tc_kernel(const __grid_constant__ CUtensorMap map_blocks, const __grid_co
       uint32_t pq0 = 0, pq1 = 0;
       int npend = 0;
       auto issue_scores = [&](uint32_t pe) {
-        const uint32_t psc = pe >> 8, kb = psc & 1u, pg = (pe >> 2) & 63u, pacc = (pe >> 1) & 1u;
-        if (!mbar_wait(kr_full + 8 * kb, (psc >> 1) & 1u, abort_flag)) return false;
+        const uint32_t psc = pe >> 8, kb = psc & 1u, pg = (pe >> 2) & 63u;
+        if (!mbar_wait_thin(kr_full + 8 * kb, (psc >> 1) & 1u, abort_flag)) return false;
         fence_after_sync();
-        const uint64_t qd = qdesc0 + (uint64_t)(pg * (1024 >> 4));
-        const uint32_t d = tmem_base + TM_S + 16 * pg, a = tmem_base + TM_KR + 64 * kb;
-        mma_f16_ts(d, a, qd, idesc_s, pacc);
-#pragma unroll
-        for (int ks = 1; ks < 8; ++ks)
-          mma_f16_ts(d, a + 8 * ks, qd + (ks >> 2) * (KT_Q_PANEL_BYTES >> 4) + 2 * (ks & 3), idesc_s, 1u);
+        mma_f16_ts_k128(tmem_base + TM_S + 16 * pg, tmem_base + TM_KR + 64 * kb, q_lo0 + pg * (1024 >> 4), KT_Q_PANEL_BYTES >> 4, idesc_s,
+                        (pe >> 1) & 1u);
         mma_commit(kr_empty + 8 * kb);
         if (pe & 1u) mma_commit(s_full);
         return true;
@@ -197,22 +196,20 @@ kscore_tc_kernel(const __grid_constant__ CUtensorMap map_blocks, const __grid_co
           for (int sl = 0; sl < Hkv && ok; ++sl) {
             const int g = sl + g_rot < Hkv ? sl + g_rot : sl + g_rot - Hkv;
             const uint32_t buf = sc & 1u;
-            if (!(ok = mbar_wait(slab_empty + 8 * buf, ((sc >> 1) & 1u) ^ 1u, abort_flag))) break;
+            if (!(ok = mbar_wait_thin(slab_empty + 8 * buf, ((sc >> 1) & 1u) ^ 1u, abort_flag))) break;
             const uint32_t d = tmem_base + TM_SLAB + buf * 128;
-            for (int j = 0; j < np; ++j) {
-              const uint32_t an = ak + j, slot = an % KT_A_SLOTS;
-              if (sl == 0 && !(ok = mbar_wait(a_full + 8 * slot, (an / KT_A_SLOTS) & 1u, abort_flag))) break;
-              const uint32_t st = bst, ph = bph;
+            const bool first = sl == 0, last = sl == Hkv - 1;
+            uint32_t an = ak;
+            for (int j = 0; j < np; ++j, ++an) {
+              const uint32_t slot = an & (KT_A_SLOTS - 1);
+              if (first && !(ok = mbar_wait_thin(a_full + 8 * slot, (an >> 3) & 1u, abort_flag))) break;
+              const uint32_t st = bst;
+              if (!(ok = mbar_wait_thin(b_full + 8 * st, bph, abort_flag))) break;
               if (++bst == (uint32_t)nb) { bst = 0; bph ^= 1u; }
-              if (!(ok = mbar_wait(b_full + 8 * st, ph, abort_flag))) break;
               fence_after_sync();
-              const uint64_t adesc = adesc0 + (uint64_t)(slot * (PANEL_BYTES >> 4));
-              const uint64_t bdesc = bdesc0 + (uint64_t)(st * (PANEL_BYTES >> 4));
-              mma_f16_ss(d, adesc, bdesc, idesc_main, j > 0 ? 1u : 0u);
-#pragma unroll
-              for (int ks = 1; ks < 4; ++ks) mma_f16_ss(d, adesc + 2 * ks, bdesc + 2 * ks, idesc_main, 1u);
+              mma_f16_ss_panel(d, a_lo0 + slot * (PANEL_BYTES >> 4), b_lo0 + st * (PANEL_BYTES >> 4), idesc_main, j > 0 ? 1u : 0u);
               mma_commit(b_empty + 8 * st);                             // ring stage reusable when these MMAs retire
-              if (sl == Hkv - 1) mma_commit(a_empty + 8 * slot);        // last slab of the pass: the X^_K panel is done
+              if (last) mma_commit(a_empty + 8 * slot);                 // last slab of the pass: the X^_K panel is done
             }
             if (!ok) break;
             mma_commit(slab_full + 8 * buf);                            // slab accumulator complete
@@ -221,7 +218,7 @@ kscore_tc_kernel(const __grid_constant__ CUtensorMap map_blocks, const __grid_co
               pq0 = pq1;
               npend = 1;
             }
-            const uint32_t pe = (sc << 8) | ((uint32_t)g << 2) | (p0 > 0 ? 2u : 0u) | ((p0 + np >= cls && sl == Hkv - 1) ? 1u : 0u);
+            const uint32_t pe = (sc << 8) | ((uint32_t)g << 2) | (p0 > 0 ? 2u : 0u) | ((p0 + np >= cls && last) ? 1u : 0u);
             if (npend == 0) pq0 = pe; else pq1 = pe;
             ++npend;
             ++sc;

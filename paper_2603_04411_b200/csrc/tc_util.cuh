@@ -47,6 +47,16 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
   return false;
 }
 
+// The same wait for a role that runs on one thread and must spend few instructions: one attempt inline, the bounded
+// loop out of line.
+static __device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+  return mbar_wait(bar, parity, abort_flag);
+}
+__device__ __forceinline__ bool mbar_wait_thin(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+  if (mbar_try(bar, parity)) return true;
+  return mbar_wait_slow(bar, parity, abort_flag);
+}
+
 // Used only after a give-up: lets copies already in flight land before the CTA exits.
 __device__ __forceinline__ void mbar_wait_drain(uint32_t bar, uint32_t parity) {
   for (uint32_t i = 0; i < (1u << 16); ++i)
@@ -92,6 +102,54 @@ __device__ __forceinline__ void mma_f16_ss(uint32_t d_tmem, uint64_t adesc, uint
       "setp.ne.b32 p, %4, 0;\n\t"
       "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
       ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate) : "memory");
+}
+// Descriptor halves: the low word carries the start address (>> 4) and the leading byte offset, the high word the
+// stride (1024 bytes between 8-row groups), the version and the swizzle mode; K steps of 16 elements and whole
+// panels only move the low word, so a single thread can step descriptors with 32-bit adds.
+__device__ __forceinline__ uint32_t kmajor_sw128_desc_lo(uint32_t addr) { return ((addr >> 4) & 0x3fffu) | (1u << 16); }
+constexpr uint32_t KMAJOR_SW128_DESC_HI = 64u | (1u << 14) | (2u << 29);
+// Four MMAs over one 64-wide K panel (K steps of 16): D (+)= A[panel] * B[panel]^T, accumulate = 0 overwrites D first.
+__device__ __forceinline__ void mma_f16_ss_panel(uint32_t d_tmem, uint32_t a_lo, uint32_t b_lo, uint32_t idesc, uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p0, p1;\n\t.reg .b64 da, db;\n\t.reg .b32 al, bl;\n\t"
+      "setp.ne.b32 p0, %4, 0;\n\t"
+      "setp.eq.b32 p1, %4, %4;\n\t"
+      "mov.b64 da, {%1, %5};\n\tmov.b64 db, {%2, %5};\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %3, p0;\n\t"
+      "add.u32 al, %1, 2;\n\tadd.u32 bl, %2, 2;\n\tmov.b64 da, {al, %5};\n\tmov.b64 db, {bl, %5};\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %3, p1;\n\t"
+      "add.u32 al, %1, 4;\n\tadd.u32 bl, %2, 4;\n\tmov.b64 da, {al, %5};\n\tmov.b64 db, {bl, %5};\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %3, p1;\n\t"
+      "add.u32 al, %1, 6;\n\tadd.u32 bl, %2, 6;\n\tmov.b64 da, {al, %5};\n\tmov.b64 db, {bl, %5};\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %3, p1;\n\t}"
+      ::"r"(d_tmem), "r"(a_lo), "r"(b_lo), "r"(idesc), "r"(accumulate), "r"(KMAJOR_SW128_DESC_HI) : "memory");
+}
+// Eight MMAs over K = 128 with A in tensor memory (8 columns per K step) and B as two 64-wide K panels
+// `panel_step` (in 16-byte units) apart.
+__device__ __forceinline__ void mma_f16_ts_k128(uint32_t d_tmem, uint32_t a_tmem, uint32_t b_lo, uint32_t panel_step, uint32_t idesc,
+                                                uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p0, p1;\n\t.reg .b64 db;\n\t.reg .b32 bl, b2, ta;\n\t"
+      "setp.ne.b32 p0, %4, 0;\n\t"
+      "setp.eq.b32 p1, %4, %4;\n\t"
+      "add.u32 b2, %2, %6;\n\t"
+      "mov.b64 db, {%2, %5};\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], db, %3, p0;\n\t"
+      "add.u32 ta, %1, 8;\n\tadd.u32 bl, %2, 2;\n\tmov.b64 db, {bl, %5};\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], [ta], db, %3, p1;\n\t"
+      "add.u32 ta, %1, 16;\n\tadd.u32 bl, %2, 4;\n\tmov.b64 db, {bl, %5};\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], [ta], db, %3, p1;\n\t"
+      "add.u32 ta, %1, 24;\n\tadd.u32 bl, %2, 6;\n\tmov.b64 db, {bl, %5};\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], [ta], db, %3, p1;\n\t"
+      "add.u32 ta, %1, 32;\n\tmov.b64 db, {b2, %5};\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], [ta], db, %3, p1;\n\t"
+      "add.u32 ta, %1, 40;\n\tadd.u32 bl, b2, 2;\n\tmov.b64 db, {bl, %5};\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], [ta], db, %3, p1;\n\t"
+      "add.u32 ta, %1, 48;\n\tadd.u32 bl, b2, 4;\n\tmov.b64 db, {bl, %5};\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], [ta], db, %3, p1;\n\t"
+      "add.u32 ta, %1, 56;\n\tadd.u32 bl, b2, 6;\n\tmov.b64 db, {bl, %5};\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], [ta], db, %3, p1;\n\t}"
+      ::"r"(d_tmem), "r"(a_tmem), "r"(b_lo), "r"(idesc), "r"(accumulate), "r"(KMAJOR_SW128_DESC_HI), "r"(panel_step) : "memory");
 }
 // Arrive on `bar` once every tcgen05 operation issued so far by this thread has completed.
 __device__ __forceinline__ void mma_commit(uint32_t bar) {
