@@ -14,11 +14,12 @@
 // over its panels that accumulate into the same S.
 //
 // Tensor memory (512 columns): slab accumulators 2 x 128 | rotated keys 2 x 64 | S 8 x 16.
-// Warp roles (352 threads, one persistent CTA per SM working through a contiguous, cost-balanced piece of the tile list):
+// Warp roles (384 threads, one persistent CTA per SM working through a contiguous, cost-balanced piece of the tile list):
 //   warp 0      TMA producer of U_K^-1 panels (ring, one lane per stage)
-//   warp 1      MMA issuer (one lane issues; owns the TMEM allocation)
+//   warp 1      issuer of the main products (one elected lane; owns the TMEM allocation)
 //   warps 2-9   epilogue (thread = one token row x one half of the RoPE frequencies)
 //   warp 10     TMA producer of X^_K panels (ring of 8 slots served by four lanes, runs ahead into the next tile)
+//   warp 11     issuer of the score products (one elected lane)
 // All waits are bounded (tc_util.cuh); a wait that runs out ends the kernel with TWKV_ERR_TIMEOUT.
 //
 // Precision: X^_K, U_K^-1 keep the cache dtype with fp32 accumulation; rotated keys and queries enter
@@ -29,7 +30,7 @@
 namespace twkv {
 using namespace tc;
 
-constexpr int KT_THREADS = 352;
+constexpr int KT_THREADS = 384;
 constexpr int KT_EPI = 256;
 constexpr int KT_A_SLOTS = 8;                                  // power of two (slot = panel count & 7, phase = bit 3)
 constexpr uint32_t KT_TMEM_COLS = 512;
@@ -168,25 +169,9 @@ kscore_tc_kernel(const __grid_constant__ CUtensorMap map_blocks, const __grid_co
       // per few instructions), so descriptors are stepped with 32-bit adds, a panel's four MMAs are one asm block, and
       // every wait tries once inline before it falls into the bounded loop.
       const uint32_t idesc_main = idesc_f16(BF16 ? 1 : 0, 128, 128);
-      const uint32_t idesc_s = idesc_f16(0, 128, 16);
-      const uint32_t a_lo0 = kmajor_sw128_desc_lo(sA), b_lo0 = kmajor_sw128_desc_lo(sB), q_lo0 = kmajor_sw128_desc_lo(sQ);
+      const uint32_t a_lo0 = kmajor_sw128_desc_lo(sA), b_lo0 = kmajor_sw128_desc_lo(sB);
       uint32_t bst = 0, bph = 0, ak = 0, sc = 0;
       bool ok = true;
-      // The score product of slab n is issued after the main product of slab n + 2: the tensor pipe
-      // then always has a slab queued while the epilogue warps rotate an earlier one.
-      // A pending entry packs: slab counter << 8 | g << 2 | accumulate << 1 | last slab of its tile.
-      uint32_t pq0 = 0, pq1 = 0;
-      int npend = 0;
-      auto issue_scores = [&](uint32_t pe) {
-        const uint32_t psc = pe >> 8, kb = psc & 1u, pg = (pe >> 2) & 63u;
-        if (!mbar_wait_thin(kr_full + 8 * kb, (psc >> 1) & 1u, abort_flag)) return false;
-        fence_after_sync();
-        mma_f16_ts_k128(tmem_base + TM_S + 16 * pg, tmem_base + TM_KR + 64 * kb, q_lo0 + pg * (1024 >> 4), KT_Q_PANEL_BYTES >> 4, idesc_s,
-                        (pe >> 1) & 1u);
-        mma_commit(kr_empty + 8 * kb);
-        if (pe & 1u) mma_commit(s_full);
-        return true;
-      };
       int4 e = w0 < total ? klist[w0] : kt_none;
       for (int w = w0; w < total && ok; w += wstep) {
         const int4 nxt = w + wstep < total ? klist[w + wstep] : kt_none;
@@ -194,7 +179,6 @@ kscore_tc_kernel(const __grid_constant__ CUtensorMap map_blocks, const __grid_co
         for (int p0 = 0; p0 < cls && ok; p0 += KT_A_SLOTS) {
           const int np = min(KT_A_SLOTS, cls - p0);
           for (int sl = 0; sl < Hkv && ok; ++sl) {
-            const int g = sl + g_rot < Hkv ? sl + g_rot : sl + g_rot - Hkv;
             const uint32_t buf = sc & 1u;
             if (!(ok = mbar_wait_thin(slab_empty + 8 * buf, ((sc >> 1) & 1u) ^ 1u, abort_flag))) break;
             const uint32_t d = tmem_base + TM_SLAB + buf * 128;
@@ -213,22 +197,42 @@ kscore_tc_kernel(const __grid_constant__ CUtensorMap map_blocks, const __grid_co
             }
             if (!ok) break;
             mma_commit(slab_full + 8 * buf);                            // slab accumulator complete
-            if (npend == 2) {
-              if (!(ok = issue_scores(pq0))) break;
-              pq0 = pq1;
-              npend = 1;
-            }
-            const uint32_t pe = (sc << 8) | ((uint32_t)g << 2) | (p0 > 0 ? 2u : 0u) | ((p0 + np >= cls && last) ? 1u : 0u);
-            if (npend == 0) pq0 = pe; else pq1 = pe;
-            ++npend;
             ++sc;
           }
           ak += np;
         }
         e = nxt;
       }
-      if (ok && npend >= 1) ok = issue_scores(pq0);
-      if (ok && npend == 2) issue_scores(pq1);
+    }
+    __syncwarp();
+  } else if (warp == 11) {
+    // ------------------------------------------------------------- score-product issuer (one elected lane)
+    // S_g (+)= Krot_g . Q_g^T as soon as the epilogue warps have stored a rotated slab; a thread of its own, so that
+    // neither issue stream waits for the other's barriers
+    if (elect_one()) {
+      const uint32_t idesc_s = idesc_f16(0, 128, 16);
+      const uint32_t q_lo0 = kmajor_sw128_desc_lo(sQ);
+      uint32_t sc = 0;
+      bool ok = true;
+      int4 e = w0 < total ? klist[w0] : kt_none;
+      for (int w = w0; w < total && ok; w += wstep) {
+        const int4 nxt = w + wstep < total ? klist[w + wstep] : kt_none;
+        const int cls = e.y & 0xff;
+        for (int p0 = 0; p0 < cls && ok; p0 += KT_A_SLOTS) {
+          const bool last_pass = p0 + KT_A_SLOTS >= cls;
+          for (int sl = 0; sl < Hkv; ++sl, ++sc) {
+            const int g = sl + g_rot < Hkv ? sl + g_rot : sl + g_rot - Hkv;
+            const uint32_t kb = sc & 1u;
+            if (!(ok = mbar_wait_thin(kr_full + 8 * kb, (sc >> 1) & 1u, abort_flag))) break;
+            fence_after_sync();
+            mma_f16_ts_k128(tmem_base + TM_S + 16 * g, tmem_base + TM_KR + 64 * kb, q_lo0 + g * (1024 >> 4), KT_Q_PANEL_BYTES >> 4, idesc_s,
+                            p0 > 0 ? 1u : 0u);
+            mma_commit(kr_empty + 8 * kb);
+            if (last_pass && sl == Hkv - 1) mma_commit(s_full);        // the tile's scores are complete
+          }
+        }
+        e = nxt;
+      }
     }
     __syncwarp();
   } else {
