@@ -247,7 +247,7 @@ kscore_tc_kernel(const __grid_constant__ CUtensorMap map_blocks, const __grid_co
     const float2* __restrict__ rope_hi = v.rope_hi;
     const float2* __restrict__ rope_lo = v.rope_lo;
     uint32_t sc = 0, tcount = 0;
-    bool ok = true;
+    bool ok = true, slab_ready = false;                            // slab_ready: the next slab's accumulator was already seen complete
     float cs[32], sn[32];
     float tmax[4 * REP];                                            // running maxima of this thread's heads for the current query slot
 #pragma unroll
@@ -325,13 +325,16 @@ kscore_tc_kernel(const __grid_constant__ CUtensorMap map_blocks, const __grid_co
       const int pos_next = nxt.w >= 0 ? kpos[(size_t)nxt.x * TILE + row] : 0;      // fetched now, used after the tile's slabs
       for (int sl = 0; sl < n_slabs; ++sl, ++sc) {
         const uint32_t buf = sc & 1u, par = (sc >> 1) & 1u;
-        if (!(ok = __all_sync(0xffffffffu, mbar_wait(slab_full + 8 * buf, par, abort_flag)))) break;
+        // barrier probes cost a few hundred cycles of latency each, so each is issued early (the next slab's "full"
+        // during this slab's store, "rotated keys free" before the rotation) and only waited on if it had not flipped yet
+        if (!slab_ready && !(ok = __all_sync(0xffffffffu, mbar_wait(slab_full + 8 * buf, par, abort_flag)))) break;
         fence_after_sync();
         const uint32_t slab = lane_addr + TM_SLAB + buf * 128 + hf * 32;
         const uint32_t kr = lane_addr + TM_KR + buf * 64 + hf * 16;
         float lo[32], hi[32];
         tmem_ld32(slab, reinterpret_cast<uint32_t*>(lo));
         tmem_ld32(slab + 64, reinterpret_cast<uint32_t*>(hi));
+        const bool kr_probe = mbar_try(kr_empty + 8 * buf, par ^ 1u);
         tmem_ld_wait();
         fence_before_sync();
         __syncwarp();
@@ -342,14 +345,16 @@ kscore_tc_kernel(const __grid_constant__ CUtensorMap map_blocks, const __grid_co
           p1[t >> 1] = pack_f16x2_sat(lo[t] * cs[t] - hi[t] * sn[t], lo[t + 1] * cs[t + 1] - hi[t + 1] * sn[t + 1]);
           p2[t >> 1] = pack_f16x2_sat(hi[t] * cs[t] + lo[t] * sn[t], hi[t + 1] * cs[t + 1] + lo[t + 1] * sn[t + 1]);
         }
-        if (!(ok = __all_sync(0xffffffffu, mbar_wait(kr_empty + 8 * buf, par ^ 1u, abort_flag)))) break;
+        if (!__all_sync(0xffffffffu, kr_probe) && !(ok = __all_sync(0xffffffffu, mbar_wait(kr_empty + 8 * buf, par ^ 1u, abort_flag)))) break;
         fence_after_sync();
         tmem_st16(kr, p1);                                                  // dims d -> column d / 2
         tmem_st16(kr + 32, p2);                                             // dims 64 + d
+        const bool next_probe = mbar_try(slab_full + 8 * (buf ^ 1u), ((sc + 1) >> 1) & 1u);
         tmem_st_wait();
         fence_before_sync();
         __syncwarp();
         if (lane == 0) mbar_arrive(kr_full + 8 * buf);
+        slab_ready = __all_sync(0xffffffffu, next_probe);
       }
       if (!ok) break;
       // the next tile's rotation factors are fetched while this tile's last score products drain
