@@ -116,19 +116,22 @@ __global__ void __launch_bounds__(1024) plan_kernel(DevView v, int layer, const 
 
 // ------------------------------------------------------------------------ V accumulate
 constexpr int VA_STAGES = 6;
-constexpr int VA_THREADS = 256;
 
-// One CTA per (query slot, split, head group of <= 32 heads).  Warp w owns the w-th group of 8
-// columns of every 64-column panel, so every rank class keeps all eight warps busy.
-template <bool BF16, int MTW>
-__global__ void __launch_bounds__(VA_THREADS, 1)
+// One CTA per (query slot, split, head group of <= 32 heads).  A warp owns one 16-head row tile (warp / 8) and the
+// (warp % 8)-th group of 8 columns of every 64-column panel, so every rank class keeps all warps busy and a thread
+// carries 64 accumulators.  NWG = 1 (up to 16 heads, 8 warps) or 2 (up to 32 heads, 16 warps).
+template <bool BF16, int NWG>
+__global__ void __launch_bounds__(256 * NWG, 1)
 vacc_kernel(DevView v, int layer, const int* __restrict__ seq_ids, int n_splits) {
+  constexpr int NT = 256 * NWG;                                    // threads
+  constexpr int TPT = 2 * NWG;                                     // threads per token in the probability phase, 8 heads each
   extern __shared__ __align__(128) unsigned char smem[];
   unsigned char* sV = smem;                                        // [STAGES][128 tokens][128 B]
   unsigned char* sP = smem + VA_STAGES * 16384;                    // [2][32 heads][256 B]
   float* sM = reinterpret_cast<float*>(sP + 2 * 8192);             // [32] reference max per head
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int mt = warp >> 3, cw = warp & 7;                         // row tile, column group
   const int Hq = v.Hq;
   const int qs = blockIdx.x / n_splits, split = blockIdx.x - qs * n_splits;
   const int h0 = blockIdx.y * 32, nh = min(32, Hq - h0);
@@ -139,7 +142,7 @@ vacc_kernel(DevView v, int layer, const int* __restrict__ seq_ids, int n_splits)
   const int4* desc = v.desc(layer, 1);
   const int* aux = v.aux(layer, 1);
 
-  for (int i = tid; i < 2 * 8192 / 4; i += VA_THREADS) reinterpret_cast<unsigned*>(sP)[i] = 0u;
+  for (int i = tid; i < 2 * 8192 / 4; i += NT) reinterpret_cast<unsigned*>(sP)[i] = 0u;
   if (tid < 32) sM[tid] = tid < nh ? dec_ordered(v.seqmax[qs * Hq + h0 + tid]) : 0.f;
   // Descriptors of this split's tiles (the k-th is list[split + k * n_splits]) are kept in a ring of 64 in
   // shared memory, refilled 16 at a time well ahead of both cursors, so neither the copy cursor nor the
@@ -161,14 +164,10 @@ vacc_kernel(DevView v, int layer, const int* __restrict__ seq_ids, int n_splits)
   }
   __syncthreads();
 
-  float acc[TWKV_MAX_CLASSES][MTW][4];
-  float accl[MTW][4];
+  float acc[TWKV_MAX_CLASSES][4];
+  float accl[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
-  for (int p = 0; p < TWKV_MAX_CLASSES; ++p)
-#pragma unroll
-    for (int m = 0; m < MTW; ++m) { acc[p][m][0] = acc[p][m][1] = acc[p][m][2] = acc[p][m][3] = 0.f; }
-#pragma unroll
-  for (int m = 0; m < MTW; ++m) { accl[m][0] = accl[m][1] = accl[m][2] = accl[m][3] = 0.f; }
+  for (int p = 0; p < TWKV_MAX_CLASSES; ++p) { acc[p][0] = acc[p][1] = acc[p][2] = acc[p][3] = 0.f; }
 
   // producer cursor over (tile, panel) jobs of this split
   int p_k = 0, p_j = 0, p_cls = 0, p_base = 0, p_n = 0;
@@ -181,8 +180,8 @@ vacc_kernel(DevView v, int layer, const int* __restrict__ seq_ids, int n_splits)
       const unsigned char* src = v.blocks + (size_t)(p_base + p_j) * BLOCK_BYTES;
       const unsigned dst = smem_u32(sV + (p_n % VA_STAGES) * 16384);
 #pragma unroll
-      for (int i = 0; i < 4; ++i) {
-        const int c = tid + i * VA_THREADS, row = c >> 3, ch = c & 7;
+      for (int i = 0; i < 1024 / NT; ++i) {
+        const int c = tid + i * NT, row = c >> 3, ch = c & 7;
         cp_async16(dst + row * 128 + ((ch ^ (row & 7)) << 4), src + row * 128 + ch * 16);
       }
       ++p_n;
@@ -196,8 +195,8 @@ vacc_kernel(DevView v, int layer, const int* __restrict__ seq_ids, int n_splits)
   int c_n = 0, pbuf = 0;
   // Scores of a tile are fetched one tile ahead (the V slot's link to its score row two tiles ahead),
   // so the gather's latency hides behind the previous tile's panels.
-  const int slot = tid >> 1, part = tid & 1;                       // two threads per token, 16 heads each
-  float sc_next[16];
+  const int slot = tid / TPT, part = tid % TPT;                    // TPT threads per token, 8 heads each
+  float sc_next[8];
   int link_next = -1;                                              // score row of this thread's token in the tile after next (-1: none)
   auto fetch_link = [&](int k) {
     link_next = -1;
@@ -205,11 +204,11 @@ vacc_kernel(DevView v, int layer, const int* __restrict__ seq_ids, int n_splits)
   };
   auto fetch_scores = [&]() {                                      // uses link_next
     if (link_next >= 0) {
-      const float* srow = v.scores + (size_t)link_next * Hq + h0 + part * 16;
+      const float* srow = v.scores + (size_t)link_next * Hq + h0 + part * 8;
       if ((Hq & 3) == 0) {                                         // rows are 16-byte aligned: four heads per load
 #pragma unroll
-        for (int hh = 0; hh < 16; hh += 4) {
-          if (part * 16 + hh < nh) {
+        for (int hh = 0; hh < 8; hh += 4) {
+          if (part * 8 + hh < nh) {
             const float4 t = __ldg(reinterpret_cast<const float4*>(srow + hh));
             sc_next[hh] = t.x; sc_next[hh + 1] = t.y; sc_next[hh + 2] = t.z; sc_next[hh + 3] = t.w;
           } else {
@@ -218,11 +217,11 @@ vacc_kernel(DevView v, int layer, const int* __restrict__ seq_ids, int n_splits)
         }
       } else {
 #pragma unroll
-        for (int hh = 0; hh < 16; ++hh) sc_next[hh] = (part * 16 + hh < nh) ? __ldg(srow + hh) : -INFINITY;
+        for (int hh = 0; hh < 8; ++hh) sc_next[hh] = (part * 8 + hh < nh) ? __ldg(srow + hh) : -INFINITY;
       }
     } else {
 #pragma unroll
-      for (int hh = 0; hh < 16; ++hh) sc_next[hh] = -INFINITY;
+      for (int hh = 0; hh < 8; ++hh) sc_next[hh] = -INFINITY;
     }
   };
   fetch_link(0);
@@ -236,8 +235,8 @@ vacc_kernel(DevView v, int layer, const int* __restrict__ seq_ids, int n_splits)
     {
       unsigned char* P = sP + pbuf * 8192;
 #pragma unroll
-      for (int hh = 0; hh < 16; ++hh) {
-        const int h = part * 16 + hh;
+      for (int hh = 0; hh < 8; ++hh) {
+        const int h = part * 8 + hh;
         if (h < nh) {
           const float pv = __expf(sc_next[hh] - sM[h]);             // -inf for rows past the last token: weight 0
           const int chunk = slot >> 3;
@@ -263,16 +262,13 @@ vacc_kernel(DevView v, int layer, const int* __restrict__ seq_ids, int n_splits)
           unsigned b[2];
           {
             const int kr = ks * 16 + (lane & 15);
-            ldsm_x2_t(b, vBase + kr * 128 + ((warp ^ (kr & 7)) << 4));
+            ldsm_x2_t(b, vBase + kr * 128 + ((cw ^ (kr & 7)) << 4));
           }
-#pragma unroll
-          for (int m = 0; m < MTW; ++m) {
-            unsigned a[4];
-            const int row = m * 16 + rin + (mat & 1) * 8, kc = ks * 2 + (mat >> 1);
-            ldsm_x4(a, pBase + row * 256 + ((kc ^ (row & 7)) << 4));
-            mma16816<BF16>(acc[pj][m], a, b[0], b[1]);
-            if (pj == 0 && warp == 0) mma16816<BF16>(accl[m], a, ones, ones);
-          }
+          unsigned a[4];
+          const int row = mt * 16 + rin + (mat & 1) * 8, kc = ks * 2 + (mat >> 1);
+          ldsm_x4(a, pBase + row * 256 + ((kc ^ (row & 7)) << 4));
+          mma16816<BF16>(acc[pj], a, b[0], b[1]);
+          if (pj == 0 && cw == 0) mma16816<BF16>(accl, a, ones, ones);
         }
       };
       switch (j) {
@@ -292,25 +288,18 @@ vacc_kernel(DevView v, int layer, const int* __restrict__ seq_ids, int n_splits)
   // partial results of this split
   const size_t pidx = (size_t)qs * n_splits + split;
   float* pa = v.part_acc + pidx * Hq * v.d_kv;
+  const int r0 = mt * 16 + (lane >> 2), r1 = r0 + 8;
 #pragma unroll
   for (int pj = 0; pj < TWKV_MAX_CLASSES; ++pj) {
     if (pj < v.NC) {
-#pragma unroll
-      for (int m = 0; m < MTW; ++m) {
-        const int col = pj * PANEL + warp * 8 + (lane & 3) * 2;
-        const int r0 = m * 16 + (lane >> 2), r1 = r0 + 8;
-        if (r0 < nh) *reinterpret_cast<float2*>(pa + (size_t)(h0 + r0) * v.d_kv + col) = make_float2(acc[pj][m][0], acc[pj][m][1]);
-        if (r1 < nh) *reinterpret_cast<float2*>(pa + (size_t)(h0 + r1) * v.d_kv + col) = make_float2(acc[pj][m][2], acc[pj][m][3]);
-      }
+      const int col = pj * PANEL + cw * 8 + (lane & 3) * 2;
+      if (r0 < nh) *reinterpret_cast<float2*>(pa + (size_t)(h0 + r0) * v.d_kv + col) = make_float2(acc[pj][0], acc[pj][1]);
+      if (r1 < nh) *reinterpret_cast<float2*>(pa + (size_t)(h0 + r1) * v.d_kv + col) = make_float2(acc[pj][2], acc[pj][3]);
     }
   }
-  if (warp == 0 && (lane & 3) == 0) {
-#pragma unroll
-    for (int m = 0; m < MTW; ++m) {
-      const int r0 = m * 16 + (lane >> 2), r1 = r0 + 8;
-      if (r0 < nh) v.part_l[pidx * Hq + h0 + r0] = accl[m][0];
-      if (r1 < nh) v.part_l[pidx * Hq + h0 + r1] = accl[m][2];
-    }
+  if (cw == 0 && (lane & 3) == 0) {
+    if (r0 < nh) v.part_l[pidx * Hq + h0 + r0] = accl[0];
+    if (r1 < nh) v.part_l[pidx * Hq + h0 + r1] = accl[2];
   }
 }
 
@@ -399,11 +388,11 @@ static cudaError_t launch_decode_t(const DevView& v, int layer, const LayerParam
   if (v.Hq <= 16) {
     cudaFuncSetAttribute(vacc_kernel<BF16, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)va_smem);
     ProfScope ps(TWKV_K_VACC, st);
-    vacc_kernel<BF16, 1><<<vgrid, VA_THREADS, va_smem, st>>>(v, layer, seq_ids, n_splits);
+    vacc_kernel<BF16, 1><<<vgrid, 256, va_smem, st>>>(v, layer, seq_ids, n_splits);
   } else {
     cudaFuncSetAttribute(vacc_kernel<BF16, 2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)va_smem);
     ProfScope ps(TWKV_K_VACC, st);
-    vacc_kernel<BF16, 2><<<vgrid, VA_THREADS, va_smem, st>>>(v, layer, seq_ids, n_splits);
+    vacc_kernel<BF16, 2><<<vgrid, 512, va_smem, st>>>(v, layer, seq_ids, n_splits);
   }
   const size_t mg_a = (size_t)v.rep * v.d_kv * 4, mg_b = (size_t)MG_JGROUPS * v.rep * 128 * 4;
   const size_t mg_smem = mg_a > mg_b ? mg_a : mg_b;
