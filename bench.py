@@ -167,20 +167,19 @@ def run_reference(args):
 def run_ours(args):
     import numpy as np
     import torch
-    import torch.distributed as dist
 
     from paper_2603_04411_b200 import build as lib_build
     lib_build.build()
     from paper_2603_04411_b200 import binding as B
 
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    rank = int(os.environ.get("RANK", "0"))
+    from paper_2603_04411_b200 import replicas
+    world = replicas.world_size()
+    rank = replicas.rank()
     local = int(os.environ.get("LOCAL_RANK", "0"))
     assert torch.cuda.is_available(), "bench.py needs a CUDA device; there is no CPU fallback"
     torch.cuda.set_device(local)
     dev = torch.device("cuda", local)
-    if world > 1:
-        dist.init_process_group("nccl", device_id=dev)
+    replicas.init("nccl", dev)
 
     li, gate = build_workload(dev)
     Wk, Wv, bk, bv = gate
@@ -206,8 +205,7 @@ def run_ours(args):
 
     def barrier():
         torch.cuda.synchronize()
-        if world > 1:
-            dist.barrier()
+        replicas.barrier()
         torch.cuda.synchronize()
 
     for _ in range(max(args.warmup, 3)):
@@ -236,10 +234,7 @@ def run_ours(args):
     total_ms = e0.elapsed_time(e1)
     comp_ms = sum(e[0].elapsed_time(e[1]) for e in evs) / args.steps
     dec_ms = sum(e[1].elapsed_time(e[2]) for e in evs) / args.steps
-    t = torch.tensor([total_ms, comp_ms, dec_ms], dtype=torch.float64, device=dev)
-    if world > 1:
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-    total_ms, comp_ms, dec_ms = [float(x) for x in t.tolist()]
+    total_ms, comp_ms, dec_ms = replicas.max_over_ranks([total_ms, comp_ms, dec_ms], dev)
     ms_per_step = total_ms / args.steps
 
     # end to end: host buffers in, host result out, through the same C ABI calls
@@ -269,13 +264,10 @@ def run_ours(args):
             e2e_step()
         g1.record(stream)
         barrier()
-        t = torch.tensor([g0.elapsed_time(g1) / n_e2e], dtype=torch.float64, device=dev)
-        if world > 1:
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        e2e_ms = float(t.item())
+        e2e_ms = replicas.max_over_ranks([g0.elapsed_time(g1) / n_e2e], dev)[0]
         h2d = sum(x.numel() * x.element_size() for x in (h_xk, h_xv, h_sid, h_pos, h_q))
         d2h = h_out.numel() * h_out.element_size()
-        e2e = {"value": world * n_tok / (e2e_ms * 1e-3), "unit": "KV tokens/s through compress + decode, host buffers",
+        e2e = {"value": replicas.whole_job_rate(n_tok, e2e_ms), "unit": "KV tokens/s through compress + decode, host buffers",
                "ms_per_step": e2e_ms, "steps": n_e2e, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h}
 
     if rank == 0:
@@ -311,7 +303,7 @@ def run_ours(args):
         dec_gbs = st.bytes_stored / (dec_ms * 1e-3) / 1e9
         extra = {
             "decode_ms": dec_ms, "compress_ms": comp_ms,
-            "compress_tokens_per_s": world * n_tok / (comp_ms * 1e-3),
+            "compress_tokens_per_s": replicas.whole_job_rate(n_tok, comp_ms),
             "decode_hbm_gbs_on_stored_bytes": dec_gbs,
             "decode_hbm_frac_of_8tbs": dec_gbs / NOMINAL_HBM_GBS,
             "decode_hbm_frac_of_measured": dec_gbs / peaks["hbm_gbs"],
@@ -338,7 +330,7 @@ def run_ours(args):
           cpu = {"value": reps * n_s / td, "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle",
                "sample": f"{reps} x decode attention over the first {n_s} tokens of sequence 0, all {HQ} heads, "
                          f"{td:.2f} s in total (the gate passes over the same tokens took {tg:.2f} s)"}
-        line = {"metric": METRIC, "value": world * n_tok / (dec_ms * 1e-3), "unit": UNIT, "n_gpus": world, "steps": args.steps,
+        line = {"metric": METRIC, "value": replicas.whole_job_rate(n_tok, dec_ms), "unit": UNIT, "n_gpus": world, "steps": args.steps,
                 "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
                 "vs_baseline": None, "dtype": "f16", "data": "synthetic",
                 "config": {"workload": WORKLOAD, "batch": B_SEQ, "context": CTX, "n_q_heads": HQ, "n_kv_heads": HKV,
@@ -349,8 +341,7 @@ def run_ours(args):
         line.update(extra)
         print(json.dumps(line), flush=True)
     B.twkv_cache_destroy(cache)
-    if world > 1:
-        dist.destroy_process_group()
+    replicas.finish()
 
 
 def main():
