@@ -7,6 +7,8 @@ this package never imports the product library.
 All floating point goes through float64.  16-bit inputs (fp16 / bf16 bit
 patterns, exactly as the GPU receives them) are widened with `widen16`.
 
+  project(x, U)                    Eq. 1   x~ = x U
+  narrow16(a, dtype)               float64 -> the 16-bit storage type, round to nearest even
   gate_logits(xt, W, b)            Eq. 5   z = x~ W + b
   gate_rank(z, tau)                Eq. 5, 6, 8   -> (r, margin[, soft mask])
   truncate(xt, r)                  Eq. 2   x^ = x~ (.) m_hard
@@ -33,6 +35,8 @@ def lib():
         dp = ctypes.POINTER(ctypes.c_double)
         ip = ctypes.POINTER(ctypes.c_int32)
         L.oracle_num_threads.restype = ctypes.c_int
+        L.oracle_project.argtypes = [dp, dp, ctypes.c_int64, ctypes.c_int, dp]
+        L.oracle_project.restype = None
         L.oracle_gate_logits.argtypes = [dp, dp, dp, ctypes.c_int64, ctypes.c_int, dp]
         L.oracle_gate_logits.restype = None
         L.oracle_gate_rank.argtypes = [dp, ctypes.c_int64, ctypes.c_int, ctypes.c_double, ip, dp, dp]
@@ -71,6 +75,41 @@ def widen16(bits, dtype: str) -> np.ndarray:
     if dtype == "bf16":
         return (bits.astype(np.uint32) << 16).view(np.float32).astype(np.float64)
     raise ValueError(dtype)
+
+
+def narrow16(a, dtype: str) -> np.ndarray:
+    """float64 -> uint16 bit patterns of fp16 ('f16') or bf16 ('bf16'), round to nearest even.
+
+    The states handed to the compress step are 16-bit; this is the one rounding between Eq. 1 and Eq. 2.
+    Both conversions go through a single rounding of the float64 value (no intermediate float32 rounding
+    that could double-round): numpy's float64 -> float16 cast for fp16, integer arithmetic on the float64
+    bit pattern for bf16.  Overflow gives infinity, as IEEE round-to-nearest does.
+    """
+    a = np.ascontiguousarray(a, dtype=np.float64)
+    if dtype == "f16":
+        with np.errstate(over="ignore"):
+            return a.astype(np.float16).view(np.uint16)
+    if dtype == "bf16":
+        # bf16 has float32's exponent range and 8 significand bits; values are assumed normal in float32
+        # (|a| >= 2^-126 or a == 0), which holds for every state the tests and workloads produce.
+        m, e = np.frexp(a)                                  # a = m 2^e, 0.5 <= |m| < 1
+        q = np.rint(np.ldexp(m, 8))                         # 8 significant bits, ties to even (rint)
+        v = np.ldexp(q, e - 8)                              # exactly representable in bf16 (or overflows below)
+        with np.errstate(over="ignore"):
+            f = v.astype(np.float32)                        # exact: v has 8 significant bits
+        return (f.view(np.uint32) >> 16).astype(np.uint16)
+    raise ValueError(dtype)
+
+
+def project(x, U) -> np.ndarray:
+    """Eq. 1: x~ = x U.  x [n, d] pre-RoPE states, U [d, d]."""
+    x, px = _d(x)
+    U, pU = _d(U)
+    n, d = x.shape
+    assert U.shape == (d, d)
+    xt = np.empty((n, d), dtype=np.float64)
+    lib().oracle_project(px, pU, n, d, xt.ctypes.data_as(ctypes.POINTER(ctypes.c_double)))
+    return xt
 
 
 def gate_logits(xt, W, b=None) -> np.ndarray:

@@ -7,6 +7,7 @@
  * smoke check and the benchmark's CPU-baseline leg.
  *
  * Every function follows one passage of the paper:
+ *   oracle_project       Eq. 1  (x~ = x U, projection to the spectral space)
  *   oracle_gate_logits   Eq. 5  (z = x~ W + b, the argument of the softmax)
  *   oracle_gate_rank     Eq. 5, Eq. 6, Eq. 8  (softmax, cumsum, Flip, threshold)
  *   oracle_reconstruct   Eq. 2 + Eq. 3  (hard prefix mask, dynamic low-rank reconstruction)
@@ -39,6 +40,20 @@ int oracle_num_threads(void) {
 #else
   return 1;
 #endif
+}
+
+/* Eq. 1: x~[t, :] = x[t, :] U.   U is [d x d] row-major: row j holds the weights of input
+ * dimension j, column n is the n-th axis of the spectral space. */
+void oracle_project(const double* x, const double* U, int64_t n_tok, int d, double* xt) {
+#pragma omp parallel for schedule(static)
+  for (int64_t t = 0; t < n_tok; ++t) {
+    double* o = xt + t * d;
+    for (int n = 0; n < d; ++n) {
+      double acc = 0.0;
+      for (int j = 0; j < d; ++j) acc += x[t * d + j] * U[(int64_t)j * d + n];
+      o[n] = acc;
+    }
+  }
 }
 
 /* Eq. 5 (inside the softmax): z[t, :] = x~[t, :] W + b.   W is [d x d] row-major. */

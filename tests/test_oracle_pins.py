@@ -110,12 +110,80 @@ def test_gate_logits_orientation_and_bias():
     np.testing.assert_allclose(z2 - z1, z1 - b, rtol=1e-12, atol=1e-12)
 
 
-# ---------------------------------------------------------------- truncate / reconstruct
 def _rand_orth(rng, d):
     q, _ = np.linalg.qr(rng.normal(size=(d, d)))
     return q
 
 
+# ------------------------------------------------------------------ spectral projection
+def test_project_closed_forms_pin_orientation():
+    rng = np.random.default_rng(21)
+    d = 24
+    x = rng.normal(size=(6, d))
+    # cyclic shift: U[j, (j + 1) % d] = 1 sends input dimension j to spectral axis j + 1 (x U, not x U^T)
+    P = np.zeros((d, d))
+    P[np.arange(d), (np.arange(d) + 1) % d] = 1.0
+    np.testing.assert_array_equal(oracle.project(x, P), np.roll(x, 1, axis=1))
+    # diagonal U scales axis n by s_n; identity leaves x alone
+    s_ = rng.normal(size=d)
+    np.testing.assert_array_equal(oracle.project(x, np.diag(s_)), x * s_[None, :])
+    np.testing.assert_array_equal(oracle.project(x, np.eye(d)), x)
+    # rank one U = a b^T: x~ = (x . a) b
+    a, b = rng.normal(size=d), rng.normal(size=d)
+    np.testing.assert_allclose(oracle.project(x, np.outer(a, b)), (x @ a)[:, None] * b[None, :], rtol=1e-12, atol=1e-12)
+    # one-hot input row j reads out row j of U
+    M = np.arange(d * d, dtype=np.float64).reshape(d, d)
+    np.testing.assert_array_equal(oracle.project(np.eye(d)[3:4], M)[0], M[3])
+
+
+def test_project_then_full_rank_reconstruct_is_identity_and_preserves_energy():
+    rng = np.random.default_rng(22)
+    d = 64
+    x = rng.normal(size=(9, d))
+    U = _rand_orth(rng, d)
+    xt = oracle.project(x, U)
+    np.testing.assert_allclose((xt ** 2).sum(1), (x ** 2).sum(1), rtol=1e-12)          # orthogonal U: Parseval
+    np.testing.assert_allclose(oracle.reconstruct(xt, np.full(9, d, np.int32), U.T), x, atol=1e-12)   # Eq. 3 undoes Eq. 1
+    G = rng.normal(size=(d, d)) + 5 * np.eye(d)                                        # learnable U need not stay orthogonal
+    np.testing.assert_allclose(oracle.reconstruct(oracle.project(x, G), np.full(9, d, np.int32), np.linalg.inv(G)), x, atol=1e-10)
+
+
+def test_project_with_pca_eigenvectors_orders_the_energy():
+    # U = eigenvectors of the calibration covariance, largest eigenvalue first: the projected dimensions are
+    # uncorrelated and their variances are the eigenvalues in descending order (what lets Eq. 2 prune the tail)
+    rng = np.random.default_rng(23)
+    d = 40
+    A = rng.normal(size=(d, d)) * (0.85 ** np.arange(d))[None, :]
+    x = rng.normal(size=(3000, d)) @ A.T
+    x = x - x.mean(0)
+    lam, vec = np.linalg.eigh(np.cov(x.T))
+    order = np.argsort(lam)[::-1]
+    U = vec[:, order]
+    C = np.cov(oracle.project(x, U).T)
+    np.testing.assert_allclose(np.diag(C), lam[order], rtol=1e-9)
+    assert np.all(np.diff(np.diag(C)) <= 1e-12)
+    off = C - np.diag(np.diag(C))
+    assert np.abs(off).max() < 1e-10 * lam.max()
+
+
+def test_narrow16_round_to_nearest_even():
+    # fp16: 11 significand bits; bf16: 8.  Halfway cases go to the even neighbour, everything else to the nearest.
+    f16 = oracle.narrow16(np.array([1.0, 1.0 + 2.0 ** -11, 1.0 + 3 * 2.0 ** -11, 1.0 + 2.0 ** -11 + 2.0 ** -30, -2.5, 65504.0, 65520.0, 0.0]), "f16")
+    np.testing.assert_array_equal(f16, np.array([0x3C00, 0x3C00, 0x3C02, 0x3C01, 0xC100, 0x7BFF, 0x7C00, 0x0000], dtype=np.uint16))
+    b16 = oracle.narrow16(np.array([1.0, 1.0 + 2.0 ** -8, 1.0 + 3 * 2.0 ** -8, 1.0 + 2.0 ** -8 + 2.0 ** -40, -2.5, 3.0e38, 0.0,
+                                    1.0 + 2.0 ** -8 - 2.0 ** -40]), "bf16")
+    np.testing.assert_array_equal(b16, np.array([0x3F80, 0x3F80, 0x3F82, 0x3F81, 0xC020, 0x7F62, 0x0000, 0x3F80], dtype=np.uint16))
+    # widening what was narrowed is exact, and narrowing representable values changes nothing
+    rng = np.random.default_rng(24)
+    for dt in ("f16", "bf16"):
+        bits = oracle.narrow16(rng.normal(size=1000) * 8, dt)
+        np.testing.assert_array_equal(oracle.narrow16(oracle.widen16(bits, dt), dt), bits)
+        v = rng.normal(size=1000) * 8
+        err = np.abs(oracle.widen16(oracle.narrow16(v, dt), dt) - v)
+        assert np.all(err <= np.abs(v) * 2.0 ** (-11 if dt == "f16" else -8))
+
+
+# ---------------------------------------------------------------- truncate / reconstruct
 def test_reconstruct_parseval_tail_energy():
     rng = np.random.default_rng(2)
     d = 64
