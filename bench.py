@@ -317,6 +317,27 @@ def run_ours(args):
             "kernels": kernels,
         }
         extra["frac_of_binding_bound"] = extra["binding_bound_ms"] / dec_ms
+        # the step before the path (Eq. 1, x~ = x U on the device), timed on its own: not part of `value` or `ms_per_step`.
+        # Operand values do not change a dense product's time, so the resident states and bases stand in for x and U.
+        ws = torch.empty(B.twkv_projector_required_bytes(D_KV), dtype=torch.uint8, device=dev)
+        pj = B.twkv_projector_create(li.Uinv_k, li.Uinv_v, ws)
+        p_k, p_v = torch.empty_like(li.xt_k), torch.empty_like(li.xt_v)
+        for _ in range(3):
+            B.twkv_project(pj, li.xt_k, li.xt_v, p_k, p_v)
+        pa, pb = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        pa.record(stream)
+        for _ in range(10):
+            B.twkv_project(pj, li.xt_k, li.xt_v, p_k, p_v)
+        pb.record(stream)
+        torch.cuda.synchronize()
+        assert B.twkv_projector_status(pj) == B.TWKV_OK
+        B.twkv_projector_destroy(pj)
+        pj_ms = pa.elapsed_time(pb) / 10
+        pj_tf = 4.0 * n_tok * D_KV * D_KV / (pj_ms * 1e-3) / 1e12
+        extra["project"] = {"kernel": "project_tc_kernel (tcgen05: x~ = x U for K and V, 16-bit out by TMA store)", "ms": pj_ms,
+                            "tokens_per_s": n_tok / (pj_ms * 1e-3), "achieved": pj_tf, "peak": peaks["tflops"], "unit": "TFLOP/s",
+                            "frac": pj_tf / peaks["tflops"], "bound": "tensor"}
+        del p_k, p_v, ws
         # CPU baseline: the oracle as it stands on a bounded sample of the same workload
         import oracle
         cpu = None

@@ -195,6 +195,36 @@ twkv_status twkv_gate_ranks_static(const void* K, const void* V, const void* W_k
                                    const float* b_k, const float* b_v, int n_tok, int d_kv, int dtype,
                                    float tau, uint16_t* levels, void* stream);
 
+/*
+ * Projection to the spectral space (Eq. 1): x~ = x U for the pre-RoPE key and value states, the step
+ * right before twkv_compress.  U is the layer's learnable basis (initialised from the PCA eigenvectors,
+ * largest eigenvalue first); Eq. 3's U^-1 is its inverse.  The product is accumulated in fp32 from the
+ * exact 16-bit inputs and rounded once, to nearest even, into the same 16-bit type: that is the x~ the
+ * compress step takes.  Applied to the rows of a model's key / value projection weights instead of to
+ * states, the same call folds U into those weights offline (x~ = h (W U)).
+ *
+ * A projector borrows two things from the caller for its lifetime: nothing of U itself (a transposed
+ * copy is made at creation) and `workspace`, device memory of twkv_projector_required_bytes(d_kv) bytes,
+ * 256-byte aligned, which holds the copies and a status word.  The library allocates no device memory.
+ *   U_k, U_v   [d_kv x d_kv] dtype, row-major, device, 16-byte aligned; row j = input dimension j, column n =
+ *              spectral axis n.  Either may be NULL when that side is never projected.
+ *   d_kv       multiple of 128, at most 8192
+ * twkv_project:
+ *   x_k, x_v   [n_tok x d_kv] dtype, row-major, device, 16-byte aligned (input);  NULL skips the side
+ *   xt_k, xt_v [n_tok x d_kv] dtype (output); must not overlap the inputs
+ * Errors: TWKV_ERR_INVALID_ARG for bad pointers / sizes / a side without its U, TWKV_ERR_CUDA for a failed
+ * launch; a device-side wait that ran out shows up as TWKV_ERR_TIMEOUT in twkv_projector_status, which
+ * synchronises `stream`, returns the sticky status and clears it.
+ */
+typedef struct twkv_projector twkv_projector;   /* opaque, host memory */
+size_t twkv_projector_required_bytes(int d_kv);
+twkv_status twkv_projector_create(int d_kv, twkv_dtype dtype, const void* U_k, const void* U_v, void* workspace,
+                                  size_t workspace_bytes, void* stream, twkv_projector** out);
+void twkv_projector_destroy(twkv_projector* projector);
+twkv_status twkv_project(twkv_projector* projector, const void* x_k, const void* x_v, void* xt_k, void* xt_v,
+                         int n_tok, void* stream);
+twkv_status twkv_projector_status(twkv_projector* projector, void* stream);
+
 /* Per-kernel device timing.  While enabled, every kernel the library launches for this cache is
  * bracketed by CUDA events on the launching stream (events are host-side resources; no device memory
  * is allocated).  twkv_profile_read synchronises `stream`, adds the elapsed times of the launches

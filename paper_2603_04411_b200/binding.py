@@ -22,7 +22,9 @@ TILE_TOKENS, PANEL_ELEMS, BLOCK_BYTES, PIECE_TOKENS, MAX_CLASSES = 128, 64, 1638
 EXPORTS = ["twkv_cache_required_bytes", "twkv_cache_create", "twkv_cache_destroy", "twkv_cache_reset",
            "twkv_cache_set_layer_params", "twkv_compress", "twkv_decode_attn", "twkv_cache_status",
            "twkv_cache_stats", "twkv_cache_layout", "twkv_launch_count", "twkv_status_string",
-           "twkv_profile_enable", "twkv_profile_read", "twkv_gate_ranks_static"]
+           "twkv_profile_enable", "twkv_profile_read", "twkv_gate_ranks_static",
+           "twkv_projector_required_bytes", "twkv_projector_create", "twkv_projector_destroy", "twkv_project",
+           "twkv_projector_status"]
 STATIC_GATE_MAX_ROWS = 1024
 KERNEL_KINDS = ["gate_gemm", "gate_rank", "hist", "alloc", "pack", "plan", "kscore", "vacc", "merge", "other"]
 
@@ -74,6 +76,16 @@ def _load():
     L.twkv_profile_read.argtypes = [vp, vp, ctypes.POINTER(ctypes.c_double), ctypes.POINTER(ctypes.c_uint64)]
     L.twkv_gate_ranks_static.argtypes = [vp, vp, vp, vp, vp, vp, i32, i32, i32, ctypes.c_float, vp, vp]
     L.twkv_gate_ranks_static.restype = i32
+    L.twkv_projector_required_bytes.argtypes = [i32]
+    L.twkv_projector_required_bytes.restype = sz
+    L.twkv_projector_create.argtypes = [i32, i32, vp, vp, vp, sz, vp, ctypes.POINTER(vp)]
+    L.twkv_projector_create.restype = i32
+    L.twkv_projector_destroy.argtypes = [vp]
+    L.twkv_projector_destroy.restype = None
+    L.twkv_project.argtypes = [vp, vp, vp, vp, vp, i32, vp]
+    L.twkv_project.restype = i32
+    L.twkv_projector_status.argtypes = [vp, vp]
+    L.twkv_projector_status.restype = i32
     L.twkv_launch_count.argtypes = []
     L.twkv_launch_count.restype = ctypes.c_uint64
     L.twkv_status_string.argtypes = [i32]
@@ -195,6 +207,36 @@ def twkv_gate_ranks_static(K, V, W_k, W_v, b_k, b_v, levels, tau=0.1, stream=Non
     n = K.shape[0] if n_tok is None else n_tok
     _check(lib.twkv_gate_ranks_static(_ptr(K), _ptr(V), _ptr(W_k), _ptr(W_v), _ptr(b_k), _ptr(b_v), n, K.shape[1],
                                       dtype_code(K.dtype), tau, _ptr(levels), _stream(stream)), "twkv_gate_ranks_static")
+
+
+def twkv_projector_required_bytes(d_kv: int) -> int:
+    return int(lib.twkv_projector_required_bytes(d_kv))
+
+
+def twkv_projector_create(U_k, U_v, workspace: torch.Tensor, stream=None):
+    """U_k / U_v: [d_kv, d_kv] fp16 or bf16 CUDA tensors (either may be None); workspace: 1-D uint8 CUDA tensor of
+    twkv_projector_required_bytes(d_kv) bytes owned by the caller (kept alive by the caller)."""
+    U = U_k if U_k is not None else U_v
+    h = ctypes.c_void_p()
+    _check(lib.twkv_projector_create(U.shape[0], dtype_code(U.dtype), _ptr(U_k), _ptr(U_v), _ptr(workspace),
+                                     workspace.numel() * workspace.element_size(), _stream(stream), ctypes.byref(h)),
+           "twkv_projector_create")
+    return h
+
+
+def twkv_projector_destroy(projector):
+    lib.twkv_projector_destroy(projector)
+
+
+def twkv_project(projector, x_k, x_v, xt_k, xt_v, stream=None, n_tok=None):
+    """Eq. 1 on the device: xt = x U for the pre-RoPE key and / or value states ([n_tok, d_kv], 16-bit)."""
+    x = x_k if x_k is not None else x_v
+    n = (x.shape[0] if x is not None else 0) if n_tok is None else n_tok
+    _check(lib.twkv_project(projector, _ptr(x_k), _ptr(x_v), _ptr(xt_k), _ptr(xt_v), n, _stream(stream)), "twkv_project")
+
+
+def twkv_projector_status(projector, stream=None) -> int:
+    return int(lib.twkv_projector_status(projector, _stream(stream)))
 
 
 def twkv_launch_count() -> int:

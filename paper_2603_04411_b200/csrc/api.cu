@@ -181,17 +181,6 @@ struct twkv_cache {
   std::vector<char> prepared_w;        // per layer: those copies and maps are current
 };
 
-struct DeviceGuard {
-  int prev = -1;
-  bool ok = true;
-  explicit DeviceGuard(int dev) {
-    if (cudaGetDevice(&prev) != cudaSuccess) { ok = false; return; }
-    if (prev != dev && cudaSetDevice(dev) != cudaSuccess) ok = false;
-    target = dev;
-  }
-  ~DeviceGuard() { if (prev >= 0 && prev != target) cudaSetDevice(prev); }
-  int target = -1;
-};
 
 extern "C" {
 

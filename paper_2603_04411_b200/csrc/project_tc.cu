@@ -1,0 +1,237 @@
+// Projection to the spectral space on the 5th-generation tensor cores:  X~ = X U  (Eq. 1), for the
+// pre-RoPE key and value states of a batch of tokens, result rounded once to the 16-bit storage type.
+//
+// Work item = (128-token tile, side K or V, slab of NS output columns); NS = 256, or 128 when d is not a
+// multiple of 256.  Items are dealt round-robin to one persistent CTA per SM, the slabs of one tile
+// next to each other, so neighbouring CTAs read the same token tile from L2 at about the same time and
+// a call of a few tokens still spreads over 2 d / NS CTAs.
+// Per item the [128 x NS] fp32 accumulator is built by tcgen05.mma chains (M = 128, N = NS, K = 16 per
+// instruction) in one of two alternating TMEM buffers; [128 x 64] panels of X and [NS x 64] panels of
+// U^T (pre-transposed once, so it is the K-major B operand) stream through a 4-stage TMA ring with the
+// 128-byte swizzle.  Epilogue warps read the accumulator with tcgen05.ld, round to f16 / bf16, write
+// [128 x 64] panels into shared memory in the swizzled layout and hand them to TMA stores, which also
+// clip the rows past the last token.
+//
+// Warp roles (320 threads):
+//   warp 0      TMA producer: lanes 0-3 the U^T panel of ring stage L, lanes 4-7 the X panel of stage L - 4
+//   warp 1      MMA issuer (one elected lane; owns the TMEM allocation)
+//   warps 2-9   epilogue: thread = one token row x half of the slab's columns; each half (four warps) owns
+//               one staging panel and one lane that issues its stores
+// All barrier waits are bounded (tc_util.cuh); a wait that runs out ends the kernel with TWKV_ERR_TIMEOUT.
+#include "twkv_dev.h"
+#include "tc_util.cuh"
+
+namespace twkv {
+using namespace tc;
+
+constexpr int PJ_THREADS = 320;
+constexpr int PJ_EPI = 256;
+constexpr int PJ_STAGES = 4;
+constexpr uint32_t PJ_TMEM_COLS = 512;
+constexpr uint32_t PJ_PANEL_BYTES = 16384;                      // [128 rows][64 x 16 bit]
+
+__device__ __forceinline__ void tma_store_2d(const CUtensorMap* map, uint32_t src, int x, int y) {
+  asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%2, %3}], [%1];"
+               ::"l"(map), "r"(src), "r"(x), "r"(y) : "memory");
+}
+__device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+// the stores committed by this thread have finished reading shared memory
+__device__ __forceinline__ void bulk_wait_read_all() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
+// ... and have been written out
+__device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
+// Barrier over `threads` threads that also ANDs a predicate across them.
+__device__ __forceinline__ bool named_bar_and(int id, int threads, bool pred) {
+  uint32_t r;
+  asm volatile(
+      "{\n\t.reg .pred p, q;\n\t"
+      "setp.ne.u32 q, %1, 0;\n\t"
+      "bar.red.and.pred p, %2, %3, q;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(r) : "r"((uint32_t)pred), "r"(id), "r"(threads) : "memory");
+  return r != 0;
+}
+__device__ __forceinline__ uint32_t pack_f16x2_rn(float lo, float hi) {
+  uint32_t d;
+  asm("cvt.rn.f16x2.f32 %0, %1, %2;" : "=r"(d) : "f"(hi), "f"(lo));
+  return d;
+}
+__device__ __forceinline__ uint32_t pack_bf16x2_rn(float lo, float hi) {
+  uint32_t d;
+  asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(d) : "f"(hi), "f"(lo));
+  return d;
+}
+
+__global__ void __launch_bounds__(PJ_THREADS, 1)
+project_tc_kernel(const __grid_constant__ CUtensorMap map_xk, const __grid_constant__ CUtensorMap map_xv,
+                  const __grid_constant__ CUtensorMap map_uk, const __grid_constant__ CUtensorMap map_uv,
+                  const __grid_constant__ CUtensorMap map_ok, const __grid_constant__ CUtensorMap map_ov,
+                  int n_tok, int d, int bf16, int side0, int n_sides, int* status) {
+  extern __shared__ __align__(1024) unsigned char smem_raw[];
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int KP = d / PANEL;
+  const int NS = (d % 256 == 0) ? 256 : 128;
+  const int n_slabs = d / NS;
+  const uint32_t b_stage_bytes = (uint32_t)NS * 128u;
+  const uint32_t stage_bytes = PJ_PANEL_BYTES + b_stage_bytes;           // [X panel | U^T panel]
+  const uint32_t sA = smem_addr(smem_raw);
+  if (sA & 1023u) {
+    if (tid == 0) atomicCAS(status, 0, TWKV_ERR_DEVICE_CHECK);
+    return;
+  }
+  unsigned char* out_stage = smem_raw + PJ_STAGES * stage_bytes;         // two output panels, one per column half
+  unsigned char* tail = out_stage + 2 * PJ_PANEL_BYTES;
+  const uint32_t bars = smem_addr(tail);
+  const uint32_t full = bars, empty = full + 8 * PJ_STAGES, acc_full = empty + 8 * PJ_STAGES, acc_empty = acc_full + 16;
+  uint32_t* s_tmem_base = reinterpret_cast<uint32_t*>(tail + 8 * (2 * PJ_STAGES + 4));
+  volatile int* abort_flag = reinterpret_cast<int*>(s_tmem_base + 1);
+
+  if (tid == 0) {
+    for (int i = 0; i < PJ_STAGES; ++i) { mbar_init(full + 8 * i, 2); mbar_init(empty + 8 * i, 1); }
+    for (int i = 0; i < 2; ++i) { mbar_init(acc_full + 8 * i, 1); mbar_init(acc_empty + 8 * i, PJ_EPI / 32); }
+    *abort_flag = 0;
+    mbar_init_fence();
+  }
+  if (warp == 1) tmem_alloc(smem_addr(s_tmem_base), PJ_TMEM_COLS);
+  fence_before_sync();
+  __syncthreads();
+  fence_after_sync();
+  const uint32_t tmem_base = *s_tmem_base;
+
+  // item -> (tile, side, slab): slab fastest, then side
+  const int per_tile = n_sides * n_slabs;
+  const int n_items = per_tile * ((n_tok + TILE - 1) / TILE);
+  const int it0 = blockIdx.x, itstep = gridDim.x;
+
+  if (warp == 0) {
+    // ------------------------------------------------------------- TMA producer
+    if (lane < 2 * PJ_STAGES) {
+      const bool is_x = lane >= PJ_STAGES;
+      const uint32_t my = is_x ? lane - PJ_STAGES : lane;
+      if (lane == 0) { tma_prefetch_desc(&map_uk); tma_prefetch_desc(&map_uv); }
+      if (lane == PJ_STAGES) { tma_prefetch_desc(&map_xk); tma_prefetch_desc(&map_xv); }
+      bool ok = true;
+      uint32_t st = 0, ph = 0;
+      for (int it = it0; it < n_items && ok; it += itstep) {
+        const int rem = it % per_tile, m0 = (it / per_tile) * TILE;
+        const int side = side0 + rem / n_slabs, ns = rem % n_slabs;
+        const CUtensorMap* map = is_x ? (side ? &map_xv : &map_xk) : (side ? &map_uv : &map_uk);
+        for (int p = 0; p < KP; ++p) {
+          const uint32_t cst = st, cph = ph;
+          if (++st == PJ_STAGES) { st = 0; ph ^= 1u; }
+          if (cst != my) continue;
+          if (!(ok = mbar_wait(empty + 8 * cst, cph ^ 1u, abort_flag))) break;
+          if (is_x) {
+            mbar_expect_tx(full + 8 * cst, PJ_PANEL_BYTES);
+            tma_load_2d(sA + cst * stage_bytes, map, full + 8 * cst, p * PANEL, m0);
+          } else {
+            mbar_expect_tx(full + 8 * cst, b_stage_bytes);
+            tma_load_2d(sA + cst * stage_bytes + PJ_PANEL_BYTES, map, full + 8 * cst, p * PANEL, ns * NS);
+          }
+        }
+      }
+    }
+    __syncwarp();
+  } else if (warp == 1) {
+    // ------------------------------------------------------------- MMA issuer
+    if (elect_one()) {
+      const uint32_t idesc = idesc_f16(bf16 ? 1 : 0, 128, NS);
+      const uint64_t adesc0 = kmajor_sw128_desc(sA), bdesc0 = kmajor_sw128_desc(sA + PJ_PANEL_BYTES);
+      bool ok = true;
+      uint32_t st = 0, ph = 0, ac = 0;
+      for (int it = it0; it < n_items && ok; it += itstep, ++ac) {
+        const uint32_t buf = ac & 1u;
+        if (!(ok = mbar_wait(acc_empty + 8 * buf, ((ac >> 1) & 1u) ^ 1u, abort_flag))) break;
+        const uint32_t dcol = tmem_base + buf * 256;
+        for (int p = 0; p < KP; ++p) {
+          const uint32_t cst = st, cph = ph;
+          if (++st == PJ_STAGES) { st = 0; ph ^= 1u; }
+          if (!(ok = mbar_wait(full + 8 * cst, cph, abort_flag))) break;
+          fence_after_sync();
+          const uint64_t adesc = adesc0 + (uint64_t)(cst * (stage_bytes >> 4));
+          const uint64_t bdesc = bdesc0 + (uint64_t)(cst * (stage_bytes >> 4));
+          mma_f16_ss(dcol, adesc, bdesc, idesc, p > 0 ? 1u : 0u);
+#pragma unroll
+          for (int ks = 1; ks < 4; ++ks) mma_f16_ss(dcol, adesc + 2 * ks, bdesc + 2 * ks, idesc, 1u);
+          mma_commit(empty + 8 * cst);
+        }
+        if (!ok) break;
+        mma_commit(acc_full + 8 * buf);
+      }
+    }
+    __syncwarp();
+  } else {
+    // ------------------------------------------------------------- epilogue
+    const int ew = warp - 2;                                   // 0..7
+    const int quarter = warp & 3, chalf = ew >> 2;
+    const int row = quarter * 32 + lane;
+    const uint32_t lane_addr = tmem_base + ((uint32_t)(quarter * 32) << 16);
+    const bool leader = (ew & 3) == 0 && lane == 0;            // issues this half's stores
+    unsigned char* my_panel = out_stage + chalf * PJ_PANEL_BYTES;
+    const uint32_t my_panel_addr = smem_addr(my_panel);
+    const int bar_id = 1 + chalf;
+    const int panels = NS / 128;                               // 64-column panels per half slab
+    uint32_t ac = 0;
+    for (int it = it0; it < n_items; it += itstep, ++ac) {
+      const int rem = it % per_tile, m0 = (it / per_tile) * TILE;
+      const int side = side0 + rem / n_slabs, ns = rem % n_slabs;
+      const CUtensorMap* omap = side ? &map_ov : &map_ok;
+      const uint32_t buf = ac & 1u;
+      const bool got = mbar_wait(acc_full + 8 * buf, (ac >> 1) & 1u, abort_flag);
+      if (!named_bar_and(bar_id, 128, got)) break;             // the four warps of a half leave together
+      fence_after_sync();
+      for (int pn = 0; pn < panels; ++pn) {
+        const int col = chalf * (NS / 2) + pn * 64;            // first column of the panel inside the slab
+        float a[32], b[32];
+        tmem_ld32(lane_addr + buf * 256 + col, reinterpret_cast<uint32_t*>(a));
+        tmem_ld32(lane_addr + buf * 256 + col + 32, reinterpret_cast<uint32_t*>(b));
+        tmem_ld_wait();
+        if (pn == panels - 1) {                                // last read of this accumulator
+          fence_before_sync();
+          __syncwarp();
+          if (lane == 0) mbar_arrive(acc_empty + 8 * buf);
+        }
+        uint32_t pk[32];
+#pragma unroll
+        for (int u = 0; u < 16; ++u) {
+          pk[u] = bf16 ? pack_bf16x2_rn(a[2 * u], a[2 * u + 1]) : pack_f16x2_rn(a[2 * u], a[2 * u + 1]);
+          pk[16 + u] = bf16 ? pack_bf16x2_rn(b[2 * u], b[2 * u + 1]) : pack_f16x2_rn(b[2 * u], b[2 * u + 1]);
+        }
+        if (leader) bulk_wait_read_all();                      // the previous store has left the staging panel
+        named_bar_sync(bar_id, 128);
+#pragma unroll
+        for (int c8 = 0; c8 < 8; ++c8)                         // 16-byte chunk c8 of the row sits at chunk c8 ^ (row % 8)
+          *reinterpret_cast<uint4*>(my_panel + row * 128 + ((c8 ^ (row & 7)) << 4)) =
+              make_uint4(pk[4 * c8], pk[4 * c8 + 1], pk[4 * c8 + 2], pk[4 * c8 + 3]);
+        fence_proxy_async_smem();
+        named_bar_sync(bar_id, 128);
+        if (leader) {
+          tma_store_2d(omap, my_panel_addr, ns * NS + col, m0);
+          bulk_commit();
+        }
+      }
+    }
+    if (leader) bulk_wait_all();
+  }
+
+  fence_before_sync();
+  __syncthreads();
+  fence_after_sync();
+  if (warp == 1) tmem_dealloc(tmem_base, PJ_TMEM_COLS);
+  if (tid == 0 && *abort_flag) atomicCAS(status, 0, TWKV_ERR_TIMEOUT);
+}
+
+cudaError_t launch_project_tc(const ProjectMaps& maps, int n_tok, int d, int bf16, int side0, int n_sides, int* status,
+                              int sm_count, cudaStream_t st) {
+  if (n_tok <= 0 || n_sides <= 0) return cudaSuccess;
+  const int NS = (d % 256 == 0) ? 256 : 128;
+  const size_t smem = (size_t)PJ_STAGES * (PJ_PANEL_BYTES + (size_t)NS * 128) + 2 * PJ_PANEL_BYTES + 8 * (2 * PJ_STAGES + 4) + 16;
+  cudaError_t e = cudaFuncSetAttribute(project_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  if (e != cudaSuccess) return e;
+  const long long n_items = (long long)n_sides * (d / NS) * ((n_tok + TILE - 1) / TILE);
+  const int grid = n_items < sm_count ? (int)n_items : sm_count;
+  project_tc_kernel<<<grid, PJ_THREADS, smem, st>>>(maps.xk, maps.xv, maps.uk, maps.uv, maps.ok, maps.ov, n_tok, d, bf16, side0, n_sides, status);
+  count_launch();
+  return cudaGetLastError();
+}
+
+}  // namespace twkv

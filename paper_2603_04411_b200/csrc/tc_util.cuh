@@ -232,6 +232,8 @@ __device__ __forceinline__ bool elect_one() {
 struct TcMaps { CUtensorMap blocks, uinvT_k; };
 // Tensor maps of the fused gate kernel: the call's K and V states, and the layer's transposed gate weights.
 struct GateMaps { CUtensorMap xk, xv, wk, wv; };
+// Tensor maps of the projection kernel: the call's raw states, the transposed bases, and the outputs.
+struct ProjectMaps { CUtensorMap xk, xv, uk, uv, ok, ov; };
 
 // Host side: 2-D tensor map over a row-major 16-bit matrix [rows][cols], box [box_rows][64], 128-byte swizzle.
 bool make_tmap_2d(CUtensorMap* out, const void* base, uint64_t rows, uint64_t cols, uint64_t row_stride_bytes, uint32_t box_rows);

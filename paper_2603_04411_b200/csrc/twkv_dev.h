@@ -95,6 +95,19 @@ __device__ inline float dec_ordered(unsigned u) {
 
 __device__ inline void set_status(const DevView& v, int code) { atomicCAS(v.status, 0, code); }
 
+// Makes `dev` the current device for the scope of a host call.
+struct DeviceGuard {
+  int prev = -1;
+  bool ok = true;
+  explicit DeviceGuard(int dev) {
+    if (cudaGetDevice(&prev) != cudaSuccess) { ok = false; return; }
+    if (prev != dev && cudaSetDevice(dev) != cudaSuccess) ok = false;
+    target = dev;
+  }
+  ~DeviceGuard() { if (prev >= 0 && prev != target) cudaSetDevice(prev); }
+  int target = -1;
+};
+
 // launch bookkeeping (host)
 void count_launch(int n = 1);
 // optional per-kernel event timing of the cache whose API call is running on this thread
@@ -118,6 +131,9 @@ struct GateMaps;   // tensor maps of the fused gate kernel (api.cu)
 cudaError_t launch_gate_ranks_tc(const DevView& v, const GateMaps& maps, const LayerParams& lp, int n_tok, unsigned short* levels,
                                  int sm_count, cudaStream_t st);
 size_t gate_tc_stage_bytes(int n_cta, int d);
+struct ProjectMaps;   // tensor maps of the projection kernel
+cudaError_t launch_project_tc(const ProjectMaps& maps, int n_tok, int d, int bf16, int side0, int n_sides, int* status,
+                              int sm_count, cudaStream_t st);
 cudaError_t launch_transpose16(const void* in, void* out, int n, cudaStream_t st);
 cudaError_t launch_gate_logits(const DevView& v, const LayerParams& lp, const void* K, const void* V, int n_tok,
                                float* logits, cudaStream_t st);

@@ -52,3 +52,21 @@ def test_host_only_calls(libpath):
     assert B.lib.twkv_compress(None, 0, None, None, None, None, 0, None, None, 0, None) == B.TWKV_ERR_INVALID_ARG
     assert B.lib.twkv_decode_attn(None, 0, None, None, 0, None, 0, None) == B.TWKV_ERR_INVALID_ARG
     assert B.twkv_launch_count() == 0
+
+
+def test_projector_argument_checks_need_no_device():
+    """Sizes and pointers are validated before any CUDA call."""
+    from paper_2603_04411_b200 import binding as B
+    import ctypes
+    assert B.twkv_projector_required_bytes(1024) == 256 + 2 * 1024 * 1024 * 2
+    assert B.twkv_projector_required_bytes(1000) == 0 and B.twkv_projector_required_bytes(64) == 0
+    h = ctypes.c_void_p()
+    one = ctypes.c_void_p(256)
+    assert B.lib.twkv_projector_create(1000, B.TWKV_F16, one, one, one, 1 << 30, None, ctypes.byref(h)) == B.TWKV_ERR_UNSUPPORTED
+    assert B.lib.twkv_projector_create(1024, B.TWKV_F32, one, one, one, 1 << 30, None, ctypes.byref(h)) == B.TWKV_ERR_UNSUPPORTED
+    assert B.lib.twkv_projector_create(1024, B.TWKV_F16, None, None, one, 1 << 30, None, ctypes.byref(h)) == B.TWKV_ERR_INVALID_ARG
+    assert B.lib.twkv_projector_create(1024, B.TWKV_F16, one, one, None, 1 << 30, None, ctypes.byref(h)) == B.TWKV_ERR_INVALID_ARG
+    assert B.lib.twkv_projector_create(1024, B.TWKV_F16, one, one, ctypes.c_void_p(264), 1 << 30, None, ctypes.byref(h)) == B.TWKV_ERR_INVALID_ARG
+    assert B.lib.twkv_projector_create(1024, B.TWKV_F16, one, one, one, 1024, None, ctypes.byref(h)) == B.TWKV_ERR_CAPACITY
+    assert B.lib.twkv_project(None, one, one, one, one, 4, None) == B.TWKV_ERR_INVALID_ARG
+    assert h.value is None
