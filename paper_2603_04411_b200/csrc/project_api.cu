@@ -8,11 +8,13 @@ struct twkv_projector {
   int device = 0, sm_count = 0, d = 0, bf16 = 0;
   unsigned char* ws = nullptr;                 // [status, 256 B][U_k^T][U_v^T]
   bool has[2] = {false, false};
-  CUtensorMap map_uT[2];
+  CUtensorMap map_uT[2];                       // box = one slab of U^T rows (single-CTA kernel)
+  CUtensorMap map_uT_half[2];                  // box = 128 rows (CTA-pair kernel: each CTA loads half a slab)
 };
 
 namespace twkv {
 constexpr size_t PJ_STATUS_BYTES = 256;
+constexpr int PJ_PAIR_MIN_TOKENS = 1024;      // from here on the CTA-pair kernel is used (d a multiple of 256)
 static bool dim_ok(int d) { return d >= 128 && d <= 8192 && d % 128 == 0; }
 }  // namespace twkv
 
@@ -50,7 +52,8 @@ twkv_status twkv_projector_create(int d_kv, twkv_dtype dtype, const void* U_k, c
     // K-major copy of U for the tensor cores: row n of the copy = column n of U
     unsigned char* dst = p->ws + PJ_STATUS_BYTES + (size_t)side * d_kv * d_kv * 2;
     ok = launch_transpose16(U[side], dst, d_kv, st) == cudaSuccess &&
-         make_tmap_2d(&p->map_uT[side], dst, d_kv, d_kv, (uint64_t)d_kv * 2, NS);
+         make_tmap_2d(&p->map_uT[side], dst, d_kv, d_kv, (uint64_t)d_kv * 2, NS) &&
+         make_tmap_2d(&p->map_uT_half[side], dst, d_kv, d_kv, (uint64_t)d_kv * 2, TILE);
     p->has[side] = true;
   }
   if (!ok) { delete p; return TWKV_ERR_CUDA; }
@@ -76,6 +79,7 @@ twkv_status twkv_project(twkv_projector* p, const void* x_k, const void* x_v, vo
   DeviceGuard g(p->device);
   if (!g.ok) return TWKV_ERR_CUDA;
   const int side0 = x_k ? 0 : 1, n_sides = (x_k ? 1 : 0) + (x_v ? 1 : 0);
+  const bool pairs = p->d % 256 == 0 && n_tok >= PJ_PAIR_MIN_TOKENS && p->sm_count >= 2;
   ProjectMaps maps;
   for (int side = 0; side < 2; ++side) {
     const int src = in[side] ? side : side0;              // an unused side's maps alias the used one (never dereferenced)
@@ -83,9 +87,9 @@ twkv_status twkv_project(twkv_projector* p, const void* x_k, const void* x_v, vo
     CUtensorMap* mo = side ? &maps.ov : &maps.ok;
     if (!make_tmap_2d(mx, in[src], (uint64_t)n_tok, p->d, (uint64_t)p->d * 2, TILE) ||
         !make_tmap_2d(mo, outp[src], (uint64_t)n_tok, p->d, (uint64_t)p->d * 2, TILE)) return TWKV_ERR_CUDA;
-    (side ? maps.uv : maps.uk) = p->map_uT[src];
+    (side ? maps.uv : maps.uk) = pairs ? p->map_uT_half[src] : p->map_uT[src];
   }
-  if (launch_project_tc(maps, n_tok, p->d, p->bf16, side0, n_sides, (int*)p->ws, p->sm_count, (cudaStream_t)stream) != cudaSuccess)
+  if (launch_project_tc(maps, n_tok, p->d, p->bf16, side0, n_sides, (int*)p->ws, p->sm_count, pairs, (cudaStream_t)stream) != cudaSuccess)
     return TWKV_ERR_CUDA;
   return TWKV_OK;
 }

@@ -17,6 +17,7 @@
 //   warp 1      MMA issuer (one elected lane; owns the TMEM allocation)
 //   warps 2-9   epilogue: thread = one token row x half of the slab's columns; each half (four warps) owns
 //               one staging panel and one lane that issues its stores
+// Calls of at least 1024 tokens with d a multiple of 256 run the CTA-pair variant further down instead.
 // All barrier waits are bounded (tc_util.cuh); a wait that runs out ends the kernel with TWKV_ERR_TIMEOUT.
 #include "twkv_dev.h"
 #include "tc_util.cuh"
@@ -220,9 +221,256 @@ project_tc_kernel(const __grid_constant__ CUtensorMap map_xk, const __grid_const
   if (tid == 0 && *abort_flag) atomicCAS(status, 0, TWKV_ERR_TIMEOUT);
 }
 
+// ------------------------------------------------------------------------------------------
+// The same product on CTA pairs (cta_group::2): two CTAs of a cluster, on neighbouring SMs, work on one
+// [256 x 256] item.  Each loads its own 128 token rows and its own 128 of the slab's 256 rows of U^T, one
+// tcgen05.mma of the even CTA drives both tensor cores (M = 256 over the pair, each CTA's accumulator in
+// its own TMEM), and each SM reads only half of the B operand from its shared memory: per SM, operand
+// traffic from L2 and shared-memory reads both drop from 96 to 64 bytes per tensor-core cycle, which is
+// what bounded the single-CTA kernel.  Protocol:
+//   full[stage]      lives in the even CTA; both CTAs' copies complete on it (the odd CTA addresses it through
+//                    the cluster window), the even CTA's producer lanes post the expected bytes of both
+//   empty[stage], acc_full[buf]   one in each CTA, signalled together by a multicast tcgen05.commit
+//   acc_empty[buf]   lives in the even CTA; 16 arrivals (8 epilogue warps of each CTA, the odd CTA's remote)
+// The cluster barrier brackets the kernel: nobody signals a barrier before it is initialised, nobody leaves
+// (and no TMEM is freed) while the partner can still read its shared memory or write its barriers.
+constexpr int PJ2_STAGES = 6;
+constexpr uint32_t PJ2_STAGE_BYTES = 2 * PJ_PANEL_BYTES;         // [X panel | half of the U^T panel]
+
+__device__ __forceinline__ uint32_t cluster_cta_rank() {
+  uint32_t r;
+  asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+  return r;
+}
+__device__ __forceinline__ void cluster_sync_all() {
+  asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+  asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+// address of the same shared-memory object in CTA `rank` of the cluster
+__device__ __forceinline__ uint32_t cluster_map(uint32_t addr, uint32_t rank) {
+  uint32_t r;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(addr), "r"(rank));
+  return r;
+}
+__device__ __forceinline__ void mbar_arrive_cluster(uint32_t bar_cluster_addr) {
+  asm volatile("mbarrier.arrive.shared::cluster.b64 _, [%0];" ::"r"(bar_cluster_addr) : "memory");
+}
+// TMA load whose completion is counted on a barrier that may live in the partner CTA (no multicast).
+__device__ __forceinline__ void tma_load_2d_pair(uint32_t dst, const CUtensorMap* map, uint32_t bar_cluster_addr, int x, int y) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+      ::"r"(dst), "l"(map), "r"(bar_cluster_addr), "r"(x), "r"(y) : "memory");
+}
+__device__ __forceinline__ void tmem_alloc_pair(uint32_t slot_smem, uint32_t cols) {
+  asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(slot_smem), "r"(cols) : "memory");
+  asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc_pair(uint32_t base, uint32_t cols) {
+  asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(base), "r"(cols) : "memory");
+}
+__device__ __forceinline__ void mma_f16_ss_pair(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate) : "memory");
+}
+// arrives, once the pair's MMAs issued so far have retired, on the barrier at this offset in both CTAs
+__device__ __forceinline__ void mma_commit_pair_both(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
+               ::"r"(bar), "h"((unsigned short)3) : "memory");
+}
+
+__global__ void __launch_bounds__(PJ_THREADS, 1)
+project_tc2_kernel(const __grid_constant__ CUtensorMap map_xk, const __grid_constant__ CUtensorMap map_xv,
+                   const __grid_constant__ CUtensorMap map_uk, const __grid_constant__ CUtensorMap map_uv,
+                   const __grid_constant__ CUtensorMap map_ok, const __grid_constant__ CUtensorMap map_ov,
+                   int n_tok, int d, int bf16, int side0, int n_sides, int* status) {
+  extern __shared__ __align__(1024) unsigned char smem_raw[];
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const uint32_t crank = cluster_cta_rank();                   // 0 = even CTA: issues the MMAs, owns full / acc_empty
+  const int KP = d / PANEL;
+  const int n_slabs = d / 256;
+  const uint32_t sA = smem_addr(smem_raw);
+  const bool misaligned = (sA & 1023u) != 0;
+  unsigned char* out_stage = smem_raw + PJ2_STAGES * PJ2_STAGE_BYTES;
+  unsigned char* tail = out_stage + 2 * PJ_PANEL_BYTES;
+  const uint32_t bars = smem_addr(tail);
+  const uint32_t full = bars, empty = full + 8 * PJ2_STAGES, acc_full = empty + 8 * PJ2_STAGES, acc_empty = acc_full + 16;
+  uint32_t* s_tmem_base = reinterpret_cast<uint32_t*>(tail + 8 * (2 * PJ2_STAGES + 4));
+  volatile int* abort_flag = reinterpret_cast<int*>(s_tmem_base + 1);
+
+  if (tid == 0) {
+    for (int i = 0; i < PJ2_STAGES; ++i) { mbar_init(full + 8 * i, 2); mbar_init(empty + 8 * i, 1); }
+    for (int i = 0; i < 2; ++i) { mbar_init(acc_full + 8 * i, 1); mbar_init(acc_empty + 8 * i, 2 * (PJ_EPI / 32)); }
+    *abort_flag = misaligned ? 1 : 0;
+    mbar_init_fence();
+  }
+  if (warp == 1) tmem_alloc_pair(smem_addr(s_tmem_base), PJ_TMEM_COLS);
+  fence_before_sync();
+  __syncthreads();
+  cluster_sync_all();                                          // both CTAs' barriers and TMEM are ready
+  fence_after_sync();
+  const uint32_t tmem_base = *s_tmem_base;
+
+  // item -> (pair of token tiles, side, slab): slab fastest, then side; one item per cluster at a time
+  const int per_tile = n_sides * n_slabs;
+  const int n_items = per_tile * ((n_tok + 2 * TILE - 1) / (2 * TILE));
+  const int it0 = blockIdx.x >> 1, itstep = gridDim.x >> 1;
+
+  if (misaligned) {
+    // nothing was started; fall through to the common exit
+  } else if (warp == 0) {
+    // ------------------------------------------------------------- TMA producer (both CTAs)
+    if (lane < 2 * PJ2_STAGES) {
+      const bool is_x = lane >= PJ2_STAGES;
+      const uint32_t my = is_x ? lane - PJ2_STAGES : lane;
+      if (lane == 0) { tma_prefetch_desc(&map_uk); tma_prefetch_desc(&map_uv); }
+      if (lane == PJ2_STAGES) { tma_prefetch_desc(&map_xk); tma_prefetch_desc(&map_xv); }
+      const uint32_t full_even = cluster_map(full + 8 * my, 0);            // the even CTA's barrier of this lane's stage
+      bool ok = true;
+      uint32_t st = 0, ph = 0;
+      for (int it = it0; it < n_items && ok; it += itstep) {
+        const int rem = it % per_tile, m0 = (it / per_tile) * (2 * TILE) + (int)crank * TILE;
+        const int side = side0 + rem / n_slabs, ns = rem % n_slabs;
+        const CUtensorMap* map = is_x ? (side ? &map_xv : &map_xk) : (side ? &map_uv : &map_uk);
+        for (int p = 0; p < KP; ++p) {
+          const uint32_t cst = st, cph = ph;
+          if (++st == PJ2_STAGES) { st = 0; ph ^= 1u; }
+          if (cst != my) continue;
+          if (!(ok = mbar_wait(empty + 8 * cst, cph ^ 1u, abort_flag))) break;
+          if (crank == 0) mbar_expect_tx(full + 8 * cst, 2 * PJ_PANEL_BYTES);      // this lane's copy and the partner's
+          if (is_x) tma_load_2d_pair(sA + cst * PJ2_STAGE_BYTES, map, full_even, p * PANEL, m0);
+          else tma_load_2d_pair(sA + cst * PJ2_STAGE_BYTES + PJ_PANEL_BYTES, map, full_even, p * PANEL, ns * 256 + (int)crank * TILE);
+        }
+      }
+    }
+    __syncwarp();
+  } else if (warp == 1) {
+    // ------------------------------------------------------------- MMA issuer (even CTA only)
+    if (crank == 0 && elect_one()) {
+      const uint32_t idesc = idesc_f16(bf16 ? 1 : 0, 256, 256);
+      const uint64_t adesc0 = kmajor_sw128_desc(sA), bdesc0 = kmajor_sw128_desc(sA + PJ_PANEL_BYTES);
+      bool ok = true;
+      uint32_t st = 0, ph = 0, ac = 0;
+      for (int it = it0; it < n_items && ok; it += itstep, ++ac) {
+        const uint32_t buf = ac & 1u;
+        if (!(ok = mbar_wait(acc_empty + 8 * buf, ((ac >> 1) & 1u) ^ 1u, abort_flag))) break;
+        fence_after_sync();
+        const uint32_t dcol = tmem_base + buf * 256;
+        for (int p = 0; p < KP; ++p) {
+          const uint32_t cst = st, cph = ph;
+          if (++st == PJ2_STAGES) { st = 0; ph ^= 1u; }
+          if (!(ok = mbar_wait(full + 8 * cst, cph, abort_flag))) break;
+          fence_after_sync();
+          const uint64_t adesc = adesc0 + (uint64_t)(cst * (PJ2_STAGE_BYTES >> 4));
+          const uint64_t bdesc = bdesc0 + (uint64_t)(cst * (PJ2_STAGE_BYTES >> 4));
+          mma_f16_ss_pair(dcol, adesc, bdesc, idesc, p > 0 ? 1u : 0u);
+#pragma unroll
+          for (int ks = 1; ks < 4; ++ks) mma_f16_ss_pair(dcol, adesc + 2 * ks, bdesc + 2 * ks, idesc, 1u);
+          mma_commit_pair_both(empty + 8 * cst);
+        }
+        if (!ok) break;
+        mma_commit_pair_both(acc_full + 8 * buf);
+      }
+    }
+    __syncwarp();
+  } else {
+    // ------------------------------------------------------------- epilogue (both CTAs, own 128 rows)
+    const int ew = warp - 2;
+    const int quarter = warp & 3, chalf = ew >> 2;
+    const int row = quarter * 32 + lane;
+    const uint32_t lane_addr = tmem_base + ((uint32_t)(quarter * 32) << 16);
+    const bool leader = (ew & 3) == 0 && lane == 0;
+    unsigned char* my_panel = out_stage + chalf * PJ_PANEL_BYTES;
+    const uint32_t my_panel_addr = smem_addr(my_panel);
+    const int bar_id = 1 + chalf;
+    const uint32_t acc_empty_even = cluster_map(acc_empty, 0);
+    uint32_t ac = 0;
+    for (int it = it0; it < n_items; it += itstep, ++ac) {
+      const int rem = it % per_tile, m0 = (it / per_tile) * (2 * TILE) + (int)crank * TILE;
+      const int side = side0 + rem / n_slabs, ns = rem % n_slabs;
+      const CUtensorMap* omap = side ? &map_ov : &map_ok;
+      const uint32_t buf = ac & 1u;
+      const bool got = mbar_wait(acc_full + 8 * buf, (ac >> 1) & 1u, abort_flag);
+      if (!named_bar_and(bar_id, 128, got)) break;
+      fence_after_sync();
+      for (int pn = 0; pn < 2; ++pn) {
+        const int col = chalf * 128 + pn * 64;
+        float a[32], b[32];
+        tmem_ld32(lane_addr + buf * 256 + col, reinterpret_cast<uint32_t*>(a));
+        tmem_ld32(lane_addr + buf * 256 + col + 32, reinterpret_cast<uint32_t*>(b));
+        tmem_ld_wait();
+        if (pn == 1) {                                         // last read of this accumulator
+          fence_before_sync();
+          __syncwarp();
+          if (lane == 0) mbar_arrive_cluster(acc_empty_even + 8 * buf);
+        }
+        uint32_t pk[32];
+#pragma unroll
+        for (int u = 0; u < 16; ++u) {
+          pk[u] = bf16 ? pack_bf16x2_rn(a[2 * u], a[2 * u + 1]) : pack_f16x2_rn(a[2 * u], a[2 * u + 1]);
+          pk[16 + u] = bf16 ? pack_bf16x2_rn(b[2 * u], b[2 * u + 1]) : pack_f16x2_rn(b[2 * u], b[2 * u + 1]);
+        }
+        if (leader) bulk_wait_read_all();
+        named_bar_sync(bar_id, 128);
+#pragma unroll
+        for (int c8 = 0; c8 < 8; ++c8)
+          *reinterpret_cast<uint4*>(my_panel + row * 128 + ((c8 ^ (row & 7)) << 4)) =
+              make_uint4(pk[4 * c8], pk[4 * c8 + 1], pk[4 * c8 + 2], pk[4 * c8 + 3]);
+        fence_proxy_async_smem();
+        named_bar_sync(bar_id, 128);
+        if (leader && m0 < n_tok) {                            // the pair's second tile may lie past the last token
+          tma_store_2d(omap, my_panel_addr, ns * 256 + col, m0);
+          bulk_commit();
+        }
+      }
+    }
+    if (leader) bulk_wait_all();
+  }
+
+  fence_before_sync();
+  __syncthreads();
+  cluster_sync_all();                                          // the partner is done with this CTA's memory as well
+  fence_after_sync();
+  if (warp == 1) tmem_dealloc_pair(tmem_base, PJ_TMEM_COLS);
+  if (tid == 0 && *abort_flag) atomicCAS(status, 0, misaligned ? TWKV_ERR_DEVICE_CHECK : TWKV_ERR_TIMEOUT);
+}
+
 cudaError_t launch_project_tc(const ProjectMaps& maps, int n_tok, int d, int bf16, int side0, int n_sides, int* status,
-                              int sm_count, cudaStream_t st) {
+                              int sm_count, bool pairs, cudaStream_t st) {
   if (n_tok <= 0 || n_sides <= 0) return cudaSuccess;
+  if (pairs) {
+    // maps.uk / maps.uv must have 128-row boxes here (each CTA loads half of a 256-row slab)
+    const size_t smem = (size_t)PJ2_STAGES * PJ2_STAGE_BYTES + 2 * PJ_PANEL_BYTES + 8 * (2 * PJ2_STAGES + 4) + 16;
+    cudaError_t e = cudaFuncSetAttribute(project_tc2_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+    const long long n_items = (long long)n_sides * (d / 256) * ((n_tok + 2 * TILE - 1) / (2 * TILE));
+    cudaLaunchConfig_t cfg = {};
+    cfg.blockDim = dim3(PJ_THREADS);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cudaLaunchAttribute pair_attr;
+    pair_attr.id = cudaLaunchAttributeClusterDimension;
+    pair_attr.val.clusterDim.x = 2; pair_attr.val.clusterDim.y = 1; pair_attr.val.clusterDim.z = 1;
+    cfg.attrs = &pair_attr;
+    cfg.numAttrs = 1;
+    static int max_clusters = -1;                              // co-resident CTA pairs on this device
+    if (max_clusters < 0) {
+      cfg.gridDim = dim3(sm_count & ~1);
+      int n = 0;
+      if (cudaOccupancyMaxActiveClusters(&n, project_tc2_kernel, &cfg) != cudaSuccess || n < 1) { cudaGetLastError(); n = 0; }
+      max_clusters = n;
+    }
+    if (max_clusters > 0) {
+      const int clusters = n_items < max_clusters ? (int)n_items : max_clusters;
+      cfg.gridDim = dim3(2 * clusters);
+      e = cudaLaunchKernelEx(&cfg, project_tc2_kernel, maps.xk, maps.xv, maps.uk, maps.uv, maps.ok, maps.ov, n_tok, d, bf16, side0, n_sides, status);
+      count_launch();
+      return e != cudaSuccess ? e : cudaGetLastError();
+    }
+    return cudaErrorInvalidConfiguration;
+  }
   const int NS = (d % 256 == 0) ? 256 : 128;
   const size_t smem = (size_t)PJ_STAGES * (PJ_PANEL_BYTES + (size_t)NS * 128) + 2 * PJ_PANEL_BYTES + 8 * (2 * PJ_STAGES + 4) + 16;
   cudaError_t e = cudaFuncSetAttribute(project_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);

@@ -133,7 +133,7 @@ cudaError_t launch_gate_ranks_tc(const DevView& v, const GateMaps& maps, const L
 size_t gate_tc_stage_bytes(int n_cta, int d);
 struct ProjectMaps;   // tensor maps of the projection kernel
 cudaError_t launch_project_tc(const ProjectMaps& maps, int n_tok, int d, int bf16, int side0, int n_sides, int* status,
-                              int sm_count, cudaStream_t st);
+                              int sm_count, bool pairs, cudaStream_t st);
 cudaError_t launch_transpose16(const void* in, void* out, int n, cudaStream_t st);
 cudaError_t launch_gate_logits(const DevView& v, const LayerParams& lp, const void* K, const void* V, int n_tok,
                                float* logits, cudaStream_t st);

@@ -81,6 +81,15 @@ def test_project_fp16_ragged_two_sides(B):
     run(B, 31, 1000, 1024, torch.float16)
 
 
+def test_project_pairs_fp16_ragged_last_pair_half_empty(B):
+    # 1300 = 5 x 256 + 20: the last CTA pair has 20 valid rows in its first tile and none in its second
+    run(B, 37, 1300, 1024, torch.float16)
+
+
+def test_project_pairs_bf16_two_slabs_value_side_only(B):
+    run(B, 38, 1024 + 129, 512, torch.bfloat16, sides=(False, True))
+
+
 def test_project_bf16_two_slabs(B):
     run(B, 32, 300, 512, torch.bfloat16)
 
