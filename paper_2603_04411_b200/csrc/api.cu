@@ -177,7 +177,8 @@ struct twkv_cache {
   CUtensorMap map_blocks;
   std::vector<CUtensorMap> map_uinvT;  // per layer, over the transposed copy of U_K^-1 inside the pool
   std::vector<char> prepared;          // per layer: transposed copy and its map are current
-  std::vector<CUtensorMap> map_wT;     // per layer x side, over the transposed copies of the gate weights
+  std::vector<CUtensorMap> map_wT;     // per layer x side, over the transposed copies of the gate weights (box = one slab)
+  std::vector<CUtensorMap> map_wT_half; // the same with 128-row boxes, for the CTA-pair kernel
   std::vector<char> prepared_w;        // per layer: those copies and maps are current
 };
 
@@ -275,6 +276,7 @@ twkv_status twkv_cache_create(const twkv_config* cfg, void* pool, size_t pool_by
   c->map_uinvT.resize(cfg->n_layers);
   c->prepared.assign(cfg->n_layers, 0);
   c->map_wT.resize(2 * (size_t)cfg->n_layers);
+  c->map_wT_half.resize(2 * (size_t)cfg->n_layers);
   c->prepared_w.assign(cfg->n_layers, 0);
   if (!make_tmap_2d(&c->map_blocks, c->view.blocks, (uint64_t)c->view.n_blocks * TILE, PANEL, PANEL * 2, TILE)) { delete c; return TWKV_ERR_CUDA; }
   twkv_status s = twkv_cache_reset(c, stream);
@@ -361,16 +363,18 @@ twkv_status twkv_compress(twkv_cache* c, int layer, const void* K, const void* V
       for (int side = 0; side < 2; ++side) {
         unsigned char* dst = c->pool + c->off.prep_wT + ((size_t)layer * 2 + side) * d * d * 2;
         if (launch_transpose16(side ? c->params[layer].W_v : c->params[layer].W_k, dst, d, st) != cudaSuccess) return TWKV_ERR_CUDA;
-        if (!make_tmap_2d(&c->map_wT[2 * (size_t)layer + side], dst, d, d, (uint64_t)d * 2, ns)) return TWKV_ERR_CUDA;
+        if (!make_tmap_2d(&c->map_wT[2 * (size_t)layer + side], dst, d, d, (uint64_t)d * 2, ns) ||
+            !make_tmap_2d(&c->map_wT_half[2 * (size_t)layer + side], dst, d, d, (uint64_t)d * 2, TILE)) return TWKV_ERR_CUDA;
       }
       c->prepared_w[layer] = 1;
     }
+    const bool pairs = d % 256 == 0 && gate_tc_max_pairs(c->sm_count) > 0;
     GateMaps maps;
-    maps.wk = c->map_wT[2 * (size_t)layer];
-    maps.wv = c->map_wT[2 * (size_t)layer + 1];
+    maps.wk = (pairs ? c->map_wT_half : c->map_wT)[2 * (size_t)layer];
+    maps.wv = (pairs ? c->map_wT_half : c->map_wT)[2 * (size_t)layer + 1];
     if (!make_tmap_2d(&maps.xk, K, (uint64_t)n_tok, d, (uint64_t)d * 2, TILE) ||
         !make_tmap_2d(&maps.xv, V, (uint64_t)n_tok, d, (uint64_t)d * 2, TILE)) return TWKV_ERR_CUDA;
-    if (launch_gate_ranks_tc(v, maps, c->params[layer], n_tok, levels, c->sm_count, st) != cudaSuccess) return TWKV_ERR_CUDA;
+    if (launch_gate_ranks_tc(v, maps, c->params[layer], n_tok, levels, c->sm_count, pairs, st) != cudaSuccess) return TWKV_ERR_CUDA;
   } else if (mode == TWKV_GATE_COMPUTE) {
     for (int lo = 0; lo < n_tok; lo += GATE_PIECE) {
       const int n = n_tok - lo < GATE_PIECE ? n_tok - lo : GATE_PIECE;

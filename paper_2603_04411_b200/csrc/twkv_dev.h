@@ -129,7 +129,8 @@ cudaError_t launch_decode(const DevView& v, int layer, const LayerParams& lp, co
                           int n_seq, void* out, int num_splits, int sm_count, const TcMaps* maps, cudaStream_t st);
 struct GateMaps;   // tensor maps of the fused gate kernel (api.cu)
 cudaError_t launch_gate_ranks_tc(const DevView& v, const GateMaps& maps, const LayerParams& lp, int n_tok, unsigned short* levels,
-                                 int sm_count, cudaStream_t st);
+                                 int sm_count, bool pairs, cudaStream_t st);
+int gate_tc_max_pairs(int sm_count);
 size_t gate_tc_stage_bytes(int n_cta, int d);
 struct ProjectMaps;   // tensor maps of the projection kernel
 cudaError_t launch_project_tc(const ProjectMaps& maps, int n_tok, int d, int bf16, int side0, int n_sides, int* status,
