@@ -240,47 +240,30 @@ __global__ void __launch_bounds__(1024) alloc_kernel(DevView v, int layer, int n
   }
 }
 
-// Copies the first r elements of a 16-bit row into the tile's panels, +0 beyond r.
-__device__ __forceinline__ void pack_row(const DevView& v, const uint4* __restrict__ src, int r, int cls, int base, int slot, int lane, int first_chunk) {
-  const int nchunks = cls * 8;                            // 16-byte chunks of 8 elements
-  for (int ch = first_chunk + lane; ch < nchunks; ch += 32) {
-    const int e0 = ch * 8;
-    uint4 val = make_uint4(0u, 0u, 0u, 0u);
-    if (e0 < r) {
-      val = __ldg(src + ch);
-      const int keep = r - e0;                            // elements kept in this chunk (>= 1)
-      if (keep < 8) {
-        unsigned* w = reinterpret_cast<unsigned*>(&val);
-#pragma unroll
-        for (int p = 0; p < 4; ++p) {
-          const int left = keep - 2 * p;                  // elements kept in 32-bit word p
-          if (left <= 0) w[p] = 0u;
-          else if (left == 1) w[p] &= 0x0000ffffu;
-        }
-      }
-    }
-    unsigned char* dst = v.blocks + (size_t)(base + (ch >> 3)) * BLOCK_BYTES + slot * (PANEL * 2) + (ch & 7) * 16;
-    *reinterpret_cast<uint4*>(dst) = val;
-  }
-}
-
-__device__ __forceinline__ void zero_tail(const DevView& v, int cls, int base, int slot, int lane) {
-  const int rows = TILE - 1 - slot;
-  const int total = rows * cls * 8;
-  for (int i = lane; i < total; i += 32) {
-    const int panel = i / (rows * 8);
-    const int rem = i - panel * rows * 8;
-    unsigned char* dst = v.blocks + (size_t)(base + panel) * BLOCK_BYTES + (slot + 1) * (PANEL * 2) + rem * 16;
-    *reinterpret_cast<uint4*>(dst) = make_uint4(0u, 0u, 0u, 0u);
-  }
-}
-
-struct Place { int base, slot_cls_r, flags; };   // slot | cls << 8 | r << 16 ; flags bit0 = zero the tile's tail
+struct Place { int base, slot_cls_r; };   // slot | cls << 8 | r << 16
 
 __global__ void __launch_bounds__(CHUNK_TOKENS) pack_kernel(DevView v, int layer, const void* __restrict__ K, const void* __restrict__ V,
                                                             const int* __restrict__ seq_ids, const int* __restrict__ positions,
                                                             const unsigned short* __restrict__ levels, int n_tok) {
   if (v.status[2] == 0) return;                           // the piece was refused
+  const int n_chunks = (n_tok + CHUNK_TOKENS - 1) / CHUNK_TOKENS;
+  if ((int)blockIdx.x >= n_chunks) {
+    // CTAs past the token chunks, one per key: if the key's last token of this piece sits in a tile created by
+    // this piece and the tile is not full, zero the slots behind it (decode reads whole tiles).
+    const int k = blockIdx.x - n_chunks;
+    const int cnt = v.key_cnt[k];
+    if (cnt == 0) return;
+    const int old = v.key_old_fill[k], cls = k % v.NC + 1;
+    const int g = old + cnt - 1, ord = g / TILE, slot = g % TILE, old_tiles = (old + TILE - 1) / TILE;
+    if (ord < old_tiles || slot == TILE - 1) return;
+    const int base = v.key_first_base[k] + (ord - old_tiles) * cls;
+    const int n16 = (TILE - 1 - slot) * 8;                 // 16-byte chunks behind the last token, per panel
+    for (int panel = 0; panel < cls; ++panel) {
+      uint4* dst = reinterpret_cast<uint4*>(v.blocks + (size_t)(base + panel) * BLOCK_BYTES + (slot + 1) * (PANEL * 2));
+      for (int i = threadIdx.x; i < n16; i += CHUNK_TOKENS) dst[i] = make_uint4(0u, 0u, 0u, 0u);
+    }
+    return;
+  }
   __shared__ int s_key[2][CHUNK_TOKENS];
   __shared__ Place s_place[2][CHUNK_TOKENS];
   __shared__ unsigned long long s_sum[2];
@@ -321,10 +304,8 @@ __global__ void __launch_bounds__(CHUNK_TOKENS) pack_kernel(DevView v, int layer
         tile = v.key_old_last[k];
         base = v.desc(layer, side)[tile].w;
       }
-      const bool last_of_key = (g + 1 == old + v.key_cnt[k]);
       s_place[side][tid].base = base;
       s_place[side][tid].slot_cls_r = slot | (cls << 8) | (r[side] << 16);
-      s_place[side][tid].flags = (is_new && last_of_key && slot < TILE - 1) ? 1 : 0;
       v.rank(layer, side)[(size_t)tile * TILE + slot] = (unsigned short)r[side];
       if (side == 0) {
         v.aux(layer, 0)[(size_t)tile * TILE + slot] = positions[i];
@@ -342,54 +323,74 @@ __global__ void __launch_bounds__(CHUNK_TOKENS) pack_kernel(DevView v, int layer
   }
   __syncthreads();
   if (tid < 2 && s_sum[tid]) atomicAdd(&v.rank_sums[layer * 2 + tid], s_sum[tid]);
-  // warp per token: move the rows.  The first 32 chunks (256 elements) of four rows are loaded before any is stored,
-  // so a warp keeps four independent copies in flight; wider rows finish in pack_row.
-  const int warp = tid >> 5, lane = tid & 31;
-  const size_t row_bytes = (size_t)v.d_kv * 2;
-  constexpr int WARPS = CHUNK_TOKENS / 32;
-  constexpr int NQ = 4;                                                  // two tokens x two sides per round
-  for (int t0 = warp * (NQ / 2); t0 < CHUNK_TOKENS; t0 += WARPS * (NQ / 2)) {
-    uint4 val[NQ];
-    int meta[NQ], base[NQ];
-    bool live[NQ];
+  // Move the rows.  The CTA's 256 (token, side) rows are a flat list of 16-byte chunks (8 elements; a row of class c
+  // has 8 c of them, those past the rank are zero fill); thread i takes chunks i, i + 128, ... so every lane has
+  // work whatever the rows' widths, and loads PACK_UNROLL chunks before it stores any.
+  __shared__ int s_pref[2 * CHUNK_TOKENS + 1];
+  __shared__ int s_wtot[CHUNK_TOKENS / 32];
+  {
+    const int c0 = valid ? ((s_place[0][tid].slot_cls_r >> 8) & 0xff) * 8 : 0;
+    const int c1 = valid ? ((s_place[1][tid].slot_cls_r >> 8) & 0xff) * 8 : 0;
+    int inc = c0 + c1;
 #pragma unroll
-    for (int q = 0; q < NQ; ++q) {
-      const int t = t0 + (q >> 1), side = q & 1, tok = blockIdx.x * CHUNK_TOKENS + t;
-      live[q] = tok < n_tok;
-      val[q] = make_uint4(0u, 0u, 0u, 0u);
-      meta[q] = 0; base[q] = 0;
-      if (live[q]) {
+    for (int o = 1; o < 32; o <<= 1) {
+      const int n = __shfl_up_sync(0xffffffffu, inc, o);
+      if ((tid & 31) >= o) inc += n;
+    }
+    if ((tid & 31) == 31) s_wtot[tid >> 5] = inc;
+    __syncthreads();
+    int off = 0;
+    for (int w = 0; w < (tid >> 5); ++w) off += s_wtot[w];
+    const int excl = off + inc - (c0 + c1);
+    s_pref[2 * tid] = excl;
+    s_pref[2 * tid + 1] = excl + c0;
+    if (tid == CHUNK_TOKENS - 1) s_pref[2 * CHUNK_TOKENS] = excl + c0 + c1;
+  }
+  __syncthreads();
+  const int total = s_pref[2 * CHUNK_TOKENS];
+  const size_t row_bytes = (size_t)v.d_kv * 2;
+  constexpr int PACK_UNROLL = 4;
+  for (int cb = tid; cb < total; cb += CHUNK_TOKENS * PACK_UNROLL) {
+    uint4 val[PACK_UNROLL];
+    unsigned char* dst[PACK_UNROLL];
+    int keep[PACK_UNROLL];
+#pragma unroll
+    for (int u = 0; u < PACK_UNROLL; ++u) {
+      const int c = cb + u * CHUNK_TOKENS;
+      val[u] = make_uint4(0u, 0u, 0u, 0u);
+      dst[u] = nullptr;
+      keep[u] = 8;
+      if (c < total) {
+        int lo = 0, hi = 2 * CHUNK_TOKENS;                       // largest row q with s_pref[q] <= c
+#pragma unroll
+        for (int it = 0; it < 8; ++it) {
+          const int mid = (lo + hi) >> 1;
+          if (s_pref[mid] <= c) lo = mid; else hi = mid;
+        }
+        const int t = lo >> 1, side = lo & 1, j = c - s_pref[lo];
         const Place p = s_place[side][t];
-        meta[q] = p.slot_cls_r; base[q] = p.base;
-        const int cls = (p.slot_cls_r >> 8) & 0xff, rr = p.slot_cls_r >> 16;
-        if (lane < cls * 8 && lane * 8 < rr)
-          val[q] = __ldg(reinterpret_cast<const uint4*>(reinterpret_cast<const unsigned char*>(side ? V : K) + (size_t)tok * row_bytes) + lane);
+        const int slot = p.slot_cls_r & 0xff, rr = p.slot_cls_r >> 16;
+        keep[u] = rr - j * 8;
+        if (keep[u] > 0)
+          val[u] = __ldg(reinterpret_cast<const uint4*>(reinterpret_cast<const unsigned char*>(side ? V : K) +
+                                                        (size_t)(blockIdx.x * CHUNK_TOKENS + t) * row_bytes) + j);
+        dst[u] = v.blocks + (size_t)(p.base + (j >> 3)) * BLOCK_BYTES + slot * (PANEL * 2) + (j & 7) * 16;
       }
     }
 #pragma unroll
-    for (int q = 0; q < NQ; ++q) {
-      if (!live[q]) continue;
-      const int t = t0 + (q >> 1), side = q & 1, tok = blockIdx.x * CHUNK_TOKENS + t;
-      const int slot = meta[q] & 0xff, cls = (meta[q] >> 8) & 0xff, rr = meta[q] >> 16;
-      if (lane < cls * 8) {
-        uint4 o = val[q];
-        const int keep = rr - lane * 8;                       // elements kept in this chunk
-        if (keep < 8) {
-          unsigned* w = reinterpret_cast<unsigned*>(&o);
+    for (int u = 0; u < PACK_UNROLL; ++u) {
+      if (!dst[u]) continue;
+      uint4 o = val[u];
+      if (keep[u] < 8) {                                         // elements kept in this chunk
+        unsigned* w = reinterpret_cast<unsigned*>(&o);
 #pragma unroll
-          for (int p = 0; p < 4; ++p) {
-            const int left = keep - 2 * p;
-            if (left <= 0) w[p] = 0u;
-            else if (left == 1) w[p] &= 0x0000ffffu;
-          }
+        for (int p = 0; p < 4; ++p) {
+          const int left = keep[u] - 2 * p;
+          if (left <= 0) w[p] = 0u;
+          else if (left == 1) w[p] &= 0x0000ffffu;
         }
-        *reinterpret_cast<uint4*>(v.blocks + (size_t)(base[q] + (lane >> 3)) * BLOCK_BYTES + slot * (PANEL * 2) + (lane & 7) * 16) = o;
       }
-      if (cls > 4) {
-        const unsigned char* src = reinterpret_cast<const unsigned char*>(side ? V : K) + (size_t)tok * row_bytes;
-        pack_row(v, reinterpret_cast<const uint4*>(src), rr, cls, base[q], slot, lane, 32);
-      }
-      if (s_place[side][t].flags & 1) zero_tail(v, cls, base[q], slot, lane);
+      *reinterpret_cast<uint4*>(dst[u]) = o;
     }
   }
 }
@@ -407,7 +408,7 @@ cudaError_t launch_compress_piece(const DevView& v, int layer, const void* K, co
     scan_kernel<<<(v.NK + 7) / 8, 256, 0, st>>>(v, layer, n_chunks);
     alloc_kernel<<<1, 1024, 0, st>>>(v, layer, n_chunks);
   }
-  { ProfScope ps(TWKV_K_PACK, st); pack_kernel<<<n_chunks, CHUNK_TOKENS, 0, st>>>(v, layer, K, V, seq_ids, positions, levels, n_tok); }
+  { ProfScope ps(TWKV_K_PACK, st); pack_kernel<<<n_chunks + v.NK, CHUNK_TOKENS, 0, st>>>(v, layer, K, V, seq_ids, positions, levels, n_tok); }
   count_launch(4);
   return cudaGetLastError();
 }
