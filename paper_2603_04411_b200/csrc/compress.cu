@@ -349,7 +349,7 @@ __global__ void __launch_bounds__(CHUNK_TOKENS) pack_kernel(DevView v, int layer
   __syncthreads();
   const int total = s_pref[2 * CHUNK_TOKENS];
   const size_t row_bytes = (size_t)v.d_kv * 2;
-  constexpr int PACK_UNROLL = 4;
+  constexpr int PACK_UNROLL = 8;
   for (int cb = tid; cb < total; cb += CHUNK_TOKENS * PACK_UNROLL) {
     uint4 val[PACK_UNROLL];
     unsigned char* dst[PACK_UNROLL];
