@@ -23,10 +23,11 @@ namespace twkv {
 // n_cta contiguous pieces of about equal estimated cost, so a CTA of the K-score kernel mostly
 // stays inside one (class, sequence) run.
 __device__ __forceinline__ unsigned ktile_cost(int cls) {
-  // cycles, roughly: per slab max(epilogue, panels * MMA time) + score product; per tile a fixed part
-  const int passes = (cls + 7) / 8, np = (cls + passes - 1) / passes;
-  const int slab = max(700, np * 280 + 250);
-  return 3000u + (unsigned)(passes * 8 * slab);
+  // cycles per tile of the K-score kernel, measured on one-class workloads (8 KV heads): a fixed part (rotation
+  // tables, score read-out, the per-slab epilogue chain) plus a per-panel part; classes above 8 run as two passes
+  if (cls <= 1) return 18000u;
+  if (cls <= 8) return 13300u + 3550u * (unsigned)cls;
+  return 15000u + 4030u * (unsigned)cls;
 }
 
 __global__ void __launch_bounds__(1024) plan_kernel(DevView v, int layer, const int* __restrict__ seq_ids, int n_seq, int n_cta) {
