@@ -118,6 +118,28 @@ def test_project_key_side_only_single_token_and_empty(B):
     B.twkv_projector_destroy(pj)
 
 
+def test_project_benchmark_size_sampled_rows(B):
+    # the launch bench.py times (524 288 tokens, both sides, CTA-pair kernel), checked on sampled rows: the first and last
+    # tile, tile and pair boundaries, and a seeded random draw
+    n, d, dtype = 16 * 32768, 1024, torch.float16
+    ch = workloads.outlier_channels(51, d, 8)
+    ck, cv = workloads.raw_states(52, 4096, d, k_outliers=ch)
+    U_k, U_v = workloads.pca_basis(ck).to(dtype), workloads.pca_basis(cv).to(dtype)
+    xk, xv = workloads.raw_states(53, n, d, device="cuda", k_outliers=ch)
+    xk, xv = xk.to(dtype), xv.to(dtype)
+    ws = torch.empty(B.twkv_projector_required_bytes(d), dtype=torch.uint8, device="cuda")
+    pj = B.twkv_projector_create(U_k.cuda(), U_v.cuda(), ws)
+    ok_, ov_ = torch.empty_like(xk), torch.empty_like(xv)
+    B.twkv_project(pj, xk, xv, ok_, ov_)
+    assert B.twkv_projector_status(pj) == B.TWKV_OK
+    B.twkv_projector_destroy(pj)
+    rng = np.random.default_rng(54)
+    rows = np.unique(np.concatenate([np.arange(0, 130), np.arange(255, 258), np.arange(n - 130, n), rng.integers(0, n, 256)]))
+    idx = torch.from_numpy(rows).cuda()
+    for out, x, U in ((ok_, xk, U_k), (ov_, xv, U_v)):
+        check_side(bits16(out[idx].cpu()), x[idx].cpu(), U, dtype)
+
+
 def test_project_identity_and_permutation_are_exact(B):
     d, n = 1024, 260
     g = torch.Generator().manual_seed(36)
