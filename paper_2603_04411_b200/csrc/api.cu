@@ -117,7 +117,7 @@ static Offsets layout_of(const twkv_config* c, const Dims& d) {
   Offsets o;
   const size_t Ls = c->n_layers, S = c->max_seqs, NT = d.NT, NK = d.NK, Hq = c->n_q_heads;
   o.status = L.alloc(8 * sizeof(int));
-  o.rope_lo = L.alloc((size_t)ROPE_LO * 64 * sizeof(float2));
+  o.rope_lo = L.alloc((size_t)ROPE_SMALL_ROWS * 64 * sizeof(float2));
   o.rope_hi = L.alloc((size_t)ROPE_HI * 64 * sizeof(float2));
   o.n_tiles = L.alloc(Ls * 2 * sizeof(int));
   o.tile_desc = L.alloc(Ls * 2 * NT * sizeof(int4));

@@ -414,27 +414,27 @@ cudaError_t launch_compress_piece(const DevView& v, int layer, const void* K, co
 }
 
 // ------------------------------------------------------------------------------------------
-// Two-level RoPE tables, built once per cache in fp64: angle(pos, i) = pos * base^(-2i/128),
-// pos = hi * 512 + lo.  cos/sin of the sum come from the angle-addition formulas at use.
+// Three-level RoPE tables, built once per cache in fp64: angle(pos, i) = pos * base^(-2i/128),
+// pos = hi * 256 + mid * 16 + lo.  cos/sin of the sum come from the angle-addition formulas at use; the
+// 32 rows of the two small tables fit in shared memory, a tile's rows share a handful of `hi` rows.
 // ------------------------------------------------------------------------------------------
-__global__ void rope_tables_kernel(float2* lo, float2* hi, double base) {
+__global__ void rope_tables_kernel(float2* small, float2* hi, double base) {
   const int i = threadIdx.x;                                   // frequency 0..63
   const int row = blockIdx.x;
   const double theta = pow(base, -2.0 * (double)i / (double)HEAD_DIM);
-  if (row < ROPE_LO) {
-    double s, c;
-    sincos((double)row * theta, &s, &c);
-    lo[row * 64 + i] = make_float2((float)c, (float)s);
+  double s, c;
+  if (row < ROPE_SMALL_ROWS) {
+    sincos(row < 16 ? (double)(row * 16) * theta : (double)(row - 16) * theta, &s, &c);
+    small[row * 64 + i] = make_float2((float)c, (float)s);
   }
   if (row < ROPE_HI) {
-    double s, c;
     sincos((double)row * (double)ROPE_LO * theta, &s, &c);
     hi[row * 64 + i] = make_float2((float)c, (float)s);
   }
 }
 
 cudaError_t launch_rope_tables(const DevView& v, float rope_base, cudaStream_t st) {
-  rope_tables_kernel<<<(ROPE_HI > ROPE_LO ? ROPE_HI : ROPE_LO), 64, 0, st>>>(v.rope_lo, v.rope_hi, (double)rope_base);
+  rope_tables_kernel<<<ROPE_HI, 64, 0, st>>>(v.rope_lo, v.rope_hi, (double)rope_base);
   count_launch();
   return cudaGetLastError();
 }

@@ -38,7 +38,8 @@ constexpr uint32_t TM_SLAB = 0, TM_KR = 256, TM_S = 384;      // column offsets 
 constexpr uint32_t PANEL_BYTES = 16384;
 constexpr int KT_Q_ROWS = 72;                                 // 8 rows per KV head + 8 rows of padding
 constexpr uint32_t KT_Q_PANEL_BYTES = KT_Q_ROWS * 128;        // one 64-wide K panel of the query operand
-constexpr uint32_t KT_ROPE_STAGE_BYTES = 8 * 32 * 8 * 8;      // per epilogue warp: 32 rows x 8 frequencies x (cos, sin)
+constexpr int KT_ROPE_STRIDE = 65;                            // float2 per row of the small RoPE tables in shared memory (64 + 1 against bank conflicts)
+constexpr uint32_t KT_ROPE_STAGE_BYTES = ROPE_SMALL_ROWS * KT_ROPE_STRIDE * 8;
 
 template <bool BF16> __device__ __forceinline__ float kt_to_f32(unsigned short bits) {
   if constexpr (BF16) return __uint_as_float((unsigned)bits << 16);
@@ -61,7 +62,7 @@ kscore_tc_kernel(const __grid_constant__ CUtensorMap map_blocks, const __grid_co
   const uint32_t sB = sA + KT_A_SLOTS * PANEL_BYTES;
   const uint32_t sQ = sB + nb * PANEL_BYTES;
   unsigned char* sQ_ptr = smem_raw + (KT_A_SLOTS + nb) * PANEL_BYTES;
-  float2* sRope = reinterpret_cast<float2*>(sQ_ptr + 2 * KT_Q_PANEL_BYTES);   // [8 epilogue warps][32 rows][8 frequencies]
+  float2* sRope = reinterpret_cast<float2*>(sQ_ptr + 2 * KT_Q_PANEL_BYTES);   // [32 rows][65]: the two small RoPE tables
   unsigned char* tail = sQ_ptr + 2 * KT_Q_PANEL_BYTES + KT_ROPE_STAGE_BYTES;
   const uint32_t bars = smem_addr(tail);
   // barrier map (8 bytes each)
@@ -85,6 +86,7 @@ kscore_tc_kernel(const __grid_constant__ CUtensorMap map_blocks, const __grid_co
   if (warp == 1) tmem_alloc(smem_addr(s_tmem_base), KT_TMEM_COLS);
   for (int i = tid; i < 2 * (int)KT_Q_PANEL_BYTES / 16; i += KT_THREADS)        // padding rows of the query operand stay zero
     reinterpret_cast<uint4*>(sQ_ptr)[i] = make_uint4(0u, 0u, 0u, 0u);
+  for (int i = tid; i < ROPE_SMALL_ROWS * 64; i += KT_THREADS) sRope[(i >> 6) * KT_ROPE_STRIDE + (i & 63)] = v.rope_lo[i];
   fence_proxy_async_smem();
   fence_before_sync();
   __syncthreads();
@@ -245,7 +247,6 @@ kscore_tc_kernel(const __grid_constant__ CUtensorMap map_blocks, const __grid_co
     const float sm_scale = v.sm_scale;
     const int* kpos = v.aux(layer, 0);
     const float2* __restrict__ rope_hi = v.rope_hi;
-    const float2* __restrict__ rope_lo = v.rope_lo;
     uint32_t sc = 0, tcount = 0;
     bool ok = true, slab_ready = false;                            // slab_ready: the next slab's accumulator was already seen complete
     float cs[32], sn[32];
@@ -253,47 +254,24 @@ kscore_tc_kernel(const __grid_constant__ CUtensorMap map_blocks, const __grid_co
 #pragma unroll
     for (int i = 0; i < 4 * REP; ++i) tmax[i] = -INFINITY;
 
-    // cos / sin of (row, frequency): pos = hi * 512 + lo, the two table rows combine by the angle-addition
-    // formulas.  Table rows are read coalesced (8 lanes per row) and handed to the row's lane through a
-    // per-warp staging buffer, 8 frequencies at a time.
+    // cos / sin of (row, frequency): pos = hi * 256 + mid * 16 + lo, the three table rows combine by the angle-addition
+    // formulas.  The mid and lo rows come from shared memory (padded rows: lanes with different rows hit different
+    // banks), the hi row from global memory: a tile's 128 rows share a few hi rows, so those reads stay in L1.
     auto rope_setup = [&](int pos) {
-      float2* stage = sRope + (warp - 2) * 256;
-      const int rs = lane >> 3, t8 = lane & 7;
-      int off_hi[8], off_lo[8];
+      const float2* __restrict__ th = rope_hi + (size_t)((pos >> 8) & (ROPE_HI - 1)) * 64 + hf * 32;
+      const float2* tm = sRope + ((pos >> 4) & 15) * KT_ROPE_STRIDE + hf * 32;
+      const float2* tl = sRope + (16 + (pos & 15)) * KT_ROPE_STRIDE + hf * 32;
 #pragma unroll
-      for (int it = 0; it < 8; ++it) {
-        const int p = __shfl_sync(0xffffffffu, pos, it * 4 + rs);
-        off_hi[it] = ((p >> 9) & (ROPE_HI - 1)) * 64 + hf * 32 + t8;
-        off_lo[it] = (p & (ROPE_LO - 1)) * 64 + hf * 32 + t8;
+      for (int t = 0; t < 32; t += 2) {                        // all hi-row reads in flight before any is used
+        const float4 h = __ldg(reinterpret_cast<const float4*>(th + t));
+        cs[t] = h.x; sn[t] = h.y; cs[t + 1] = h.z; sn[t + 1] = h.w;
       }
 #pragma unroll
-      for (int k2 = 0; k2 < 2; ++k2) {
-        float2 a[2][8], b[2][8];
-#pragma unroll
-        for (int kk = 0; kk < 2; ++kk)
-#pragma unroll
-          for (int it = 0; it < 8; ++it) {
-            a[kk][it] = __ldg(rope_hi + off_hi[it] + (k2 * 2 + kk) * 8);
-            b[kk][it] = __ldg(rope_lo + off_lo[it] + (k2 * 2 + kk) * 8);
-          }
-#pragma unroll
-        for (int kk = 0; kk < 2; ++kk) {
-          const int k = k2 * 2 + kk;
-#pragma unroll
-          for (int it = 0; it < 8; ++it) {
-            const int r = it * 4 + rs;
-            stage[r * 8 + (t8 ^ (r & 7))] = make_float2(a[kk][it].x * b[kk][it].x - a[kk][it].y * b[kk][it].y,
-                                                        a[kk][it].y * b[kk][it].x + a[kk][it].x * b[kk][it].y);
-          }
-          __syncwarp();
-#pragma unroll
-          for (int t = 0; t < 8; ++t) {
-            const float2 c = stage[lane * 8 + (t ^ (lane & 7))];
-            cs[k * 8 + t] = c.x;
-            sn[k * 8 + t] = c.y;
-          }
-          __syncwarp();
-        }
+      for (int t = 0; t < 32; ++t) {
+        const float2 m = tm[t], l = tl[t];
+        const float hx = cs[t] * m.x - sn[t] * m.y, hy = sn[t] * m.x + cs[t] * m.y;
+        cs[t] = hx * l.x - hy * l.y;
+        sn[t] = hy * l.x + hx * l.y;
       }
     };
     // The group's queries as the K-major, 128-byte-swizzled B operand: row 8 g + h, two 64-wide panels.

@@ -79,7 +79,7 @@ twkv_status twkv_project(twkv_projector* p, const void* x_k, const void* x_v, vo
   DeviceGuard g(p->device);
   if (!g.ok) return TWKV_ERR_CUDA;
   const int side0 = x_k ? 0 : 1, n_sides = (x_k ? 1 : 0) + (x_v ? 1 : 0);
-  const bool pairs = p->d % 256 == 0 && n_tok >= PJ_PAIR_MIN_TOKENS && p->sm_count >= 2;
+  const bool pairs = p->d % 256 == 0 && n_tok >= PJ_PAIR_MIN_TOKENS && project_tc_max_pairs(p->sm_count) > 0;
   ProjectMaps maps;
   for (int side = 0; side < 2; ++side) {
     const int src = in[side] ? side : side0;              // an unused side's maps alias the used one (never dereferenced)

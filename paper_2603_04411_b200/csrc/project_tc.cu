@@ -393,39 +393,49 @@ project_tc2_kernel(const __grid_constant__ CUtensorMap map_xk, const __grid_cons
   if (tid == 0 && *abort_flag) atomicCAS(status, 0, misaligned ? TWKV_ERR_DEVICE_CHECK : TWKV_ERR_TIMEOUT);
 }
 
+static void project_pair_config(cudaLaunchConfig_t* cfg, cudaLaunchAttribute* attr, size_t smem, cudaStream_t st) {
+  *cfg = cudaLaunchConfig_t{};
+  cfg->blockDim = dim3(PJ_THREADS);
+  cfg->dynamicSmemBytes = smem;
+  cfg->stream = st;
+  attr->id = cudaLaunchAttributeClusterDimension;
+  attr->val.clusterDim.x = 2; attr->val.clusterDim.y = 1; attr->val.clusterDim.z = 1;
+  cfg->attrs = attr;
+  cfg->numAttrs = 1;
+}
+constexpr size_t PJ2_SMEM = (size_t)PJ2_STAGES * PJ2_STAGE_BYTES + 2 * PJ_PANEL_BYTES + 8 * (2 * PJ2_STAGES + 4) + 16;
+
+// CTA pairs of project_tc2_kernel that can be resident at once on the current device (0: the pair kernel cannot run).
+int project_tc_max_pairs(int sm_count) {
+  static int cached = -1;
+  if (cached >= 0) return cached;
+  if (cudaFuncSetAttribute(project_tc2_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)PJ2_SMEM) != cudaSuccess) { cudaGetLastError(); return cached = 0; }
+  cudaLaunchConfig_t cfg;
+  cudaLaunchAttribute attr;
+  project_pair_config(&cfg, &attr, PJ2_SMEM, nullptr);
+  cfg.gridDim = dim3(sm_count & ~1);
+  int n = 0;
+  if (cudaOccupancyMaxActiveClusters(&n, project_tc2_kernel, &cfg) != cudaSuccess || n < 1) { cudaGetLastError(); n = 0; }
+  return cached = n;
+}
+
 cudaError_t launch_project_tc(const ProjectMaps& maps, int n_tok, int d, int bf16, int side0, int n_sides, int* status,
                               int sm_count, bool pairs, cudaStream_t st) {
   if (n_tok <= 0 || n_sides <= 0) return cudaSuccess;
   if (pairs) {
     // maps.uk / maps.uv must have 128-row boxes here (each CTA loads half of a 256-row slab)
-    const size_t smem = (size_t)PJ2_STAGES * PJ2_STAGE_BYTES + 2 * PJ_PANEL_BYTES + 8 * (2 * PJ2_STAGES + 4) + 16;
-    cudaError_t e = cudaFuncSetAttribute(project_tc2_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    const int max_clusters = project_tc_max_pairs(sm_count);
+    if (max_clusters < 1) return cudaErrorInvalidConfiguration;
+    cudaError_t e = cudaFuncSetAttribute(project_tc2_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)PJ2_SMEM);
     if (e != cudaSuccess) return e;
     const long long n_items = (long long)n_sides * (d / 256) * ((n_tok + 2 * TILE - 1) / (2 * TILE));
-    cudaLaunchConfig_t cfg = {};
-    cfg.blockDim = dim3(PJ_THREADS);
-    cfg.dynamicSmemBytes = smem;
-    cfg.stream = st;
-    cudaLaunchAttribute pair_attr;
-    pair_attr.id = cudaLaunchAttributeClusterDimension;
-    pair_attr.val.clusterDim.x = 2; pair_attr.val.clusterDim.y = 1; pair_attr.val.clusterDim.z = 1;
-    cfg.attrs = &pair_attr;
-    cfg.numAttrs = 1;
-    static int max_clusters = -1;                              // co-resident CTA pairs on this device
-    if (max_clusters < 0) {
-      cfg.gridDim = dim3(sm_count & ~1);
-      int n = 0;
-      if (cudaOccupancyMaxActiveClusters(&n, project_tc2_kernel, &cfg) != cudaSuccess || n < 1) { cudaGetLastError(); n = 0; }
-      max_clusters = n;
-    }
-    if (max_clusters > 0) {
-      const int clusters = n_items < max_clusters ? (int)n_items : max_clusters;
-      cfg.gridDim = dim3(2 * clusters);
-      e = cudaLaunchKernelEx(&cfg, project_tc2_kernel, maps.xk, maps.xv, maps.uk, maps.uv, maps.ok, maps.ov, n_tok, d, bf16, side0, n_sides, status);
-      count_launch();
-      return e != cudaSuccess ? e : cudaGetLastError();
-    }
-    return cudaErrorInvalidConfiguration;
+    cudaLaunchConfig_t cfg;
+    cudaLaunchAttribute attr;
+    project_pair_config(&cfg, &attr, PJ2_SMEM, st);
+    cfg.gridDim = dim3(2 * (n_items < max_clusters ? (int)n_items : max_clusters));
+    e = cudaLaunchKernelEx(&cfg, project_tc2_kernel, maps.xk, maps.xv, maps.uk, maps.uv, maps.ok, maps.ov, n_tok, d, bf16, side0, n_sides, status);
+    count_launch();
+    return e != cudaSuccess ? e : cudaGetLastError();
   }
   const int NS = (d % 256 == 0) ? 256 : 128;
   const size_t smem = (size_t)PJ_STAGES * (PJ_PANEL_BYTES + (size_t)NS * 128) + 2 * PJ_PANEL_BYTES + 8 * (2 * PJ_STAGES + 4) + 16;

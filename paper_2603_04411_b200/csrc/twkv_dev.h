@@ -14,8 +14,9 @@ constexpr int BLOCK_BYTES = TWKV_BLOCK_BYTES;
 constexpr int HEAD_DIM = 128;
 constexpr int CHUNK_TOKENS = 128;           // tokens per compress CTA
 constexpr int PIECE_CHUNKS = TWKV_PIECE_TOKENS / CHUNK_TOKENS;
-constexpr int ROPE_LO = 512;                // pos = hi * 512 + lo
-constexpr int ROPE_HI = 1024;               // positions up to 512 * 1024 - 1
+constexpr int ROPE_LO = 256;                // pos = hi * 256 + mid * 16 + lo
+constexpr int ROPE_HI = 2048;               // positions up to 256 * 2048 - 1
+constexpr int ROPE_SMALL_ROWS = 32;         // rows 0..15: mid * 16 * theta, rows 16..31: lo * theta
 constexpr int MAX_PARTIALS_EXTRA = 320;     // V-side partial slots beyond max_seqs
 constexpr int MAX_PLAN_CTAS = 1024;         // upper bound on the K-score kernel's grid
 
@@ -24,8 +25,8 @@ struct DevView {
   int L, Hq, Hkv, rep, d_kv, NC, S, tmax, NT, TPS, n_blocks, dtype, out_dtype, NK, max_partials;
   float tau, sm_scale;
   int* status;               // [8]: [0] sticky status, [1] next free block, [2] piece_ok, [3] piece flags
-  float2* rope_lo;           // [ROPE_LO][64] (cos, sin) of lo * theta_i
-  float2* rope_hi;           // [ROPE_HI][64] (cos, sin) of hi * 512 * theta_i
+  float2* rope_lo;           // [ROPE_SMALL_ROWS][64] (cos, sin) of mid * 16 * theta_i (rows 0..15) and lo * theta_i (rows 16..31)
+  float2* rope_hi;           // [ROPE_HI][64] (cos, sin) of hi * 256 * theta_i
   unsigned char* blocks;     // n_blocks x 16 KiB
   // per-layer tables (index with the helpers below)
   int* n_tiles;              // [L][2]
@@ -135,6 +136,7 @@ size_t gate_tc_stage_bytes(int n_cta, int d);
 struct ProjectMaps;   // tensor maps of the projection kernel
 cudaError_t launch_project_tc(const ProjectMaps& maps, int n_tok, int d, int bf16, int side0, int n_sides, int* status,
                               int sm_count, bool pairs, cudaStream_t st);
+int project_tc_max_pairs(int sm_count);
 cudaError_t launch_transpose16(const void* in, void* out, int n, cudaStream_t st);
 cudaError_t launch_gate_logits(const DevView& v, const LayerParams& lp, const void* K, const void* V, int n_tok,
                                float* logits, cudaStream_t st);
