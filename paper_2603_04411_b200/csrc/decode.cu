@@ -116,7 +116,8 @@ __global__ void __launch_bounds__(1024) plan_kernel(DevView v, int layer, const 
 }
 
 // ------------------------------------------------------------------------ V accumulate
-constexpr int VA_STAGES = 6;
+constexpr int VA_GROUP = 4;                                        // panels of a tile that share one read of the probabilities
+constexpr int VA_STAGES = 2 * VA_GROUP + 1;                       // the group being read + the group being refilled + one
 
 // One CTA per (query slot, split, head group of <= 32 heads).  A warp owns one 16-head row tile (warp / 8) and the
 // (warp % 8)-th group of 8 columns of every 64-column panel, so every rank class keeps all warps busy and a thread
@@ -176,16 +177,18 @@ vacc_kernel(DevView v, int layer, const int* __restrict__ seq_ids, int n_splits)
     if (p_k < n_mine) { const int4 d = s_desc[p_k & 63]; p_cls = d.y; p_base = d.w; }
   };
   p_load_desc();
+  // this thread's 16-byte chunks of a panel: rows tid / 8 + i * NT / 8 (same row % 8, so one swizzle term), chunk tid % 8
+  const unsigned cp_src_off = (unsigned)tid * 16u;
+  const unsigned cp_dst_off = smem_u32(sV) + (unsigned)(tid >> 3) * 128u + ((((unsigned)tid & 7u) ^ ((unsigned)(tid >> 3) & 7u)) << 4);
+  unsigned p_stage_off = 0;                                         // byte offset of the ring stage the next copy fills
   auto issue = [&]() {
     if (p_k < n_mine) {
-      const unsigned char* src = v.blocks + (size_t)(p_base + p_j) * BLOCK_BYTES;
-      const unsigned dst = smem_u32(sV + (p_n % VA_STAGES) * 16384);
+      const unsigned char* src = v.blocks + (size_t)(p_base + p_j) * BLOCK_BYTES + cp_src_off;
+      const unsigned dst = cp_dst_off + p_stage_off;
 #pragma unroll
-      for (int i = 0; i < 1024 / NT; ++i) {
-        const int c = tid + i * NT, row = c >> 3, ch = c & 7;
-        cp_async16(dst + row * 128 + ((ch ^ (row & 7)) << 4), src + row * 128 + ch * 16);
-      }
+      for (int i = 0; i < 1024 / NT; ++i) cp_async16(dst + i * (NT * 16), src + i * (NT * 16));
       ++p_n;
+      p_stage_off = p_stage_off == (VA_STAGES - 1) * 16384u ? 0u : p_stage_off + 16384u;
       if (++p_j == p_cls) { p_j = 0; ++p_k; p_load_desc(); }
     }
     cp_async_commit();
@@ -194,6 +197,18 @@ vacc_kernel(DevView v, int layer, const int* __restrict__ seq_ids, int n_splits)
 
   const unsigned ones = BF16 ? 0x3f803f80u : 0x3c003c00u;
   int c_n = 0, pbuf = 0;
+  unsigned c_stage_off = 0;                                         // byte offset of the ring stage the next panel is read from
+  int g_prev = 0;                                                   // panels of the previous group: their stages are refilled next
+  // per-lane fragment addresses, fixed for the kernel.  B (V panel, transposed loads): lanes 0-15 address the 16 token
+  // rows of k-step 2 i, lanes 16-31 those of k-step 2 i + 1, so one x4 load brings two k-steps; the swizzle term only
+  // depends on row % 8 = lane % 8.  A (probabilities): row and 16-byte chunk of the lane's 8 x 8 matrix per k-step.
+  const unsigned frag_b_off = smem_u32(sV) + (unsigned)((lane & 15) + (lane >> 4) * 16) * 128u + (((unsigned)cw ^ ((unsigned)lane & 7u)) << 4);
+  unsigned frag_a_off[8];
+  {
+    const int mat = lane >> 3, rin = lane & 7, row = mt * 16 + rin + (mat & 1) * 8;
+#pragma unroll
+    for (int ks = 0; ks < 8; ++ks) frag_a_off[ks] = smem_u32(sP) + (unsigned)row * 256u + ((unsigned)((ks * 2 + (mat >> 1)) ^ rin) << 4);
+  }
   // Scores of a tile are fetched one tile ahead (the V slot's link to its score row two tiles ahead),
   // so the gather's latency hides behind the previous tile's panels.
   const int slot = tid / TPT, part = tid % TPT;                    // TPT threads per token, 8 heads each
@@ -247,39 +262,68 @@ vacc_kernel(DevView v, int layer, const int* __restrict__ seq_ids, int n_splits)
     }
     fetch_scores();                                                // next tile's scores (link fetched one tile ago)
     fetch_link(k + 2);
-    for (int j = 0; j < cls; ++j) {
-      cp_async_wait<VA_STAGES - 2>();
+    // The tile's panels are taken in groups of up to VA_GROUP: the probability fragments of a k-step are read from
+    // shared memory once per group instead of once per panel (they were two thirds of the shared-memory reads, which
+    // bound this kernel).  The stages the previous group occupied are refilled while this one is read.
+    for (int j0 = 0; j0 < cls; j0 += VA_GROUP) {
+      const int g = min(VA_GROUP, cls - j0);
+      // copies still allowed in flight once this group's panels have landed: everything issued after them
+      switch (VA_STAGES - 1 - g_prev - g) {
+        case 0: cp_async_wait<0>(); break;
+        case 1: cp_async_wait<1>(); break;
+        case 2: cp_async_wait<2>(); break;
+        case 3: cp_async_wait<3>(); break;
+        case 4: cp_async_wait<4>(); break;
+        case 5: cp_async_wait<5>(); break;
+        default: cp_async_wait<6>(); break;
+      }
       __syncthreads();
-      issue();
-      const unsigned vBase = smem_u32(sV + (c_n % VA_STAGES) * 16384);
-      const unsigned pBase = smem_u32(sP + pbuf * 8192);
-      ++c_n;
-      // the panel index selects the accumulator at compile time so it stays in registers
-      auto do_panel = [&](auto PJ) {
-        constexpr int pj = decltype(PJ)::value;
-        const int mat = lane >> 3, rin = lane & 7;
+      for (int i = 0; i < g_prev; ++i) issue();
+      g_prev = g;
+      unsigned vAddr[VA_GROUP];
 #pragma unroll
-        for (int ks = 0; ks < 8; ++ks) {
-          unsigned b[2];
-          {
-            const int kr = ks * 16 + (lane & 15);
-            ldsm_x2_t(b, vBase + kr * 128 + ((cw ^ (kr & 7)) << 4));
+      for (int jj = 0; jj < VA_GROUP; ++jj) {
+        unsigned o = c_stage_off + jj * 16384u;
+        if (o >= VA_STAGES * 16384u) o -= VA_STAGES * 16384u;
+        vAddr[jj] = frag_b_off + o;
+      }
+      c_stage_off += (unsigned)g * 16384u;
+      if (c_stage_off >= VA_STAGES * 16384u) c_stage_off -= VA_STAGES * 16384u;
+      c_n += g;
+      const unsigned pOff = (unsigned)pbuf * 8192u;
+      // first panel and group size select the accumulators at compile time so they stay in registers
+      auto do_group = [&](auto J0, auto G) {
+        constexpr int jbase = decltype(J0)::value, gn = decltype(G)::value;
+#pragma unroll
+        for (int k2 = 0; k2 < 4; ++k2) {                           // two k-steps (32 tokens) per iteration
+          unsigned a0[4], a1[4];
+          ldsm_x4(a0, frag_a_off[2 * k2] + pOff);
+          ldsm_x4(a1, frag_a_off[2 * k2 + 1] + pOff);
+#pragma unroll
+          for (int jj = 0; jj < gn; ++jj) {
+            if (jbase + jj < TWKV_MAX_CLASSES) {
+              unsigned b[4];
+              ldsm_x4_t(b, vAddr[jj] + k2 * 4096);
+              mma16816<BF16>(acc[jbase + jj < TWKV_MAX_CLASSES ? jbase + jj : 0], a0, b[0], b[1]);
+              mma16816<BF16>(acc[jbase + jj < TWKV_MAX_CLASSES ? jbase + jj : 0], a1, b[2], b[3]);
+            }
           }
-          unsigned a[4];
-          const int row = mt * 16 + rin + (mat & 1) * 8, kc = ks * 2 + (mat >> 1);
-          ldsm_x4(a, pBase + row * 256 + ((kc ^ (row & 7)) << 4));
-          mma16816<BF16>(acc[pj], a, b[0], b[1]);
-          if (pj == 0 && cw == 0) mma16816<BF16>(accl, a, ones, ones);
+          if (jbase == 0 && cw == 0) { mma16816<BF16>(accl, a0, ones, ones); mma16816<BF16>(accl, a1, ones, ones); }
         }
       };
-      switch (j) {
-#define TWKV_PANEL_CASE(N) case N: do_panel(std::integral_constant<int, N>{}); break;
-        TWKV_PANEL_CASE(0) TWKV_PANEL_CASE(1) TWKV_PANEL_CASE(2) TWKV_PANEL_CASE(3)
-        TWKV_PANEL_CASE(4) TWKV_PANEL_CASE(5) TWKV_PANEL_CASE(6) TWKV_PANEL_CASE(7)
-        TWKV_PANEL_CASE(8) TWKV_PANEL_CASE(9) TWKV_PANEL_CASE(10) TWKV_PANEL_CASE(11)
-        TWKV_PANEL_CASE(12) TWKV_PANEL_CASE(13) TWKV_PANEL_CASE(14) TWKV_PANEL_CASE(15)
-#undef TWKV_PANEL_CASE
-        default: break;
+      auto by_size = [&](auto J0) {
+        switch (g) {
+          case 1: do_group(J0, std::integral_constant<int, 1>{}); break;
+          case 2: do_group(J0, std::integral_constant<int, 2>{}); break;
+          case 3: do_group(J0, std::integral_constant<int, 3>{}); break;
+          default: do_group(J0, std::integral_constant<int, 4>{}); break;
+        }
+      };
+      switch (j0) {
+        case 0: by_size(std::integral_constant<int, 0>{}); break;
+        case 4: by_size(std::integral_constant<int, 4>{}); break;
+        case 8: by_size(std::integral_constant<int, 8>{}); break;
+        default: by_size(std::integral_constant<int, 12>{}); break;
       }
     }
     pbuf ^= 1;
