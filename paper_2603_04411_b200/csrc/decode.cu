@@ -246,8 +246,9 @@ vacc_kernel(DevView v, int layer, const int* __restrict__ seq_ids, int n_splits)
   for (int k = 0; k < n_mine; ++k) {
     if ((k & 15) == 0) refill(k + 48);                             // used from tile k + 16 on; many barriers in between
     const int cls = s_desc[k & 63].y;
-    // probabilities of this tile's tokens: p = exp(s - max), rounded to the storage type
-    __syncthreads();
+    // probabilities of this tile's tokens: p = exp(s - max), rounded to the storage type.  No barrier is needed here:
+    // the buffer was last read two tiles ago, and every warp has since passed a group barrier of the previous tile;
+    // the first group barrier below publishes the new values.
     {
       unsigned char* P = sP + pbuf * 8192;
 #pragma unroll
