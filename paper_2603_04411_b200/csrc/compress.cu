@@ -201,22 +201,25 @@ __global__ void __launch_bounds__(1024) alloc_kernel(DevView v, int layer, int n
     off_b += nnew * cls;
   }
   __syncthreads();
-  // tile lists: K per class (ascending sequence), V per sequence (ascending class)
-  if (tid < v.NC) {
+  // tile lists: K per class (ascending sequence), V per sequence (ascending class); one warp per list, the lanes
+  // write a key's run of consecutive tile ids together
+  const int warp = tid >> 5, lane = tid & 31;
+  if (warp < v.NC) {
     int* cnt = v.kcc(layer);
-    int* list = v.kct(layer) + (size_t)tid * v.NT;
-    int run = cnt[tid];
+    int* list = v.kct(layer) + (size_t)warp * v.NT;
+    int run = cnt[warp];
     for (int s = 0; s < v.S; ++s) {
-      const int k = s * v.NC + tid;
+      const int k = s * v.NC + warp;
       const int c = v.key_cnt[k], old = v.key_old_fill[k];
       const int nnew = ceil_div(old + c, TILE) - ceil_div(old, TILE);
       const int first = v.key_first_id[k];
-      for (int j = 0; j < nnew; ++j) list[run + j] = first + j;
+      for (int j = lane; j < nnew; j += 32) list[run + j] = first + j;
       run += nnew;
     }
-    cnt[tid] = run;
+    __syncwarp();
+    if (lane == 0) cnt[warp] = run;
   }
-  for (int s = tid; s < v.S; s += 1024) {
+  for (int s = warp; s < v.S; s += 32) {
     int* list = v.svt(layer) + (size_t)s * v.TPS;
     int run = v.svc(layer)[s];
     int add = 0;
@@ -225,12 +228,15 @@ __global__ void __launch_bounds__(1024) alloc_kernel(DevView v, int layer, int n
       const int cn = v.key_cnt[k], old = v.key_old_fill[k];
       const int nnew = ceil_div(old + cn, TILE) - ceil_div(old, TILE);
       const int first = v.key_first_id[k];
-      for (int j = 0; j < nnew; ++j) list[run + j] = first + j;
+      for (int j = lane; j < nnew; j += 32) list[run + j] = first + j;
       run += nnew;
       add += v.key_cnt[s * v.NC + c];
     }
-    v.svc(layer)[s] = run;
-    stok[s] += add;
+    __syncwarp();
+    if (lane == 0) {
+      v.svc(layer)[s] = run;
+      stok[s] += add;
+    }
   }
   if (tid == 0) {
     v.status[1] = next_block + tot_b;
