@@ -369,12 +369,24 @@ merge_kernel(DevView v, const unsigned short* __restrict__ Uinv_v, int n_splits,
     sInvL[tid] = l > 0.f ? 1.f / l : 0.f;
   }
   __syncthreads();
-  for (int i = tid; i < REP * d_kv; i += MG_THREADS) {
-    const int hh = i / d_kv, j = i - hh * d_kv;
-    const float* p = v.part_acc + (((size_t)qs * n_splits) * Hq + g * REP + hh) * d_kv + j;
-    float a = 0.f;
-    for (int s = 0; s < n_splits; ++s) a += p[(size_t)s * Hq * d_kv];
-    sAcc[i] = a * sInvL[hh];
+  // split sums in split order; four elements per thread at a time so that four reads per split are in flight
+  for (int i0 = tid; i0 < REP * d_kv; i0 += 4 * MG_THREADS) {
+    const float* p[4];
+    float a[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      const int i = min(i0 + u * MG_THREADS, REP * d_kv - 1), hh = i / d_kv, j = i - hh * d_kv;
+      p[u] = v.part_acc + (((size_t)qs * n_splits) * Hq + g * REP + hh) * d_kv + j;
+    }
+    for (int s = 0; s < n_splits; ++s) {
+#pragma unroll
+      for (int u = 0; u < 4; ++u) a[u] += __ldg(p[u] + (size_t)s * Hq * d_kv);
+    }
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      const int i = i0 + u * MG_THREADS;
+      if (i < REP * d_kv) sAcc[i] = a[u] * sInvL[i / d_kv];
+    }
   }
   __syncthreads();
   const int dp = tid & 63, jg = tid >> 6;
@@ -383,12 +395,12 @@ merge_kernel(DevView v, const unsigned short* __restrict__ Uinv_v, int n_splits,
 #pragma unroll
   for (int h = 0; h < 8; ++h) { o[h][0] = 0.f; o[h][1] = 0.f; }
   const unsigned* ucol = reinterpret_cast<const unsigned*>(Uinv_v + g * HEAD_DIM) + dp;    // two 16-bit columns per load
-  for (int jb = 0; jb < jn; jb += 8) {
-    unsigned u[8];
+  for (int jb = 0; jb < jn; jb += 16) {                // jn is a multiple of 16 (d_kv a multiple of 128)
+    unsigned u[16];
 #pragma unroll
-    for (int t = 0; t < 8; ++t) u[t] = __ldg(ucol + (size_t)(j0 + jb + t) * (d_kv / 2));
+    for (int t = 0; t < 16; ++t) u[t] = __ldg(ucol + (size_t)(j0 + jb + t) * (d_kv / 2));
 #pragma unroll
-    for (int t = 0; t < 8; ++t) {
+    for (int t = 0; t < 16; ++t) {
       const float u0 = to_f32<BF16>((unsigned short)(u[t] & 0xffffu)), u1 = to_f32<BF16>((unsigned short)(u[t] >> 16));
 #pragma unroll
       for (int h = 0; h < 8; ++h)
