@@ -58,45 +58,62 @@ __global__ void __launch_bounds__(1024) plan_kernel(DevView v, int layer, const 
   const int4* desc = v.desc(layer, 0);
   const int* kct = v.kct(layer);
   const int n_all = s_cls_off[v.NC];
-  for (int f0 = 0; f0 < n_all; f0 += 1024) {
-    const int f = f0 + tid;
-    int4 e = make_int4(0, 0, 0, -1);
-    if (f < n_all) {
-      int k = 0;
-      while (f >= s_cls_off[k + 1]) ++k;
-      const int cls = v.NC - k;
-      const int tile = kct[(size_t)(cls - 1) * v.NT + (f - s_cls_off[k])];
-      const int4 d = desc[tile];
-      e = make_int4(tile, d.y | (d.z << 8), d.w, v.qslot[d.x]);
-    }
-    const unsigned keep = e.w >= 0 ? 1u : 0u;
-    const unsigned cost = keep ? ktile_cost(e.y & 0xff) : 0u;
-    unsigned ik = keep, ic = cost;                              // inclusive scans inside the warp
+  constexpr int PL_BATCH = 4;                                     // list chunks of 1024 whose table reads are issued together
+  for (int f0 = 0; f0 < n_all; f0 += 1024 * PL_BATCH) {
+    // the three dependent reads (tile id -> descriptor -> query slot) of PL_BATCH chunks go out level by level
+    int tile[PL_BATCH], cls_[PL_BATCH];
+    int4 d[PL_BATCH];
+    int4 ent[PL_BATCH];
 #pragma unroll
-    for (int o = 1; o < 32; o <<= 1) {
-      const unsigned a = __shfl_up_sync(0xffffffffu, ik, o), b = __shfl_up_sync(0xffffffffu, ic, o);
-      if (lane >= o) { ik += a; ic += b; }
+    for (int u = 0; u < PL_BATCH; ++u) {
+      const int f = f0 + u * 1024 + tid;
+      tile[u] = -1; cls_[u] = 0;
+      if (f < n_all) {
+        int k = 0;
+        while (f >= s_cls_off[k + 1]) ++k;
+        cls_[u] = v.NC - k;
+        tile[u] = kct[(size_t)(cls_[u] - 1) * v.NT + (f - s_cls_off[k])];
+      }
     }
-    if (lane == 31) { s_wsum[warp][0] = ik; s_wsum[warp][1] = ic; }
-    __syncthreads();
-    if (warp == 0) {
-      unsigned wk = s_wsum[lane][0], wc = s_wsum[lane][1];
+#pragma unroll
+    for (int u = 0; u < PL_BATCH; ++u) d[u] = tile[u] >= 0 ? desc[tile[u]] : make_int4(0, 0, 0, 0);
+#pragma unroll
+    for (int u = 0; u < PL_BATCH; ++u)
+      ent[u] = tile[u] >= 0 ? make_int4(tile[u], d[u].y | (d[u].z << 8), d[u].w, v.qslot[d[u].x]) : make_int4(0, 0, 0, -1);
+#pragma unroll
+    for (int u = 0; u < PL_BATCH; ++u) {
+      if (f0 + u * 1024 >= n_all) break;                         // uniform across the CTA
+      const int4 e = ent[u];
+      const unsigned keep = e.w >= 0 ? 1u : 0u;
+      const unsigned cost = keep ? ktile_cost(e.y & 0xff) : 0u;
+      unsigned ik = keep, ic = cost;                              // inclusive scans inside the warp
 #pragma unroll
       for (int o = 1; o < 32; o <<= 1) {
-        const unsigned a = __shfl_up_sync(0xffffffffu, wk, o), b = __shfl_up_sync(0xffffffffu, wc, o);
-        if (lane >= o) { wk += a; wc += b; }
+        const unsigned a = __shfl_up_sync(0xffffffffu, ik, o), b = __shfl_up_sync(0xffffffffu, ic, o);
+        if (lane >= o) { ik += a; ic += b; }
       }
-      s_wsum[lane][0] = wk; s_wsum[lane][1] = wc;               // inclusive over warps
+      if (lane == 31) { s_wsum[warp][0] = ik; s_wsum[warp][1] = ic; }
+      __syncthreads();
+      if (warp == 0) {
+        unsigned wk = s_wsum[lane][0], wc = s_wsum[lane][1];
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+          const unsigned a = __shfl_up_sync(0xffffffffu, wk, o), b = __shfl_up_sync(0xffffffffu, wc, o);
+          if (lane >= o) { wk += a; wc += b; }
+        }
+        s_wsum[lane][0] = wk; s_wsum[lane][1] = wc;               // inclusive over warps
+      }
+      __syncthreads();
+      const unsigned pk = s_base[0] + (warp ? s_wsum[warp - 1][0] : 0u) + ik - keep;      // exclusive position
+      const unsigned pc = s_base[1] + (warp ? s_wsum[warp - 1][1] : 0u) + ic - cost;      // exclusive cost prefix
+      if (keep) { v.klist[pk] = e; v.klist_cost[pk] = pc; }
+      __syncthreads();
+      if (tid == 0) { s_base[0] += s_wsum[31][0]; s_base[1] += s_wsum[31][1]; }
+      __syncthreads();
     }
-    __syncthreads();
-    const unsigned pk = s_base[0] + (warp ? s_wsum[warp - 1][0] : 0u) + ik - keep;      // exclusive position
-    const unsigned pc = s_base[1] + (warp ? s_wsum[warp - 1][1] : 0u) + ic - cost;      // exclusive cost prefix
-    if (keep) { v.klist[pk] = e; v.klist_cost[pk] = pc; }
-    __syncthreads();
-    if (tid == 0) { s_base[0] += s_wsum[31][0]; s_base[1] += s_wsum[31][1]; }
-    __syncthreads();
   }
-  // cut points: piece b starts at the first entry whose cost prefix reaches b / n_cta of the total
+  // cut points: piece b starts at the entry whose cost interval [lo, hi) holds b / n_cta of the total, i.e. the last
+  // entry with lo * n_cta <= b * total (64-bit products, no division); a binary search per piece
   const unsigned n_keep = s_base[0];
   const unsigned long long total = s_base[1];
   if (tid == 0) { *v.klist_count = (int)n_keep; v.cta_start[n_cta] = (int)n_keep; }
@@ -104,14 +121,14 @@ __global__ void __launch_bounds__(1024) plan_kernel(DevView v, int layer, const 
     for (int b = tid; b < n_cta; b += blockDim.x) v.cta_start[b] = 0;
     return;
   }
-  for (unsigned i = tid; i < n_keep; i += blockDim.x) {
-    const unsigned long long lo = v.klist_cost[i];
-    const unsigned long long hi = i + 1 < n_keep ? v.klist_cost[i + 1] : total;
-    // pieces b with lo <= b * total / n_cta < hi, i.e. b in [ceil(lo n / T), ceil(hi n / T) - 1]
-    const int b0 = (int)((lo * n_cta + total - 1) / total);
-    int b1 = (int)((hi * n_cta + total - 1) / total) - 1;
-    if (b1 > n_cta - 1) b1 = n_cta - 1;
-    for (int b = b0; b <= b1; ++b) v.cta_start[b] = (int)i;
+  for (int b = tid; b < n_cta; b += blockDim.x) {
+    const unsigned long long key = (unsigned long long)b * total;
+    unsigned lo = 0, hi = n_keep;                                   // invariant: cost[lo] * n_cta <= key (cost[0] = 0)
+    while (hi - lo > 1) {
+      const unsigned mid = (lo + hi) >> 1;
+      if ((unsigned long long)v.klist_cost[mid] * (unsigned long long)n_cta <= key) lo = mid; else hi = mid;
+    }
+    v.cta_start[b] = (int)lo;
   }
 }
 
