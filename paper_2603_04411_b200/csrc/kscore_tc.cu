@@ -41,6 +41,18 @@ constexpr uint32_t KT_Q_PANEL_BYTES = KT_Q_ROWS * 128;        // one 64-wide K p
 constexpr int KT_ROPE_STRIDE = 65;                            // float2 per row of the small RoPE tables in shared memory (64 + 1 against bank conflicts)
 constexpr uint32_t KT_ROPE_STAGE_BYTES = ROPE_SMALL_ROWS * KT_ROPE_STRIDE * 8;
 
+// Packed fp32 pairs (two lanes per 64-bit register, one instruction for both): the rotation is issue-bound.
+__device__ __forceinline__ uint64_t f2_pack(float a, float b) { uint64_t r; asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(a), "f"(b)); return r; }
+__device__ __forceinline__ uint64_t f2_pack_bits(uint32_t a, uint32_t b) { uint64_t r; asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "r"(a), "r"(b)); return r; }
+__device__ __forceinline__ uint64_t f2_mul(uint64_t a, uint64_t b) { uint64_t r; asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b)); return r; }
+__device__ __forceinline__ uint64_t f2_sub(uint64_t a, uint64_t b) { uint64_t r; asm("sub.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(a), "l"(b)); return r; }
+__device__ __forceinline__ uint64_t f2_fma(uint64_t a, uint64_t b, uint64_t c) { uint64_t r; asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(r) : "l"(a), "l"(b), "l"(c)); return r; }
+__device__ __forceinline__ uint32_t f2_to_f16x2_sat(uint64_t v) {       // (lo lane -> bits 0..15), saturating
+  uint32_t d;
+  asm("{\n\t.reg .f32 a, b;\n\tmov.b64 {a, b}, %1;\n\tcvt.rn.satfinite.f16x2.f32 %0, b, a;\n\t}" : "=r"(d) : "l"(v));
+  return d;
+}
+
 template <bool BF16> __device__ __forceinline__ float kt_to_f32(unsigned short bits) {
   if constexpr (BF16) return __uint_as_float((unsigned)bits << 16);
   else return __half2float(__ushort_as_half(bits));
@@ -249,7 +261,8 @@ kscore_tc_kernel(const __grid_constant__ CUtensorMap map_blocks, const __grid_co
     const float2* __restrict__ rope_hi = v.rope_hi;
     uint32_t sc = 0, tcount = 0;
     bool ok = true, slab_ready = false;                            // slab_ready: the next slab's accumulator was already seen complete
-    float cs[32], sn[32];
+    float cs[32], sn[32];                                         // scratch of rope_setup
+    uint64_t cs2[16], sn2[16];                                    // the tile's rotation factors, frequencies (2 t, 2 t + 1) packed
     float tmax[4 * REP];                                            // running maxima of this thread's heads for the current query slot
 #pragma unroll
     for (int i = 0; i < 4 * REP; ++i) tmax[i] = -INFINITY;
@@ -273,6 +286,8 @@ kscore_tc_kernel(const __grid_constant__ CUtensorMap map_blocks, const __grid_co
         cs[t] = hx * l.x - hy * l.y;
         sn[t] = hy * l.x + hx * l.y;
       }
+#pragma unroll
+      for (int t = 0; t < 16; ++t) { cs2[t] = f2_pack(cs[2 * t], cs[2 * t + 1]); sn2[t] = f2_pack(sn[2 * t], sn[2 * t + 1]); }
     };
     // The group's queries as the K-major, 128-byte-swizzled B operand: row 8 g + h, two 64-wide panels.
     // Only called when no score product that reads the rows can still be in flight.
@@ -309,9 +324,9 @@ kscore_tc_kernel(const __grid_constant__ CUtensorMap map_blocks, const __grid_co
         fence_after_sync();
         const uint32_t slab = lane_addr + TM_SLAB + buf * 128 + hf * 32;
         const uint32_t kr = lane_addr + TM_KR + buf * 64 + hf * 16;
-        float lo[32], hi[32];
-        tmem_ld32(slab, reinterpret_cast<uint32_t*>(lo));
-        tmem_ld32(slab + 64, reinterpret_cast<uint32_t*>(hi));
+        uint32_t lo[32], hi[32];
+        tmem_ld32(slab, lo);
+        tmem_ld32(slab + 64, hi);
         const bool kr_probe = mbar_try(kr_empty + 8 * buf, par ^ 1u);
         tmem_ld_wait();
         fence_before_sync();
@@ -319,9 +334,10 @@ kscore_tc_kernel(const __grid_constant__ CUtensorMap map_blocks, const __grid_co
         if (lane == 0) mbar_arrive(slab_empty + 8 * buf);                    // the slab accumulator is free for slab n + 2
         uint32_t p1[16], p2[16];
 #pragma unroll
-        for (int t = 0; t < 32; t += 2) {
-          p1[t >> 1] = pack_f16x2_sat(lo[t] * cs[t] - hi[t] * sn[t], lo[t + 1] * cs[t + 1] - hi[t + 1] * sn[t + 1]);
-          p2[t >> 1] = pack_f16x2_sat(hi[t] * cs[t] + lo[t] * sn[t], hi[t + 1] * cs[t + 1] + lo[t + 1] * sn[t + 1]);
+        for (int t = 0; t < 16; ++t) {
+          const uint64_t L = f2_pack_bits(lo[2 * t], lo[2 * t + 1]), H = f2_pack_bits(hi[2 * t], hi[2 * t + 1]);
+          p1[t] = f2_to_f16x2_sat(f2_sub(f2_mul(L, cs2[t]), f2_mul(H, sn2[t])));      // lo cos - hi sin
+          p2[t] = f2_to_f16x2_sat(f2_fma(L, sn2[t], f2_mul(H, cs2[t])));              // hi cos + lo sin
         }
         if (!__all_sync(0xffffffffu, kr_probe) && !(ok = __all_sync(0xffffffffu, mbar_wait(kr_empty + 8 * buf, par ^ 1u, abort_flag)))) break;
         fence_after_sync();
