@@ -376,14 +376,17 @@ constexpr int MG_JGROUPS = MG_THREADS / 64;
 
 template <bool BF16>
 __global__ void __launch_bounds__(MG_THREADS)
-merge_kernel(DevView v, const unsigned short* __restrict__ Uinv_v, int n_splits, void* __restrict__ out) {
-  extern __shared__ float sAcc[];                    // [REP][d_kv] normalised spectral accumulators, then [MG_JGROUPS][REP][128]
+merge_kernel(DevView v, const unsigned short* __restrict__ Uinv_v, int n_splits, int hp, void* __restrict__ out) {
+  extern __shared__ float sAcc[];                    // [hp][d_kv] normalised spectral accumulators, then [MG_JGROUPS][hp][128]
   __shared__ float sInvL[8];
-  const int qs = blockIdx.x, g = blockIdx.y, tid = threadIdx.x;
-  const int Hq = v.Hq, d_kv = v.d_kv, REP = v.rep;
+  // blockIdx.y = KV head g and which hp of its query heads (hp divides the group size; small batches use hp < group
+  // size so that the grid still fills the device)
+  const int qs = blockIdx.x, parts = v.rep / hp, g = blockIdx.y / parts, tid = threadIdx.x;
+  const int Hq = v.Hq, d_kv = v.d_kv, REP = hp;
+  const int head0 = g * v.rep + (blockIdx.y % parts) * hp;      // first query head of this CTA
   if (tid < REP) {
     float l = 0.f;
-    for (int s = 0; s < n_splits; ++s) l += v.part_l[((size_t)qs * n_splits + s) * Hq + g * REP + tid];
+    for (int s = 0; s < n_splits; ++s) l += v.part_l[((size_t)qs * n_splits + s) * Hq + head0 + tid];
     sInvL[tid] = l > 0.f ? 1.f / l : 0.f;
   }
   __syncthreads();
@@ -394,7 +397,7 @@ merge_kernel(DevView v, const unsigned short* __restrict__ Uinv_v, int n_splits,
 #pragma unroll
     for (int u = 0; u < 4; ++u) {
       const int i = min(i0 + u * MG_THREADS, REP * d_kv - 1), hh = i / d_kv, j = i - hh * d_kv;
-      p[u] = v.part_acc + (((size_t)qs * n_splits) * Hq + g * REP + hh) * d_kv + j;
+      p[u] = v.part_acc + (((size_t)qs * n_splits) * Hq + head0 + hh) * d_kv + j;
     }
     for (int s = 0; s < n_splits; ++s) {
 #pragma unroll
@@ -440,7 +443,7 @@ merge_kernel(DevView v, const unsigned short* __restrict__ Uinv_v, int n_splits,
 #pragma unroll
     for (int k = 0; k < MG_JGROUPS; ++k) val += red[k * REP * 128 + i];        // fixed order
     const int h = i >> 7, dc = i & 127;
-    const size_t oi = ((size_t)qs * Hq + g * REP + h) * HEAD_DIM + dc;
+    const size_t oi = ((size_t)qs * Hq + head0 + h) * HEAD_DIM + dc;
     if (v.out_dtype == TWKV_F32) reinterpret_cast<float*>(out)[oi] = val;
     else if (v.out_dtype == TWKV_BF16) reinterpret_cast<unsigned short*>(out)[oi] = from_f32<true>(val);
     else reinterpret_cast<unsigned short*>(out)[oi] = from_f32<false>(val);
@@ -470,11 +473,14 @@ static cudaError_t launch_decode_t(const DevView& v, int layer, const LayerParam
     ProfScope ps(TWKV_K_VACC, st);
     vacc_kernel<BF16, 2><<<vgrid, 512, va_smem, st>>>(v, layer, seq_ids, n_splits);
   }
-  const size_t mg_a = (size_t)v.rep * v.d_kv * 4, mg_b = (size_t)MG_JGROUPS * v.rep * 128 * 4;
+  // query heads per merge CTA: the whole group when the batch fills the device, fewer (a divisor) for small batches
+  int hp = v.rep;
+  while (hp % 2 == 0 && 2 * n_seq * v.Hkv * (v.rep / hp) < sm_count) hp /= 2;
+  const size_t mg_a = (size_t)hp * v.d_kv * 4, mg_b = (size_t)MG_JGROUPS * hp * 128 * 4;
   const size_t mg_smem = mg_a > mg_b ? mg_a : mg_b;
   {
     ProfScope ps(TWKV_K_MERGE, st);
-    merge_kernel<BF16><<<dim3(n_seq, v.Hkv), MG_THREADS, mg_smem, st>>>(v, reinterpret_cast<const unsigned short*>(lp.Uinv_v), n_splits, out);
+    merge_kernel<BF16><<<dim3(n_seq, v.Hkv * (v.rep / hp)), MG_THREADS, mg_smem, st>>>(v, reinterpret_cast<const unsigned short*>(lp.Uinv_v), n_splits, hp, out);
   }
   count_launch(4);
   return cudaGetLastError();

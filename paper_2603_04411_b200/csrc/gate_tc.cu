@@ -494,11 +494,9 @@ cudaError_t launch_gate_ranks_tc(const DevView& v, const GateMaps& maps, const L
 }
 
 // CTA pairs of gate_tc2_kernel that can be resident at once on the current device (0: the pair kernel cannot run).
-int gate_tc_max_pairs(int sm_count) {
-  static int cached = -1;
-  if (cached >= 0) return cached;
+static int gate_tc_query_pairs(int sm_count) {
   const size_t smem = (size_t)GT2_STAGES * 2 * GT_PANEL_BYTES + TILE * GT_BLK_STRIDE * sizeof(float2) + 8 * (2 * GT2_STAGES + 5) + 16;
-  if (cudaFuncSetAttribute(gate_tc2_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) { cudaGetLastError(); return cached = 0; }
+  if (cudaFuncSetAttribute(gate_tc2_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) { cudaGetLastError(); return 0; }
   cudaLaunchConfig_t cfg = {};
   cfg.blockDim = dim3(GT_THREADS);
   cfg.dynamicSmemBytes = smem;
@@ -510,7 +508,11 @@ int gate_tc_max_pairs(int sm_count) {
   cfg.numAttrs = 1;
   int n = 0;
   if (cudaOccupancyMaxActiveClusters(&n, gate_tc2_kernel, &cfg) != cudaSuccess || n < 1) { cudaGetLastError(); n = 0; }
-  return cached = n;
+  return n;
+}
+int gate_tc_max_pairs(int sm_count) {
+  static const int cached = gate_tc_query_pairs(sm_count);     // queried once per process (thread-safe initialisation)
+  return cached;
 }
 
 }  // namespace twkv

@@ -406,17 +406,19 @@ static void project_pair_config(cudaLaunchConfig_t* cfg, cudaLaunchAttribute* at
 constexpr size_t PJ2_SMEM = (size_t)PJ2_STAGES * PJ2_STAGE_BYTES + 2 * PJ_PANEL_BYTES + 8 * (2 * PJ2_STAGES + 4) + 16;
 
 // CTA pairs of project_tc2_kernel that can be resident at once on the current device (0: the pair kernel cannot run).
-int project_tc_max_pairs(int sm_count) {
-  static int cached = -1;
-  if (cached >= 0) return cached;
-  if (cudaFuncSetAttribute(project_tc2_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)PJ2_SMEM) != cudaSuccess) { cudaGetLastError(); return cached = 0; }
+static int project_tc_query_pairs(int sm_count) {
+  if (cudaFuncSetAttribute(project_tc2_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)PJ2_SMEM) != cudaSuccess) { cudaGetLastError(); return 0; }
   cudaLaunchConfig_t cfg;
   cudaLaunchAttribute attr;
   project_pair_config(&cfg, &attr, PJ2_SMEM, nullptr);
   cfg.gridDim = dim3(sm_count & ~1);
   int n = 0;
   if (cudaOccupancyMaxActiveClusters(&n, project_tc2_kernel, &cfg) != cudaSuccess || n < 1) { cudaGetLastError(); n = 0; }
-  return cached = n;
+  return n;
+}
+int project_tc_max_pairs(int sm_count) {
+  static const int cached = project_tc_query_pairs(sm_count);  // queried once per process (thread-safe initialisation)
+  return cached;
 }
 
 cudaError_t launch_project_tc(const ProjectMaps& maps, int n_tok, int d, int bf16, int side0, int n_sides, int* status,
