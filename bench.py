@@ -321,6 +321,15 @@ def run_ours(args):
             "kernels": kernels,
         }
         extra["frac_of_binding_bound"] = extra["binding_bound_ms"] / dec_ms
+        # the two HBM-side kernels against the measured copy bandwidth (algorithmic bytes, CUDA-event launch times)
+        if extra["vacc_gbs"]:
+            extra["roofline_vacc"] = {"kernel": "vacc_kernel (softmax weights + absorbed V accumulate)", "bound": "hbm", "achieved": extra["vacc_gbs"],
+                                      "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": extra["vacc_gbs"] / peaks["hbm_gbs"],
+                                      "bytes": "stored V rows + 4 Hq bytes of scores per token"}
+        if extra["pack_gbs"]:
+            extra["roofline_pack"] = {"kernel": "pack_kernel (truncate + pack)", "bound": "hbm", "achieved": extra["pack_gbs"],
+                                      "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": extra["pack_gbs"] / peaks["hbm_gbs"],
+                                      "bytes": "2 (r_K + r_V) read + class-padded rows written per token"}
         # the step before the path (Eq. 1, x~ = x U on the device), timed on its own: not part of `value` or `ms_per_step`.
         # Operand values do not change a dense product's time, so the resident states and bases stand in for x and U.
         ws = torch.empty(B.twkv_projector_required_bytes(D_KV), dtype=torch.uint8, device=dev)
