@@ -140,6 +140,8 @@ constexpr int VA_STAGES = 2 * VA_GROUP + 1;                       // the group b
 // One CTA per (query slot, split, head group of <= 32 heads).  A warp owns one 16-head row tile (warp / 8) and the
 // (warp % 8)-th group of 8 columns of every 64-column panel, so every rank class keeps all warps busy and a thread
 // carries 64 accumulators.  NWG = 1 (up to 16 heads, 8 warps) or 2 (up to 32 heads, 16 warps).
+// Panels arrive through a ring of cp.async stages; a tile's panels are consumed in groups of up to VA_GROUP that
+// share one ldmatrix read of the tile's probability fragments (shared-memory reads bound this kernel).
 template <bool BF16, int NWG>
 __global__ void __launch_bounds__(256 * NWG, 1)
 vacc_kernel(DevView v, int layer, const int* __restrict__ seq_ids, int n_splits) {
