@@ -249,13 +249,30 @@ def run_ours(args):
         d_xk, d_xv = torch.empty_like(li.xt_k), torch.empty_like(li.xt_v)
         d_sid, d_pos, d_q = torch.empty_like(li.seq_ids), torch.empty_like(li.positions), torch.empty_like(li.q)
 
+        # The states go up in pieces of the library's own piece size on a copy stream; the compress call of a piece starts
+        # when its copy has landed, so copies and kernels overlap (the cache ends up the same as after one call).
+        copy_stream = torch.cuda.Stream(device=dev)
+        piece = B.PIECE_TOKENS
+        n_pieces = (n_tok + piece - 1) // piece
+        landed = [torch.cuda.Event() for _ in range(n_pieces)]
+        step_done = torch.cuda.Event()
+
         def e2e_step():
-            d_xk.copy_(h_xk, non_blocking=True); d_xv.copy_(h_xv, non_blocking=True)
-            d_sid.copy_(h_sid, non_blocking=True); d_pos.copy_(h_pos, non_blocking=True); d_q.copy_(h_q, non_blocking=True)
+            copy_stream.wait_event(step_done)                     # the previous step no longer reads the device buffers
+            with torch.cuda.stream(copy_stream):
+                d_sid.copy_(h_sid, non_blocking=True); d_pos.copy_(h_pos, non_blocking=True); d_q.copy_(h_q, non_blocking=True)
+                for p_ in range(n_pieces):
+                    lo, hi = p_ * piece, min(n_tok, (p_ + 1) * piece)
+                    d_xk[lo:hi].copy_(h_xk[lo:hi], non_blocking=True); d_xv[lo:hi].copy_(h_xv[lo:hi], non_blocking=True)
+                    landed[p_].record(copy_stream)
             B.twkv_cache_reset(cache)
-            B.twkv_compress(cache, 0, d_xk, d_xv, d_sid, d_pos, None, levels, B.TWKV_GATE_COMPUTE)
+            for p_ in range(n_pieces):
+                lo, hi = p_ * piece, min(n_tok, (p_ + 1) * piece)
+                stream.wait_event(landed[p_])
+                B.twkv_compress(cache, 0, d_xk[lo:hi], d_xv[lo:hi], d_sid[lo:hi], d_pos[lo:hi], None, levels[lo:hi], B.TWKV_GATE_COMPUTE)
             B.twkv_decode_attn(cache, 0, d_q, sid, out)
             h_out.copy_(out, non_blocking=True)
+            step_done.record(stream)
 
         e2e_step()
         barrier()
@@ -268,7 +285,7 @@ def run_ours(args):
         e2e_ms = replicas.max_over_ranks([g0.elapsed_time(g1) / n_e2e], dev)[0]
         h2d = sum(x.numel() * x.element_size() for x in (h_xk, h_xv, h_sid, h_pos, h_q))
         d2h = h_out.numel() * h_out.element_size()
-        e2e = {"value": replicas.whole_job_rate(n_tok, e2e_ms), "unit": "KV tokens/s through compress + decode, host buffers",
+        e2e = {"value": replicas.whole_job_rate(n_tok, e2e_ms), "unit": "KV tokens/s through compress + decode, host buffers (state copies in pieces on a copy stream, each piece compressed when it has landed)",
                "ms_per_step": e2e_ms, "steps": n_e2e, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h}
 
     if rank == 0:
