@@ -76,13 +76,13 @@ constexpr int GATE_PIECE = 8192;       // tokens per COMPUTE-mode gate piece (lo
 constexpr int GATE_TC_MIN_TOKENS = 1024;   // calls at least this large run the fused tcgen05 gate kernel
 
 struct Offsets {
-  size_t status, rope_lo, rope_hi, n_tiles, tile_desc, tile_aux, tile_rank, fill, key_last, kclass_count,
+  size_t status, pflags, rope_lo, rope_hi, n_tiles, tile_desc, tile_aux, tile_rank, fill, key_last, kclass_count,
       kclass_tiles, seq_vcount, seq_vtiles, seq_tokens, rank_sums, hist, key_cnt, key_old_fill, key_first_id,
       key_first_base, key_old_last, scores, seqmax, qslot, klist, klist_count, klist_cost, cta_start, part_acc, part_l, gate_scratch, stats_buf, tables_end, prep_uinvT, prep_wT,
       blocks, end_fixed;
 };
 
-struct Dims { int d_kv, NC, NT, TPS, NK, rep, max_partials; };
+struct Dims { int d_kv, NC, NT, TPS, NK, rep, max_partials, batch; };
 
 static bool config_ok(const twkv_config* c) {
   if (!c) return false;
@@ -109,6 +109,11 @@ static Dims dims_of(const twkv_config* c) {
   d.NK = 2 * c->max_seqs * d.NC;
   d.rep = c->n_q_heads / c->n_kv_heads;
   d.max_partials = c->max_seqs + MAX_PARTIALS_EXTRA;
+  // pieces whose bookkeeping kernels are launched together: up to 4, while their chunk-count tables stay under 64 MiB
+  const size_t hist_piece = (size_t)PIECE_CHUNKS * d.NK * sizeof(int);
+  d.batch = (int)((size_t)(64u << 20) / hist_piece);
+  if (d.batch < 1) d.batch = 1;
+  if (d.batch > 4) d.batch = 4;
   return d;
 }
 
@@ -132,12 +137,14 @@ static Offsets layout_of(const twkv_config* c, const Dims& d) {
   o.seq_tokens = L.alloc(Ls * S * sizeof(int));
   o.rank_sums = L.alloc(Ls * 2 * sizeof(unsigned long long));
   o.tables_end = L.alloc(0);
-  o.hist = L.alloc((size_t)PIECE_CHUNKS * NK * sizeof(int));
-  o.key_cnt = L.alloc(NK * sizeof(int));
-  o.key_old_fill = L.alloc(NK * sizeof(int));
-  o.key_first_id = L.alloc(NK * sizeof(int));
-  o.key_first_base = L.alloc(NK * sizeof(int));
-  o.key_old_last = L.alloc(NK * sizeof(int));
+  const size_t PB = (size_t)d.batch;
+  o.hist = L.alloc(PB * PIECE_CHUNKS * NK * sizeof(int));
+  o.key_cnt = L.alloc(PB * NK * sizeof(int));
+  o.key_old_fill = L.alloc(PB * NK * sizeof(int));
+  o.key_first_id = L.alloc(PB * NK * sizeof(int));
+  o.key_first_base = L.alloc(PB * NK * sizeof(int));
+  o.key_old_last = L.alloc(PB * NK * sizeof(int));
+  o.pflags = L.alloc(PB * 2 * sizeof(int));
   o.scores = L.alloc(NT * TILE * Hq * sizeof(float));
   o.seqmax = L.alloc(S * Hq * sizeof(unsigned));
   o.qslot = L.alloc(S * sizeof(int));
@@ -221,7 +228,7 @@ static void fill_view(twkv_cache* c) {
   v.out_dtype = cfg.out_dtype; v.NK = d.NK; v.max_partials = d.max_partials; v.tau = cfg.tau; v.sm_scale = cfg.sm_scale;
   const size_t nb = (c->pool_bytes - o.blocks) / BLOCK_BYTES;
   v.n_blocks = (int)(nb > 0x7fffffffull ? 0x7fffffffull : nb);
-  v.status = (int*)(p + o.status);
+  v.status = (int*)(p + o.status); v.pflags = (int*)(p + o.pflags); v.batch = d.batch;
   v.rope_lo = (float2*)(p + o.rope_lo); v.rope_hi = (float2*)(p + o.rope_hi);
   v.blocks = p + o.blocks;
   v.n_tiles = (int*)(p + o.n_tiles); v.tile_desc = (int4*)(p + o.tile_desc); v.tile_aux = (int*)(p + o.tile_aux);
@@ -383,10 +390,11 @@ twkv_status twkv_compress(twkv_cache* c, int layer, const void* K, const void* V
       if (launch_gate_rank(v, v.gate_scratch, levels + 2 * (size_t)lo, n, st) != cudaSuccess) return TWKV_ERR_CUDA;
     }
   }
-  for (int lo = 0; lo < n_tok; lo += TWKV_PIECE_TOKENS) {
-    const int n = n_tok - lo < TWKV_PIECE_TOKENS ? n_tok - lo : TWKV_PIECE_TOKENS;
-    if (launch_compress_piece(v, layer, (const unsigned char*)K + lo * row, (const unsigned char*)V + lo * row, seq_ids + lo,
-                              positions + lo, n, levels + 2 * (size_t)lo, st) != cudaSuccess) return TWKV_ERR_CUDA;
+  const int group = TWKV_PIECE_TOKENS * c->dims.batch;     // tokens whose pieces are handled by one set of launches
+  for (int lo = 0; lo < n_tok; lo += group) {
+    const int n = n_tok - lo < group ? n_tok - lo : group;
+    if (launch_compress_pieces(v, layer, (const unsigned char*)K + lo * row, (const unsigned char*)V + lo * row, seq_ids + lo,
+                               positions + lo, n, levels + 2 * (size_t)lo, st) != cudaSuccess) return TWKV_ERR_CUDA;
   }
   return TWKV_OK;
 }

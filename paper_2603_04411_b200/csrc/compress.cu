@@ -75,25 +75,42 @@ __device__ __forceinline__ int key_of(const DevView& v, int side, int seq, int c
   return (side * v.S + seq) * v.NC + (cls - 1);
 }
 
-__global__ void __launch_bounds__(CHUNK_TOKENS) hist_kernel(DevView v, const int* __restrict__ seq_ids, const int* __restrict__ positions,
+// A compress call is handled piece by piece (TWKV_PIECE_TOKENS tokens), but the kernels below run once for up to
+// v.batch pieces: every piece has its own copy of the per-piece scratch, selected here.
+__device__ __forceinline__ DevView piece_view(DevView v, int p) {
+  v.hist += (size_t)p * v.NK * PIECE_CHUNKS;
+  v.key_cnt += (size_t)p * v.NK; v.key_old_fill += (size_t)p * v.NK; v.key_first_id += (size_t)p * v.NK;
+  v.key_first_base += (size_t)p * v.NK; v.key_old_last += (size_t)p * v.NK;
+  v.pflags += 2 * p;
+  return v;
+}
+
+// grid: the chunks of all pieces of the launch group (chunk b belongs to piece b / PIECE_CHUNKS)
+__global__ void __launch_bounds__(CHUNK_TOKENS) hist_kernel(DevView v0, const int* __restrict__ seq_ids, const int* __restrict__ positions,
                                                             const unsigned short* __restrict__ levels, int n_tok) {
+  const DevView v = piece_view(v0, blockIdx.x / PIECE_CHUNKS);
+  const int chunk = blockIdx.x % PIECE_CHUNKS;
   const int i = blockIdx.x * CHUNK_TOKENS + threadIdx.x;
   if (i >= n_tok) return;
   const int seq = seq_ids[i];
   const int rk = levels[2 * i], rv = levels[2 * i + 1];
   const int pos = positions[i];
   if (seq < 0 || seq >= v.S || rk < 1 || rk > v.d_kv || rv < 1 || rv > v.d_kv || pos < 0 || pos >= ROPE_LO * ROPE_HI) {
-    atomicOr(&v.status[3], 1);
+    atomicOr(&v.pflags[1], 1);
     return;
   }
-  atomicAdd(&v.hist[(size_t)key_of(v, 0, seq, (rk + PANEL - 1) / PANEL) * PIECE_CHUNKS + blockIdx.x], 1);
-  atomicAdd(&v.hist[(size_t)key_of(v, 1, seq, (rv + PANEL - 1) / PANEL) * PIECE_CHUNKS + blockIdx.x], 1);
+  atomicAdd(&v.hist[(size_t)key_of(v, 0, seq, (rk + PANEL - 1) / PANEL) * PIECE_CHUNKS + chunk], 1);
+  atomicAdd(&v.hist[(size_t)key_of(v, 1, seq, (rv + PANEL - 1) / PANEL) * PIECE_CHUNKS + chunk], 1);
 }
 
 // Warp per key: the key's per-chunk counts (contiguous, [key][chunk]) become exclusive bases, their sum the key's count.
-__global__ void __launch_bounds__(256) scan_kernel(DevView v, int layer, int n_chunks) {
-  const int key = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, lane = threadIdx.x & 31;
-  if (key >= v.NK) return;
+// grid: one warp per (piece, key); total_chunks counts the chunks of all pieces of the launch group
+__global__ void __launch_bounds__(256) scan_kernel(DevView v0, int n_pieces, int total_chunks) {
+  const int widx = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, lane = threadIdx.x & 31;
+  if (widx >= v0.NK * n_pieces) return;
+  const int piece = widx / v0.NK, key = widx - piece * v0.NK;
+  const DevView v = piece_view(v0, piece);
+  const int n_chunks = min(PIECE_CHUNKS, total_chunks - piece * PIECE_CHUNKS);
   int* h = v.hist + (size_t)key * PIECE_CHUNKS;
   int carry = 0;
   for (int c0 = 0; c0 < n_chunks; c0 += 128) {
@@ -111,161 +128,180 @@ __global__ void __launch_bounds__(256) scan_kernel(DevView v, int layer, int n_c
     if (c < n_chunks) *reinterpret_cast<int4*>(h + c) = make_int4(base, base + t.x, base + t.x + t.y, base + t.x + t.y + t.z);
     carry += __shfl_sync(0xffffffffu, incl, 31);
   }
-  if (lane == 0) {
-    v.key_cnt[key] = carry;
-    v.key_old_fill[key] = v.fill_l(layer)[key];
-  }
+  if (lane == 0) v.key_cnt[key] = carry;
 }
 
 __device__ __forceinline__ int ceil_div(int a, int b) { return (a + b - 1) / b; }
 
-// One CTA of 1024 threads.  Turns per-chunk counts into exclusive bases, checks capacity and,
-// if the whole piece fits, creates the new tiles in ascending key order.
-__global__ void __launch_bounds__(1024) alloc_kernel(DevView v, int layer, int n_chunks) {
+// One CTA of 1024 threads, the pieces of the launch group one after the other.  Per piece: checks capacity and, if
+// the whole piece fits, creates the new tiles in ascending key order; a piece that does not fit (or holds an invalid
+// token) is refused whole and the later pieces carry on from the unchanged tables.
+__global__ void __launch_bounds__(1024) alloc_kernel(DevView v0, int layer, int n_pieces) {
   __shared__ int s_scan[3][1024];
   __shared__ int s_fail;
   const int tid = threadIdx.x;
-  const int NK = v.NK;
-  int* fill = v.fill_l(layer);
-  int* key_last = v.key_last_l(layer);
-  if (tid == 0) s_fail = 0;
-  __syncthreads();
-  // (per-key counts and per-chunk bases come from scan_kernel)  new tiles / blocks per key, scanned in key order
+  const int NK = v0.NK;
+  int* fill = v0.fill_l(layer);
+  int* key_last = v0.key_last_l(layer);
   const int KPT = ceil_div(NK, 1024);
   const int k0 = tid * KPT, k1 = min(NK, k0 + KPT);
-  const int half = v.S * v.NC;                        // keys per side
-  int sum_tk = 0, sum_tv = 0, sum_b = 0;
-  for (int k = k0; k < k1; ++k) {
-    const int cnt = v.key_cnt[k], old = v.key_old_fill[k];
-    const int nnew = ceil_div(old + cnt, TILE) - ceil_div(old, TILE);
-    if (k < half) sum_tk += nnew; else sum_tv += nnew;
-    sum_b += nnew * (k % v.NC + 1);
-  }
-  s_scan[0][tid] = sum_tk; s_scan[1][tid] = sum_tv; s_scan[2][tid] = sum_b;
-  __syncthreads();
-  for (int o = 1; o < 1024; o <<= 1) {                 // inclusive Hillis-Steele scan
-    int a = 0, b = 0, c = 0;
-    if (tid >= o) { a = s_scan[0][tid - o]; b = s_scan[1][tid - o]; c = s_scan[2][tid - o]; }
-    __syncthreads();
-    s_scan[0][tid] += a; s_scan[1][tid] += b; s_scan[2][tid] += c;
-    __syncthreads();
-  }
-  const int tot_tk = s_scan[0][1023], tot_tv = s_scan[1][1023], tot_b = s_scan[2][1023];
-  const int next_block = v.status[1];
-  int* ntiles = v.ntiles(layer);
-  const int ntk = ntiles[0], ntv = ntiles[1];
-  // capacity: tokens per sequence
-  int* stok = v.stok(layer);
-  for (int s = tid; s < v.S; s += 1024) {
-    int add = 0;
-    for (int c = 0; c < v.NC; ++c) add += v.key_cnt[s * v.NC + c];
-    if (stok[s] + add > v.tmax) atomicOr(&s_fail, 1);
-  }
-  if (tid == 0) {
-    if (next_block + tot_b > v.n_blocks || ntk + tot_tk > v.NT || ntv + tot_tv > v.NT) atomicOr(&s_fail, 1);
-    if (v.status[3]) atomicOr(&s_fail, 2);
-  }
-  __syncthreads();
-  if (s_fail) {
-    if (tid == 0) {
-      v.status[2] = 0;
-      v.status[3] = 0;
-      set_status(v, (s_fail & 2) ? TWKV_ERR_INVALID_ARG : TWKV_ERR_CAPACITY);
-    }
-    return;
-  }
-  // commit
-  int off_tk = s_scan[0][tid] - sum_tk, off_tv = s_scan[1][tid] - sum_tv, off_b = s_scan[2][tid] - sum_b;
-  for (int k = k0; k < k1; ++k) {
-    const int cnt = v.key_cnt[k], old = v.key_old_fill[k];
-    const int side = k >= half ? 1 : 0;
-    const int cls = k % v.NC + 1;
-    const int seq = (k / v.NC) % v.S;
-    const int old_tiles = ceil_div(old, TILE);
-    const int nnew = ceil_div(old + cnt, TILE) - old_tiles;
-    const int first_id = (side ? ntv + off_tv : ntk + off_tk);
-    const int first_base = next_block + off_b;
-    v.key_first_id[k] = first_id;
-    v.key_first_base[k] = first_base;
-    v.key_old_last[k] = key_last[k];
-    if (cnt > 0) {
-      const int nf = old + cnt;
-      int4* desc = v.desc(layer, side);
-      if (old % TILE != 0) desc[key_last[k]].z = min(TILE, nf - (old_tiles - 1) * TILE);
-      for (int j = 0; j < nnew; ++j)
-        desc[first_id + j] = make_int4(seq, cls, min(TILE, nf - (old_tiles + j) * TILE), first_base + j * cls);
-      if (nnew > 0) key_last[k] = first_id + nnew - 1;
-      fill[k] = nf;
-    }
-    if (side) off_tv += nnew; else off_tk += nnew;
-    off_b += nnew * cls;
-  }
-  __syncthreads();
-  // tile lists: K per class (ascending sequence), V per sequence (ascending class); one warp per list, the lanes
-  // write a key's run of consecutive tile ids together
+  const int half = v0.S * v0.NC;                      // keys per side
+  int* ntiles = v0.ntiles(layer);
+  int* stok = v0.stok(layer);
   const int warp = tid >> 5, lane = tid & 31;
-  if (warp < v.NC) {
-    int* cnt = v.kcc(layer);
-    int* list = v.kct(layer) + (size_t)warp * v.NT;
-    int run = cnt[warp];
-    for (int s = 0; s < v.S; ++s) {
-      const int k = s * v.NC + warp;
-      const int c = v.key_cnt[k], old = v.key_old_fill[k];
-      const int nnew = ceil_div(old + c, TILE) - ceil_div(old, TILE);
-      const int first = v.key_first_id[k];
-      for (int j = lane; j < nnew; j += 32) list[run + j] = first + j;
-      run += nnew;
+  for (int piece = 0; piece < n_pieces; ++piece) {
+    const DevView v = piece_view(v0, piece);
+    if (tid == 0) s_fail = 0;
+    __syncthreads();                                   // also: the previous piece's table updates are visible
+    // (per-key counts and per-chunk bases come from scan_kernel)  new tiles / blocks per key, scanned in key order
+    int sum_tk = 0, sum_tv = 0, sum_b = 0;
+    for (int k = k0; k < k1; ++k) {
+      const int cnt = v.key_cnt[k], old = fill[k];
+      v.key_old_fill[k] = old;
+      const int nnew = ceil_div(old + cnt, TILE) - ceil_div(old, TILE);
+      if (k < half) sum_tk += nnew; else sum_tv += nnew;
+      sum_b += nnew * (k % v.NC + 1);
     }
-    __syncwarp();
-    if (lane == 0) cnt[warp] = run;
-  }
-  for (int s = warp; s < v.S; s += 32) {
-    int* list = v.svt(layer) + (size_t)s * v.TPS;
-    int run = v.svc(layer)[s];
-    int add = 0;
-    for (int c = 0; c < v.NC; ++c) {
-      const int k = half + s * v.NC + c;
-      const int cn = v.key_cnt[k], old = v.key_old_fill[k];
-      const int nnew = ceil_div(old + cn, TILE) - ceil_div(old, TILE);
-      const int first = v.key_first_id[k];
-      for (int j = lane; j < nnew; j += 32) list[run + j] = first + j;
-      run += nnew;
-      add += v.key_cnt[s * v.NC + c];
+    s_scan[0][tid] = sum_tk; s_scan[1][tid] = sum_tv; s_scan[2][tid] = sum_b;
+    __syncthreads();
+    for (int o = 1; o < 1024; o <<= 1) {                 // inclusive Hillis-Steele scan
+      int a = 0, b = 0, c = 0;
+      if (tid >= o) { a = s_scan[0][tid - o]; b = s_scan[1][tid - o]; c = s_scan[2][tid - o]; }
+      __syncthreads();
+      s_scan[0][tid] += a; s_scan[1][tid] += b; s_scan[2][tid] += c;
+      __syncthreads();
     }
-    __syncwarp();
-    if (lane == 0) {
-      v.svc(layer)[s] = run;
-      stok[s] += add;
+    const int tot_tk = s_scan[0][1023], tot_tv = s_scan[1][1023], tot_b = s_scan[2][1023];
+    const int next_block = v.status[1];
+    const int ntk = ntiles[0], ntv = ntiles[1];
+    // capacity: tokens per sequence
+    for (int s = tid; s < v.S; s += 1024) {
+      int add = 0;
+      for (int c = 0; c < v.NC; ++c) add += v.key_cnt[s * v.NC + c];
+      if (stok[s] + add > v.tmax) atomicOr(&s_fail, 1);
     }
-  }
-  if (tid == 0) {
-    v.status[1] = next_block + tot_b;
-    ntiles[0] = ntk + tot_tk;
-    ntiles[1] = ntv + tot_tv;
-    v.status[2] = 1;
+    if (tid == 0) {
+      if (next_block + tot_b > v.n_blocks || ntk + tot_tk > v.NT || ntv + tot_tv > v.NT) atomicOr(&s_fail, 1);
+      if (v.pflags[1]) atomicOr(&s_fail, 2);
+    }
+    __syncthreads();
+    if (s_fail) {
+      if (tid == 0) {
+        v.pflags[0] = 0;
+        set_status(v, (s_fail & 2) ? TWKV_ERR_INVALID_ARG : TWKV_ERR_CAPACITY);
+      }
+      __syncthreads();                                 // s_fail is reset at the top of the next round
+      continue;
+    }
+    // commit
+    int off_tk = s_scan[0][tid] - sum_tk, off_tv = s_scan[1][tid] - sum_tv, off_b = s_scan[2][tid] - sum_b;
+    for (int k = k0; k < k1; ++k) {
+      const int cnt = v.key_cnt[k], old = v.key_old_fill[k];
+      const int side = k >= half ? 1 : 0;
+      const int cls = k % v.NC + 1;
+      const int seq = (k / v.NC) % v.S;
+      const int old_tiles = ceil_div(old, TILE);
+      const int nnew = ceil_div(old + cnt, TILE) - old_tiles;
+      const int first_id = (side ? ntv + off_tv : ntk + off_tk);
+      const int first_base = next_block + off_b;
+      v.key_first_id[k] = first_id;
+      v.key_first_base[k] = first_base;
+      v.key_old_last[k] = key_last[k];
+      if (cnt > 0) {
+        const int nf = old + cnt;
+        int4* desc = v.desc(layer, side);
+        if (old % TILE != 0) desc[key_last[k]].z = min(TILE, nf - (old_tiles - 1) * TILE);
+        for (int j = 0; j < nnew; ++j)
+          desc[first_id + j] = make_int4(seq, cls, min(TILE, nf - (old_tiles + j) * TILE), first_base + j * cls);
+        if (nnew > 0) key_last[k] = first_id + nnew - 1;
+        fill[k] = nf;
+      }
+      if (side) off_tv += nnew; else off_tk += nnew;
+      off_b += nnew * cls;
+    }
+    __syncthreads();
+    // tile lists: K per class (ascending sequence), V per sequence (ascending class); one warp per list, the lanes
+    // write a key's run of consecutive tile ids together
+    if (warp < v.NC) {
+      int* cnt = v.kcc(layer);
+      int* list = v.kct(layer) + (size_t)warp * v.NT;
+      int run = cnt[warp];
+      for (int s = 0; s < v.S; ++s) {
+        const int k = s * v.NC + warp;
+        const int c = v.key_cnt[k], old = v.key_old_fill[k];
+        const int nnew = ceil_div(old + c, TILE) - ceil_div(old, TILE);
+        const int first = v.key_first_id[k];
+        for (int j = lane; j < nnew; j += 32) list[run + j] = first + j;
+        run += nnew;
+      }
+      __syncwarp();
+      if (lane == 0) cnt[warp] = run;
+    }
+    for (int s = warp; s < v.S; s += 32) {
+      int* list = v.svt(layer) + (size_t)s * v.TPS;
+      int run = v.svc(layer)[s];
+      int add = 0;
+      for (int c = 0; c < v.NC; ++c) {
+        const int k = half + s * v.NC + c;
+        const int cn = v.key_cnt[k], old = v.key_old_fill[k];
+        const int nnew = ceil_div(old + cn, TILE) - ceil_div(old, TILE);
+        const int first = v.key_first_id[k];
+        for (int j = lane; j < nnew; j += 32) list[run + j] = first + j;
+        run += nnew;
+        add += v.key_cnt[s * v.NC + c];
+      }
+      __syncwarp();
+      if (lane == 0) {
+        v.svc(layer)[s] = run;
+        stok[s] += add;
+      }
+    }
+    if (tid == 0) {
+      v.status[1] = next_block + tot_b;
+      ntiles[0] = ntk + tot_tk;
+      ntiles[1] = ntv + tot_tv;
+      v.pflags[0] = 1;
+    }
+    __syncthreads();
   }
 }
 
 struct Place { int base, slot_cls_r; };   // slot | cls << 8 | r << 16
 
-__global__ void __launch_bounds__(CHUNK_TOKENS) pack_kernel(DevView v, int layer, const void* __restrict__ K, const void* __restrict__ V,
+// grid: the chunks of all pieces of the launch group (chunk b belongs to piece b / PIECE_CHUNKS), then one CTA per
+// (piece, key) for the tile tails
+__global__ void __launch_bounds__(CHUNK_TOKENS) pack_kernel(DevView v0, int layer, const void* __restrict__ K, const void* __restrict__ V,
                                                             const int* __restrict__ seq_ids, const int* __restrict__ positions,
                                                             const unsigned short* __restrict__ levels, int n_tok) {
-  if (v.status[2] == 0) return;                           // the piece was refused
   const int n_chunks = (n_tok + CHUNK_TOKENS - 1) / CHUNK_TOKENS;
-  if ((int)blockIdx.x >= n_chunks) {
-    // CTAs past the token chunks, one per key: if the key's last token of this piece sits in a tile created by
-    // this piece and the tile is not full, zero the slots behind it (decode reads whole tiles).
-    const int k = blockIdx.x - n_chunks;
+  const bool tail_cta = (int)blockIdx.x >= n_chunks;
+  const int piece = tail_cta ? (blockIdx.x - n_chunks) / v0.NK : blockIdx.x / PIECE_CHUNKS;
+  const DevView v = piece_view(v0, piece);
+  if (v.pflags[0] == 0) return;                           // the piece was refused
+  const int chunk = blockIdx.x % PIECE_CHUNKS;            // of a token CTA, inside its piece
+  if (tail_cta) {
+    // one CTA per (piece, key): if the key's last token of the piece sits in a tile created by the piece and the
+    // tile is not full, zero the slots behind it (decode reads whole tiles).
+    const int k = (blockIdx.x - n_chunks) % v.NK;
     const int cnt = v.key_cnt[k];
     if (cnt == 0) return;
     const int old = v.key_old_fill[k], cls = k % v.NC + 1;
     const int g = old + cnt - 1, ord = g / TILE, slot = g % TILE, old_tiles = (old + TILE - 1) / TILE;
-    if (ord < old_tiles || slot == TILE - 1) return;
+    if (ord < old_tiles) return;
+    // later pieces of this launch group keep filling the same tile (their CTAs run beside this one): leave them
+    // their slots and zero from behind the key's last token of the whole group
+    int later = 0;
+    const int n_pieces = (n_chunks + PIECE_CHUNKS - 1) / PIECE_CHUNKS;
+    for (int q = piece + 1; q < n_pieces; ++q) {
+      const DevView w = piece_view(v0, q);
+      if (w.pflags[0]) later += w.key_cnt[k];
+    }
+    const int first_zero = slot + 1 + later;
+    if (first_zero >= TILE) return;
     const int base = v.key_first_base[k] + (ord - old_tiles) * cls;
-    const int n16 = (TILE - 1 - slot) * 8;                 // 16-byte chunks behind the last token, per panel
+    const int n16 = (TILE - first_zero) * 8;               // 16-byte chunks behind the last token, per panel
     for (int panel = 0; panel < cls; ++panel) {
-      uint4* dst = reinterpret_cast<uint4*>(v.blocks + (size_t)(base + panel) * BLOCK_BYTES + (slot + 1) * (PANEL * 2));
+      uint4* dst = reinterpret_cast<uint4*>(v.blocks + (size_t)(base + panel) * BLOCK_BYTES + first_zero * (PANEL * 2));
       for (int i = threadIdx.x; i < n16; i += CHUNK_TOKENS) dst[i] = make_uint4(0u, 0u, 0u, 0u);
     }
     return;
@@ -298,7 +334,7 @@ __global__ void __launch_bounds__(CHUNK_TOKENS) pack_kernel(DevView v, int layer
       const int k = key[side];
       const int cls = k % v.NC + 1;
       const int old = v.key_old_fill[k];
-      const int g = old + v.hist[(size_t)k * PIECE_CHUNKS + blockIdx.x] + before[side];
+      const int g = old + v.hist[(size_t)k * PIECE_CHUNKS + chunk] + before[side];
       const int ord = g / TILE, slot = g % TILE;
       const int old_tiles = (old + TILE - 1) / TILE;
       int tile, base;
@@ -401,20 +437,26 @@ __global__ void __launch_bounds__(CHUNK_TOKENS) pack_kernel(DevView v, int layer
   }
 }
 
-cudaError_t launch_compress_piece(const DevView& v, int layer, const void* K, const void* V, const int* seq_ids,
-                                  const int* positions, int n_tok, const unsigned short* levels, cudaStream_t st) {
+// The pieces of up to v.batch * TWKV_PIECE_TOKENS tokens: one launch each of the histogram, the per-key scan, the
+// allocator (which takes the pieces in order) and the packer.
+cudaError_t launch_compress_pieces(const DevView& v, int layer, const void* K, const void* V, const int* seq_ids,
+                                   const int* positions, int n_tok, const unsigned short* levels, cudaStream_t st) {
   if (n_tok <= 0) return cudaSuccess;
   const int n_chunks = (n_tok + CHUNK_TOKENS - 1) / CHUNK_TOKENS;
-  const int n_cols = (n_chunks + 3) & ~3;                  // scan_kernel reads the counts four at a time
-  cudaError_t e = cudaMemset2DAsync(v.hist, (size_t)PIECE_CHUNKS * sizeof(int), 0, (size_t)n_cols * sizeof(int), (size_t)v.NK, st);
+  const int n_pieces = (n_chunks + PIECE_CHUNKS - 1) / PIECE_CHUNKS;
+  // scan_kernel reads the counts four at a time; a launch group of several pieces clears its tables whole
+  const int n_cols = n_pieces > 1 ? PIECE_CHUNKS : (n_chunks + 3) & ~3;
+  cudaError_t e = cudaMemset2DAsync(v.hist, (size_t)PIECE_CHUNKS * sizeof(int), 0, (size_t)n_cols * sizeof(int), (size_t)v.NK * n_pieces, st);
+  if (e != cudaSuccess) return e;
+  e = cudaMemsetAsync(v.pflags, 0, (size_t)v.batch * 2 * sizeof(int), st);
   if (e != cudaSuccess) return e;
   { ProfScope ps(TWKV_K_HIST, st); hist_kernel<<<n_chunks, CHUNK_TOKENS, 0, st>>>(v, seq_ids, positions, levels, n_tok); }
   {
     ProfScope ps(TWKV_K_ALLOC, st);
-    scan_kernel<<<(v.NK + 7) / 8, 256, 0, st>>>(v, layer, n_chunks);
-    alloc_kernel<<<1, 1024, 0, st>>>(v, layer, n_chunks);
+    scan_kernel<<<(v.NK * n_pieces + 7) / 8, 256, 0, st>>>(v, n_pieces, n_chunks);
+    alloc_kernel<<<1, 1024, 0, st>>>(v, layer, n_pieces);
   }
-  { ProfScope ps(TWKV_K_PACK, st); pack_kernel<<<n_chunks + v.NK, CHUNK_TOKENS, 0, st>>>(v, layer, K, V, seq_ids, positions, levels, n_tok); }
+  { ProfScope ps(TWKV_K_PACK, st); pack_kernel<<<n_chunks + v.NK * n_pieces, CHUNK_TOKENS, 0, st>>>(v, layer, K, V, seq_ids, positions, levels, n_tok); }
   count_launch(4);
   return cudaGetLastError();
 }

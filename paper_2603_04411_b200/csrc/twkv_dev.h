@@ -24,7 +24,9 @@ constexpr int MAX_PLAN_CTAS = 1024;         // upper bound on the K-score kernel
 struct DevView {
   int L, Hq, Hkv, rep, d_kv, NC, S, tmax, NT, TPS, n_blocks, dtype, out_dtype, NK, max_partials;
   float tau, sm_scale;
-  int* status;               // [8]: [0] sticky status, [1] next free block, [2] piece_ok, [3] piece flags
+  int* status;               // [8]: [0] sticky status, [1] next free block
+  int* pflags;               // [batch][2]: piece accepted, piece holds an invalid token (scratch of one compress call)
+  int batch;                 // pieces of a compress call whose bookkeeping is launched together
   float2* rope_lo;           // [ROPE_SMALL_ROWS][64] (cos, sin) of mid * 16 * theta_i (rows 0..15) and lo * theta_i (rows 16..31)
   float2* rope_hi;           // [ROPE_HI][64] (cos, sin) of hi * 256 * theta_i
   unsigned char* blocks;     // n_blocks x 16 KiB
@@ -42,9 +44,10 @@ struct DevView {
   int* seq_tokens;           // [L][S]
   unsigned long long* rank_sums;  // [L][2]  sum of r_K, r_V
   // scratch shared by all layers
+  // per-piece scratch of a compress call, [batch] copies each (piece_view() selects one)
   int* hist;                 // [NK][PIECE_CHUNKS]   per-chunk key counts -> exclusive bases
-  int* key_cnt;              // [NK]  tokens of the key in the current piece
-  int* key_old_fill;         // [NK]
+  int* key_cnt;              // [NK]  tokens of the key in the piece
+  int* key_old_fill;         // [NK]  tokens of the key before the piece
   int* key_first_id;         // [NK]  id of the key's first new tile
   int* key_first_base;       // [NK]  base block of the key's first new tile
   int* key_old_last;         // [NK]  the key's newest tile before the piece
@@ -123,7 +126,7 @@ struct ProfScope {
 cudaError_t launch_rope_tables(const DevView& v, float rope_base, cudaStream_t st);
 cudaError_t launch_clear_tables(const DevView& v, cudaStream_t st);
 cudaError_t launch_gate_rank(const DevView& v, const float* logits, unsigned short* levels, int n_tok, cudaStream_t st);
-cudaError_t launch_compress_piece(const DevView& v, int layer, const void* K, const void* V, const int* seq_ids,
+cudaError_t launch_compress_pieces(const DevView& v, int layer, const void* K, const void* V, const int* seq_ids,
                                   const int* positions, int n_tok, const unsigned short* levels, cudaStream_t st);
 struct TcMaps;   // tensor maps of the K-score kernel (api.cu)
 cudaError_t launch_decode(const DevView& v, int layer, const LayerParams& lp, const void* q, const int* seq_ids,
