@@ -404,6 +404,41 @@ def test_compress_spanning_two_pieces(B):
     gc.close()
 
 
+def test_three_pieces_middle_one_refused(B):
+    # One call of three pieces whose bookkeeping is launched together.  The middle piece would push sequence 0 past
+    # max_tokens_per_seq: it is skipped whole (sticky TWKV_ERR_CAPACITY), the pieces before and after it are stored, and
+    # the third one continues the tiles of nothing the refused piece touched.
+    P = B.PIECE_TOKENS
+    half, tmax, d = P // 2, 70000, 1024
+    seq = torch.cat([torch.full((half,), 0), torch.full((half,), 1), torch.full((half,), 0), torch.full((half,), 2),
+                     torch.full((500,), 2)]).to(torch.int32)
+    n = seq.numel()
+    pos = torch.zeros(n, dtype=torch.int32)
+    for s_ in range(3):
+        m = seq == s_
+        pos[m] = torch.arange(int(m.sum()), dtype=torch.int32)
+    g = torch.Generator().manual_seed(91)
+    xk = (torch.randn(n, d, generator=g) * 0.5).to(torch.float16)
+    xv = (torch.randn(n, d, generator=g) * 0.5).to(torch.float16)
+    ranks = torch.randint(1, 129, (n, 2), generator=g).numpy().astype(np.int64)        # classes 1 and 2 keep the case light
+    gc = GpuCache(B, n_layers=1, n_q_heads=8, n_kv_heads=8, dtype=torch.float16, out_dtype=torch.float32,
+                  max_seqs=3, max_tokens_per_seq=tmax, payload_bytes=int((-(-ranks // 64) * 128).sum()))
+    U = torch.eye(d, dtype=torch.float16).cuda()
+    B.twkv_cache_set_layer_params(gc.h, 0, U, U)
+    B.twkv_compress(gc.h, 0, xk.cuda(), xv.cuda(), seq.cuda(), pos.cuda(), None, levels_tensor(ranks), B.TWKV_GATE_FORCED)
+    assert B.twkv_cache_status(gc.h) == B.TWKV_ERR_CAPACITY                            # read once: cleared
+    img = CacheImage(1, d, 3, tmax, int(gc.lay.n_blocks))
+    got = []
+    for lo in range(0, n, P):                                                           # the image takes the pieces one by one
+        hi = min(n, lo + P)
+        got.append(img.append(0, bits16(xk[lo:hi]), bits16(xv[lo:hi]), seq[lo:hi].numpy(), pos[lo:hi].numpy(), ranks[lo:hi]))
+    assert got == [True, False, True]
+    compare_cache_with_image(gc, img)
+    st = B.twkv_cache_stats(gc.h, 0)
+    assert st.tokens == P + 500
+    gc.close()
+
+
 def test_benchmark_workload_full_size_sampled(B):
     # the workload and launch configuration bench.py times (B = 16, T = 32768, GQA 4, fp16, COMPUTE gate), checked
     # on what the oracle can afford: the ranks of every token of one sequence, and that sequence's attention output
