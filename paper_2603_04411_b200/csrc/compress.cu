@@ -136,7 +136,11 @@ __device__ __forceinline__ int ceil_div(int a, int b) { return (a + b - 1) / b; 
 // One CTA of 1024 threads, the pieces of the launch group one after the other.  Per piece: checks capacity and, if
 // the whole piece fits, creates the new tiles in ascending key order; a piece that does not fit (or holds an invalid
 // token) is refused whole and the later pieces carry on from the unchanged tables.
-__global__ void __launch_bounds__(1024) alloc_kernel(DevView v0, int layer, int n_pieces) {
+// A call of at most one chunk (the decode-time append) skips the histogram and scan launches: `count_tok` > 0 makes
+// this kernel count the call's tokens per key itself (one piece, one chunk, so every per-chunk base is 0).
+__global__ void __launch_bounds__(1024) alloc_kernel(DevView v0, int layer, int n_pieces, const int* __restrict__ seq_ids,
+                                                     const int* __restrict__ positions, const unsigned short* __restrict__ levels,
+                                                     int count_tok) {
   __shared__ int s_scan[3][1024];
   __shared__ int s_fail;
   const int tid = threadIdx.x;
@@ -149,6 +153,24 @@ __global__ void __launch_bounds__(1024) alloc_kernel(DevView v0, int layer, int 
   int* ntiles = v0.ntiles(layer);
   int* stok = v0.stok(layer);
   const int warp = tid >> 5, lane = tid & 31;
+  if (count_tok > 0) {
+    for (int k = k0; k < k1; ++k) v0.key_cnt[k] = 0;
+    if (tid < 2) v0.pflags[tid] = 0;
+    __syncthreads();
+    if (tid < count_tok) {
+      const int seq = seq_ids[tid], rk = levels[2 * tid], rv = levels[2 * tid + 1], pos = positions[tid];
+      if (seq < 0 || seq >= v0.S || rk < 1 || rk > v0.d_kv || rv < 1 || rv > v0.d_kv || pos < 0 || pos >= ROPE_LO * ROPE_HI) {
+        atomicOr(&v0.pflags[1], 1);
+      } else {
+        const int kk = key_of(v0, 0, seq, (rk + PANEL - 1) / PANEL), kv = key_of(v0, 1, seq, (rv + PANEL - 1) / PANEL);
+        atomicAdd(&v0.key_cnt[kk], 1);
+        atomicAdd(&v0.key_cnt[kv], 1);
+        v0.hist[(size_t)kk * PIECE_CHUNKS] = 0;                // the chunk's base inside the piece
+        v0.hist[(size_t)kv * PIECE_CHUNKS] = 0;
+      }
+    }
+    // the barrier at the top of the piece loop publishes the counts
+  }
   for (int piece = 0; piece < n_pieces; ++piece) {
     const DevView v = piece_view(v0, piece);
     if (tid == 0) s_fail = 0;
@@ -445,6 +467,13 @@ cudaError_t launch_compress_pieces(const DevView& v, int layer, const void* K, c
   const int n_chunks = (n_tok + CHUNK_TOKENS - 1) / CHUNK_TOKENS;
   const int n_pieces = (n_chunks + PIECE_CHUNKS - 1) / PIECE_CHUNKS;
   // scan_kernel reads the counts four at a time; a launch group of several pieces clears its tables whole
+  if (n_chunks == 1) {
+    // decode-time append: the allocator counts the tokens itself, two launches in all
+    { ProfScope ps(TWKV_K_ALLOC, st); alloc_kernel<<<1, 1024, 0, st>>>(v, layer, 1, seq_ids, positions, levels, n_tok); }
+    { ProfScope ps(TWKV_K_PACK, st); pack_kernel<<<1 + v.NK, CHUNK_TOKENS, 0, st>>>(v, layer, K, V, seq_ids, positions, levels, n_tok); }
+    count_launch(2);
+    return cudaGetLastError();
+  }
   const int n_cols = n_pieces > 1 ? PIECE_CHUNKS : (n_chunks + 3) & ~3;
   cudaError_t e = cudaMemset2DAsync(v.hist, (size_t)PIECE_CHUNKS * sizeof(int), 0, (size_t)n_cols * sizeof(int), (size_t)v.NK * n_pieces, st);
   if (e != cudaSuccess) return e;
@@ -454,7 +483,7 @@ cudaError_t launch_compress_pieces(const DevView& v, int layer, const void* K, c
   {
     ProfScope ps(TWKV_K_ALLOC, st);
     scan_kernel<<<(v.NK * n_pieces + 7) / 8, 256, 0, st>>>(v, n_pieces, n_chunks);
-    alloc_kernel<<<1, 1024, 0, st>>>(v, layer, n_pieces);
+    alloc_kernel<<<1, 1024, 0, st>>>(v, layer, n_pieces, nullptr, nullptr, nullptr, 0);
   }
   { ProfScope ps(TWKV_K_PACK, st); pack_kernel<<<n_chunks + v.NK * n_pieces, CHUNK_TOKENS, 0, st>>>(v, layer, K, V, seq_ids, positions, levels, n_tok); }
   count_launch(4);
