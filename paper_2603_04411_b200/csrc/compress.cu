@@ -292,7 +292,7 @@ struct Place { int base, slot_cls_r; };   // slot | cls << 8 | r << 16
 
 // grid: the chunks of all pieces of the launch group (chunk b belongs to piece b / PIECE_CHUNKS), then one CTA per
 // (piece, key) for the tile tails
-__global__ void __launch_bounds__(CHUNK_TOKENS) pack_kernel(DevView v0, int layer, const void* __restrict__ K, const void* __restrict__ V,
+__global__ void __launch_bounds__(CHUNK_TOKENS, 7) pack_kernel(DevView v0, int layer, const void* __restrict__ K, const void* __restrict__ V,
                                                             const int* __restrict__ seq_ids, const int* __restrict__ positions,
                                                             const unsigned short* __restrict__ levels, int n_tok) {
   const int n_chunks = (n_tok + CHUNK_TOKENS - 1) / CHUNK_TOKENS;
@@ -390,7 +390,10 @@ __global__ void __launch_bounds__(CHUNK_TOKENS) pack_kernel(DevView v0, int laye
   // Move the rows.  The CTA's 256 (token, side) rows are a flat list of 16-byte chunks (8 elements; a row of class c
   // has 8 c of them, those past the rank are zero fill); thread i takes chunks i, i + 128, ... so every lane has
   // work whatever the rows' widths, and loads PACK_UNROLL chunks before it stores any.
-  __shared__ int s_pref[2 * CHUNK_TOKENS + 1];
+  // Every row is a whole number of 8-chunk groups (one 128-byte panel row each); s_oct maps a group to its row and to
+  // the panel inside the row, so finding a chunk's row is one shared-memory read.
+  __shared__ unsigned short s_oct[2 * CHUNK_TOKENS * TWKV_MAX_CLASSES];      // (row << 4) | panel
+  __shared__ int s_total;
   __shared__ int s_wtot[CHUNK_TOKENS / 32];
   {
     const int c0 = valid ? ((s_place[0][tid].slot_cls_r >> 8) & 0xff) * 8 : 0;
@@ -406,12 +409,12 @@ __global__ void __launch_bounds__(CHUNK_TOKENS) pack_kernel(DevView v0, int laye
     int off = 0;
     for (int w = 0; w < (tid >> 5); ++w) off += s_wtot[w];
     const int excl = off + inc - (c0 + c1);
-    s_pref[2 * tid] = excl;
-    s_pref[2 * tid + 1] = excl + c0;
-    if (tid == CHUNK_TOKENS - 1) s_pref[2 * CHUNK_TOKENS] = excl + c0 + c1;
+    for (int pnl = 0; pnl < (c0 >> 3); ++pnl) s_oct[(excl >> 3) + pnl] = (unsigned short)(((2 * tid) << 4) | pnl);
+    for (int pnl = 0; pnl < (c1 >> 3); ++pnl) s_oct[((excl + c0) >> 3) + pnl] = (unsigned short)(((2 * tid + 1) << 4) | pnl);
+    if (tid == CHUNK_TOKENS - 1) s_total = excl + c0 + c1;
   }
   __syncthreads();
-  const int total = s_pref[2 * CHUNK_TOKENS];
+  const int total = s_total;
   const size_t row_bytes = (size_t)v.d_kv * 2;
   constexpr int PACK_UNROLL = 8;
   for (int cb = tid; cb < total; cb += CHUNK_TOKENS * PACK_UNROLL) {
@@ -425,13 +428,8 @@ __global__ void __launch_bounds__(CHUNK_TOKENS) pack_kernel(DevView v0, int laye
       dst[u] = nullptr;
       keep[u] = 8;
       if (c < total) {
-        int lo = 0, hi = 2 * CHUNK_TOKENS;                       // largest row q with s_pref[q] <= c
-#pragma unroll
-        for (int it = 0; it < 8; ++it) {
-          const int mid = (lo + hi) >> 1;
-          if (s_pref[mid] <= c) lo = mid; else hi = mid;
-        }
-        const int t = lo >> 1, side = lo & 1, j = c - s_pref[lo];
+        const int info = s_oct[c >> 3];
+        const int t = info >> 5, side = (info >> 4) & 1, j = (info & 15) * 8 + (c & 7);
         const Place p = s_place[side][t];
         const int slot = p.slot_cls_r & 0xff, rr = p.slot_cls_r >> 16;
         keep[u] = rr - j * 8;
