@@ -242,39 +242,55 @@ __global__ void __launch_bounds__(1024) alloc_kernel(DevView v0, int layer, int 
       off_b += nnew * cls;
     }
     __syncthreads();
-    // tile lists: K per class (ascending sequence), V per sequence (ascending class); one warp per list, the lanes
-    // write a key's run of consecutive tile ids together
+    // tile lists: K per class (ascending sequence), V per sequence (ascending class); one warp per list, one lane per
+    // key of the list: the lanes read their keys' tables together, a warp scan places their runs of tile ids
     if (warp < v.NC) {
       int* cnt = v.kcc(layer);
       int* list = v.kct(layer) + (size_t)warp * v.NT;
       int run = cnt[warp];
-      for (int s = 0; s < v.S; ++s) {
-        const int k = s * v.NC + warp;
-        const int c = v.key_cnt[k], old = v.key_old_fill[k];
-        const int nnew = ceil_div(old + c, TILE) - ceil_div(old, TILE);
-        const int first = v.key_first_id[k];
-        for (int j = lane; j < nnew; j += 32) list[run + j] = first + j;
-        run += nnew;
+      for (int s0 = 0; s0 < v.S; s0 += 32) {
+        const int s = s0 + lane;
+        int nnew = 0, first = 0;
+        if (s < v.S) {
+          const int k = s * v.NC + warp;
+          const int c = v.key_cnt[k], old = v.key_old_fill[k];
+          nnew = ceil_div(old + c, TILE) - ceil_div(old, TILE);
+          first = v.key_first_id[k];
+        }
+        int incl = nnew;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+          const int u = __shfl_up_sync(0xffffffffu, incl, o);
+          if (lane >= o) incl += u;
+        }
+        int* dst = list + run + incl - nnew;
+        for (int j = 0; j < nnew; ++j) dst[j] = first + j;
+        run += __shfl_sync(0xffffffffu, incl, 31);
       }
-      __syncwarp();
       if (lane == 0) cnt[warp] = run;
     }
     for (int s = warp; s < v.S; s += 32) {
       int* list = v.svt(layer) + (size_t)s * v.TPS;
-      int run = v.svc(layer)[s];
-      int add = 0;
-      for (int c = 0; c < v.NC; ++c) {
-        const int k = half + s * v.NC + c;
+      const int run0 = v.svc(layer)[s];
+      int nnew = 0, first = 0, add = 0;
+      if (lane < v.NC) {
+        const int k = half + s * v.NC + lane;
         const int cn = v.key_cnt[k], old = v.key_old_fill[k];
-        const int nnew = ceil_div(old + cn, TILE) - ceil_div(old, TILE);
-        const int first = v.key_first_id[k];
-        for (int j = lane; j < nnew; j += 32) list[run + j] = first + j;
-        run += nnew;
-        add += v.key_cnt[s * v.NC + c];
+        nnew = ceil_div(old + cn, TILE) - ceil_div(old, TILE);
+        first = v.key_first_id[k];
+        add = v.key_cnt[s * v.NC + lane];
       }
-      __syncwarp();
-      if (lane == 0) {
-        v.svc(layer)[s] = run;
+      int incl = nnew;
+#pragma unroll
+      for (int o = 1; o < 32; o <<= 1) {
+        const int u = __shfl_up_sync(0xffffffffu, incl, o);
+        if (lane >= o) incl += u;
+        add += __shfl_xor_sync(0xffffffffu, add, o);              // butterfly: every lane ends with the total
+      }
+      int* dst = list + run0 + incl - nnew;
+      for (int j = 0; j < nnew; ++j) dst[j] = first + j;
+      if (lane == 31) {
+        v.svc(layer)[s] = run0 + incl;
         stok[s] += add;
       }
     }
