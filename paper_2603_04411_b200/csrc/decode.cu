@@ -378,17 +378,20 @@ constexpr int MG_JGROUPS = MG_THREADS / 64;
 
 template <bool BF16>
 __global__ void __launch_bounds__(MG_THREADS)
-merge_kernel(DevView v, const unsigned short* __restrict__ Uinv_v, int n_splits, int hp, void* __restrict__ out) {
-  extern __shared__ float sAcc[];                    // [hp][d_kv] normalised spectral accumulators, then [MG_JGROUPS][hp][128]
+merge_kernel(DevView v, const unsigned short* __restrict__ Uinv_v, int n_splits, int hp, int ns, int n_seq, void* __restrict__ out) {
+  extern __shared__ float sAcc[];                    // [rows][d_kv] normalised spectral accumulators, then [MG_JGROUPS][rows][128]
   __shared__ float sInvL[8];
   // blockIdx.y = KV head g and which hp of its query heads (hp divides the group size; small batches use hp < group
-  // size so that the grid still fills the device)
-  const int qs = blockIdx.x, parts = v.rep / hp, g = blockIdx.y / parts, tid = threadIdx.x;
-  const int Hq = v.Hq, d_kv = v.d_kv, REP = hp;
+  // size so that the grid still fills the device); blockIdx.x = ns query slots that share the reads of U_V^-1 (large
+  // batches).  A row of this CTA is (slot, head): at most 8 rows.
+  const int qs0 = blockIdx.x * ns, parts = v.rep / hp, g = blockIdx.y / parts, tid = threadIdx.x;
+  const int Hq = v.Hq, d_kv = v.d_kv;
+  const int REP = min(ns, n_seq - qs0) * hp;                    // rows
   const int head0 = g * v.rep + (blockIdx.y % parts) * hp;      // first query head of this CTA
   if (tid < REP) {
+    const int qs = qs0 + tid / hp, head = head0 + tid % hp;
     float l = 0.f;
-    for (int s = 0; s < n_splits; ++s) l += v.part_l[((size_t)qs * n_splits + s) * Hq + head0 + tid];
+    for (int s = 0; s < n_splits; ++s) l += v.part_l[((size_t)qs * n_splits + s) * Hq + head];
     sInvL[tid] = l > 0.f ? 1.f / l : 0.f;
   }
   __syncthreads();
@@ -399,7 +402,7 @@ merge_kernel(DevView v, const unsigned short* __restrict__ Uinv_v, int n_splits,
 #pragma unroll
     for (int u = 0; u < 4; ++u) {
       const int i = min(i0 + u * MG_THREADS, REP * d_kv - 1), hh = i / d_kv, j = i - hh * d_kv;
-      p[u] = v.part_acc + (((size_t)qs * n_splits) * Hq + head0 + hh) * d_kv + j;
+      p[u] = v.part_acc + (((size_t)(qs0 + hh / hp) * n_splits) * Hq + head0 + hh % hp) * d_kv + j;
     }
     for (int s = 0; s < n_splits; ++s) {
 #pragma unroll
@@ -445,7 +448,7 @@ merge_kernel(DevView v, const unsigned short* __restrict__ Uinv_v, int n_splits,
 #pragma unroll
     for (int k = 0; k < MG_JGROUPS; ++k) val += red[k * REP * 128 + i];        // fixed order
     const int h = i >> 7, dc = i & 127;
-    const size_t oi = ((size_t)qs * Hq + head0 + h) * HEAD_DIM + dc;
+    const size_t oi = ((size_t)(qs0 + h / hp) * Hq + head0 + h % hp) * HEAD_DIM + dc;
     if (v.out_dtype == TWKV_F32) reinterpret_cast<float*>(out)[oi] = val;
     else if (v.out_dtype == TWKV_BF16) reinterpret_cast<unsigned short*>(out)[oi] = from_f32<true>(val);
     else reinterpret_cast<unsigned short*>(out)[oi] = from_f32<false>(val);
@@ -475,14 +478,18 @@ static cudaError_t launch_decode_t(const DevView& v, int layer, const LayerParam
     ProfScope ps(TWKV_K_VACC, st);
     vacc_kernel<BF16, 2><<<vgrid, 512, va_smem, st>>>(v, layer, seq_ids, n_splits);
   }
-  // query heads per merge CTA: the whole group when the batch fills the device, fewer (a divisor) for small batches
+  // query heads per merge CTA: the whole group when the batch fills the device, fewer (a divisor) for small batches;
+  // query slots per CTA: more than one (they share the reads of U_V^-1) while the grid still fills most of the device
   int hp = v.rep;
   while (hp % 2 == 0 && 2 * n_seq * v.Hkv * (v.rep / hp) < sm_count) hp /= 2;
-  const size_t mg_a = (size_t)hp * v.d_kv * 4, mg_b = (size_t)MG_JGROUPS * hp * 128 * 4;
+  int ns = 1;
+  while (2 * ns * hp <= 8 && 4 * (n_seq * v.Hkv * (v.rep / hp) / (2 * ns)) >= 3 * sm_count) ns *= 2;
+  const size_t mg_a = (size_t)ns * hp * v.d_kv * 4, mg_b = (size_t)MG_JGROUPS * ns * hp * 128 * 4;
   const size_t mg_smem = mg_a > mg_b ? mg_a : mg_b;
   {
     ProfScope ps(TWKV_K_MERGE, st);
-    merge_kernel<BF16><<<dim3(n_seq, v.Hkv * (v.rep / hp)), MG_THREADS, mg_smem, st>>>(v, reinterpret_cast<const unsigned short*>(lp.Uinv_v), n_splits, hp, out);
+    merge_kernel<BF16><<<dim3((n_seq + ns - 1) / ns, v.Hkv * (v.rep / hp)), MG_THREADS, mg_smem, st>>>(
+        v, reinterpret_cast<const unsigned short*>(lp.Uinv_v), n_splits, hp, ns, n_seq, out);
   }
   count_launch(4);
   return cudaGetLastError();

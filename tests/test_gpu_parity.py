@@ -166,6 +166,17 @@ def test_config3_shape_shuffled_positions_and_append(B):
     assert max_abs < MAX_ABS and rel_l2 < REL_L2, (max_abs, rel_l2)
 
 
+def test_large_batch_of_short_sequences(B):
+    # 37 sequences x 150 tokens: the merge kernel then takes two query slots per CTA (they share the reads of U_V^-1),
+    # with a last group of one; the V pass runs with few splits per sequence
+    li = to_cuda(workloads.build_layer(61, n_seq=37, ctx=150, n_q_heads=32, mode="forced",
+                                       level_probs=(0.10, 0.20, 0.40, 0.30), shuffle_positions=True))
+    ranks = li.ranks.cpu().numpy().astype(np.int64)
+    (max_abs, rel_l2), got, _ = run_case(B, li, ranks, mode=B.TWKV_GATE_FORCED)
+    assert np.all(np.isfinite(got))
+    assert max_abs < MAX_ABS and rel_l2 < REL_L2, (max_abs, rel_l2)
+
+
 def test_tile_boundaries_and_single_token(B):
     for ctx in (1, 127, 128, 129):
         li = to_cuda(workloads.build_layer(20 + ctx, n_seq=2, ctx=ctx, n_q_heads=16, n_kv_heads=4, mode="forced",
