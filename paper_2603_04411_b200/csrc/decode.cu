@@ -26,8 +26,8 @@ __device__ __forceinline__ unsigned ktile_cost(int cls) {
   // cycles per tile of the K-score kernel by rank class, measured inside the kernel on the benchmark's mix of classes
   // (8 KV heads): a fixed part (rotation factors, score read-out, the per-slab epilogue chain) plus a per-panel part;
   // classes above 8 run as two passes.  Only the ratios matter.
-  constexpr unsigned kCost[TWKV_MAX_CLASSES] = {13900u, 16400u, 19900u, 22800u, 26900u, 29300u, 32600u, 35600u,
-                                                45100u, 46800u, 50700u, 54000u, 58200u, 63300u, 64700u, 68300u};
+  constexpr unsigned kCost[TWKV_MAX_CLASSES] = {17800u, 19400u, 22100u, 25100u, 29100u, 31700u, 34900u, 37900u,
+                                                50200u, 51200u, 55300u, 58800u, 62800u, 67500u, 68500u, 71700u};
   return kCost[min(max(cls, 1), TWKV_MAX_CLASSES) - 1];
 }
 

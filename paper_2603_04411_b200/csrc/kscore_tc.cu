@@ -7,13 +7,14 @@
 // The first product is a tcgen05.mma chain (M = 128, N = 128, K = 16 per instruction) whose fp32
 // accumulator lives in TMEM; X^_K panels and panels of the pre-transposed U_K^-1 arrive by TMA with
 // the 128-byte swizzle, which is the K-major operand layout the MMA reads from shared memory.
-// Epilogue warps pull the slab out of TMEM, rotate it in fp32, round it to f16 and store it back to
-// TMEM, from where it is the A operand of the second product (N = 16, the group's heads padded);
+// Epilogue warps pull the slab out of TMEM, rotate it in fp32, split it into a high and a low f16 part and
+// store both back to TMEM, from where they are the A operands of the second product (N = 16, the group's
+// heads padded; one product per part);
 // its accumulator S stays in TMEM until the tile's last slab, so RoPE is the only per-element
 // CUDA-core work.  Both sums are linear in X^_K, so a class wider than 8 panels runs as two passes
 // over its panels that accumulate into the same S.
 //
-// Tensor memory (512 columns): slab accumulators 2 x 128 | rotated keys 2 x 64 | S 8 x 16.
+// Tensor memory (512 columns): slab accumulators 2 x 128 | rotated keys, high and low part, 64 each | S 8 x 16.
 // Warp roles (384 threads, one persistent CTA per SM working through a contiguous, cost-balanced piece of the tile list):
 //   warp 0      TMA producer of U_K^-1 panels (ring, one lane per stage)
 //   warp 1      issuer of the main products (one elected lane; owns the TMEM allocation)
@@ -22,8 +23,9 @@
 //   warp 11     issuer of the score products (one elected lane)
 // All waits are bounded (tc_util.cuh); a wait that runs out ends the kernel with TWKV_ERR_TIMEOUT.
 //
-// Precision: X^_K, U_K^-1 keep the cache dtype with fp32 accumulation; rotated keys and queries enter
-// the score product as f16 (keys saturate at +-65504; a bf16 query must be finite in f16).
+// Precision: X^_K, U_K^-1 keep the cache dtype with fp32 accumulation; queries enter the score product as
+// f16 (a bf16 query must be finite in f16), rotated keys as the sum of two f16 (21 significant bits; they
+// saturate at +-65504).
 #include "twkv_dev.h"
 #include "tc_util.cuh"
 
@@ -236,12 +238,13 @@ kscore_tc_kernel(const __grid_constant__ CUtensorMap map_blocks, const __grid_co
           const bool last_pass = p0 + KT_A_SLOTS >= cls;
           for (int sl = 0; sl < Hkv; ++sl, ++sc) {
             const int g = sl + g_rot < Hkv ? sl + g_rot : sl + g_rot - Hkv;
-            const uint32_t kb = sc & 1u;
-            if (!(ok = mbar_wait_thin(kr_full + 8 * kb, (sc >> 1) & 1u, abort_flag))) break;
+            if (!(ok = mbar_wait_thin(kr_full, sc & 1u, abort_flag))) break;
             fence_after_sync();
-            mma_f16_ts_k128(tmem_base + TM_S + 16 * g, tmem_base + TM_KR + 64 * kb, q_lo0 + g * (1024 >> 4), KT_Q_PANEL_BYTES >> 4, idesc_s,
+            // the rotated keys come as a high and a low f16 part (their sum carries 21 bits): two products into the same S
+            mma_f16_ts_k128(tmem_base + TM_S + 16 * g, tmem_base + TM_KR, q_lo0 + g * (1024 >> 4), KT_Q_PANEL_BYTES >> 4, idesc_s,
                             p0 > 0 ? 1u : 0u);
-            mma_commit(kr_empty + 8 * kb);
+            mma_f16_ts_k128(tmem_base + TM_S + 16 * g, tmem_base + TM_KR + 64, q_lo0 + g * (1024 >> 4), KT_Q_PANEL_BYTES >> 4, idesc_s, 1u);
+            mma_commit(kr_empty);
             if (last_pass && sl == Hkv - 1) mma_commit(s_full);        // the tile's scores are complete
           }
         }
@@ -323,31 +326,49 @@ kscore_tc_kernel(const __grid_constant__ CUtensorMap map_blocks, const __grid_co
         if (!slab_ready && !(ok = __all_sync(0xffffffffu, mbar_wait(slab_full + 8 * buf, par, abort_flag)))) break;
         fence_after_sync();
         const uint32_t slab = lane_addr + TM_SLAB + buf * 128 + hf * 32;
-        const uint32_t kr = lane_addr + TM_KR + buf * 64 + hf * 16;
+        const uint32_t kr = lane_addr + TM_KR + hf * 16;                     // high parts; the low parts 64 columns on
+        const uint32_t kr_par = (sc & 1u) ^ 1u;
         uint32_t lo[32], hi[32];
         tmem_ld32(slab, lo);
         tmem_ld32(slab + 64, hi);
-        const bool kr_probe = mbar_try(kr_empty + 8 * buf, par ^ 1u);
+        const bool kr_probe = mbar_try(kr_empty, kr_par);
         tmem_ld_wait();
         fence_before_sync();
         __syncwarp();
         if (lane == 0) mbar_arrive(slab_empty + 8 * buf);                    // the slab accumulator is free for slab n + 2
-        uint32_t p1[16], p2[16];
+        // a rotated value v leaves as two f16: v with its low 13 mantissa bits cleared (exact in f16) and the rest
+        // (rounded to f16: 2^-21 of v instead of the 2^-11 of one f16), so that the score error stays far below the bar
+        // even where a few key channels carry most of the magnitude
 #pragma unroll
-        for (int t = 0; t < 16; ++t) {
-          const uint64_t L = f2_pack_bits(lo[2 * t], lo[2 * t + 1]), H = f2_pack_bits(hi[2 * t], hi[2 * t + 1]);
-          p1[t] = f2_to_f16x2_sat(f2_sub(f2_mul(L, cs2[t]), f2_mul(H, sn2[t])));      // lo cos - hi sin
-          p2[t] = f2_to_f16x2_sat(f2_fma(L, sn2[t], f2_mul(H, cs2[t])));              // hi cos + lo sin
+        for (int hb = 0; hb < 2; ++hb) {
+          uint32_t p1[8], p2[8], l1[8], l2[8];
+#pragma unroll
+          for (int t8 = 0; t8 < 8; ++t8) {
+            const int t = hb * 8 + t8;
+            const uint64_t L = f2_pack_bits(lo[2 * t], lo[2 * t + 1]), H = f2_pack_bits(hi[2 * t], hi[2 * t + 1]);
+            const uint64_t a = f2_sub(f2_mul(L, cs2[t]), f2_mul(H, sn2[t]));           // lo cos - hi sin
+            const uint64_t b = f2_fma(L, sn2[t], f2_mul(H, cs2[t]));                   // hi cos + lo sin
+            const uint64_t ah = a & 0xFFFFE000FFFFE000ull, bh = b & 0xFFFFE000FFFFE000ull;
+            p1[t8] = f2_to_f16x2_sat(ah);
+            p2[t8] = f2_to_f16x2_sat(bh);
+            l1[t8] = f2_to_f16x2_sat(f2_sub(a, ah));
+            l2[t8] = f2_to_f16x2_sat(f2_sub(b, bh));
+          }
+          if (hb == 0) {
+            if (!__all_sync(0xffffffffu, kr_probe) && !(ok = __all_sync(0xffffffffu, mbar_wait(kr_empty, kr_par, abort_flag)))) break;
+            fence_after_sync();
+          }
+          tmem_st8(kr + 8 * hb, p1);                                        // dims d -> column d / 2
+          tmem_st8(kr + 32 + 8 * hb, p2);                                   // dims 64 + d
+          tmem_st8(kr + 64 + 8 * hb, l1);
+          tmem_st8(kr + 96 + 8 * hb, l2);
         }
-        if (!__all_sync(0xffffffffu, kr_probe) && !(ok = __all_sync(0xffffffffu, mbar_wait(kr_empty + 8 * buf, par ^ 1u, abort_flag)))) break;
-        fence_after_sync();
-        tmem_st16(kr, p1);                                                  // dims d -> column d / 2
-        tmem_st16(kr + 32, p2);                                             // dims 64 + d
+        if (!ok) break;
         const bool next_probe = mbar_try(slab_full + 8 * (buf ^ 1u), ((sc + 1) >> 1) & 1u);
         tmem_st_wait();
         fence_before_sync();
         __syncwarp();
-        if (lane == 0) mbar_arrive(kr_full + 8 * buf);
+        if (lane == 0) mbar_arrive(kr_full);
         slab_ready = __all_sync(0xffffffffu, next_probe);
       }
       if (!ok) break;

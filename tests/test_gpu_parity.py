@@ -177,6 +177,26 @@ def test_large_batch_of_short_sequences(B):
     assert max_abs < MAX_ABS and rel_l2 < REL_L2, (max_abs, rel_l2)
 
 
+def test_long_context_full_size(B):
+    # the long-context workload at its full size: one sequence of 131072 tokens, 64 query heads on 8 KV heads, bf16,
+    # heavy-tailed outlier channels, full rank at the sink and the recent window and low rank between
+    li = to_cuda(workloads.config(4))
+    ranks = li.ranks.cpu().numpy().astype(np.int64)
+    (max_abs, rel_l2), got, _ = run_case(B, li, ranks, mode=B.TWKV_GATE_FORCED)
+    assert np.all(np.isfinite(got))
+    assert max_abs < MAX_ABS and rel_l2 < REL_L2, (max_abs, rel_l2)
+
+
+def test_high_batch_full_size_sampled(B):
+    # the high-batch workload at its full size (64 sequences x 8192 tokens, shuffled positions, one compress call of
+    # four pieces); the cache image is compared in full, the attention output on three sequences
+    li = to_cuda(workloads.config(3))
+    ranks = li.ranks.cpu().numpy().astype(np.int64)
+    (max_abs, rel_l2), got, _ = run_case(B, li, ranks, mode=B.TWKV_GATE_FORCED, decode_seqs=[0, 41, 63])
+    assert np.all(np.isfinite(got))
+    assert max_abs < MAX_ABS and rel_l2 < REL_L2, (max_abs, rel_l2)
+
+
 def test_tile_boundaries_and_single_token(B):
     for ctx in (1, 127, 128, 129):
         li = to_cuda(workloads.build_layer(20 + ctx, n_seq=2, ctx=ctx, n_q_heads=16, n_kv_heads=4, mode="forced",
