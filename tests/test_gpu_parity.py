@@ -169,8 +169,7 @@ def test_config3_shape_shuffled_positions_and_append(B):
 def test_large_batch_of_short_sequences(B):
     # 37 sequences x 150 tokens: the merge kernel then takes two query slots per CTA (they share the reads of U_V^-1),
     # with a last group of one; the V pass runs with few splits per sequence
-    li = to_cuda(workloads.build_layer(61, n_seq=37, ctx=150, n_q_heads=32, mode="forced",
-                                       level_probs=(0.10, 0.20, 0.40, 0.30), shuffle_positions=True))
+    li = to_cuda(workloads.config(3, ctx=150, n_seq=37))
     ranks = li.ranks.cpu().numpy().astype(np.int64)
     (max_abs, rel_l2), got, _ = run_case(B, li, ranks, mode=B.TWKV_GATE_FORCED)
     assert np.all(np.isfinite(got))
@@ -193,6 +192,16 @@ def test_high_batch_full_size_sampled(B):
     li = to_cuda(workloads.config(3))
     ranks = li.ranks.cpu().numpy().astype(np.int64)
     (max_abs, rel_l2), got, _ = run_case(B, li, ranks, mode=B.TWKV_GATE_FORCED, decode_seqs=[0, 41, 63])
+    assert np.all(np.isfinite(got))
+    assert max_abs < MAX_ABS and rel_l2 < REL_L2, (max_abs, rel_l2)
+
+
+def test_mixed_layer_workload_full_size_sampled(B):
+    # one layer of the 32-layer decode workload at its full size (32 sequences x 16384 tokens, Dirichlet level mix);
+    # levels and statistics on every token, the attention output on two sequences
+    li = to_cuda(workloads.config(5))
+    ranks = li.ranks.cpu().numpy().astype(np.int64)
+    (max_abs, rel_l2), got, _ = run_case(B, li, ranks, mode=B.TWKV_GATE_FORCED, decode_seqs=[3, 30], check_image=False)
     assert np.all(np.isfinite(got))
     assert max_abs < MAX_ABS and rel_l2 < REL_L2, (max_abs, rel_l2)
 
