@@ -175,8 +175,9 @@ twkv_status twkv_cache_stats(twkv_cache* cache, int layer, void* stream, twkv_st
 twkv_status twkv_cache_layout(const twkv_cache* cache, twkv_layout* out /*host*/);
 /*
  * Gate ranks without any caller-provided scratch (the paper has no counterpart; this is a
- * convenience of the library).  Computes, for n_tok tokens, the same (r_K, r_V) that twkv_compress
- * produces in TWKV_GATE_COMPUTE mode (Eq. 5, 6, 8), but needs no cache and allocates nothing: the
+ * convenience of the library).  Computes, for n_tok tokens, the (r_K, r_V) of Eq. 5, 6, 8 as twkv_compress
+ * does in TWKV_GATE_COMPUTE mode (both evaluate the formulas in fp32; they give the same rank except where a
+ * cumulative softmax sum lies within fp32 rounding of tau), but needs no cache and allocates nothing: the
  * fp32 logits are staged in a 4 MiB array that is part of the library image and is resident on
  * every GPU that loads the library, until the process exits.  It is meant for callers that cannot
  * obtain device memory at the point of the call, for instance a scheduler that sizes cache blocks

@@ -78,7 +78,7 @@ constexpr int GATE_TC_MIN_TOKENS = 1024;   // calls at least this large run the 
 struct Offsets {
   size_t status, pflags, rope_lo, rope_hi, n_tiles, tile_desc, tile_aux, tile_rank, fill, key_last, kclass_count,
       kclass_tiles, seq_vcount, seq_vtiles, seq_tokens, rank_sums, hist, key_cnt, key_old_fill, key_first_id,
-      key_first_base, key_old_last, scores, seqmax, qslot, klist, klist_count, klist_cost, cta_start, part_acc, part_l, gate_scratch, stats_buf, tables_end, prep_uinvT, prep_wT,
+      key_first_base, key_old_last, scores, seqmax, qslot, klist, klist_count, klist_cost, cta_start, part_acc, part_l, gate_scratch, gate_fix, stats_buf, tables_end, prep_uinvT, prep_wT,
       blocks, end_fixed;
 };
 
@@ -122,8 +122,8 @@ static Offsets layout_of(const twkv_config* c, const Dims& d) {
   Offsets o;
   const size_t Ls = c->n_layers, S = c->max_seqs, NT = d.NT, NK = d.NK, Hq = c->n_q_heads;
   o.status = L.alloc(8 * sizeof(int));
-  o.rope_lo = L.alloc((size_t)ROPE_SMALL_ROWS * 64 * sizeof(float2));
-  o.rope_hi = L.alloc((size_t)ROPE_HI * 64 * sizeof(float2));
+  o.rope_lo = L.alloc((size_t)ROPE_LO * 32 * sizeof(float4));
+  o.rope_hi = L.alloc((size_t)ROPE_HI * 32 * sizeof(float4));
   o.n_tiles = L.alloc(Ls * 2 * sizeof(int));
   o.tile_desc = L.alloc(Ls * 2 * NT * sizeof(int4));
   o.tile_aux = L.alloc(Ls * 2 * NT * TILE * sizeof(int));
@@ -158,6 +158,7 @@ static Offsets layout_of(const twkv_config* c, const Dims& d) {
     const size_t small = (size_t)GATE_PIECE * 2 * d.d_kv * sizeof(float), fused = gate_tc_stage_bytes(MAX_PLAN_CTAS < 160 ? MAX_PLAN_CTAS : 160, d.d_kv);
     o.gate_scratch = L.alloc(small > fused ? small : fused);
   }
+  o.gate_fix = L.alloc(gate_tc_fix_bytes());
   o.stats_buf = L.alloc(64 * sizeof(unsigned long long));
   o.prep_uinvT = L.alloc(Ls * (size_t)d.d_kv * d.d_kv * 2, 1024);
   o.prep_wT = L.alloc(Ls * 2 * (size_t)d.d_kv * d.d_kv * 2, 1024);
@@ -229,7 +230,7 @@ static void fill_view(twkv_cache* c) {
   const size_t nb = (c->pool_bytes - o.blocks) / BLOCK_BYTES;
   v.n_blocks = (int)(nb > 0x7fffffffull ? 0x7fffffffull : nb);
   v.status = (int*)(p + o.status); v.pflags = (int*)(p + o.pflags); v.batch = d.batch;
-  v.rope_lo = (float2*)(p + o.rope_lo); v.rope_hi = (float2*)(p + o.rope_hi);
+  v.rope_lo = (float4*)(p + o.rope_lo); v.rope_hi = (float4*)(p + o.rope_hi);
   v.blocks = p + o.blocks;
   v.n_tiles = (int*)(p + o.n_tiles); v.tile_desc = (int4*)(p + o.tile_desc); v.tile_aux = (int*)(p + o.tile_aux);
   v.tile_rank = (unsigned short*)(p + o.tile_rank); v.fill = (int*)(p + o.fill); v.key_last = (int*)(p + o.key_last);
@@ -244,6 +245,7 @@ static void fill_view(twkv_cache* c) {
   v.klist_cost = (unsigned*)(p + o.klist_cost); v.cta_start = (int*)(p + o.cta_start);
   v.part_acc = (float*)(p + o.part_acc); v.part_l = (float*)(p + o.part_l);
   v.gate_scratch = (float*)(p + o.gate_scratch);
+  v.gate_fix = (int4*)(p + o.gate_fix);
 }
 
 twkv_status twkv_cache_reset(twkv_cache* c, void* stream) {
@@ -381,6 +383,9 @@ twkv_status twkv_compress(twkv_cache* c, int layer, const void* K, const void* V
     maps.wv = (pairs ? c->map_wT_half : c->map_wT)[2 * (size_t)layer + 1];
     if (!make_tmap_2d(&maps.xk, K, (uint64_t)n_tok, d, (uint64_t)d * 2, TILE) ||
         !make_tmap_2d(&maps.xv, V, (uint64_t)n_tok, d, (uint64_t)d * 2, TILE)) return TWKV_ERR_CUDA;
+    const unsigned char* wT = c->pool + c->off.prep_wT + (size_t)layer * 2 * d * d * 2;
+    maps.raw = GateRaw{(const unsigned short*)K, (const unsigned short*)V, (const unsigned short*)wT,
+                       (const unsigned short*)(wT + (size_t)d * d * 2), v.gate_fix, v.status + 2};
     if (launch_gate_ranks_tc(v, maps, c->params[layer], n_tok, levels, c->sm_count, pairs, st) != cudaSuccess) return TWKV_ERR_CUDA;
   } else if (mode == TWKV_GATE_COMPUTE) {
     for (int lo = 0; lo < n_tok; lo += GATE_PIECE) {

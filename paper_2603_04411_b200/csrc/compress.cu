@@ -505,27 +505,28 @@ cudaError_t launch_compress_pieces(const DevView& v, int layer, const void* K, c
 }
 
 // ------------------------------------------------------------------------------------------
-// Three-level RoPE tables, built once per cache in fp64: angle(pos, i) = pos * base^(-2i/128),
-// pos = hi * 256 + mid * 16 + lo.  cos/sin of the sum come from the angle-addition formulas at use; the
-// 32 rows of the two small tables fit in shared memory, a tile's rows share a handful of `hi` rows.
+// Two-level RoPE tables, built once per cache in fp64: angle(pos, i) = pos * base^(-2i/128), pos = hi * 16 + lo.
+// cos/sin of the sum come from the angle-addition formulas at use (one complex product per frequency); the 16 `lo`
+// rows fit in shared memory, the 8 KB-apart `hi` rows a tile touches stay in L2 (1 MiB per 32768 positions).
+// Entries are stored per pair of frequencies as (cos, cos, sin, sin), the packed form the K-score kernel multiplies.
 // ------------------------------------------------------------------------------------------
-__global__ void rope_tables_kernel(float2* small, float2* hi, double base) {
-  const int i = threadIdx.x;                                   // frequency 0..63
+__global__ void rope_tables_kernel(float4* lo, float4* hi, double base) {
+  const int t = threadIdx.x;                                   // frequency pair (2 t, 2 t + 1)
   const int row = blockIdx.x;
-  const double theta = pow(base, -2.0 * (double)i / (double)HEAD_DIM);
-  double s, c;
-  if (row < ROPE_SMALL_ROWS) {
-    sincos(row < 16 ? (double)(row * 16) * theta : (double)(row - 16) * theta, &s, &c);
-    small[row * 64 + i] = make_float2((float)c, (float)s);
+  const double th0 = pow(base, -2.0 * (double)(2 * t) / (double)HEAD_DIM), th1 = pow(base, -2.0 * (double)(2 * t + 1) / (double)HEAD_DIM);
+  double s0, c0, s1, c1;
+  if (row < ROPE_LO) {
+    sincos((double)row * th0, &s0, &c0);
+    sincos((double)row * th1, &s1, &c1);
+    lo[row * 32 + t] = make_float4((float)c0, (float)c1, (float)s0, (float)s1);
   }
-  if (row < ROPE_HI) {
-    sincos((double)row * (double)ROPE_LO * theta, &s, &c);
-    hi[row * 64 + i] = make_float2((float)c, (float)s);
-  }
+  sincos((double)row * (double)ROPE_LO * th0, &s0, &c0);
+  sincos((double)row * (double)ROPE_LO * th1, &s1, &c1);
+  hi[(size_t)row * 32 + t] = make_float4((float)c0, (float)c1, (float)s0, (float)s1);
 }
 
 cudaError_t launch_rope_tables(const DevView& v, float rope_base, cudaStream_t st) {
-  rope_tables_kernel<<<ROPE_HI, 64, 0, st>>>(v.rope_lo, v.rope_hi, (double)rope_base);
+  rope_tables_kernel<<<ROPE_HI, 32, 0, st>>>(v.rope_lo, v.rope_hi, (double)rope_base);
   count_launch();
   return cudaGetLastError();
 }

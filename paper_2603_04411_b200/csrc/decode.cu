@@ -149,8 +149,10 @@ vacc_kernel(DevView v, int layer, const int* __restrict__ seq_ids, int n_splits)
   constexpr int TPT = 2 * NWG;                                     // threads per token in the probability phase, 8 heads each
   extern __shared__ __align__(128) unsigned char smem[];
   unsigned char* sV = smem;                                        // [STAGES][128 tokens][128 B]
-  unsigned char* sP = smem + VA_STAGES * 16384;                    // [2][32 heads][256 B]
-  float* sM = reinterpret_cast<float*>(sP + 2 * 8192);             // [32] reference max per head
+  // [2][32 heads][256 B]; bf16 keeps a second pair of buffers for the low parts of the weights (see below)
+  unsigned char* sP = smem + VA_STAGES * 16384;
+  constexpr int P_BYTES = (BF16 ? 4 : 2) * 8192;
+  float* sM = reinterpret_cast<float*>(sP + P_BYTES);              // [32] reference max per head
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int mt = warp >> 3, cw = warp & 7;                         // row tile, column group
@@ -164,7 +166,7 @@ vacc_kernel(DevView v, int layer, const int* __restrict__ seq_ids, int n_splits)
   const int4* desc = v.desc(layer, 1);
   const int* aux = v.aux(layer, 1);
 
-  for (int i = tid; i < 2 * 8192 / 4; i += NT) reinterpret_cast<unsigned*>(sP)[i] = 0u;
+  for (int i = tid; i < P_BYTES / 4; i += NT) reinterpret_cast<unsigned*>(sP)[i] = 0u;
   if (tid < 32) sM[tid] = tid < nh ? dec_ordered(v.seqmax[qs * Hq + h0 + tid]) : 0.f;
   // Descriptors of this split's tiles (the k-th is list[split + k * n_splits]) are kept in a ring of 64 in
   // shared memory, refilled 16 at a time well ahead of both cursors, so neither the copy cursor nor the
@@ -277,7 +279,13 @@ vacc_kernel(DevView v, int layer, const int* __restrict__ seq_ids, int n_splits)
         if (h < nh) {
           const float pv = __expf(sc_next[hh] - sM[h]);             // -inf for rows past the last token: weight 0
           const int chunk = slot >> 3;
-          *reinterpret_cast<unsigned short*>(P + h * 256 + ((chunk ^ (h & 7)) << 4) + (slot & 7) * 2) = from_f32<BF16>(pv);
+          const unsigned short ph = from_f32<BF16>(pv);
+          *reinterpret_cast<unsigned short*>(P + h * 256 + ((chunk ^ (h & 7)) << 4) + (slot & 7) * 2) = ph;
+          // bf16 keeps 8 bits of a weight: with few tokens per sequence that rounding alone reaches 1e-3 of the output,
+          // so the remainder goes into a second operand (16 bits in all, like an f16 weight's 11 where it matters)
+          if constexpr (BF16)
+            *reinterpret_cast<unsigned short*>(P + 16384 + h * 256 + ((chunk ^ (h & 7)) << 4) + (slot & 7) * 2) =
+                from_f32<true>(pv - to_f32<true>(ph));
         }
       }
     }
@@ -318,8 +326,13 @@ vacc_kernel(DevView v, int layer, const int* __restrict__ seq_ids, int n_splits)
 #pragma unroll
         for (int k2 = 0; k2 < 4; ++k2) {                           // two k-steps (32 tokens) per iteration
           unsigned a0[4], a1[4];
+          [[maybe_unused]] unsigned l0[4], l1[4];
           ldsm_x4(a0, frag_a_off[2 * k2] + pOff);
           ldsm_x4(a1, frag_a_off[2 * k2 + 1] + pOff);
+          if constexpr (BF16) {
+            ldsm_x4(l0, frag_a_off[2 * k2] + pOff + 16384u);
+            ldsm_x4(l1, frag_a_off[2 * k2 + 1] + pOff + 16384u);
+          }
 #pragma unroll
           for (int jj = 0; jj < gn; ++jj) {
             if (jbase + jj < TWKV_MAX_CLASSES) {
@@ -327,9 +340,16 @@ vacc_kernel(DevView v, int layer, const int* __restrict__ seq_ids, int n_splits)
               ldsm_x4_t(b, vAddr[jj] + k2 * 4096);
               mma16816<BF16>(acc[jbase + jj < TWKV_MAX_CLASSES ? jbase + jj : 0], a0, b[0], b[1]);
               mma16816<BF16>(acc[jbase + jj < TWKV_MAX_CLASSES ? jbase + jj : 0], a1, b[2], b[3]);
+              if constexpr (BF16) {
+                mma16816<BF16>(acc[jbase + jj < TWKV_MAX_CLASSES ? jbase + jj : 0], l0, b[0], b[1]);
+                mma16816<BF16>(acc[jbase + jj < TWKV_MAX_CLASSES ? jbase + jj : 0], l1, b[2], b[3]);
+              }
             }
           }
-          if (jbase == 0 && cw == 0) { mma16816<BF16>(accl, a0, ones, ones); mma16816<BF16>(accl, a1, ones, ones); }
+          if (jbase == 0 && cw == 0) {
+            mma16816<BF16>(accl, a0, ones, ones); mma16816<BF16>(accl, a1, ones, ones);
+            if constexpr (BF16) { mma16816<BF16>(accl, l0, ones, ones); mma16816<BF16>(accl, l1, ones, ones); }
+          }
         }
       };
       auto by_size = [&](auto J0) {
@@ -467,7 +487,7 @@ static cudaError_t launch_decode_t(const DevView& v, int layer, const LayerParam
     cudaError_t e = launch_kscore_tc(v, layer, maps->blocks, maps->uinvT_k, q, sm_count, st);
     if (e != cudaSuccess) return e;
   }
-  const size_t va_smem = VA_STAGES * 16384 + 2 * 8192 + 32 * 4;
+  const size_t va_smem = VA_STAGES * 16384 + (BF16 ? 4 : 2) * 8192 + 32 * 4;
   const dim3 vgrid(n_seq * n_splits, (v.Hq + 31) / 32);
   if (v.Hq <= 16) {
     cudaFuncSetAttribute(vacc_kernel<BF16, 1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)va_smem);

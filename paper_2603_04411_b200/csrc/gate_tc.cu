@@ -61,6 +61,91 @@ __device__ __forceinline__ float2 unpack_f16x2(uint32_t v) {
   return r;
 }
 
+// One row decided again in fp32 by a whole warp (Eq. 5, 6, 8 for the 32 logits of the block in which the cumulative
+// sum crosses tau): every logit is a dot product over d spread across the lanes (coalesced reads of the transposed
+// weights, butterfly sum), the terms exp(z - M) continue the cumulative sum from `base`, the block summaries before
+// the crossing block having been taken in fp32 already.
+__device__ __forceinline__ void gate_redo_row(const GateRaw& raw, int bf16, int d, const float* __restrict__ bias_k,
+                                              const float* __restrict__ bias_v, int side, int row, int b_s, float base, float thr,
+                                              float M, unsigned short* __restrict__ levels, int lane) {
+  const int n16 = d >> 3;                                      // 16-byte pieces per row; lane takes pieces lane, lane + 32, ...
+  auto widen = [&](const uint4 q, float* f) {
+    const uint32_t w4[4] = {q.x, q.y, q.z, q.w};
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+      if (bf16) { f[2 * k] = __uint_as_float(w4[k] << 16); f[2 * k + 1] = __uint_as_float(w4[k] & 0xffff0000u); }
+      else { const float2 t = unpack_f16x2(w4[k]); f[2 * k] = t.x; f[2 * k + 1] = t.y; }
+    }
+  };
+  float xf[32];
+  {
+    const uint4* xr = reinterpret_cast<const uint4*>((side ? raw.xv : raw.xk) + (size_t)row * d);
+#pragma unroll
+    for (int k = 0; k < 4; ++k) widen(lane + 32 * k < n16 ? __ldg(xr + lane + 32 * k) : make_uint4(0u, 0u, 0u, 0u), xf + 8 * k);
+  }
+  const unsigned short* wbase = (side ? raw.wvT : raw.wkT) + (size_t)(b_s * 32) * d;
+  float z = 0.f;
+#pragma unroll 1
+  for (int j0 = 0; j0 < 32; j0 += 4) {
+    uint4 wq[4][4];
+#pragma unroll
+    for (int jj = 0; jj < 4; ++jj) {
+      const uint4* wr = reinterpret_cast<const uint4*>(wbase + (size_t)(j0 + jj) * d);
+#pragma unroll
+      for (int k = 0; k < 4; ++k) wq[jj][k] = lane + 32 * k < n16 ? __ldg(wr + lane + 32 * k) : make_uint4(0u, 0u, 0u, 0u);
+    }
+#pragma unroll
+    for (int jj = 0; jj < 4; ++jj) {
+      float acc = 0.f;
+#pragma unroll
+      for (int k = 0; k < 4; ++k) {
+        float wf[8];
+        widen(wq[jj][k], wf);
+#pragma unroll
+        for (int e = 0; e < 8; ++e) acc = fmaf(xf[8 * k + e], wf[e], acc);
+      }
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, o);
+      if (lane == j0 + jj) z = acc;
+    }
+  }
+  const float* bias = side ? bias_v : bias_k;
+  if (bias) z += __ldg(bias + b_s * 32 + lane);
+  float incl = __expf(z - M);
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    const float t = __shfl_up_sync(0xffffffffu, incl, o);
+    if (lane >= o) incl += t;
+  }
+  const int cnt = __popc(__ballot_sync(0xffffffffu, base + incl <= thr));
+  if (lane == 0) {
+    int r = d - (b_s * 32 + cnt);
+    if (r < 1) r = 1;
+    levels[(size_t)row * 2 + side] = (unsigned short)r;
+  }
+}
+
+// The rows the fused kernel could not decide from its f16-staged terms, one warp per row.  The list's counter is
+// cleared by the last CTA to finish, so the next launch of the fused kernel starts from an empty list.
+constexpr int GT_FIX_CAP = 1 << 18;                            // list entries; rows beyond are decided inside the fused kernel
+constexpr int GT_FIX_THREADS = 128;
+__global__ void __launch_bounds__(GT_FIX_THREADS)
+gate_fixup_kernel(const GateRaw raw, int bf16, int d, const float* __restrict__ bias_k, const float* __restrict__ bias_v,
+                  const int4* __restrict__ list, int* counters, unsigned short* __restrict__ levels) {
+  const int lane = threadIdx.x & 31;
+  const int n = min(counters[0], GT_FIX_CAP);
+  for (int i = (blockIdx.x * GT_FIX_THREADS + threadIdx.x) >> 5; i < n; i += (gridDim.x * GT_FIX_THREADS) >> 5) {
+    const int4 e0 = list[2 * i], e1 = list[2 * i + 1];
+    gate_redo_row(raw, bf16, d, bias_k, bias_v, e0.y & 1, e0.x, e0.y >> 1, __int_as_float(e0.z), __int_as_float(e0.w),
+                  __int_as_float(e1.x), levels, lane);
+  }
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    __threadfence();
+    if (atomicAdd(&counters[1], 1) == (int)gridDim.x - 1) { counters[0] = 0; counters[1] = 0; __threadfence(); }
+  }
+}
+
 // Epilogue and rank role of both gate kernels (warps 2-9, 256 threads).
 //   Per slab: thread = (token row, half of the slab's columns).  Every block of 32 logits is reduced to
 //   (maximum bm, sum of exp(z - bm)) in shared memory, and the 32 terms exp(z - bm), which lie in (0, 1], are
@@ -69,7 +154,9 @@ __device__ __forceinline__ float2 unpack_f16x2(uint32_t v) {
 //   Both combine the block summaries into the softmax denominator S_d, the half that holds the block in which
 //   the running sum crosses tau * S_d finishes inside it from the block's 32 staged terms (64 bytes per row).
 //   The f16 rounding of the staged terms moves a cumulative sum by at most 2^-11 of its block's share of S_d,
-//   i.e. by less than 0.5 % of tau = 0.1: it can only change a rank whose decision was closer than that.
+//   i.e. by less than 0.5 % of tau = 0.1.  A row whose decision is closer than that bound is decided again from
+//   fp32 terms (the warp recomputes the crossing block's 32 logits from the 16-bit operands), so the rank this
+//   kernel writes has the accuracy of an fp32 evaluation of Eq. 5, 6 and 8, like the small-call path.
 // PAIR: the kernel runs on CTA pairs; the accumulator-free barrier lives in the even CTA and rows start at
 // the CTA's own half of the 256-token item.
 template <bool PAIR>
@@ -77,7 +164,8 @@ __device__ __forceinline__ void gate_epilogue_role(uint32_t tmem_base, uint32_t 
                                                    float2* sBlk, volatile int* abort_flag, unsigned short* stage,
                                                    const float* __restrict__ bias_k, const float* __restrict__ bias_v,
                                                    unsigned short* __restrict__ levels, int n_tok, int d, int NS, int n_slabs,
-                                                   int ns_rot, int it0, int itstep, int n_items, float tau, uint32_t crank) {
+                                                   int ns_rot, int it0, int itstep, int n_items, float tau, uint32_t crank,
+                                                   const GateRaw raw, int bf16) {
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int ew = warp - 2;                                   // 0..7
   const int quarter = warp & 3, chalf = ew >> 2;
@@ -162,12 +250,15 @@ __device__ __forceinline__ void gate_epilogue_role(uint32_t tmem_base, uint32_t 
       }
       const bool lower_found = __shfl_sync(0xffffffffu, bstar >= 0 ? 1 : 0, lane & ~1) != 0;
       const bool mine = hh ? !lower_found : bstar >= 0;      // the upper half also reports "nothing crossed" (NaN logits: r = 1)
+      bool redo = false;                                     // decided closer to tau than the f16 staging can tell
       if (mine && m0 + rr < n_tok) {
         int below = d;
         if (bstar >= 0) {
           const float scale = __expf(blk[bstar].x - M);
+          // a staged term is off by at most 2^-11 of itself (round to nearest), or 2^-25 once it is subnormal in f16,
+          // so the cumulative sum after k terms is off by at most 2^-11 of the block's partial sum + k 2^-25
           const unsigned short* zb = stage + ((size_t)(bstar * 4) * TILE + rr) * 8;
-          float sn = base;
+          float sn = base, part = 0x1p-20f;                  // part: the block's partial sum (+ the subnormal allowance)
           int cnt = 0;
 #pragma unroll
           for (int u = 0; u < 4; ++u) {
@@ -176,15 +267,33 @@ __device__ __forceinline__ void gate_epilogue_role(uint32_t tmem_base, uint32_t 
 #pragma unroll
             for (int k = 0; k < 4; ++k) {
               const float2 e = unpack_f16x2(w[k]);
-              sn += e.x * scale; cnt += sn <= thr ? 1 : 0;
-              sn += e.y * scale; cnt += sn <= thr ? 1 : 0;
+              sn += e.x * scale; part += e.x; cnt += sn <= thr ? 1 : 0; redo |= fabsf(sn - thr) <= part * scale * 0x1.2p-11f;
+              sn += e.y * scale; part += e.y; cnt += sn <= thr ? 1 : 0; redo |= fabsf(sn - thr) <= part * scale * 0x1.2p-11f;
             }
           }
           below = bstar * 32 + cnt;
         }
         int r = d - below;
         if (r < 1) r = 1;
-        levels[(size_t)(m0 + rr) * 2 + side] = (unsigned short)r;
+        if (!redo) levels[(size_t)(m0 + rr) * 2 + side] = (unsigned short)r;
+      }
+      // Rows flagged above are decided again in fp32 (gate_redo_row) by the small kernel that follows this one; the
+      // list holds what it needs.  Should the list ever be full, the warp does the row here instead.
+      if (redo) {
+        const int slot = atomicAdd(raw.fix_counters, 1);
+        if (slot < GT_FIX_CAP) {
+          raw.fix_list[2 * slot] = make_int4(m0 + rr, side | (bstar << 1), __float_as_int(base), __float_as_int(thr));
+          raw.fix_list[2 * slot + 1] = make_int4(__float_as_int(M), 0, 0, 0);
+          redo = false;
+        }
+      }
+      unsigned todo = __ballot_sync(0xffffffffu, redo);
+      while (todo) {
+        const int src = __ffs(todo) - 1;
+        todo &= todo - 1;
+        gate_redo_row(raw, bf16, d, bias_k, bias_v, side, m0 + __shfl_sync(0xffffffffu, rr, src), __shfl_sync(0xffffffffu, bstar, src),
+                      __shfl_sync(0xffffffffu, base, src), __shfl_sync(0xffffffffu, thr, src), __shfl_sync(0xffffffffu, M, src),
+                      levels, lane);
       }
     }
     if (!(ok = epi_sync())) break;                           // the staging block may be overwritten by the next item
@@ -195,7 +304,7 @@ __global__ void __launch_bounds__(GT_THREADS, 1)
 gate_tc_kernel(const __grid_constant__ CUtensorMap map_xk, const __grid_constant__ CUtensorMap map_xv,
                const __grid_constant__ CUtensorMap map_wk, const __grid_constant__ CUtensorMap map_wv,
                const float* __restrict__ bias_k, const float* __restrict__ bias_v, int n_tok, int d, int bf16, float tau,
-               float* __restrict__ stage_all, unsigned short* __restrict__ levels, int* status) {
+               float* __restrict__ stage_all, unsigned short* __restrict__ levels, int* status, const GateRaw raw) {
   extern __shared__ __align__(1024) unsigned char smem_raw[];
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int KP = d / PANEL;                                   // K panels of the token tile
@@ -301,7 +410,7 @@ gate_tc_kernel(const __grid_constant__ CUtensorMap map_xk, const __grid_constant
     // ------------------------------------------------------------- epilogue + rank
     gate_epilogue_role<false>(tmem_base, acc_full, acc_empty, epi_bar, sBlk, abort_flag,
                               reinterpret_cast<unsigned short*>(stage_all) + (size_t)blockIdx.x * TILE * d, bias_k, bias_v, levels,
-                              n_tok, d, NS, n_slabs, ns_rot, it0, itstep, n_items, tau, 0u);
+                              n_tok, d, NS, n_slabs, ns_rot, it0, itstep, n_items, tau, 0u, raw, bf16);
   }
 
   fence_before_sync();
@@ -329,7 +438,7 @@ __global__ void __launch_bounds__(GT_THREADS, 1)
 gate_tc2_kernel(const __grid_constant__ CUtensorMap map_xk, const __grid_constant__ CUtensorMap map_xv,
                const __grid_constant__ CUtensorMap map_wk, const __grid_constant__ CUtensorMap map_wv,
                const float* __restrict__ bias_k, const float* __restrict__ bias_v, int n_tok, int d, int bf16, float tau,
-               float* __restrict__ stage_all, unsigned short* __restrict__ levels, int* status) {
+               float* __restrict__ stage_all, unsigned short* __restrict__ levels, int* status, const GateRaw raw) {
   extern __shared__ __align__(1024) unsigned char smem_raw[];
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const uint32_t crank = cluster_cta_rank();                  // 0 = even CTA: issues the MMAs, owns full / acc_empty
@@ -433,7 +542,7 @@ gate_tc2_kernel(const __grid_constant__ CUtensorMap map_xk, const __grid_constan
     // ------------------------------------------------------------- epilogue + rank
     gate_epilogue_role<true>(tmem_base, acc_full, acc_empty, epi_bar, sBlk, abort_flag,
                               reinterpret_cast<unsigned short*>(stage_all) + (size_t)blockIdx.x * TILE * d, bias_k, bias_v, levels,
-                              n_tok, d, NS, n_slabs, ns_rot, it0, itstep, n_items, tau, crank);
+                              n_tok, d, NS, n_slabs, ns_rot, it0, itstep, n_items, tau, crank, raw, bf16);
   }
 
   fence_before_sync();
@@ -446,6 +555,17 @@ gate_tc2_kernel(const __grid_constant__ CUtensorMap map_xk, const __grid_constan
 
 int gate_tc_max_pairs(int sm_count);
 size_t gate_tc_stage_bytes(int n_cta, int d) { return (size_t)n_cta * TILE * d * sizeof(unsigned short); }
+
+size_t gate_tc_fix_bytes() { return (size_t)GT_FIX_CAP * 2 * sizeof(int4); }
+
+static cudaError_t launch_gate_fixup(const DevView& v, const GateMaps& maps, const LayerParams& lp, int bf16, unsigned short* levels,
+                                     int sm_count, cudaStream_t st) {
+  ProfScope ps(TWKV_K_GATE_RANK, st);
+  gate_fixup_kernel<<<2 * sm_count, GT_FIX_THREADS, 0, st>>>(maps.raw, bf16, v.d_kv, lp.b_k, lp.b_v, maps.raw.fix_list,
+                                                             maps.raw.fix_counters, levels);
+  count_launch();
+  return cudaGetLastError();
+}
 
 cudaError_t launch_gate_ranks_tc(const DevView& v, const GateMaps& maps, const LayerParams& lp, int n_tok, unsigned short* levels,
                                  int sm_count, bool pairs, cudaStream_t st) {
@@ -473,10 +593,11 @@ cudaError_t launch_gate_ranks_tc(const DevView& v, const GateMaps& maps, const L
     {
       ProfScope ps(TWKV_K_GATE_GEMM, st);
       e = cudaLaunchKernelEx(&cfg, gate_tc2_kernel, maps.xk, maps.xv, maps.wk, maps.wv, lp.b_k, lp.b_v, n_tok, d, bf16, v.tau,
-                             v.gate_scratch, levels, v.status);
+                             v.gate_scratch, levels, v.status, maps.raw);
     }
     count_launch();
-    return e != cudaSuccess ? e : cudaGetLastError();
+    if (e != cudaSuccess) return e;
+    return launch_gate_fixup(v, maps, lp, bf16, levels, sm_count, st);
   }
   const int NS = (d % 256 == 0) ? 256 : 128;
   const size_t smem = (size_t)GT_STAGES * (GT_PANEL_BYTES + (size_t)NS * 128) + TILE * GT_BLK_STRIDE * sizeof(float2) + 8 * (2 * GT_STAGES + 5) + 16;
@@ -487,10 +608,11 @@ cudaError_t launch_gate_ranks_tc(const DevView& v, const GateMaps& maps, const L
   {
     ProfScope ps(TWKV_K_GATE_GEMM, st);
     gate_tc_kernel<<<grid, GT_THREADS, smem, st>>>(maps.xk, maps.xv, maps.wk, maps.wv, lp.b_k, lp.b_v, n_tok, d, bf16, v.tau,
-                                                   v.gate_scratch, levels, v.status);
+                                                   v.gate_scratch, levels, v.status, maps.raw);
   }
   count_launch();
-  return cudaGetLastError();
+  if (cudaError_t e2 = cudaGetLastError(); e2 != cudaSuccess) return e2;
+  return launch_gate_fixup(v, maps, lp, bf16, levels, sm_count, st);
 }
 
 // CTA pairs of gate_tc2_kernel that can be resident at once on the current device (0: the pair kernel cannot run).

@@ -5,22 +5,26 @@
 //   Krot_g = RoPE(Kbar_g, position of each token)                             (keys are rotated after reconstruction)
 //   S_g    = Krot_g . Q_g^T,  Q_g = the REP query heads that share KV head g   (the GQA group makes this a dense contraction)
 // The first product is a tcgen05.mma chain (M = 128, N = 128, K = 16 per instruction) whose fp32
-// accumulator lives in TMEM; X^_K panels and panels of the pre-transposed U_K^-1 arrive by TMA with
+// accumulator (a "slab") lives in TMEM; X^_K panels and panels of the pre-transposed U_K^-1 arrive by TMA with
 // the 128-byte swizzle, which is the K-major operand layout the MMA reads from shared memory.
-// Epilogue warps pull the slab out of TMEM, rotate it in fp32, split it into a high and a low f16 part and
-// store both back to TMEM, from where they are the A operands of the second product (N = 16, the group's
-// heads padded; one product per part);
-// its accumulator S stays in TMEM until the tile's last slab, so RoPE is the only per-element
-// CUDA-core work.  Both sums are linear in X^_K, so a class wider than 8 panels runs as two passes
-// over its panels that accumulate into the same S.
+// Epilogue warps pull the slab out of TMEM sixteen columns at a time, rotate it in fp32, split every value into a
+// high and a low f16 part and store both back IN PLACE (a thread overwrites only columns it has already read: 64
+// fp32 columns become 32 columns of high parts and 32 of low parts), from where they are the A operands of the second
+// product (N = 16, the group's heads padded; one product per part).  The order of the 128 dimensions along the
+// contraction is whatever that in-place layout gives; the query operand is written in the same order.
+// Each slab's scores land in one of four 16-column accumulators and are read out by the epilogue warps two slabs
+// later (scaled, masked, stored, folded into the per-(sequence, head) maximum), so that a tile has no tail:
+// RoPE is the only per-element CUDA-core work.  Both products are linear in X^_K, so a class wider than 8 panels runs
+// as two passes over its panels; the second pass adds to the scores the first one stored.
 //
-// Tensor memory (512 columns): slab accumulators 2 x 128 | rotated keys, high and low part, 64 each | S 8 x 16.
+// Tensor memory (512 columns): slabs 3 x 128 | score accumulators 4 x 16.
 // Warp roles (384 threads, one persistent CTA per SM working through a contiguous, cost-balanced piece of the tile list):
 //   warp 0      TMA producer of U_K^-1 panels (ring, one lane per stage)
 //   warp 1      issuer of the main products (one elected lane; owns the TMEM allocation)
 //   warps 2-9   epilogue (thread = one token row x one half of the RoPE frequencies)
-//   warp 10     TMA producer of X^_K panels (ring of 8 slots served by four lanes, runs ahead into the next tile)
+//   warp 10     TMA producer of X^_K panels (ring of 8 slots served by four lanes, runs ahead into the next tiles)
 //   warp 11     issuer of the score products (one elected lane)
+// A slab buffer goes round: main products (slab_full) -> epilogue (kr_full) -> score products (slab_empty).
 // All waits are bounded (tc_util.cuh); a wait that runs out ends the kernel with TWKV_ERR_TIMEOUT.
 //
 // Precision: X^_K, U_K^-1 keep the cache dtype with fp32 accumulation; queries enter the score product as
@@ -35,13 +39,16 @@ using namespace tc;
 constexpr int KT_THREADS = 384;
 constexpr int KT_EPI = 256;
 constexpr int KT_A_SLOTS = 8;                                  // power of two (slot = panel count & 7, phase = bit 3)
+constexpr int KT_SLABS = 3;                                    // slab buffers
+constexpr int KT_S_SLOTS = 4;                                  // score accumulators
 constexpr uint32_t KT_TMEM_COLS = 512;
-constexpr uint32_t TM_SLAB = 0, TM_KR = 256, TM_S = 384;      // column offsets inside the allocation
+constexpr uint32_t TM_SLAB = 0, TM_S = 128 * KT_SLABS;        // column offsets inside the allocation
 constexpr uint32_t PANEL_BYTES = 16384;
 constexpr int KT_Q_ROWS = 72;                                 // 8 rows per KV head + 8 rows of padding
 constexpr uint32_t KT_Q_PANEL_BYTES = KT_Q_ROWS * 128;        // one 64-wide K panel of the query operand
-constexpr int KT_ROPE_STRIDE = 65;                            // float2 per row of the small RoPE tables in shared memory (64 + 1 against bank conflicts)
-constexpr uint32_t KT_ROPE_STAGE_BYTES = ROPE_SMALL_ROWS * KT_ROPE_STRIDE * 8;
+constexpr int KT_ROPE_STRIDE = 33;                            // float4 per row of the small RoPE table in shared memory (32 + 1 against bank conflicts)
+constexpr uint32_t KT_ROPE_STAGE_BYTES = ROPE_LO * KT_ROPE_STRIDE * 16;
+constexpr int KT_N_BARS = 2 * KT_A_SLOTS + 3 * KT_SLABS + 2 * KT_S_SLOTS;     // + 2 nb for the U_K^-1 ring
 
 // Packed fp32 pairs (two lanes per 64-bit register, one instruction for both): the rotation is issue-bound.
 __device__ __forceinline__ uint64_t f2_pack(float a, float b) { uint64_t r; asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(a), "f"(b)); return r; }
@@ -54,11 +61,25 @@ __device__ __forceinline__ uint32_t f2_to_f16x2_sat(uint64_t v) {       // (lo l
   asm("{\n\t.reg .f32 a, b;\n\tmov.b64 {a, b}, %1;\n\tcvt.rn.satfinite.f16x2.f32 %0, b, a;\n\t}" : "=r"(d) : "l"(v));
   return d;
 }
+__device__ __forceinline__ unsigned warp_max_u32(unsigned x) {
+  unsigned r;
+  asm volatile("redux.sync.max.u32 %0, %1, 0xffffffff;" : "=r"(r) : "r"(x));
+  return r;
+}
 
 template <bool BF16> __device__ __forceinline__ float kt_to_f32(unsigned short bits) {
   if constexpr (BF16) return __uint_as_float((unsigned)bits << 16);
   else return __half2float(__ushort_as_half(bits));
 }
+
+// A score read-out that is still owed: which accumulator, where the scores go, how they combine.
+struct KtPending {
+  float* out;            // this thread's row of the score scratch, at the group's first head
+  int mxi;               // index of the group's first head in the running-max table
+  uint32_t meta;         // bit 0 valid | bit 1 reader half | bits 2-3 mode | bits 4-5 accumulator | bit 6 its parity | bit 7 row is a token
+};
+constexpr uint32_t KP_VALID = 1u, KP_LIVE = 128u;
+constexpr uint32_t KP_STORE_PART = 0u, KP_STORE_FINAL = 1u, KP_ADD_FINAL = 2u;      // modes
 
 template <bool BF16, int REP>
 __global__ void __launch_bounds__(KT_THREADS, 1)
@@ -76,31 +97,30 @@ kscore_tc_kernel(const __grid_constant__ CUtensorMap map_blocks, const __grid_co
   const uint32_t sB = sA + KT_A_SLOTS * PANEL_BYTES;
   const uint32_t sQ = sB + nb * PANEL_BYTES;
   unsigned char* sQ_ptr = smem_raw + (KT_A_SLOTS + nb) * PANEL_BYTES;
-  float2* sRope = reinterpret_cast<float2*>(sQ_ptr + 2 * KT_Q_PANEL_BYTES);   // [32 rows][65]: the two small RoPE tables
+  float4* sRope = reinterpret_cast<float4*>(sQ_ptr + 2 * KT_Q_PANEL_BYTES);   // [16 rows][33]: the small RoPE table
   unsigned char* tail = sQ_ptr + 2 * KT_Q_PANEL_BYTES + KT_ROPE_STAGE_BYTES;
   const uint32_t bars = smem_addr(tail);
   // barrier map (8 bytes each)
   const uint32_t a_full = bars, a_empty = a_full + 8 * KT_A_SLOTS, b_full = a_empty + 8 * KT_A_SLOTS;
-  const uint32_t b_empty = b_full + 8 * nb, slab_full = b_empty + 8 * nb, slab_empty = slab_full + 16;
-  const uint32_t kr_full = slab_empty + 16, kr_empty = kr_full + 16, s_full = kr_empty + 16;
-  uint32_t* s_tmem_base = reinterpret_cast<uint32_t*>(tail + 8 * (2 * KT_A_SLOTS + 2 * nb + 9));
+  const uint32_t b_empty = b_full + 8 * nb, slab_full = b_empty + 8 * nb, kr_full = slab_full + 8 * KT_SLABS;
+  const uint32_t slab_empty = kr_full + 8 * KT_SLABS, s_full = slab_empty + 8 * KT_SLABS, s_empty = s_full + 8 * KT_S_SLOTS;
+  uint32_t* s_tmem_base = reinterpret_cast<uint32_t*>(tail + 8 * (KT_N_BARS + 2 * nb));
   volatile int* abort_flag = reinterpret_cast<int*>(s_tmem_base + 1);
 
   if (tid == 0) {
     for (int i = 0; i < KT_A_SLOTS; ++i) { mbar_init(a_full + 8 * i, 1); mbar_init(a_empty + 8 * i, 1); }
     for (int i = 0; i < nb; ++i) { mbar_init(b_full + 8 * i, 1); mbar_init(b_empty + 8 * i, 1); }
-    for (int i = 0; i < 2; ++i) {
-      mbar_init(slab_full + 8 * i, 1); mbar_init(slab_empty + 8 * i, KT_EPI / 32);
-      mbar_init(kr_full + 8 * i, KT_EPI / 32); mbar_init(kr_empty + 8 * i, 1);
+    for (int i = 0; i < KT_SLABS; ++i) {
+      mbar_init(slab_full + 8 * i, 1); mbar_init(kr_full + 8 * i, KT_EPI / 32); mbar_init(slab_empty + 8 * i, 1);
     }
-    mbar_init(s_full, 1);
+    for (int i = 0; i < KT_S_SLOTS; ++i) { mbar_init(s_full + 8 * i, 1); mbar_init(s_empty + 8 * i, KT_EPI / 64); }
     *abort_flag = 0;
     mbar_init_fence();
   }
   if (warp == 1) tmem_alloc(smem_addr(s_tmem_base), KT_TMEM_COLS);
   for (int i = tid; i < 2 * (int)KT_Q_PANEL_BYTES / 16; i += KT_THREADS)        // padding rows of the query operand stay zero
     reinterpret_cast<uint4*>(sQ_ptr)[i] = make_uint4(0u, 0u, 0u, 0u);
-  for (int i = tid; i < ROPE_SMALL_ROWS * 64; i += KT_THREADS) sRope[(i >> 6) * KT_ROPE_STRIDE + (i & 63)] = v.rope_lo[i];
+  for (int i = tid; i < ROPE_LO * 32; i += KT_THREADS) sRope[(i >> 5) * KT_ROPE_STRIDE + (i & 31)] = v.rope_lo[i];
   fence_proxy_async_smem();
   fence_before_sync();
   __syncthreads();
@@ -112,7 +132,6 @@ kscore_tc_kernel(const __grid_constant__ CUtensorMap map_blocks, const __grid_co
   const int w0 = v.cta_start[blockIdx.x], total = v.cta_start[blockIdx.x + 1];
   const int4* klist = v.klist;
   const int4 kt_none = make_int4(0, 0, 0, -1);
-  constexpr int wstep = 1;
   // CTAs walk the KV heads in rotated order, so that at any moment they read different panels of U_K^-1 from L2
   const int g_rot = blockIdx.x % Hkv;
 
@@ -125,8 +144,8 @@ kscore_tc_kernel(const __grid_constant__ CUtensorMap map_blocks, const __grid_co
       uint32_t ak = 0;                                          // panels so far; slot = ak % 8
       bool ok = true;
       int4 e = w0 < total ? klist[w0] : kt_none;
-      for (int w = w0; w < total && ok; w += wstep) {
-        const int4 nxt = w + wstep < total ? klist[w + wstep] : kt_none;
+      for (int w = w0; w < total && ok; ++w) {
+        const int4 nxt = w + 1 < total ? klist[w + 1] : kt_none;
         const int cls = e.y & 0xff, blk = e.z;
         for (int j = 0; j < cls; ++j, ++ak) {
           const uint32_t slot = ak % KT_A_SLOTS, ph = (ak / KT_A_SLOTS) & 1u;
@@ -152,8 +171,8 @@ kscore_tc_kernel(const __grid_constant__ CUtensorMap map_blocks, const __grid_co
       uint32_t bk = 0, bst = 0, bph = 0;                        // panels so far; ring stage and its phase
       bool ok = true;
       int4 e = w0 < total ? klist[w0] : kt_none;
-      for (int w = w0; w < total && ok; w += wstep) {
-        const int4 nxt = w + wstep < total ? klist[w + wstep] : kt_none;
+      for (int w = w0; w < total && ok; ++w) {
+        const int4 nxt = w + 1 < total ? klist[w + 1] : kt_none;
         const int cls = e.y & 0xff;
         for (int p0 = 0; p0 < cls && ok; p0 += KT_A_SLOTS) {
           const int np = min(KT_A_SLOTS, cls - p0);
@@ -186,18 +205,19 @@ kscore_tc_kernel(const __grid_constant__ CUtensorMap map_blocks, const __grid_co
       // every wait tries once inline before it falls into the bounded loop.
       const uint32_t idesc_main = idesc_f16(BF16 ? 1 : 0, 128, 128);
       const uint32_t a_lo0 = kmajor_sw128_desc_lo(sA), b_lo0 = kmajor_sw128_desc_lo(sB);
-      uint32_t bst = 0, bph = 0, ak = 0, sc = 0;
+      uint32_t bst = 0, bph = 0, ak = 0, sbuf = 0, sph = 0;
       bool ok = true;
       int4 e = w0 < total ? klist[w0] : kt_none;
-      for (int w = w0; w < total && ok; w += wstep) {
-        const int4 nxt = w + wstep < total ? klist[w + wstep] : kt_none;
+      for (int w = w0; w < total && ok; ++w) {
+        const int4 nxt = w + 1 < total ? klist[w + 1] : kt_none;
         const int cls = e.y & 0xff;
         for (int p0 = 0; p0 < cls && ok; p0 += KT_A_SLOTS) {
           const int np = min(KT_A_SLOTS, cls - p0);
           for (int sl = 0; sl < Hkv && ok; ++sl) {
-            const uint32_t buf = sc & 1u;
-            if (!(ok = mbar_wait_thin(slab_empty + 8 * buf, ((sc >> 1) & 1u) ^ 1u, abort_flag))) break;
-            const uint32_t d = tmem_base + TM_SLAB + buf * 128;
+            // the buffer is free once the score products over its previous contents have retired
+            if (!(ok = mbar_wait_thin(slab_empty + 8 * sbuf, sph ^ 1u, abort_flag))) break;
+            fence_after_sync();
+            const uint32_t d = tmem_base + TM_SLAB + sbuf * 128;
             const bool first = sl == 0, last = sl == Hkv - 1;
             uint32_t an = ak;
             for (int j = 0; j < np; ++j, ++an) {
@@ -212,8 +232,8 @@ kscore_tc_kernel(const __grid_constant__ CUtensorMap map_blocks, const __grid_co
               if (last) mma_commit(a_empty + 8 * slot);                 // last slab of the pass: the X^_K panel is done
             }
             if (!ok) break;
-            mma_commit(slab_full + 8 * buf);                            // slab accumulator complete
-            ++sc;
+            mma_commit(slab_full + 8 * sbuf);                           // slab accumulator complete
+            if (++sbuf == (uint32_t)KT_SLABS) { sbuf = 0; sph ^= 1u; }
           }
           ak += np;
         }
@@ -223,29 +243,31 @@ kscore_tc_kernel(const __grid_constant__ CUtensorMap map_blocks, const __grid_co
     __syncwarp();
   } else if (warp == 11) {
     // ------------------------------------------------------------- score-product issuer (one elected lane)
-    // S_g (+)= Krot_g . Q_g^T as soon as the epilogue warps have stored a rotated slab; a thread of its own, so that
+    // S (+)= Krot_g . Q_g^T as soon as the epilogue warps have stored a rotated slab; a thread of its own, so that
     // neither issue stream waits for the other's barriers
     if (elect_one()) {
       const uint32_t idesc_s = idesc_f16(0, 128, 16);
       const uint32_t q_lo0 = kmajor_sw128_desc_lo(sQ);
-      uint32_t sc = 0;
+      uint32_t sbuf = 0, sph = 0, slot = 0, slph = 0;
       bool ok = true;
       int4 e = w0 < total ? klist[w0] : kt_none;
-      for (int w = w0; w < total && ok; w += wstep) {
-        const int4 nxt = w + wstep < total ? klist[w + wstep] : kt_none;
+      for (int w = w0; w < total && ok; ++w) {
+        const int4 nxt = w + 1 < total ? klist[w + 1] : kt_none;
         const int cls = e.y & 0xff;
         for (int p0 = 0; p0 < cls && ok; p0 += KT_A_SLOTS) {
-          const bool last_pass = p0 + KT_A_SLOTS >= cls;
-          for (int sl = 0; sl < Hkv; ++sl, ++sc) {
+          for (int sl = 0; sl < Hkv; ++sl) {
             const int g = sl + g_rot < Hkv ? sl + g_rot : sl + g_rot - Hkv;
-            if (!(ok = mbar_wait_thin(kr_full, sc & 1u, abort_flag))) break;
+            if (!(ok = mbar_wait_thin(kr_full + 8 * sbuf, sph, abort_flag))) break;
+            if (!(ok = mbar_wait_thin(s_empty + 8 * slot, slph ^ 1u, abort_flag))) break;
             fence_after_sync();
             // the rotated keys come as a high and a low f16 part (their sum carries 21 bits): two products into the same S
-            mma_f16_ts_k128(tmem_base + TM_S + 16 * g, tmem_base + TM_KR, q_lo0 + g * (1024 >> 4), KT_Q_PANEL_BYTES >> 4, idesc_s,
-                            p0 > 0 ? 1u : 0u);
-            mma_f16_ts_k128(tmem_base + TM_S + 16 * g, tmem_base + TM_KR + 64, q_lo0 + g * (1024 >> 4), KT_Q_PANEL_BYTES >> 4, idesc_s, 1u);
-            mma_commit(kr_empty);
-            if (last_pass && sl == Hkv - 1) mma_commit(s_full);        // the tile's scores are complete
+            const uint32_t kr = tmem_base + TM_SLAB + sbuf * 128, sd = tmem_base + TM_S + 16 * slot;
+            mma_f16_ts_k128(sd, kr, q_lo0 + g * (1024 >> 4), KT_Q_PANEL_BYTES >> 4, idesc_s, 0u);
+            mma_f16_ts_k128(sd, kr + 64, q_lo0 + g * (1024 >> 4), KT_Q_PANEL_BYTES >> 4, idesc_s, 1u);
+            mma_commit(slab_empty + 8 * sbuf);                          // the slab buffer may be overwritten
+            mma_commit(s_full + 8 * slot);                              // this slab's scores are complete
+            if (++sbuf == (uint32_t)KT_SLABS) { sbuf = 0; sph ^= 1u; }
+            if (++slot == (uint32_t)KT_S_SLOTS) { slot = 0; slph ^= 1u; }
           }
         }
         e = nxt;
@@ -258,41 +280,33 @@ kscore_tc_kernel(const __grid_constant__ CUtensorMap map_blocks, const __grid_co
     const int quarter = warp & 3, hf = (warp - 2) >> 2;
     const int row = quarter * 32 + lane;
     const uint32_t lane_addr = tmem_base + ((uint32_t)(quarter * 32) << 16);
-    const int g_lo = hf ? (Hkv + 1) / 2 : 0, g_hi = hf ? Hkv : (Hkv + 1) / 2;      // this thread's KV-head groups (at most 4)
     const float sm_scale = v.sm_scale;
     const int* kpos = v.aux(layer, 0);
-    const float2* __restrict__ rope_hi = v.rope_hi;
-    uint32_t sc = 0, tcount = 0;
-    bool ok = true, slab_ready = false;                            // slab_ready: the next slab's accumulator was already seen complete
-    float cs[32], sn[32];                                         // scratch of rope_setup
+    const float4* __restrict__ rope_hi = v.rope_hi;
+    uint32_t sbuf = 0, sph = 0, slot = 0, slph = 0;
+    bool ok = true;
     uint64_t cs2[16], sn2[16];                                    // the tile's rotation factors, frequencies (2 t, 2 t + 1) packed
-    float tmax[4 * REP];                                            // running maxima of this thread's heads for the current query slot
-#pragma unroll
-    for (int i = 0; i < 4 * REP; ++i) tmax[i] = -INFINITY;
 
-    // cos / sin of (row, frequency): pos = hi * 256 + mid * 16 + lo, the three table rows combine by the angle-addition
-    // formulas.  The mid and lo rows come from shared memory (padded rows: lanes with different rows hit different
-    // banks), the hi row from global memory: a tile's 128 rows share a few hi rows, so those reads stay in L1.
+    // cos / sin of (row, frequency): pos = hi * 16 + lo, the two table rows combine by the angle-addition formulas.
+    // The lo row comes from shared memory (padded rows: lanes with different rows hit different banks), the hi row
+    // from global memory (L2; neighbouring positions share it).
     auto rope_setup = [&](int pos) {
-      const float2* __restrict__ th = rope_hi + (size_t)((pos >> 8) & (ROPE_HI - 1)) * 64 + hf * 32;
-      const float2* tm = sRope + ((pos >> 4) & 15) * KT_ROPE_STRIDE + hf * 32;
-      const float2* tl = sRope + (16 + (pos & 15)) * KT_ROPE_STRIDE + hf * 32;
+      const float4* __restrict__ th = rope_hi + (size_t)((pos >> 4) & (ROPE_HI - 1)) * 32 + hf * 16;
+      const float4* tl = sRope + (pos & 15) * KT_ROPE_STRIDE + hf * 16;
+      float4 h[16];
 #pragma unroll
-      for (int t = 0; t < 32; t += 2) {                        // all hi-row reads in flight before any is used
-        const float4 h = __ldg(reinterpret_cast<const float4*>(th + t));
-        cs[t] = h.x; sn[t] = h.y; cs[t + 1] = h.z; sn[t + 1] = h.w;
+      for (int t = 0; t < 16; ++t) h[t] = __ldg(th + t);        // all hi-row reads in flight before any is used
+#pragma unroll
+      for (int t = 0; t < 16; ++t) {
+        const float4 l = tl[t];
+        const uint64_t ch = f2_pack(h[t].x, h[t].y), sh = f2_pack(h[t].z, h[t].w), cl = f2_pack(l.x, l.y), sl = f2_pack(l.z, l.w);
+        cs2[t] = f2_sub(f2_mul(ch, cl), f2_mul(sh, sl));
+        sn2[t] = f2_fma(sh, cl, f2_mul(ch, sl));
       }
-#pragma unroll
-      for (int t = 0; t < 32; ++t) {
-        const float2 m = tm[t], l = tl[t];
-        const float hx = cs[t] * m.x - sn[t] * m.y, hy = sn[t] * m.x + cs[t] * m.y;
-        cs[t] = hx * l.x - hy * l.y;
-        sn[t] = hy * l.x + hx * l.y;
-      }
-#pragma unroll
-      for (int t = 0; t < 16; ++t) { cs2[t] = f2_pack(cs[2 * t], cs[2 * t + 1]); sn2[t] = f2_pack(sn[2 * t], sn[2 * t + 1]); }
     };
-    // The group's queries as the K-major, 128-byte-swizzled B operand: row 8 g + h, two 64-wide panels.
+    // The group's queries as the K-major, 128-byte-swizzled B operand: row 8 g + h, two 64-wide panels.  The
+    // contraction runs over the dimensions in the order the epilogue leaves the rotated keys in: 16-byte piece
+    // 8 hf + 2 c holds dimensions 32 hf + 8 c .. + 7, piece 8 hf + 2 c + 1 the dimensions 64 above them.
     // Only called when no score product that reads the rows can still be in flight.
     auto write_q = [&](int qs) {
       for (int i = et; i < Hq * 16; i += KT_EPI) {
@@ -306,122 +320,137 @@ kscore_tc_kernel(const __grid_constant__ CUtensorMap map_blocks, const __grid_co
           val.z = pack_f16x2_sat(kt_to_f32<true>(e[4]), kt_to_f32<true>(e[5]));
           val.w = pack_f16x2_sat(kt_to_f32<true>(e[6]), kt_to_f32<true>(e[7]));
         }
-        const int qrow = (head / REP) * 8 + head % REP, c8 = ch & 7;
-        *reinterpret_cast<uint4*>(sQ_ptr + (ch >> 3) * KT_Q_PANEL_BYTES + qrow * 128 + ((c8 ^ (qrow & 7)) << 4)) = val;
+        const int kc = ((ch & 7) >> 2) * 8 + (ch & 3) * 2 + (ch >> 3);     // position of the piece along the contraction
+        const int qrow = (head / REP) * 8 + head % REP, c8 = kc & 7;
+        *reinterpret_cast<uint4*>(sQ_ptr + (kc >> 3) * KT_Q_PANEL_BYTES + qrow * 128 + ((c8 ^ (qrow & 7)) << 4)) = val;
       }
       fence_proxy_async_smem();
     };
+    // Scores of one slab: REP columns of its accumulator, scaled, rows past the tile's last token masked; the reading
+    // half of the epilogue warps alternates from slab to slab.
+    auto read_out = [&](const KtPending& p) -> bool {
+      if (!(p.meta & KP_VALID) || (int)((p.meta >> 1) & 1u) != hf) return true;       // uniform over the warp
+      const uint32_t sl_ = (p.meta >> 4) & 3u, par = (p.meta >> 6) & 1u, mode = (p.meta >> 2) & 3u;
+      if (!__all_sync(0xffffffffu, mbar_wait(s_full + 8 * sl_, par, abort_flag))) return false;
+      fence_after_sync();
+      float sv[REP];
+      {
+        uint32_t* dst = reinterpret_cast<uint32_t*>(sv);
+        const uint32_t src = lane_addr + TM_S + 16 * sl_;
+        if constexpr (REP == 1) tmem_ld1(src, dst);
+        else if constexpr (REP == 2) tmem_ld2(src, dst);
+        else if constexpr (REP == 4) tmem_ld4(src, dst);
+        else tmem_ld8(src, dst);
+      }
+      tmem_ld_wait();
+      fence_before_sync();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(s_empty + 8 * sl_);
+      const bool live = (p.meta & KP_LIVE) != 0;
+      float* out = p.out;
+#pragma unroll
+      for (int i = 0; i < REP; ++i) {
+        float x = sv[i] * sm_scale;
+        if (mode == KP_ADD_FINAL) x += out[i];                                       // the first pass stored its part
+        sv[i] = live ? x : -INFINITY;
+      }
+      if constexpr (REP >= 4) {
+#pragma unroll
+        for (int i = 0; i < REP; i += 4) *reinterpret_cast<float4*>(out + i) = make_float4(sv[i], sv[i + 1], sv[i + 2], sv[i + 3]);
+      } else {
+#pragma unroll
+        for (int i = 0; i < REP; ++i) out[i] = sv[i];
+      }
+      if (mode != KP_STORE_PART) {
+        // maximum over the warp's rows, one atomic per head (max is order-independent, so the result is deterministic)
+        unsigned mine = 0u;
+#pragma unroll
+        for (int i = 0; i < REP; ++i) {
+          const unsigned m = warp_max_u32(enc_ordered(sv[i]));
+          if (lane == i) mine = m;
+        }
+        if (lane < REP) atomicMax(&v.seqmax[p.mxi + lane], mine);
+      }
+      return true;
+    };
 
+    KtPending p_old{nullptr, 0, 0u}, p_new{nullptr, 0, 0u};
     int4 e = w0 < total ? klist[w0] : kt_none;
     if (w0 < total) { write_q(e.w); rope_setup(kpos[(size_t)e.x * TILE + row]); }
-    for (int w = w0; w < total && ok; w += wstep) {
-      const int4 nxt = w + wstep < total ? klist[w + wstep] : kt_none;
+    for (int w = w0; w < total && ok; ++w) {
+      const int4 nxt = w + 1 < total ? klist[w + 1] : kt_none;
       const int tile = e.x, cls = e.y & 0xff, n_valid = e.y >> 8, qs = e.w;
-      const int n_slabs = ((cls + KT_A_SLOTS - 1) / KT_A_SLOTS) * Hkv;
+      const int passes = (cls + KT_A_SLOTS - 1) / KT_A_SLOTS;
       const int pos_next = nxt.w >= 0 ? kpos[(size_t)nxt.x * TILE + row] : 0;      // fetched now, used after the tile's slabs
-      for (int sl = 0; sl < n_slabs; ++sl, ++sc) {
-        const uint32_t buf = sc & 1u, par = (sc >> 1) & 1u;
-        // barrier probes cost a few hundred cycles of latency each, so each is issued early (the next slab's "full"
-        // during this slab's store, "rotated keys free" before the rotation) and only waited on if it had not flipped yet
-        if (!slab_ready && !(ok = __all_sync(0xffffffffu, mbar_wait(slab_full + 8 * buf, par, abort_flag)))) break;
-        fence_after_sync();
-        const uint32_t slab = lane_addr + TM_SLAB + buf * 128 + hf * 32;
-        const uint32_t kr = lane_addr + TM_KR + hf * 16;                     // high parts; the low parts 64 columns on
-        const uint32_t kr_par = (sc & 1u) ^ 1u;
-        uint32_t lo[32], hi[32];
-        tmem_ld32(slab, lo);
-        tmem_ld32(slab + 64, hi);
-        const bool kr_probe = mbar_try(kr_empty, kr_par);
-        tmem_ld_wait();
-        fence_before_sync();
-        __syncwarp();
-        if (lane == 0) mbar_arrive(slab_empty + 8 * buf);                    // the slab accumulator is free for slab n + 2
-        // a rotated value v leaves as two f16: v with its low 13 mantissa bits cleared (exact in f16) and the rest
-        // (rounded to f16: 2^-21 of v instead of the 2^-11 of one f16), so that the score error stays far below the bar
-        // even where a few key channels carry most of the magnitude
+      float* const out_row = v.scores + ((size_t)tile * TILE + row) * Hq;
+      const uint32_t live_bit = row < n_valid ? KP_LIVE : 0u;
+      for (int ps = 0; ps < passes && ok; ++ps) {
+        const uint32_t mode = passes == 1 ? KP_STORE_FINAL : (ps == 0 ? KP_STORE_PART : KP_ADD_FINAL);
+        for (int sli = 0; sli < Hkv; ++sli) {
+          const int g = sli + g_rot < Hkv ? sli + g_rot : sli + g_rot - Hkv;
+          if (!(ok = __all_sync(0xffffffffu, mbar_wait(slab_full + 8 * sbuf, sph, abort_flag)))) break;
+          fence_after_sync();
+          const uint32_t sl_addr = lane_addr + TM_SLAB + sbuf * 128 + hf * 32;
+          // the slab goes through the registers sixteen columns at a time (8 low dims + the 8 dims 64 above them), the
+          // next piece's load in flight while this one is rotated; a piece's results overwrite the columns it came from
+          uint32_t va[16], vb[16];
+          tmem_ld8(sl_addr, va);
+          tmem_ld8(sl_addr + 64, va + 8);
+          if (!(ok = read_out(p_old))) break;                                // the scores of the slab before last
 #pragma unroll
-        for (int hb = 0; hb < 2; ++hb) {
-          uint32_t p1[8], p2[8], l1[8], l2[8];
+          for (int c = 0; c < 4; ++c) {
+            uint32_t* cur = (c & 1) ? vb : va;
+            uint32_t* nx = (c & 1) ? va : vb;
+            tmem_ld_wait();
+            if (c < 3) {
+              tmem_ld8(sl_addr + 8 * (c + 1), nx);
+              tmem_ld8(sl_addr + 64 + 8 * (c + 1), nx + 8);
+            }
+            // a rotated value leaves as two f16: the value with its low 13 mantissa bits cleared (exact in f16) and the
+            // rest (rounded to f16: 2^-21 of the value instead of the 2^-11 of one f16), so that the score error stays
+            // far below the bar even where a few key channels carry most of the magnitude
+            uint32_t oh[8], ol[8];
 #pragma unroll
-          for (int t8 = 0; t8 < 8; ++t8) {
-            const int t = hb * 8 + t8;
-            const uint64_t L = f2_pack_bits(lo[2 * t], lo[2 * t + 1]), H = f2_pack_bits(hi[2 * t], hi[2 * t + 1]);
-            const uint64_t a = f2_sub(f2_mul(L, cs2[t]), f2_mul(H, sn2[t]));           // lo cos - hi sin
-            const uint64_t b = f2_fma(L, sn2[t], f2_mul(H, cs2[t]));                   // hi cos + lo sin
-            const uint64_t ah = a & 0xFFFFE000FFFFE000ull, bh = b & 0xFFFFE000FFFFE000ull;
-            p1[t8] = f2_to_f16x2_sat(ah);
-            p2[t8] = f2_to_f16x2_sat(bh);
-            l1[t8] = f2_to_f16x2_sat(f2_sub(a, ah));
-            l2[t8] = f2_to_f16x2_sat(f2_sub(b, bh));
+            for (int u = 0; u < 4; ++u) {
+              const int t = 4 * c + u;
+              const uint64_t L = f2_pack_bits(cur[2 * u], cur[2 * u + 1]), H = f2_pack_bits(cur[8 + 2 * u], cur[8 + 2 * u + 1]);
+              const uint64_t a = f2_sub(f2_mul(L, cs2[t]), f2_mul(H, sn2[t]));           // lo cos - hi sin
+              const uint64_t b = f2_fma(L, sn2[t], f2_mul(H, cs2[t]));                   // hi cos + lo sin
+              const uint64_t ah = a & 0xFFFFE000FFFFE000ull, bh = b & 0xFFFFE000FFFFE000ull;
+              oh[u] = f2_to_f16x2_sat(ah);
+              oh[4 + u] = f2_to_f16x2_sat(bh);
+              ol[u] = f2_to_f16x2_sat(f2_sub(a, ah));
+              ol[4 + u] = f2_to_f16x2_sat(f2_sub(b, bh));
+            }
+            tmem_st8(sl_addr + 8 * c, oh);                                    // high parts: columns 0 .. 63 of the slab
+            tmem_st8(sl_addr + 64 + 8 * c, ol);                               // low parts: columns 64 .. 127
           }
-          if (hb == 0) {
-            if (!__all_sync(0xffffffffu, kr_probe) && !(ok = __all_sync(0xffffffffu, mbar_wait(kr_empty, kr_par, abort_flag)))) break;
-            fence_after_sync();
-          }
-          tmem_st8(kr + 8 * hb, p1);                                        // dims d -> column d / 2
-          tmem_st8(kr + 32 + 8 * hb, p2);                                   // dims 64 + d
-          tmem_st8(kr + 64 + 8 * hb, l1);
-          tmem_st8(kr + 96 + 8 * hb, l2);
+          tmem_st_wait();
+          fence_before_sync();
+          __syncwarp();
+          if (lane == 0) mbar_arrive(kr_full + 8 * sbuf);
+          p_old = p_new;
+          p_new.out = out_row + g * REP;
+          p_new.mxi = qs * Hq + g * REP;
+          p_new.meta = KP_VALID | ((uint32_t)(sli & 1) << 1) | (mode << 2) | (slot << 4) | (slph << 6) | live_bit;
+          if (++sbuf == (uint32_t)KT_SLABS) { sbuf = 0; sph ^= 1u; }
+          if (++slot == (uint32_t)KT_S_SLOTS) { slot = 0; slph ^= 1u; }
         }
-        if (!ok) break;
-        const bool next_probe = mbar_try(slab_full + 8 * (buf ^ 1u), ((sc + 1) >> 1) & 1u);
-        tmem_st_wait();
-        fence_before_sync();
-        __syncwarp();
-        if (lane == 0) mbar_arrive(kr_full);
-        slab_ready = __all_sync(0xffffffffu, next_probe);
       }
       if (!ok) break;
-      // the next tile's rotation factors are fetched while this tile's last score products drain
       if (nxt.w >= 0) rope_setup(pos_next);
-      // all score products of the tile have retired: scale, mask the rows past the last token, store
-      if (!(ok = __all_sync(0xffffffffu, mbar_wait(s_full, tcount & 1u, abort_flag)))) break;
-      ++tcount;
-      fence_after_sync();
-      {
-        // this thread's groups g_lo .. g_hi - 1: REP columns of each group's 16-column region, all loads in flight at once
-        float sv[4 * REP];
-#pragma unroll
-        for (int gi = 0; gi < 4; ++gi)
-          if (g_lo + gi < g_hi) {
-            uint32_t* dst = reinterpret_cast<uint32_t*>(sv + gi * REP);
-            const uint32_t src = lane_addr + TM_S + 16 * (g_lo + gi);
-            if constexpr (REP == 1) tmem_ld1(src, dst);
-            else if constexpr (REP == 2) tmem_ld2(src, dst);
-            else if constexpr (REP == 4) tmem_ld4(src, dst);
-            else tmem_ld8(src, dst);
-          }
-        tmem_ld_wait();
-        const int h0 = g_lo * REP, nh = (g_hi - g_lo) * REP;
-        float* out = v.scores + ((size_t)tile * TILE + row) * Hq + h0;
-        const bool live = row < n_valid;
-#pragma unroll
-        for (int i = 0; i < 4 * REP; ++i) sv[i] = (live && i < nh) ? sv[i] * sm_scale : -INFINITY;
-        if constexpr (REP >= 4) {
-#pragma unroll
-          for (int i = 0; i < 4 * REP; i += 4)
-            if (i < nh) *reinterpret_cast<float4*>(out + i) = make_float4(sv[i], sv[i + 1], sv[i + 2], sv[i + 3]);
-        } else {
-#pragma unroll
-          for (int i = 0; i < 4 * REP; ++i) if (i < nh) out[i] = sv[i];
-        }
-#pragma unroll
-        for (int i = 0; i < 4 * REP; ++i) tmax[i] = fmaxf(tmax[i], sv[i]);
-        if (nxt.w != qs) {
-          // last tile of this query slot in the piece: maximum over the warp's rows, one atomic per head
-#pragma unroll
-          for (int i = 0; i < 4 * REP; ++i) {
-            float m = tmax[i];
-#pragma unroll
-            for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
-            if (lane == i && i < nh) atomicMax(&v.seqmax[qs * Hq + h0 + i], enc_ordered(m));
-            tmax[i] = -INFINITY;
-          }
-        }
+      if (nxt.w >= 0 && nxt.w != qs) {
+        // the query operand changes: every score product that reads the old one must have retired first
+        if (!(ok = read_out(p_old))) break;
+        p_old.meta = 0u;
+        if (!(ok = __all_sync(0xffffffffu, mbar_wait(s_full + 8 * ((p_new.meta >> 4) & 3u), (p_new.meta >> 6) & 1u, abort_flag)))) break;
+        write_q(nxt.w);
       }
-      if (nxt.w >= 0 && nxt.w != qs) write_q(nxt.w);
       e = nxt;
     }
+    if (ok) ok = read_out(p_old);
+    if (ok) ok = read_out(p_new);
+    tmem_ld_wait();                                                          // nothing of this thread is in flight when TMEM is freed
   }
 
   fence_before_sync();
@@ -451,7 +480,7 @@ cudaError_t launch_transpose16(const void* in, void* out, int n, cudaStream_t st
 }
 
 size_t kscore_tc_smem_bytes(int nb) {
-  return (size_t)(KT_A_SLOTS + nb) * PANEL_BYTES + 2 * KT_Q_PANEL_BYTES + KT_ROPE_STAGE_BYTES + 8 * (2 * KT_A_SLOTS + 2 * nb + 9) +
+  return (size_t)(KT_A_SLOTS + nb) * PANEL_BYTES + 2 * KT_Q_PANEL_BYTES + KT_ROPE_STAGE_BYTES + 8 * (KT_N_BARS + 2 * nb) +
          2 * sizeof(int);
 }
 

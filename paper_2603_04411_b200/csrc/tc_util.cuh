@@ -276,7 +276,11 @@ __device__ __forceinline__ void mma_commit_pair_both(uint32_t bar) {
 // Tensor maps the decode path needs: the block pool as rows of 64 elements, and the layer's transposed U_K^-1.
 struct TcMaps { CUtensorMap blocks, uinvT_k; };
 // Tensor maps of the fused gate kernel: the call's K and V states, and the layer's transposed gate weights.
-struct GateMaps { CUtensorMap xk, xv, wk, wv; };
+// `raw`: the same four operands as plain pointers (states row-major, weights transposed), for the rows the kernel
+// decides again in fp32.
+// fix_list / fix_counters: rows handed to the fix-up kernel (two int4 per row) and {entries, finished CTAs}.
+struct GateRaw { const unsigned short *xk, *xv, *wkT, *wvT; int4* fix_list; int* fix_counters; };
+struct GateMaps { CUtensorMap xk, xv, wk, wv; GateRaw raw; };
 // Tensor maps of the projection kernel: the call's raw states, the transposed bases, and the outputs.
 struct ProjectMaps { CUtensorMap xk, xv, uk, uv, ok, ov; };
 

@@ -14,9 +14,8 @@ constexpr int BLOCK_BYTES = TWKV_BLOCK_BYTES;
 constexpr int HEAD_DIM = 128;
 constexpr int CHUNK_TOKENS = 128;           // tokens per compress CTA
 constexpr int PIECE_CHUNKS = TWKV_PIECE_TOKENS / CHUNK_TOKENS;
-constexpr int ROPE_LO = 256;                // pos = hi * 256 + mid * 16 + lo
-constexpr int ROPE_HI = 2048;               // positions up to 256 * 2048 - 1
-constexpr int ROPE_SMALL_ROWS = 32;         // rows 0..15: mid * 16 * theta, rows 16..31: lo * theta
+constexpr int ROPE_LO = 16;                 // pos = hi * 16 + lo
+constexpr int ROPE_HI = 32768;              // positions up to 16 * 32768 - 1
 constexpr int MAX_PARTIALS_EXTRA = 320;     // V-side partial slots beyond max_seqs
 constexpr int MAX_PLAN_CTAS = 1024;         // upper bound on the K-score kernel's grid
 
@@ -24,11 +23,12 @@ constexpr int MAX_PLAN_CTAS = 1024;         // upper bound on the K-score kernel
 struct DevView {
   int L, Hq, Hkv, rep, d_kv, NC, S, tmax, NT, TPS, n_blocks, dtype, out_dtype, NK, max_partials;
   float tau, sm_scale;
-  int* status;               // [8]: [0] sticky status, [1] next free block
+  int* status;               // [8]: [0] sticky status, [1] next free block, [2] rows listed for the gate fix-up, [3] its finished CTAs
   int* pflags;               // [batch][2]: piece accepted, piece holds an invalid token (scratch of one compress call)
   int batch;                 // pieces of a compress call whose bookkeeping is launched together
-  float2* rope_lo;           // [ROPE_SMALL_ROWS][64] (cos, sin) of mid * 16 * theta_i (rows 0..15) and lo * theta_i (rows 16..31)
-  float2* rope_hi;           // [ROPE_HI][64] (cos, sin) of hi * 256 * theta_i
+  // RoPE tables, one float4 per pair of frequencies (2t, 2t + 1): (cos_2t, cos_2t+1, sin_2t, sin_2t+1)
+  float4* rope_lo;           // [ROPE_LO][32]  angles lo * theta_i
+  float4* rope_hi;           // [ROPE_HI][32]  angles hi * 16 * theta_i
   unsigned char* blocks;     // n_blocks x 16 KiB
   // per-layer tables (index with the helpers below)
   int* n_tiles;              // [L][2]
@@ -60,6 +60,7 @@ struct DevView {
   int* cta_start;            // [MAX_PLAN_CTAS + 1]  first list entry of every K-score CTA
   float* part_acc;           // [max_partials][Hq][d_kv]
   float* part_l;             // [max_partials][Hq]
+  int4* gate_fix;            // rows the fused gate kernel hands to its fix-up kernel
   float* gate_scratch;       // COMPUTE mode logits: [GATE_PIECE][2][d_kv] (small calls) or one [128][d_kv] block per CTA (fused kernel)
 
   __host__ __device__ int4* desc(int l, int side) const { return tile_desc + ((size_t)l * 2 + side) * NT; }
@@ -136,6 +137,7 @@ cudaError_t launch_gate_ranks_tc(const DevView& v, const GateMaps& maps, const L
                                  int sm_count, bool pairs, cudaStream_t st);
 int gate_tc_max_pairs(int sm_count);
 size_t gate_tc_stage_bytes(int n_cta, int d);
+size_t gate_tc_fix_bytes();
 struct ProjectMaps;   // tensor maps of the projection kernel
 cudaError_t launch_project_tc(const ProjectMaps& maps, int n_tok, int d, int bf16, int side0, int n_sides, int* status,
                               int sm_count, bool pairs, cudaStream_t st);

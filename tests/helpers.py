@@ -89,6 +89,37 @@ def compare_cache_with_image(gc: GpuCache, img: CacheImage):
         np.testing.assert_array_equal(gc.blocks(img.next_block), img.blocks[:img.next_block])
 
 
+# COMPUTE-mode gate: the library forms z = x~ W + b in fp32 from exact 16-bit products and evaluates Eq. 5, 6, 8 in fp32
+# (rows the fused kernel cannot decide from its f16-staged terms are redone from fp32 terms).  With |z| up to a few
+# tens, the accumulation error of a logit is below 1e-4 absolute, i.e. below 1e-4 relative on exp(z) and on every
+# cumulative sum; decisions the fp64 oracle takes with a relative margin of at least 1e-3 must therefore agree.
+GATE_MARGIN_COMPUTE = 1e-3
+GATE_MARGIN_LOGITS = 1e-4        # logits given in fp32: only the fp32 softmax and prefix sums differ from fp64
+
+
+def check_gate_levels(got, z_k, z_v, tau, margin):
+    """Per-token ranks of the library against the oracle's gate on the oracle's own logits (Eq. 5, 6, 8).
+
+    Tokens the oracle decides with a relative distance of at least `margin` between every cumulative sum and tau
+    must carry the oracle's rank, bit for bit.  For the others several ranks are valid; the rank is non-increasing
+    in tau, so the library's rank must lie between the oracle's ranks at tau (1 + margin) and tau (1 - margin).
+    Returns the number of (token, side) decisions that fell under the second rule."""
+    got = np.asarray(got).astype(np.int64)
+    n_loose = 0
+    for side, z in enumerate((z_k, z_v)):
+        r, m = oracle.gate_rank(z, tau)
+        safe = m >= margin
+        np.testing.assert_array_equal(got[safe, side], r[safe])
+        if not safe.all():
+            zz = z[~safe]
+            r_lo, _ = oracle.gate_rank(zz, tau * (1.0 + margin))
+            r_hi, _ = oracle.gate_rank(zz, tau * (1.0 - margin))
+            g = got[~safe, side]
+            assert np.all((r_lo <= g) & (g <= r_hi)), (side, g[(g < r_lo) | (g > r_hi)][:8])
+            n_loose += int((~safe).sum())
+    return n_loose
+
+
 def oracle_decode(li, ranks, seq_list, layer_tokens=None, rope_base=500000.0):
     """Oracle attention for the listed sequences.  li: LayerInputs (any device); ranks [n, 2] numpy."""
     dn = dtype_name(li.dtype)
