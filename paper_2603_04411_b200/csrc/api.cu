@@ -160,7 +160,7 @@ static Offsets layout_of(const twkv_config* c, const Dims& d) {
   }
   o.gate_fix = L.alloc(gate_tc_fix_bytes());
   o.stats_buf = L.alloc(64 * sizeof(unsigned long long));
-  o.prep_uinvT = L.alloc(Ls * (size_t)d.d_kv * d.d_kv * 2, 1024);
+  o.prep_uinvT = L.alloc(Ls * ((kscore_uinv_bytes(d.d_kv) + 1023) / 1024 * 1024), 1024);
   o.prep_wT = L.alloc(Ls * 2 * (size_t)d.d_kv * d.d_kv * 2, 1024);
   o.blocks = L.alloc(0, 1024);
   o.end_fixed = o.blocks;
@@ -422,10 +422,10 @@ twkv_status twkv_decode_attn(twkv_cache* c, int layer, const void* q, const int3
   if (!g.ok) return TWKV_ERR_CUDA;
   ProfBind pb(&c->prof);
   if (!c->prepared[layer]) {
-    // first decode after the parameters were (re)set: K-major copy of U_K^-1 for the tensor cores
-    unsigned char* dst = c->pool + c->off.prep_uinvT + (size_t)layer * c->dims.d_kv * c->dims.d_kv * 2;
-    if (launch_transpose16(c->params[layer].Uinv_k, dst, c->dims.d_kv, (cudaStream_t)stream) != cudaSuccess) return TWKV_ERR_CUDA;
-    if (!make_tmap_2d(&c->map_uinvT[layer], dst, c->dims.d_kv, c->dims.d_kv, (uint64_t)c->dims.d_kv * 2, HEAD_DIM)) return TWKV_ERR_CUDA;
+    // first decode after the parameters were (re)set: U_K^-1 re-tiled into the contiguous K-major panels the tensor cores read
+    unsigned char* dst = c->pool + c->off.prep_uinvT + (size_t)layer * ((kscore_uinv_bytes(c->dims.d_kv) + 1023) / 1024 * 1024);
+    if (launch_uinv_panels(c->params[layer].Uinv_k, dst, c->dims.d_kv, (cudaStream_t)stream) != cudaSuccess) return TWKV_ERR_CUDA;
+    if (!make_tmap_2d(&c->map_uinvT[layer], dst, kscore_uinv_panel_rows(c->dims.d_kv), PANEL, PANEL * 2, HEAD_DIM)) return TWKV_ERR_CUDA;
     c->prepared[layer] = 1;
   }
   TcMaps maps;

@@ -5,8 +5,9 @@
 //   Krot_g = RoPE(Kbar_g, position of each token)                             (keys are rotated after reconstruction)
 //   S_g    = Krot_g . Q_g^T,  Q_g = the REP query heads that share KV head g   (the GQA group makes this a dense contraction)
 // The first product is a tcgen05.mma chain (M = 128, N = 128, K = 16 per instruction) whose fp32
-// accumulator (a "slab") lives in TMEM; X^_K panels and panels of the pre-transposed U_K^-1 arrive by TMA with
-// the 128-byte swizzle, which is the K-major operand layout the MMA reads from shared memory.
+// accumulator (a "slab") lives in TMEM; X^_K panels and panels of U_K^-1 (re-tiled once per layer into contiguous
+// [128 x 64] transposed panels) arrive by TMA with the 128-byte swizzle, which is the K-major operand layout the MMA
+// reads from shared memory.
 // Epilogue warps pull the slab out of TMEM sixteen columns at a time, rotate it in fp32, split every value into a
 // high and a low f16 part and store both back IN PLACE (a thread overwrites only columns it has already read: 64
 // fp32 columns become 32 columns of high parts and 32 of low parts), from where they are the A operands of the second
@@ -48,6 +49,8 @@ constexpr int KT_Q_ROWS = 72;                                 // 8 rows per KV h
 constexpr uint32_t KT_Q_PANEL_BYTES = KT_Q_ROWS * 128;        // one 64-wide K panel of the query operand
 constexpr int KT_ROPE_STRIDE = 33;                            // float4 per row of the small RoPE table in shared memory (32 + 1 against bank conflicts)
 constexpr uint32_t KT_ROPE_STAGE_BYTES = ROPE_LO * KT_ROPE_STRIDE * 16;
+constexpr int KT_HOT_PANELS = 4;                              // panel rows of U_K^-1 (64 spectral components each) kept in several copies
+constexpr int KT_UINV_COPIES = 8;
 constexpr int KT_N_BARS = 2 * KT_A_SLOTS + 3 * KT_SLABS + 2 * KT_S_SLOTS;     // + 2 nb for the U_K^-1 ring
 
 // Packed fp32 pairs (two lanes per 64-bit register, one instruction for both): the rotation is issue-bound.
@@ -75,7 +78,7 @@ template <bool BF16> __device__ __forceinline__ float kt_to_f32(unsigned short b
 // A score read-out that is still owed: which accumulator, where the scores go, how they combine.
 struct KtPending {
   float* out;            // this thread's row of the score scratch, at the group's first head
-  int mxi;               // index of the group's first head in the running-max table
+  int mxi;               // which of the reading thread's running maxima the scores fold into (slab index / 2)
   uint32_t meta;         // bit 0 valid | bit 1 reader half | bits 2-3 mode | bits 4-5 accumulator | bit 6 its parity | bit 7 row is a token
 };
 constexpr uint32_t KP_VALID = 1u, KP_LIVE = 128u;
@@ -137,8 +140,10 @@ kscore_tc_kernel(const __grid_constant__ CUtensorMap map_blocks, const __grid_co
 
   if (warp == 10) {
     // ------------------------------------------------------------- TMA producer: X^_K panels
-    // A thread's TMA copies complete one after the other, so the ring is served by four lanes
-    // (lane L owns slots L and L + 4) that each keep their own copy in flight.
+    // A thread's TMA copies complete one after the other, so the ring is served by four lanes (lane L issues the
+    // copies of slots L and L + 4) that each keep their own copy in flight.  The four lanes walk the panel sequence
+    // together and wait on the same barrier (slots free up in order): lanes of one warp blocked on different barriers
+    // would run one after the other, each one's wait holding up the others' copies.
     if (lane < 4) {
       if (lane == 0) tma_prefetch_desc(&map_blocks);
       uint32_t ak = 0;                                          // panels so far; slot = ak % 8
@@ -149,10 +154,12 @@ kscore_tc_kernel(const __grid_constant__ CUtensorMap map_blocks, const __grid_co
         const int cls = e.y & 0xff, blk = e.z;
         for (int j = 0; j < cls; ++j, ++ak) {
           const uint32_t slot = ak % KT_A_SLOTS, ph = (ak / KT_A_SLOTS) & 1u;
-          if ((slot & 3u) != (uint32_t)lane) continue;
-          if (!(ok = mbar_wait(a_empty + 8 * slot, ph ^ 1u, abort_flag))) break;
-          mbar_expect_tx(a_full + 8 * slot, PANEL_BYTES);
-          tma_load_2d(sA + slot * PANEL_BYTES, &map_blocks, a_full + 8 * slot, 0, (blk + j) * TILE);
+          if (!(ok = __all_sync(0xfu, mbar_wait(a_empty + 8 * slot, ph ^ 1u, abort_flag)))) break;
+          if ((slot & 3u) == (uint32_t)lane) {
+            mbar_expect_tx(a_full + 8 * slot, PANEL_BYTES);
+            tma_load_2d(sA + slot * PANEL_BYTES, &map_blocks, a_full + 8 * slot, 0, (blk + j) * TILE);
+          }
+          __syncwarp(0xfu);
         }
         e = nxt;
       }
@@ -165,11 +172,15 @@ kscore_tc_kernel(const __grid_constant__ CUtensorMap map_blocks, const __grid_co
     __syncwarp();
   } else if (warp == 0) {
     // ------------------------------------------------------------- TMA producer: U_K^-1 panels
-    // one lane per ring stage, for the same reason
+    // one lane per ring stage, walking the panel sequence together, for the same reasons
     if (lane < nb) {
+      const unsigned lanes = (1u << nb) - 1u;
       if (lane == 0) tma_prefetch_desc(&map_uinvT);
       uint32_t bk = 0, bst = 0, bph = 0;                        // panels so far; ring stage and its phase
       bool ok = true;
+      // this CTA's copy of the hot panel rows (copy 0 is the full matrix itself)
+      const int hot_copy = (blockIdx.x / Hkv) % KT_UINV_COPIES;
+      const int hot_base = v.NC * Hkv + (hot_copy - 1) * KT_HOT_PANELS * Hkv;
       int4 e = w0 < total ? klist[w0] : kt_none;
       for (int w = w0; w < total && ok; ++w) {
         const int4 nxt = w + 1 < total ? klist[w + 1] : kt_none;
@@ -181,10 +192,14 @@ kscore_tc_kernel(const __grid_constant__ CUtensorMap map_blocks, const __grid_co
             for (int j = 0; j < np; ++j, ++bk) {
               const uint32_t st = bst, ph = bph;
               if (++bst == (uint32_t)nb) { bst = 0; bph ^= 1u; }
-              if (st != (uint32_t)lane) continue;
-              if (!(ok = mbar_wait(b_empty + 8 * st, ph ^ 1u, abort_flag))) break;
-              mbar_expect_tx(b_full + 8 * st, PANEL_BYTES);
-              tma_load_2d(sB + st * PANEL_BYTES, &map_uinvT, b_full + 8 * st, (p0 + j) * PANEL, g * HEAD_DIM);
+              if (!(ok = __all_sync(lanes, mbar_wait(b_empty + 8 * st, ph ^ 1u, abort_flag)))) break;
+              if (st == (uint32_t)lane) {
+                const int pj = p0 + j;
+                const int prow = pj < KT_HOT_PANELS && hot_copy ? hot_base + pj * Hkv + g : pj * Hkv + g;     // panel index in the re-tiled copy
+                mbar_expect_tx(b_full + 8 * st, PANEL_BYTES);
+                tma_load_2d(sB + st * PANEL_BYTES, &map_uinvT, b_full + 8 * st, 0, prow * HEAD_DIM);
+              }
+              __syncwarp(lanes);
             }
           }
         }
@@ -286,6 +301,11 @@ kscore_tc_kernel(const __grid_constant__ CUtensorMap map_blocks, const __grid_co
     uint32_t sbuf = 0, sph = 0, slot = 0, slph = 0;
     bool ok = true;
     uint64_t cs2[16], sn2[16];                                    // the tile's rotation factors, frequencies (2 t, 2 t + 1) packed
+    float tmax[4][REP];                                           // running maxima of the heads this thread reads out (slab index / 2)
+#pragma unroll
+    for (int a = 0; a < 4; ++a)
+#pragma unroll
+      for (int i = 0; i < REP; ++i) tmax[a][i] = -INFINITY;
 
     // cos / sin of (row, frequency): pos = hi * 16 + lo, the two table rows combine by the angle-addition formulas.
     // The lo row comes from shared memory (padded rows: lanes with different rows hit different banks), the hi row
@@ -362,16 +382,32 @@ kscore_tc_kernel(const __grid_constant__ CUtensorMap map_blocks, const __grid_co
         for (int i = 0; i < REP; ++i) out[i] = sv[i];
       }
       if (mode != KP_STORE_PART) {
-        // maximum over the warp's rows, one atomic per head (max is order-independent, so the result is deterministic)
-        unsigned mine = 0u;
+        const int a_ = p.mxi;                                                        // slab index / 2: which maxima
 #pragma unroll
-        for (int i = 0; i < REP; ++i) {
-          const unsigned m = warp_max_u32(enc_ordered(sv[i]));
-          if (lane == i) mine = m;
-        }
-        if (lane < REP) atomicMax(&v.seqmax[p.mxi + lane], mine);
+        for (int a = 0; a < 4; ++a)
+#pragma unroll
+          for (int i = 0; i < REP; ++i) tmax[a][i] = a == a_ ? fmaxf(tmax[a][i], sv[i]) : tmax[a][i];
       }
       return true;
+    };
+    // Folds this thread's running maxima into the per-(sequence, head) maximum: over the warp's rows first, then one
+    // atomic per head (max is order-independent, so the result is deterministic).
+    auto flush_max = [&](int qs) {
+#pragma unroll
+      for (int a = 0; a < 4; ++a) {
+        const int sli = 2 * a + hf;
+        if (sli < Hkv) {
+          const int g = sli + g_rot < Hkv ? sli + g_rot : sli + g_rot - Hkv;
+          unsigned mine = 0u;
+#pragma unroll
+          for (int i = 0; i < REP; ++i) {
+            const unsigned m = warp_max_u32(enc_ordered(tmax[a][i]));
+            if (lane == i) mine = m;
+            tmax[a][i] = -INFINITY;
+          }
+          if (lane < REP) atomicMax(&v.seqmax[qs * Hq + g * REP + lane], mine);
+        }
+      }
     };
 
     KtPending p_old{nullptr, 0, 0u}, p_new{nullptr, 0, 0u};
@@ -431,7 +467,7 @@ kscore_tc_kernel(const __grid_constant__ CUtensorMap map_blocks, const __grid_co
           if (lane == 0) mbar_arrive(kr_full + 8 * sbuf);
           p_old = p_new;
           p_new.out = out_row + g * REP;
-          p_new.mxi = qs * Hq + g * REP;
+          p_new.mxi = sli >> 1;
           p_new.meta = KP_VALID | ((uint32_t)(sli & 1) << 1) | (mode << 2) | (slot << 4) | (slph << 6) | live_bit;
           if (++sbuf == (uint32_t)KT_SLABS) { sbuf = 0; sph ^= 1u; }
           if (++slot == (uint32_t)KT_S_SLOTS) { slot = 0; slph ^= 1u; }
@@ -439,17 +475,19 @@ kscore_tc_kernel(const __grid_constant__ CUtensorMap map_blocks, const __grid_co
       }
       if (!ok) break;
       if (nxt.w >= 0) rope_setup(pos_next);
-      if (nxt.w >= 0 && nxt.w != qs) {
-        // the query operand changes: every score product that reads the old one must have retired first
+      if (nxt.w != qs) {
+        // last tile of this query slot in the piece: the owed read-outs belong to it; the query operand may only change
+        // once every score product that reads the old one has retired
         if (!(ok = read_out(p_old))) break;
-        p_old.meta = 0u;
         if (!(ok = __all_sync(0xffffffffu, mbar_wait(s_full + 8 * ((p_new.meta >> 4) & 3u), (p_new.meta >> 6) & 1u, abort_flag)))) break;
-        write_q(nxt.w);
+        if (!(ok = read_out(p_new))) break;
+        p_old.meta = 0u;
+        p_new.meta = 0u;
+        flush_max(qs);
+        if (nxt.w >= 0) write_q(nxt.w);
       }
       e = nxt;
     }
-    if (ok) ok = read_out(p_old);
-    if (ok) ok = read_out(p_new);
     tmem_ld_wait();                                                          // nothing of this thread is in flight when TMEM is freed
   }
 
@@ -471,6 +509,41 @@ __global__ void transpose16_kernel(const unsigned short* __restrict__ in, unsign
   for (int r = threadIdx.y; r < 32; r += blockDim.y) out[(size_t)(bx + r) * n + by + threadIdx.x] = t[threadIdx.x][r];
 }
 
+// U_K^-1 [d x d] (row j = spectral component j) -> the B operand panels of the K-score kernel, each one contiguous:
+// panel (j64, g) = rows n = 0..127 of 128 bytes, out[((j64 * Hkv + g) * 128 + n) * 64 + k] = in[(j64 * 64 + k) * d + g * 128 + n].
+// A panel whose rows lie 2 d bytes apart (the plain transpose) sits in very few L2 slices, and with many CTAs asking
+// for the same panel its copy took thousands of cycles; 16 KiB of consecutive lines spread over all of them.
+// The first KT_HOT_PANELS panel rows (all that tiles of the narrow rank classes read) are stored KT_UINV_COPIES
+// times, blockIdx.z selecting the copy: when every CTA of the K-score kernel works on narrow tiles they all ask L2
+// for the same 8 .. 32 panels, and a panel's copy then took ~400 cycles per CTA asking for it (7 k cycles for a class-1
+// tile's panel); with each CTA on one of eight copies the requests spread over eight times as many lines.
+__global__ void uinv_panels_kernel(const unsigned short* __restrict__ in, unsigned short* __restrict__ out, int d) {
+  __shared__ unsigned short t[64][129];
+  const int j64 = blockIdx.x, g = blockIdx.y, tid = threadIdx.x;
+  if (blockIdx.z > 0) {
+    if (j64 >= KT_HOT_PANELS) return;
+    out += (size_t)d * d + (size_t)(blockIdx.z - 1) * KT_HOT_PANELS * d * 64;
+  }
+  for (int i = tid; i < 64 * 128; i += blockDim.x) {
+    const int k = i >> 7, n = i & 127;
+    t[k][n] = in[(size_t)(j64 * 64 + k) * d + g * 128 + n];
+  }
+  __syncthreads();
+  unsigned short* o = out + ((size_t)(j64 * gridDim.y + g) * 128) * 64;
+  for (int i = tid; i < 64 * 128; i += blockDim.x) {
+    const int n = i >> 6, k = i & 63;
+    o[i] = t[k][n];
+  }
+}
+
+cudaError_t launch_uinv_panels(const void* in, void* out, int d, cudaStream_t st) {
+  ProfScope ps(TWKV_K_OTHER, st);
+  uinv_panels_kernel<<<dim3(d / 64, d / 128, KT_UINV_COPIES), 256, 0, st>>>(reinterpret_cast<const unsigned short*>(in),
+                                                           reinterpret_cast<unsigned short*>(out), d);
+  count_launch();
+  return cudaGetLastError();
+}
+
 cudaError_t launch_transpose16(const void* in, void* out, int n, cudaStream_t st) {
   ProfScope ps(TWKV_K_OTHER, st);
   transpose16_kernel<<<dim3(n / 32, n / 32), dim3(32, 8), 0, st>>>(reinterpret_cast<const unsigned short*>(in),
@@ -478,6 +551,10 @@ cudaError_t launch_transpose16(const void* in, void* out, int n, cudaStream_t st
   count_launch();
   return cudaGetLastError();
 }
+
+// bytes of the re-tiled copy of one layer's U_K^-1 and the panel rows (of 128 x 64) it holds
+size_t kscore_uinv_bytes(int d) { return (size_t)d * d * 2 + (size_t)(KT_UINV_COPIES - 1) * KT_HOT_PANELS * d * 64 * 2; }
+size_t kscore_uinv_panel_rows(int d) { return (size_t)(d / 64) * d + (size_t)(KT_UINV_COPIES - 1) * KT_HOT_PANELS * d; }
 
 size_t kscore_tc_smem_bytes(int nb) {
   return (size_t)(KT_A_SLOTS + nb) * PANEL_BYTES + 2 * KT_Q_PANEL_BYTES + KT_ROPE_STAGE_BYTES + 8 * (KT_N_BARS + 2 * nb) +

@@ -143,6 +143,9 @@ cudaError_t launch_project_tc(const ProjectMaps& maps, int n_tok, int d, int bf1
                               int sm_count, bool pairs, cudaStream_t st);
 int project_tc_max_pairs(int sm_count);
 cudaError_t launch_transpose16(const void* in, void* out, int n, cudaStream_t st);
+cudaError_t launch_uinv_panels(const void* in, void* out, int d, cudaStream_t st);
+size_t kscore_uinv_bytes(int d);
+size_t kscore_uinv_panel_rows(int d);
 cudaError_t launch_gate_logits(const DevView& v, const LayerParams& lp, const void* K, const void* V, int n_tok,
                                float* logits, cudaStream_t st);
 cudaError_t launch_stats(const DevView& v, int layer, unsigned long long* out_dev, cudaStream_t st);
