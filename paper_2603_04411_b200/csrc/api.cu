@@ -1,6 +1,7 @@
 // C ABI of libtwkv: cache lifetime, argument checks, piece loop, launch bookkeeping.
 #include <atomic>
 #include <cstdio>
+#include <cstdlib>
 #include <cstring>
 #include <new>
 #include <vector>
@@ -78,7 +79,7 @@ constexpr int GATE_TC_MIN_TOKENS = 1024;   // calls at least this large run the 
 struct Offsets {
   size_t status, pflags, rope_lo, rope_hi, n_tiles, tile_desc, tile_aux, tile_rank, fill, key_last, kclass_count,
       kclass_tiles, seq_vcount, seq_vtiles, seq_tokens, rank_sums, hist, key_cnt, key_old_fill, key_first_id,
-      key_first_base, key_old_last, scores, seqmax, qslot, klist, klist_count, klist_cost, cta_start, part_acc, part_l, gate_scratch, gate_fix, stats_buf, tables_end, prep_uinvT, prep_wT,
+      key_first_base, key_old_last, scores, seqmax, qslot, klist, kpairs, klist_count, cta_start, part_acc, part_l, gate_scratch, gate_fix, stats_buf, tables_end, prep_uinvT, prep_wT,
       blocks, end_fixed;
 };
 
@@ -150,7 +151,7 @@ static Offsets layout_of(const twkv_config* c, const Dims& d) {
   o.qslot = L.alloc(S * sizeof(int));
   o.klist = L.alloc(NT * sizeof(int4));
   o.klist_count = L.alloc(sizeof(int));
-  o.klist_cost = L.alloc(NT * sizeof(unsigned));
+  o.kpairs = L.alloc((NT + 64) * sizeof(int4));
   o.cta_start = L.alloc((MAX_PLAN_CTAS + 1) * sizeof(int));
   o.part_acc = L.alloc((size_t)d.max_partials * Hq * d.d_kv * sizeof(float));
   o.part_l = L.alloc((size_t)d.max_partials * Hq * sizeof(float));
@@ -160,7 +161,7 @@ static Offsets layout_of(const twkv_config* c, const Dims& d) {
   }
   o.gate_fix = L.alloc(gate_tc_fix_bytes());
   o.stats_buf = L.alloc(64 * sizeof(unsigned long long));
-  o.prep_uinvT = L.alloc(Ls * ((kscore_uinv_bytes(d.d_kv) + 1023) / 1024 * 1024), 1024);
+  o.prep_uinvT = L.alloc(Ls * (size_t)d.d_kv * d.d_kv * 2, 1024);
   o.prep_wT = L.alloc(Ls * 2 * (size_t)d.d_kv * d.d_kv * 2, 1024);
   o.blocks = L.alloc(0, 1024);
   o.end_fixed = o.blocks;
@@ -188,6 +189,7 @@ struct twkv_cache {
   std::vector<CUtensorMap> map_wT;     // per layer x side, over the transposed copies of the gate weights (box = one slab)
   std::vector<CUtensorMap> map_wT_half; // the same with 128-row boxes, for the CTA-pair kernel
   std::vector<char> prepared_w;        // per layer: those copies and maps are current
+  bool kscore_pairs = false;           // the K-score kernel runs on CTA pairs (the device can co-schedule them)
 };
 
 
@@ -242,7 +244,7 @@ static void fill_view(twkv_cache* c) {
   v.key_old_last = (int*)(p + o.key_old_last);
   v.scores = (float*)(p + o.scores); v.seqmax = (unsigned*)(p + o.seqmax); v.qslot = (int*)(p + o.qslot);
   v.klist = (int4*)(p + o.klist); v.klist_count = (int*)(p + o.klist_count);
-  v.klist_cost = (unsigned*)(p + o.klist_cost); v.cta_start = (int*)(p + o.cta_start);
+  v.kpairs = (int4*)(p + o.kpairs); v.cta_start = (int*)(p + o.cta_start);
   v.part_acc = (float*)(p + o.part_acc); v.part_l = (float*)(p + o.part_l);
   v.gate_scratch = (float*)(p + o.gate_scratch);
   v.gate_fix = (int4*)(p + o.gate_fix);
@@ -281,6 +283,11 @@ twkv_status twkv_cache_create(const twkv_config* cfg, void* pool, size_t pool_by
   if (!g.ok) { delete c; return TWKV_ERR_CUDA; }
   if (cudaDeviceGetAttribute(&c->sm_count, cudaDevAttrMultiProcessorCount, c->device) != cudaSuccess) { delete c; return TWKV_ERR_CUDA; }
   if (c->sm_count > MAX_PLAN_CTAS) c->sm_count = MAX_PLAN_CTAS;
+  {
+    // TWKV_KSCORE_SINGLE=1 keeps the K-score kernel on single CTAs (the fallback where CTA pairs cannot be scheduled)
+    const char* single = getenv("TWKV_KSCORE_SINGLE");
+    c->kscore_pairs = !(single && single[0] == '1') && kscore_max_pairs(c->sm_count) > 0;
+  }
   fill_view(c);
   c->map_uinvT.resize(cfg->n_layers);
   c->prepared.assign(cfg->n_layers, 0);
@@ -423,15 +430,17 @@ twkv_status twkv_decode_attn(twkv_cache* c, int layer, const void* q, const int3
   ProfBind pb(&c->prof);
   if (!c->prepared[layer]) {
     // first decode after the parameters were (re)set: U_K^-1 re-tiled into the contiguous K-major panels the tensor cores read
-    unsigned char* dst = c->pool + c->off.prep_uinvT + (size_t)layer * ((kscore_uinv_bytes(c->dims.d_kv) + 1023) / 1024 * 1024);
+    unsigned char* dst = c->pool + c->off.prep_uinvT + (size_t)layer * c->dims.d_kv * c->dims.d_kv * 2;
     if (launch_uinv_panels(c->params[layer].Uinv_k, dst, c->dims.d_kv, (cudaStream_t)stream) != cudaSuccess) return TWKV_ERR_CUDA;
-    if (!make_tmap_2d(&c->map_uinvT[layer], dst, kscore_uinv_panel_rows(c->dims.d_kv), PANEL, PANEL * 2, HEAD_DIM)) return TWKV_ERR_CUDA;
+    // box = a whole panel for the single-CTA kernel, the CTA's half of its rows for the pair kernel
+    if (!make_tmap_2d(&c->map_uinvT[layer], dst, (uint64_t)c->dims.NC * c->dims.d_kv, PANEL, PANEL * 2,
+                      c->kscore_pairs ? HEAD_DIM / 2 : HEAD_DIM)) return TWKV_ERR_CUDA;
     c->prepared[layer] = 1;
   }
   TcMaps maps;
   maps.blocks = c->map_blocks;
   maps.uinvT_k = c->map_uinvT[layer];
-  if (launch_decode(c->view, layer, c->params[layer], q, seq_ids, n_seq, out, num_splits, c->sm_count, &maps,
+  if (launch_decode(c->view, layer, c->params[layer], q, seq_ids, n_seq, out, num_splits, c->sm_count, &maps, c->kscore_pairs,
                     (cudaStream_t)stream) != cudaSuccess) return TWKV_ERR_CUDA;
   return TWKV_OK;
 }

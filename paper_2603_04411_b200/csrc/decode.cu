@@ -19,30 +19,34 @@ namespace twkv {
 // ------------------------------------------------------------------------------ plan
 // One CTA: sequence id -> query slot map, running-max reset, and the K-score work list: the K tiles
 // of the listed sequences in class order (widest first, inside a class in table order), compacted
-// with block-wide scans so the order does not depend on thread timing.  The list is then cut into
-// n_cta contiguous pieces of about equal estimated cost, so a CTA of the K-score kernel mostly
-// stays inside one (class, sequence) run.
+// with block-wide scans so the order does not depend on thread timing.  For the CTA-pair kernel the list
+// is rewritten as items of two tiles of one class.  The list is then cut into n_cta contiguous pieces of
+// about equal estimated cost, so a CTA (pair) of the K-score kernel mostly stays inside one (class, sequence) run.
 __device__ __forceinline__ unsigned ktile_cost(int cls) {
-  // cycles per tile of the K-score kernel by rank class, measured inside the kernel on the benchmark's mix of classes
-  // (8 KV heads): a fixed part (rotation factors, score read-out, the per-slab epilogue chain) plus a per-panel part;
-  // classes above 8 run as two passes.  Only the ratios matter.
-  constexpr unsigned kCost[TWKV_MAX_CLASSES] = {17800u, 19400u, 22100u, 25100u, 29100u, 31700u, 34900u, 37900u,
-                                                50200u, 51200u, 55300u, 58800u, 62800u, 67500u, 68500u, 71700u};
+  // cycles per tile of the K-score kernel by rank class, measured on one-class workloads (8 KV heads): a fixed part
+  // (rotation factors, the per-slab epilogue and score products) plus a per-panel part; classes above 8 run as two
+  // passes.  Only the ratios matter.
+  constexpr unsigned kCost[TWKV_MAX_CLASSES] = {17100u, 17100u, 17900u, 19700u, 22700u, 25700u, 28600u, 31600u,
+                                                44000u, 46000u, 49000u, 52000u, 55000u, 58000u, 61000u, 63300u};
   return kCost[min(max(cls, 1), TWKV_MAX_CLASSES) - 1];
 }
 
-__global__ void __launch_bounds__(1024) plan_kernel(DevView v, int layer, const int* __restrict__ seq_ids, int n_seq, int n_cta) {
+__global__ void __launch_bounds__(1024) plan_kernel(DevView v, int layer, const int* __restrict__ seq_ids, int n_seq, int n_cta, int pairs) {
   __shared__ int s_cls_off[TWKV_MAX_CLASSES + 1];
-  __shared__ unsigned s_wsum[32][2];
-  __shared__ unsigned s_base[2];                                  // entries kept so far, their cost
+  __shared__ unsigned s_wsum[32];
+  __shared__ unsigned s_base;                                     // entries kept so far
+  __shared__ int s_keep[TWKV_MAX_CLASSES];                        // kept tiles per class run (run k = class NC - k)
+  __shared__ int s_koff[TWKV_MAX_CLASSES + 1], s_ioff[TWKV_MAX_CLASSES + 1];    // start of run k in the tile list / in the item list
+  __shared__ unsigned long long s_coff[TWKV_MAX_CLASSES + 1];     // estimated cost of everything before run k
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   for (int s = tid; s < v.S; s += blockDim.x) v.qslot[s] = -1;
+  if (tid < TWKV_MAX_CLASSES) s_keep[tid] = 0;
   if (tid == 0) {
     const int* kcc = v.kcc(layer);
     int run = 0;
     for (int c = v.NC; c >= 1; --c) { s_cls_off[v.NC - c] = run; run += kcc[c - 1]; }    // widest class first
     s_cls_off[v.NC] = run;
-    s_base[0] = 0u; s_base[1] = 0u;
+    s_base = 0u;
   }
   __syncthreads();
   for (int i = tid; i < n_seq; i += blockDim.x) {
@@ -62,18 +66,18 @@ __global__ void __launch_bounds__(1024) plan_kernel(DevView v, int layer, const 
   constexpr int PL_BATCH = 4;                                     // list chunks of 1024 whose table reads are issued together
   for (int f0 = 0; f0 < n_all; f0 += 1024 * PL_BATCH) {
     // the three dependent reads (tile id -> descriptor -> query slot) of PL_BATCH chunks go out level by level
-    int tile[PL_BATCH], cls_[PL_BATCH];
+    int tile[PL_BATCH], run_[PL_BATCH];
     int4 d[PL_BATCH];
     int4 ent[PL_BATCH];
 #pragma unroll
     for (int u = 0; u < PL_BATCH; ++u) {
       const int f = f0 + u * 1024 + tid;
-      tile[u] = -1; cls_[u] = 0;
+      tile[u] = -1; run_[u] = 0;
       if (f < n_all) {
         int k = 0;
         while (f >= s_cls_off[k + 1]) ++k;
-        cls_[u] = v.NC - k;
-        tile[u] = kct[(size_t)(cls_[u] - 1) * v.NT + (f - s_cls_off[k])];
+        run_[u] = k;
+        tile[u] = kct[(size_t)(v.NC - k - 1) * v.NT + (f - s_cls_off[k])];
       }
     }
 #pragma unroll
@@ -86,50 +90,72 @@ __global__ void __launch_bounds__(1024) plan_kernel(DevView v, int layer, const 
       if (f0 + u * 1024 >= n_all) break;                         // uniform across the CTA
       const int4 e = ent[u];
       const unsigned keep = e.w >= 0 ? 1u : 0u;
-      const unsigned cost = keep ? ktile_cost(e.y & 0xff) : 0u;
-      unsigned ik = keep, ic = cost;                              // inclusive scans inside the warp
+      unsigned ik = keep;                                         // inclusive scan inside the warp
 #pragma unroll
       for (int o = 1; o < 32; o <<= 1) {
-        const unsigned a = __shfl_up_sync(0xffffffffu, ik, o), b = __shfl_up_sync(0xffffffffu, ic, o);
-        if (lane >= o) { ik += a; ic += b; }
+        const unsigned a = __shfl_up_sync(0xffffffffu, ik, o);
+        if (lane >= o) ik += a;
       }
-      if (lane == 31) { s_wsum[warp][0] = ik; s_wsum[warp][1] = ic; }
+      if (lane == 31) s_wsum[warp] = ik;
       __syncthreads();
       if (warp == 0) {
-        unsigned wk = s_wsum[lane][0], wc = s_wsum[lane][1];
+        unsigned wk = s_wsum[lane];
 #pragma unroll
         for (int o = 1; o < 32; o <<= 1) {
-          const unsigned a = __shfl_up_sync(0xffffffffu, wk, o), b = __shfl_up_sync(0xffffffffu, wc, o);
-          if (lane >= o) { wk += a; wc += b; }
+          const unsigned a = __shfl_up_sync(0xffffffffu, wk, o);
+          if (lane >= o) wk += a;
         }
-        s_wsum[lane][0] = wk; s_wsum[lane][1] = wc;               // inclusive over warps
+        s_wsum[lane] = wk;                                        // inclusive over warps
       }
       __syncthreads();
-      const unsigned pk = s_base[0] + (warp ? s_wsum[warp - 1][0] : 0u) + ik - keep;      // exclusive position
-      const unsigned pc = s_base[1] + (warp ? s_wsum[warp - 1][1] : 0u) + ic - cost;      // exclusive cost prefix
-      if (keep) { v.klist[pk] = e; v.klist_cost[pk] = pc; }
+      const unsigned pk = s_base + (warp ? s_wsum[warp - 1] : 0u) + ik - keep;      // exclusive position
+      if (keep) { v.klist[pk] = e; atomicAdd(&s_keep[run_[u]], 1); }
       __syncthreads();
-      if (tid == 0) { s_base[0] += s_wsum[31][0]; s_base[1] += s_wsum[31][1]; }
+      if (tid == 0) s_base += s_wsum[31];
       __syncthreads();
     }
   }
-  // cut points: piece b starts at the entry whose cost interval [lo, hi) holds b / n_cta of the total, i.e. the last
-  // entry with lo * n_cta <= b * total (64-bit products, no division); a binary search per piece
-  const unsigned n_keep = s_base[0];
-  const unsigned long long total = s_base[1];
-  if (tid == 0) { *v.klist_count = (int)n_keep; v.cta_start[n_cta] = (int)n_keep; }
-  if (n_keep == 0 || total == 0ull) {
-    for (int b = tid; b < n_cta; b += blockDim.x) v.cta_start[b] = 0;
-    return;
+  // class runs of the kept list: tiles, items (a pair item holds two tiles) and estimated cost before each run
+  if (tid == 0) {
+    int ko = 0, io = 0;
+    unsigned long long co = 0ull;
+    for (int k = 0; k < v.NC; ++k) {
+      s_koff[k] = ko; s_ioff[k] = io; s_coff[k] = co;
+      const int items = pairs ? (s_keep[k] + 1) / 2 : s_keep[k];
+      ko += s_keep[k]; io += items;
+      co += (unsigned long long)items * ktile_cost(v.NC - k);
+    }
+    s_koff[v.NC] = ko; s_ioff[v.NC] = io; s_coff[v.NC] = co;
+    *v.klist_count = ko;
+    v.cta_start[n_cta] = io;
   }
+  __syncthreads();
+  const int n_items = s_ioff[v.NC];
+  const unsigned long long total = s_coff[v.NC];
+  if (pairs) {
+    for (int i = tid; i < n_items; i += blockDim.x) {
+      int k = 0;
+      while (i >= s_ioff[k + 1]) ++k;
+      const int t0 = s_koff[k] + 2 * (i - s_ioff[k]);
+      const int4 e0 = v.klist[t0];
+      // a run of odd length ends with a filler: the same tile again, flagged so that its scores are dropped
+      v.kpairs[2 * i] = e0;
+      v.kpairs[2 * i + 1] = t0 + 1 < s_koff[k + 1] ? v.klist[t0 + 1] : make_int4(e0.x, e0.y | 0x80, e0.z, e0.w);
+    }
+  }
+  // cut points: piece b starts at the item whose cost interval holds b / n_cta of the total (64-bit arithmetic; inside
+  // a run every item costs the same, so the item follows from a division)
   for (int b = tid; b < n_cta; b += blockDim.x) {
-    const unsigned long long key = (unsigned long long)b * total;
-    unsigned lo = 0, hi = n_keep;                                   // invariant: cost[lo] * n_cta <= key (cost[0] = 0)
-    while (hi - lo > 1) {
-      const unsigned mid = (lo + hi) >> 1;
-      if ((unsigned long long)v.klist_cost[mid] * (unsigned long long)n_cta <= key) lo = mid; else hi = mid;
+    int start = 0;
+    if (n_items > 0 && total > 0ull) {
+      const unsigned long long key = (unsigned long long)b * total / (unsigned long long)n_cta;
+      int k = 0;
+      while (k + 1 < v.NC && s_coff[k + 1] <= key) ++k;
+      const unsigned long long within = (key - s_coff[k]) / ktile_cost(v.NC - k);
+      const int cap = s_ioff[k + 1] - s_ioff[k];
+      start = s_ioff[k] + (int)(within < (unsigned long long)cap ? within : (unsigned long long)cap);
     }
-    v.cta_start[b] = (int)lo;
+    v.cta_start[b] = start;
   }
 }
 
@@ -477,14 +503,16 @@ merge_kernel(DevView v, const unsigned short* __restrict__ Uinv_v, int n_splits,
 
 // ------------------------------------------------------------------------- host side
 cudaError_t launch_kscore_tc(const DevView& v, int layer, const CUtensorMap& map_blocks, const CUtensorMap& map_uinvT,
-                             const void* q, int sm_count, cudaStream_t st);
+                             const void* q, int n_pieces, bool pairs, cudaStream_t st);
 
 template <bool BF16>
 static cudaError_t launch_decode_t(const DevView& v, int layer, const LayerParams& lp, const void* q, const int* seq_ids,
-                                   int n_seq, void* out, int n_splits, int sm_count, const TcMaps* maps, cudaStream_t st) {
-  { ProfScope ps(TWKV_K_PLAN, st); plan_kernel<<<1, 1024, 0, st>>>(v, layer, seq_ids, n_seq, sm_count); }
+                                   int n_seq, void* out, int n_splits, int sm_count, const TcMaps* maps, bool pairs, cudaStream_t st) {
+  // the K-score kernel's work is cut into one piece per persistent CTA, or per CTA pair
+  const int n_pieces = pairs ? kscore_max_pairs(sm_count) : sm_count;
+  { ProfScope ps(TWKV_K_PLAN, st); plan_kernel<<<1, 1024, 0, st>>>(v, layer, seq_ids, n_seq, n_pieces, pairs ? 1 : 0); }
   {
-    cudaError_t e = launch_kscore_tc(v, layer, maps->blocks, maps->uinvT_k, q, sm_count, st);
+    cudaError_t e = launch_kscore_tc(v, layer, maps->blocks, maps->uinvT_k, q, n_pieces, pairs, st);
     if (e != cudaSuccess) return e;
   }
   const size_t va_smem = VA_STAGES * 16384 + (BF16 ? 4 : 2) * 8192 + 32 * 4;
@@ -516,10 +544,10 @@ static cudaError_t launch_decode_t(const DevView& v, int layer, const LayerParam
 }
 
 cudaError_t launch_decode(const DevView& v, int layer, const LayerParams& lp, const void* q, const int* seq_ids,
-                          int n_seq, void* out, int num_splits, int sm_count, const TcMaps* maps, cudaStream_t st) {
+                          int n_seq, void* out, int num_splits, int sm_count, const TcMaps* maps, bool pairs, cudaStream_t st) {
   if (n_seq <= 0) return cudaSuccess;
-  return v.dtype == TWKV_BF16 ? launch_decode_t<true>(v, layer, lp, q, seq_ids, n_seq, out, num_splits, sm_count, maps, st)
-                              : launch_decode_t<false>(v, layer, lp, q, seq_ids, n_seq, out, num_splits, sm_count, maps, st);
+  return v.dtype == TWKV_BF16 ? launch_decode_t<true>(v, layer, lp, q, seq_ids, n_seq, out, num_splits, sm_count, maps, pairs, st)
+                              : launch_decode_t<false>(v, layer, lp, q, seq_ids, n_seq, out, num_splits, sm_count, maps, pairs, st);
 }
 
 }  // namespace twkv

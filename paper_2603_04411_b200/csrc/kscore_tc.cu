@@ -20,10 +20,10 @@
 //
 // Tensor memory (512 columns): slabs 3 x 128 | score accumulators 4 x 16.
 // Warp roles (384 threads, one persistent CTA per SM working through a contiguous, cost-balanced piece of the tile list):
-//   warp 0      TMA producer of U_K^-1 panels (ring, one lane per stage)
+//   warp 0      TMA producer of U_K^-1 panels (ring; one elected lane)
 //   warp 1      issuer of the main products (one elected lane; owns the TMEM allocation)
 //   warps 2-9   epilogue (thread = one token row x one half of the RoPE frequencies)
-//   warp 10     TMA producer of X^_K panels (ring of 8 slots served by four lanes, runs ahead into the next tiles)
+//   warp 10     TMA producer of X^_K panels (ring of 8 slots; one elected lane, runs ahead into the next tiles)
 //   warp 11     issuer of the score products (one elected lane)
 // A slab buffer goes round: main products (slab_full) -> epilogue (kr_full) -> score products (slab_empty).
 // All waits are bounded (tc_util.cuh); a wait that runs out ends the kernel with TWKV_ERR_TIMEOUT.
@@ -49,8 +49,6 @@ constexpr int KT_Q_ROWS = 72;                                 // 8 rows per KV h
 constexpr uint32_t KT_Q_PANEL_BYTES = KT_Q_ROWS * 128;        // one 64-wide K panel of the query operand
 constexpr int KT_ROPE_STRIDE = 33;                            // float4 per row of the small RoPE table in shared memory (32 + 1 against bank conflicts)
 constexpr uint32_t KT_ROPE_STAGE_BYTES = ROPE_LO * KT_ROPE_STRIDE * 16;
-constexpr int KT_HOT_PANELS = 4;                              // panel rows of U_K^-1 (64 spectral components each) kept in several copies
-constexpr int KT_UINV_COPIES = 8;
 constexpr int KT_N_BARS = 2 * KT_A_SLOTS + 3 * KT_SLABS + 2 * KT_S_SLOTS;     // + 2 nb for the U_K^-1 ring
 
 // Packed fp32 pairs (two lanes per 64-bit register, one instruction for both): the rotation is issue-bound.
@@ -82,24 +80,34 @@ struct KtPending {
   uint32_t meta;         // bit 0 valid | bit 1 reader half | bits 2-3 mode | bits 4-5 accumulator | bit 6 its parity | bit 7 row is a token
 };
 constexpr uint32_t KP_VALID = 1u, KP_LIVE = 128u;
-constexpr uint32_t KP_STORE_PART = 0u, KP_STORE_FINAL = 1u, KP_ADD_FINAL = 2u;      // modes
+constexpr uint32_t KP_STORE_PART = 0u, KP_STORE_FINAL = 1u, KP_ADD_FINAL = 2u, KP_DISCARD = 3u;      // modes
+constexpr int KE_DISCARD = 0x80;                               // list entry, .y bit 7: a filler tile whose scores are not kept
 
-template <bool BF16, int REP>
+// PAIR: the kernel runs on CTA pairs (clusters of two, cta_group::2).  The two CTAs take two tiles of the same class
+// at a time: each loads its own tile's panels and its own 64 of the 128 rows of every U_K^-1 panel, one
+// tcgen05.mma of the even CTA (M = 256 over the pair) drives both tensor cores, each CTA's accumulator in its own
+// TMEM.  Per SM the panels of U_K^-1 read from L2, and the shared-memory operand reads, drop by half; both bound the
+// single-CTA kernel on the wide classes.  Epilogue, rotation factors and queries stay per CTA; the score product
+// takes 8 query rows from each CTA (N = 16), so each CTA finds its own scores in its own 8 columns.
+// Barriers: a_full / b_full / kr_full / slab_empty / s_empty live in the even CTA (the odd CTA's copies complete on
+// them and its epilogue warps arrive on them through the cluster window); a_empty / b_empty / slab_full / s_full exist in
+// both and are signalled together by a multicast tcgen05.commit (a commit, not a load).
+template <bool BF16, int REP, bool PAIR>
 __global__ void __launch_bounds__(KT_THREADS, 1)
 kscore_tc_kernel(const __grid_constant__ CUtensorMap map_blocks, const __grid_constant__ CUtensorMap map_uinvT,
                  DevView v, int layer, const unsigned short* __restrict__ q, int nb) {
   extern __shared__ __align__(1024) unsigned char smem_raw[];
+  constexpr int CG = PAIR ? 2 : 1;
+  constexpr uint32_t B_STAGE_BYTES = PAIR ? PANEL_BYTES / 2 : PANEL_BYTES;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int Hq = v.Hq, Hkv = v.Hkv;
+  const uint32_t crank = PAIR ? cluster_cta_rank() : 0u;
   // operand tiles need 1024-byte alignment for the 128-byte swizzle
   const uint32_t sA = smem_addr(smem_raw);
-  if (sA & 1023u) {
-    if (tid == 0) set_status(v, TWKV_ERR_DEVICE_CHECK);
-    return;
-  }
+  const bool misaligned = (sA & 1023u) != 0;
   const uint32_t sB = sA + KT_A_SLOTS * PANEL_BYTES;
-  const uint32_t sQ = sB + nb * PANEL_BYTES;
-  unsigned char* sQ_ptr = smem_raw + (KT_A_SLOTS + nb) * PANEL_BYTES;
+  const uint32_t sQ = sB + nb * B_STAGE_BYTES;
+  unsigned char* sQ_ptr = smem_raw + KT_A_SLOTS * PANEL_BYTES + nb * B_STAGE_BYTES;
   float4* sRope = reinterpret_cast<float4*>(sQ_ptr + 2 * KT_Q_PANEL_BYTES);   // [16 rows][33]: the small RoPE table
   unsigned char* tail = sQ_ptr + 2 * KT_Q_PANEL_BYTES + KT_ROPE_STAGE_BYTES;
   const uint32_t bars = smem_addr(tail);
@@ -109,82 +117,87 @@ kscore_tc_kernel(const __grid_constant__ CUtensorMap map_blocks, const __grid_co
   const uint32_t slab_empty = kr_full + 8 * KT_SLABS, s_full = slab_empty + 8 * KT_SLABS, s_empty = s_full + 8 * KT_S_SLOTS;
   uint32_t* s_tmem_base = reinterpret_cast<uint32_t*>(tail + 8 * (KT_N_BARS + 2 * nb));
   volatile int* abort_flag = reinterpret_cast<int*>(s_tmem_base + 1);
+  // the even CTA's copies of the barriers both CTAs signal
+  const uint32_t a_full_own = PAIR ? cluster_map(a_full, 0) : a_full, b_full_own = PAIR ? cluster_map(b_full, 0) : b_full;
+  const uint32_t kr_full_own = PAIR ? cluster_map(kr_full, 0) : kr_full, s_empty_own = PAIR ? cluster_map(s_empty, 0) : s_empty;
 
   if (tid == 0) {
     for (int i = 0; i < KT_A_SLOTS; ++i) { mbar_init(a_full + 8 * i, 1); mbar_init(a_empty + 8 * i, 1); }
     for (int i = 0; i < nb; ++i) { mbar_init(b_full + 8 * i, 1); mbar_init(b_empty + 8 * i, 1); }
     for (int i = 0; i < KT_SLABS; ++i) {
-      mbar_init(slab_full + 8 * i, 1); mbar_init(kr_full + 8 * i, KT_EPI / 32); mbar_init(slab_empty + 8 * i, 1);
+      mbar_init(slab_full + 8 * i, 1); mbar_init(kr_full + 8 * i, CG * (KT_EPI / 32)); mbar_init(slab_empty + 8 * i, 1);
     }
-    for (int i = 0; i < KT_S_SLOTS; ++i) { mbar_init(s_full + 8 * i, 1); mbar_init(s_empty + 8 * i, KT_EPI / 64); }
-    *abort_flag = 0;
+    for (int i = 0; i < KT_S_SLOTS; ++i) { mbar_init(s_full + 8 * i, 1); mbar_init(s_empty + 8 * i, CG * (KT_EPI / 64)); }
+    *abort_flag = misaligned ? 1 : 0;
     mbar_init_fence();
   }
-  if (warp == 1) tmem_alloc(smem_addr(s_tmem_base), KT_TMEM_COLS);
+  if (warp == 1) {
+    if constexpr (PAIR) tmem_alloc_pair(smem_addr(s_tmem_base), KT_TMEM_COLS);
+    else tmem_alloc(smem_addr(s_tmem_base), KT_TMEM_COLS);
+  }
   for (int i = tid; i < 2 * (int)KT_Q_PANEL_BYTES / 16; i += KT_THREADS)        // padding rows of the query operand stay zero
     reinterpret_cast<uint4*>(sQ_ptr)[i] = make_uint4(0u, 0u, 0u, 0u);
   for (int i = tid; i < ROPE_LO * 32; i += KT_THREADS) sRope[(i >> 5) * KT_ROPE_STRIDE + (i & 31)] = v.rope_lo[i];
   fence_proxy_async_smem();
   fence_before_sync();
   __syncthreads();
+  if constexpr (PAIR) cluster_sync_all();                       // both CTAs' barriers and TMEM are ready
   fence_after_sync();
   const uint32_t tmem_base = *s_tmem_base;
 
-  // work list written by plan_kernel: the K tiles of the sequences being decoded, widest class first
-  // this CTA's contiguous piece [w0, total) of the list (cut by estimated cost)
-  const int w0 = v.cta_start[blockIdx.x], total = v.cta_start[blockIdx.x + 1];
-  const int4* klist = v.klist;
+  // Work list written by plan_kernel: the K tiles of the sequences being decoded, widest class first; this CTA's (this
+  // pair's) contiguous piece [w0, total) of it, cut by estimated cost.  The pair list holds two entries per item, the
+  // even CTA's and the odd CTA's tile, always of one class (a class with an odd number of tiles ends with a filler).
+  const int piece = PAIR ? (int)(blockIdx.x >> 1) : (int)blockIdx.x;
+  const int w0 = v.cta_start[piece], total = v.cta_start[piece + 1];
+  const int4* klist = PAIR ? v.kpairs + crank : v.klist;
+  constexpr int KSTEP = PAIR ? 2 : 1;
   const int4 kt_none = make_int4(0, 0, 0, -1);
   // CTAs walk the KV heads in rotated order, so that at any moment they read different panels of U_K^-1 from L2
-  const int g_rot = blockIdx.x % Hkv;
+  const int g_rot = piece % Hkv;
 
-  if (warp == 10) {
+  if (misaligned) {
+    // nothing was started; fall through to the common exit
+  } else if (warp == 10) {
     // ------------------------------------------------------------- TMA producer: X^_K panels
-    // A thread's TMA copies complete one after the other, so the ring is served by four lanes (lane L issues the
-    // copies of slots L and L + 4) that each keep their own copy in flight.  The four lanes walk the panel sequence
-    // together and wait on the same barrier (slots free up in order): lanes of one warp blocked on different barriers
-    // would run one after the other, each one's wait holding up the others' copies.
-    if (lane < 4) {
-      if (lane == 0) tma_prefetch_desc(&map_blocks);
+    // One elected thread issues every copy, in ring order (slots free up in that order, so waiting for the oldest one
+    // never holds back a copy that could go out), and runs ahead into the next tiles.  Only a thread picked by
+    // elect.sync issues the copy instruction directly; from lanes picked by their index each issue took hundreds of cycles.
+    if (elect_one()) {
+      tma_prefetch_desc(&map_blocks);
       uint32_t ak = 0;                                          // panels so far; slot = ak % 8
       bool ok = true;
-      int4 e = w0 < total ? klist[w0] : kt_none;
+      int4 e = w0 < total ? klist[KSTEP * w0] : kt_none;
       for (int w = w0; w < total && ok; ++w) {
-        const int4 nxt = w + 1 < total ? klist[w + 1] : kt_none;
-        const int cls = e.y & 0xff, blk = e.z;
+        const int4 nxt = w + 1 < total ? klist[KSTEP * (w + 1)] : kt_none;
+        const int cls = e.y & 0x7f, blk = e.z;
         for (int j = 0; j < cls; ++j, ++ak) {
           const uint32_t slot = ak % KT_A_SLOTS, ph = (ak / KT_A_SLOTS) & 1u;
-          if (!(ok = __all_sync(0xfu, mbar_wait(a_empty + 8 * slot, ph ^ 1u, abort_flag)))) break;
-          if ((slot & 3u) == (uint32_t)lane) {
-            mbar_expect_tx(a_full + 8 * slot, PANEL_BYTES);
-            tma_load_2d(sA + slot * PANEL_BYTES, &map_blocks, a_full + 8 * slot, 0, (blk + j) * TILE);
-          }
-          __syncwarp(0xfu);
+          if (!(ok = mbar_wait_thin(a_empty + 8 * slot, ph ^ 1u, abort_flag))) break;
+          if (crank == 0) mbar_expect_tx(a_full + 8 * slot, CG * PANEL_BYTES);          // this CTA's copy and the partner's
+          if constexpr (PAIR) tma_load_2d_pair(sA + slot * PANEL_BYTES, &map_blocks, a_full_own + 8 * slot, 0, (blk + j) * TILE);
+          else tma_load_2d(sA + slot * PANEL_BYTES, &map_blocks, a_full + 8 * slot, 0, (blk + j) * TILE);
         }
         e = nxt;
       }
-      if (!ok)                                                  // let copies in flight land before the CTA goes away
+      if (!ok && !PAIR)                                         // let copies in flight land before the CTA goes away
         for (uint32_t i = 0; i < (uint32_t)KT_A_SLOTS && i < ak; ++i) {
           const uint32_t n = ak - 1 - i;
-          if (((n % KT_A_SLOTS) & 3u) == (uint32_t)lane) mbar_wait_drain(a_full + 8 * (n % KT_A_SLOTS), (n / KT_A_SLOTS) & 1u);
+          mbar_wait_drain(a_full + 8 * (n % KT_A_SLOTS), (n / KT_A_SLOTS) & 1u);
         }
     }
     __syncwarp();
   } else if (warp == 0) {
     // ------------------------------------------------------------- TMA producer: U_K^-1 panels
-    // one lane per ring stage, walking the panel sequence together, for the same reasons
-    if (lane < nb) {
-      const unsigned lanes = (1u << nb) - 1u;
-      if (lane == 0) tma_prefetch_desc(&map_uinvT);
+    // one elected thread, ring order, as above; a pair CTA loads its own half of every panel's rows
+    if (elect_one()) {
+      tma_prefetch_desc(&map_uinvT);
       uint32_t bk = 0, bst = 0, bph = 0;                        // panels so far; ring stage and its phase
       bool ok = true;
-      // this CTA's copy of the hot panel rows (copy 0 is the full matrix itself)
-      const int hot_copy = (blockIdx.x / Hkv) % KT_UINV_COPIES;
-      const int hot_base = v.NC * Hkv + (hot_copy - 1) * KT_HOT_PANELS * Hkv;
-      int4 e = w0 < total ? klist[w0] : kt_none;
+      int4 e = w0 < total ? klist[KSTEP * w0] : kt_none;
       for (int w = w0; w < total && ok; ++w) {
-        const int4 nxt = w + 1 < total ? klist[w + 1] : kt_none;
-        const int cls = e.y & 0xff;
+        const int4 nxt = w + 1 < total ? klist[KSTEP * (w + 1)] : kt_none;
+        const int cls = e.y & 0x7f;
         for (int p0 = 0; p0 < cls && ok; p0 += KT_A_SLOTS) {
           const int np = min(KT_A_SLOTS, cls - p0);
           for (int sl = 0; sl < Hkv && ok; ++sl) {
@@ -192,40 +205,37 @@ kscore_tc_kernel(const __grid_constant__ CUtensorMap map_blocks, const __grid_co
             for (int j = 0; j < np; ++j, ++bk) {
               const uint32_t st = bst, ph = bph;
               if (++bst == (uint32_t)nb) { bst = 0; bph ^= 1u; }
-              if (!(ok = __all_sync(lanes, mbar_wait(b_empty + 8 * st, ph ^ 1u, abort_flag)))) break;
-              if (st == (uint32_t)lane) {
-                const int pj = p0 + j;
-                const int prow = pj < KT_HOT_PANELS && hot_copy ? hot_base + pj * Hkv + g : pj * Hkv + g;     // panel index in the re-tiled copy
-                mbar_expect_tx(b_full + 8 * st, PANEL_BYTES);
-                tma_load_2d(sB + st * PANEL_BYTES, &map_uinvT, b_full + 8 * st, 0, prow * HEAD_DIM);
-              }
-              __syncwarp(lanes);
+              if (!(ok = mbar_wait_thin(b_empty + 8 * st, ph ^ 1u, abort_flag))) break;
+              const int y = ((p0 + j) * Hkv + g) * HEAD_DIM + (PAIR ? (int)crank * (HEAD_DIM / 2) : 0);     // rows of the re-tiled copy
+              if (crank == 0) mbar_expect_tx(b_full + 8 * st, CG * B_STAGE_BYTES);
+              if constexpr (PAIR) tma_load_2d_pair(sB + st * B_STAGE_BYTES, &map_uinvT, b_full_own + 8 * st, 0, y);
+              else tma_load_2d(sB + st * B_STAGE_BYTES, &map_uinvT, b_full + 8 * st, 0, y);
             }
           }
         }
         e = nxt;
       }
-      if (!ok)
+      if (!ok && !PAIR)
         for (uint32_t i = 0; i < (uint32_t)nb && i < bk; ++i) {
           const uint32_t n = bk - 1 - i;
-          if (n % nb == (uint32_t)lane) mbar_wait_drain(b_full + 8 * (n % nb), (n / nb) & 1u);
+          mbar_wait_drain(b_full + 8 * (n % nb), (n / nb) & 1u);
         }
     }
     __syncwarp();
   } else if (warp == 1) {
     // ------------------------------------------------------------- MMA issuer (one elected lane runs the whole role)
-    if (elect_one()) {
+    if (crank == 0 && elect_one()) {
       // This role is one thread issuing asynchronous work; what it costs is its own instruction stream (a 64-cycle MMA
       // per few instructions), so descriptors are stepped with 32-bit adds, a panel's four MMAs are one asm block, and
       // every wait tries once inline before it falls into the bounded loop.
-      const uint32_t idesc_main = idesc_f16(BF16 ? 1 : 0, 128, 128);
+      const uint32_t idesc_main = idesc_f16(BF16 ? 1 : 0, PAIR ? 256 : 128, 128);
       const uint32_t a_lo0 = kmajor_sw128_desc_lo(sA), b_lo0 = kmajor_sw128_desc_lo(sB);
       uint32_t bst = 0, bph = 0, ak = 0, sbuf = 0, sph = 0;
       bool ok = true;
-      int4 e = w0 < total ? klist[w0] : kt_none;
+      int4 e = w0 < total ? klist[KSTEP * w0] : kt_none;
       for (int w = w0; w < total && ok; ++w) {
-        const int4 nxt = w + 1 < total ? klist[w + 1] : kt_none;
-        const int cls = e.y & 0xff;
+        const int4 nxt = w + 1 < total ? klist[KSTEP * (w + 1)] : kt_none;
+        const int cls = e.y & 0x7f;
         for (int p0 = 0; p0 < cls && ok; p0 += KT_A_SLOTS) {
           const int np = min(KT_A_SLOTS, cls - p0);
           for (int sl = 0; sl < Hkv && ok; ++sl) {
@@ -242,12 +252,14 @@ kscore_tc_kernel(const __grid_constant__ CUtensorMap map_blocks, const __grid_co
               if (!(ok = mbar_wait_thin(b_full + 8 * st, bph, abort_flag))) break;
               if (++bst == (uint32_t)nb) { bst = 0; bph ^= 1u; }
               fence_after_sync();
-              mma_f16_ss_panel(d, a_lo0 + slot * (PANEL_BYTES >> 4), b_lo0 + st * (PANEL_BYTES >> 4), idesc_main, j > 0 ? 1u : 0u);
-              mma_commit(b_empty + 8 * st);                             // ring stage reusable when these MMAs retire
-              if (last) mma_commit(a_empty + 8 * slot);                 // last slab of the pass: the X^_K panel is done
+              mma_f16_ss_panel_cg<CG>(d, a_lo0 + slot * (PANEL_BYTES >> 4), b_lo0 + st * (B_STAGE_BYTES >> 4), idesc_main, j > 0 ? 1u : 0u);
+              // ring stage reusable when these MMAs retire; after the last slab of the pass the X^_K panel is done too
+              if constexpr (PAIR) { mma_commit_pair_both(b_empty + 8 * st); if (last) mma_commit_pair_both(a_empty + 8 * slot); }
+              else { mma_commit(b_empty + 8 * st); if (last) mma_commit(a_empty + 8 * slot); }
             }
             if (!ok) break;
-            mma_commit(slab_full + 8 * sbuf);                           // slab accumulator complete
+            if constexpr (PAIR) mma_commit_pair_both(slab_full + 8 * sbuf);     // slab accumulator complete
+            else mma_commit(slab_full + 8 * sbuf);
             if (++sbuf == (uint32_t)KT_SLABS) { sbuf = 0; sph ^= 1u; }
           }
           ak += np;
@@ -260,15 +272,15 @@ kscore_tc_kernel(const __grid_constant__ CUtensorMap map_blocks, const __grid_co
     // ------------------------------------------------------------- score-product issuer (one elected lane)
     // S (+)= Krot_g . Q_g^T as soon as the epilogue warps have stored a rotated slab; a thread of its own, so that
     // neither issue stream waits for the other's barriers
-    if (elect_one()) {
-      const uint32_t idesc_s = idesc_f16(0, 128, 16);
+    if (crank == 0 && elect_one()) {
+      const uint32_t idesc_s = idesc_f16(0, PAIR ? 256 : 128, 16);
       const uint32_t q_lo0 = kmajor_sw128_desc_lo(sQ);
       uint32_t sbuf = 0, sph = 0, slot = 0, slph = 0;
       bool ok = true;
-      int4 e = w0 < total ? klist[w0] : kt_none;
+      int4 e = w0 < total ? klist[KSTEP * w0] : kt_none;
       for (int w = w0; w < total && ok; ++w) {
-        const int4 nxt = w + 1 < total ? klist[w + 1] : kt_none;
-        const int cls = e.y & 0xff;
+        const int4 nxt = w + 1 < total ? klist[KSTEP * (w + 1)] : kt_none;
+        const int cls = e.y & 0x7f;
         for (int p0 = 0; p0 < cls && ok; p0 += KT_A_SLOTS) {
           for (int sl = 0; sl < Hkv; ++sl) {
             const int g = sl + g_rot < Hkv ? sl + g_rot : sl + g_rot - Hkv;
@@ -277,10 +289,10 @@ kscore_tc_kernel(const __grid_constant__ CUtensorMap map_blocks, const __grid_co
             fence_after_sync();
             // the rotated keys come as a high and a low f16 part (their sum carries 21 bits): two products into the same S
             const uint32_t kr = tmem_base + TM_SLAB + sbuf * 128, sd = tmem_base + TM_S + 16 * slot;
-            mma_f16_ts_k128(sd, kr, q_lo0 + g * (1024 >> 4), KT_Q_PANEL_BYTES >> 4, idesc_s, 0u);
-            mma_f16_ts_k128(sd, kr + 64, q_lo0 + g * (1024 >> 4), KT_Q_PANEL_BYTES >> 4, idesc_s, 1u);
-            mma_commit(slab_empty + 8 * sbuf);                          // the slab buffer may be overwritten
-            mma_commit(s_full + 8 * slot);                              // this slab's scores are complete
+            mma_f16_ts_k128_cg<CG>(sd, kr, q_lo0 + g * (1024 >> 4), KT_Q_PANEL_BYTES >> 4, idesc_s, 0u);
+            mma_f16_ts_k128_cg<CG>(sd, kr + 64, q_lo0 + g * (1024 >> 4), KT_Q_PANEL_BYTES >> 4, idesc_s, 1u);
+            if constexpr (PAIR) { mma_commit_pair(slab_empty + 8 * sbuf); mma_commit_pair_both(s_full + 8 * slot); }
+            else { mma_commit(slab_empty + 8 * sbuf); mma_commit(s_full + 8 * slot); }   // buffer reusable; scores complete
             if (++sbuf == (uint32_t)KT_SLABS) { sbuf = 0; sph ^= 1u; }
             if (++slot == (uint32_t)KT_S_SLOTS) { slot = 0; slph ^= 1u; }
           }
@@ -289,12 +301,13 @@ kscore_tc_kernel(const __grid_constant__ CUtensorMap map_blocks, const __grid_co
       }
     }
     __syncwarp();
-  } else {
+  } else if (warp >= 2 && warp <= 9) {
     // ------------------------------------------------------------- epilogue
     const int et = tid - 64;
     const int quarter = warp & 3, hf = (warp - 2) >> 2;
     const int row = quarter * 32 + lane;
     const uint32_t lane_addr = tmem_base + ((uint32_t)(quarter * 32) << 16);
+    const uint32_t s_col0 = TM_S + (PAIR ? 8u * crank : 0u);     // this CTA's columns of a score accumulator
     const float sm_scale = v.sm_scale;
     const int* kpos = v.aux(layer, 0);
     const float4* __restrict__ rope_hi = v.rope_hi;
@@ -356,7 +369,7 @@ kscore_tc_kernel(const __grid_constant__ CUtensorMap map_blocks, const __grid_co
       float sv[REP];
       {
         uint32_t* dst = reinterpret_cast<uint32_t*>(sv);
-        const uint32_t src = lane_addr + TM_S + 16 * sl_;
+        const uint32_t src = lane_addr + s_col0 + 16 * sl_;
         if constexpr (REP == 1) tmem_ld1(src, dst);
         else if constexpr (REP == 2) tmem_ld2(src, dst);
         else if constexpr (REP == 4) tmem_ld4(src, dst);
@@ -365,7 +378,11 @@ kscore_tc_kernel(const __grid_constant__ CUtensorMap map_blocks, const __grid_co
       tmem_ld_wait();
       fence_before_sync();
       __syncwarp();
-      if (lane == 0) mbar_arrive(s_empty + 8 * sl_);
+      if (lane == 0) {
+        if constexpr (PAIR) mbar_arrive_cluster(s_empty_own + 8 * sl_);
+        else mbar_arrive(s_empty + 8 * sl_);
+      }
+      if (mode == KP_DISCARD) return true;
       const bool live = (p.meta & KP_LIVE) != 0;
       float* out = p.out;
 #pragma unroll
@@ -411,17 +428,18 @@ kscore_tc_kernel(const __grid_constant__ CUtensorMap map_blocks, const __grid_co
     };
 
     KtPending p_old{nullptr, 0, 0u}, p_new{nullptr, 0, 0u};
-    int4 e = w0 < total ? klist[w0] : kt_none;
+    int4 e = w0 < total ? klist[KSTEP * w0] : kt_none;
     if (w0 < total) { write_q(e.w); rope_setup(kpos[(size_t)e.x * TILE + row]); }
     for (int w = w0; w < total && ok; ++w) {
-      const int4 nxt = w + 1 < total ? klist[w + 1] : kt_none;
-      const int tile = e.x, cls = e.y & 0xff, n_valid = e.y >> 8, qs = e.w;
+      const int4 nxt = w + 1 < total ? klist[KSTEP * (w + 1)] : kt_none;
+      const int tile = e.x, cls = e.y & 0x7f, n_valid = e.y >> 8, qs = e.w;
+      const bool discard = (e.y & KE_DISCARD) != 0;
       const int passes = (cls + KT_A_SLOTS - 1) / KT_A_SLOTS;
       const int pos_next = nxt.w >= 0 ? kpos[(size_t)nxt.x * TILE + row] : 0;      // fetched now, used after the tile's slabs
       float* const out_row = v.scores + ((size_t)tile * TILE + row) * Hq;
       const uint32_t live_bit = row < n_valid ? KP_LIVE : 0u;
       for (int ps = 0; ps < passes && ok; ++ps) {
-        const uint32_t mode = passes == 1 ? KP_STORE_FINAL : (ps == 0 ? KP_STORE_PART : KP_ADD_FINAL);
+        const uint32_t mode = discard ? KP_DISCARD : passes == 1 ? KP_STORE_FINAL : (ps == 0 ? KP_STORE_PART : KP_ADD_FINAL);
         for (int sli = 0; sli < Hkv; ++sli) {
           const int g = sli + g_rot < Hkv ? sli + g_rot : sli + g_rot - Hkv;
           if (!(ok = __all_sync(0xffffffffu, mbar_wait(slab_full + 8 * sbuf, sph, abort_flag)))) break;
@@ -464,7 +482,10 @@ kscore_tc_kernel(const __grid_constant__ CUtensorMap map_blocks, const __grid_co
           tmem_st_wait();
           fence_before_sync();
           __syncwarp();
-          if (lane == 0) mbar_arrive(kr_full + 8 * sbuf);
+          if (lane == 0) {
+            if constexpr (PAIR) mbar_arrive_cluster(kr_full_own + 8 * sbuf);
+            else mbar_arrive(kr_full + 8 * sbuf);
+          }
           p_old = p_new;
           p_new.out = out_row + g * REP;
           p_new.mxi = sli >> 1;
@@ -493,9 +514,13 @@ kscore_tc_kernel(const __grid_constant__ CUtensorMap map_blocks, const __grid_co
 
   fence_before_sync();
   __syncthreads();
+  if constexpr (PAIR) cluster_sync_all();                       // the partner is done with this CTA's memory and barriers as well
   fence_after_sync();
-  if (warp == 1) tmem_dealloc(tmem_base, KT_TMEM_COLS);
-  if (tid == 0 && *abort_flag) set_status(v, TWKV_ERR_TIMEOUT);
+  if (warp == 1) {
+    if constexpr (PAIR) tmem_dealloc_pair(tmem_base, KT_TMEM_COLS);
+    else tmem_dealloc(tmem_base, KT_TMEM_COLS);
+  }
+  if (tid == 0 && *abort_flag) set_status(v, misaligned ? TWKV_ERR_DEVICE_CHECK : TWKV_ERR_TIMEOUT);
 }
 
 // ------------------------------------------------------------------------------------------
@@ -511,19 +536,10 @@ __global__ void transpose16_kernel(const unsigned short* __restrict__ in, unsign
 
 // U_K^-1 [d x d] (row j = spectral component j) -> the B operand panels of the K-score kernel, each one contiguous:
 // panel (j64, g) = rows n = 0..127 of 128 bytes, out[((j64 * Hkv + g) * 128 + n) * 64 + k] = in[(j64 * 64 + k) * d + g * 128 + n].
-// A panel whose rows lie 2 d bytes apart (the plain transpose) sits in very few L2 slices, and with many CTAs asking
-// for the same panel its copy took thousands of cycles; 16 KiB of consecutive lines spread over all of them.
-// The first KT_HOT_PANELS panel rows (all that tiles of the narrow rank classes read) are stored KT_UINV_COPIES
-// times, blockIdx.z selecting the copy: when every CTA of the K-score kernel works on narrow tiles they all ask L2
-// for the same 8 .. 32 panels, and a panel's copy then took ~400 cycles per CTA asking for it (7 k cycles for a class-1
-// tile's panel); with each CTA on one of eight copies the requests spread over eight times as many lines.
+// One TMA box then reads 16 KiB of consecutive lines (a half panel for the CTA-pair kernel: rows 0..63 or 64..127).
 __global__ void uinv_panels_kernel(const unsigned short* __restrict__ in, unsigned short* __restrict__ out, int d) {
   __shared__ unsigned short t[64][129];
   const int j64 = blockIdx.x, g = blockIdx.y, tid = threadIdx.x;
-  if (blockIdx.z > 0) {
-    if (j64 >= KT_HOT_PANELS) return;
-    out += (size_t)d * d + (size_t)(blockIdx.z - 1) * KT_HOT_PANELS * d * 64;
-  }
   for (int i = tid; i < 64 * 128; i += blockDim.x) {
     const int k = i >> 7, n = i & 127;
     t[k][n] = in[(size_t)(j64 * 64 + k) * d + g * 128 + n];
@@ -538,7 +554,7 @@ __global__ void uinv_panels_kernel(const unsigned short* __restrict__ in, unsign
 
 cudaError_t launch_uinv_panels(const void* in, void* out, int d, cudaStream_t st) {
   ProfScope ps(TWKV_K_OTHER, st);
-  uinv_panels_kernel<<<dim3(d / 64, d / 128, KT_UINV_COPIES), 256, 0, st>>>(reinterpret_cast<const unsigned short*>(in),
+  uinv_panels_kernel<<<dim3(d / 64, d / 128), 256, 0, st>>>(reinterpret_cast<const unsigned short*>(in),
                                                            reinterpret_cast<unsigned short*>(out), d);
   count_launch();
   return cudaGetLastError();
@@ -552,28 +568,57 @@ cudaError_t launch_transpose16(const void* in, void* out, int n, cudaStream_t st
   return cudaGetLastError();
 }
 
-// bytes of the re-tiled copy of one layer's U_K^-1 and the panel rows (of 128 x 64) it holds
-size_t kscore_uinv_bytes(int d) { return (size_t)d * d * 2 + (size_t)(KT_UINV_COPIES - 1) * KT_HOT_PANELS * d * 64 * 2; }
-size_t kscore_uinv_panel_rows(int d) { return (size_t)(d / 64) * d + (size_t)(KT_UINV_COPIES - 1) * KT_HOT_PANELS * d; }
-
-size_t kscore_tc_smem_bytes(int nb) {
-  return (size_t)(KT_A_SLOTS + nb) * PANEL_BYTES + 2 * KT_Q_PANEL_BYTES + KT_ROPE_STAGE_BYTES + 8 * (KT_N_BARS + 2 * nb) +
+size_t kscore_tc_smem_bytes(int nb, size_t stage_bytes) {
+  return (size_t)KT_A_SLOTS * PANEL_BYTES + (size_t)nb * stage_bytes + 2 * KT_Q_PANEL_BYTES + KT_ROPE_STAGE_BYTES + 8 * (KT_N_BARS + 2 * nb) +
          2 * sizeof(int);
 }
+constexpr int KT_NB_SINGLE = 4, KT_NB_PAIR = 8;                // ring stages of U_K^-1 panels (16 KiB) / half panels (8 KiB)
 
-template <bool BF16>
+// CTA pairs of the pair kernel that can be resident at once on the current device (0: it cannot run).
+static int kscore_query_pairs(int sm_count) {
+  const size_t smem = kscore_tc_smem_bytes(KT_NB_PAIR, PANEL_BYTES / 2);
+  if (cudaFuncSetAttribute(kscore_tc_kernel<false, 4, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) { cudaGetLastError(); return 0; }
+  cudaLaunchConfig_t cfg = {};
+  cfg.blockDim = dim3(KT_THREADS);
+  cfg.dynamicSmemBytes = smem;
+  cfg.gridDim = dim3(sm_count & ~1);
+  cudaLaunchAttribute pair_attr;
+  pair_attr.id = cudaLaunchAttributeClusterDimension;
+  pair_attr.val.clusterDim.x = 2; pair_attr.val.clusterDim.y = 1; pair_attr.val.clusterDim.z = 1;
+  cfg.attrs = &pair_attr;
+  cfg.numAttrs = 1;
+  int n = 0;
+  if (cudaOccupancyMaxActiveClusters(&n, kscore_tc_kernel<false, 4, true>, &cfg) != cudaSuccess || n < 1) { cudaGetLastError(); n = 0; }
+  return n;
+}
+int kscore_max_pairs(int sm_count) {
+  static const int cached = kscore_query_pairs(sm_count);       // queried once per process (thread-safe initialisation)
+  return cached;
+}
+
+template <bool BF16, bool PAIR>
 static cudaError_t launch_kscore_tc_t(const DevView& v, int layer, const CUtensorMap& map_blocks, const CUtensorMap& map_uinvT,
-                                      const void* q, int sm_count, cudaStream_t st) {
-  int nb = 5;
-  while (nb > 2 && kscore_tc_smem_bytes(nb) > 227 * 1024) --nb;
-  const size_t smem = kscore_tc_smem_bytes(nb);
+                                      const void* q, int n_pieces, cudaStream_t st) {
+  const int nb = PAIR ? KT_NB_PAIR : KT_NB_SINGLE;
+  const size_t smem = kscore_tc_smem_bytes(nb, PAIR ? PANEL_BYTES / 2 : PANEL_BYTES);
   const unsigned short* qq = reinterpret_cast<const unsigned short*>(q);
+  cudaLaunchConfig_t cfg = {};
+  cfg.blockDim = dim3(KT_THREADS);
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = st;
+  cfg.gridDim = dim3(PAIR ? 2 * n_pieces : n_pieces);
+  cudaLaunchAttribute pair_attr;
+  pair_attr.id = cudaLaunchAttributeClusterDimension;
+  pair_attr.val.clusterDim.x = 2; pair_attr.val.clusterDim.y = 1; pair_attr.val.clusterDim.z = 1;
+  cfg.attrs = PAIR ? &pair_attr : nullptr;
+  cfg.numAttrs = PAIR ? 1 : 0;
   ProfScope ps(TWKV_K_KSCORE, st);
+  cudaError_t e = cudaSuccess;
 #define TWKV_KT(REP)                                                                                                  \
   {                                                                                                                   \
-    cudaError_t e = cudaFuncSetAttribute(kscore_tc_kernel<BF16, REP>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem); \
+    e = cudaFuncSetAttribute(kscore_tc_kernel<BF16, REP, PAIR>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem); \
     if (e != cudaSuccess) return e;                                                                                   \
-    kscore_tc_kernel<BF16, REP><<<sm_count, KT_THREADS, smem, st>>>(map_blocks, map_uinvT, v, layer, qq, nb);         \
+    e = cudaLaunchKernelEx(&cfg, kscore_tc_kernel<BF16, REP, PAIR>, map_blocks, map_uinvT, v, layer, qq, nb);        \
   }
   switch (v.rep) {
     case 1: TWKV_KT(1) break;
@@ -583,13 +628,17 @@ static cudaError_t launch_kscore_tc_t(const DevView& v, int layer, const CUtenso
   }
 #undef TWKV_KT
   count_launch();
-  return cudaGetLastError();
+  return e != cudaSuccess ? e : cudaGetLastError();
 }
 
+// `pairs`: run on CTA pairs (n_pieces pairs, map_uinvT with 64-row boxes) instead of single CTAs (128-row boxes).
 cudaError_t launch_kscore_tc(const DevView& v, int layer, const CUtensorMap& map_blocks, const CUtensorMap& map_uinvT,
-                             const void* q, int sm_count, cudaStream_t st) {
-  return v.dtype == TWKV_BF16 ? launch_kscore_tc_t<true>(v, layer, map_blocks, map_uinvT, q, sm_count, st)
-                              : launch_kscore_tc_t<false>(v, layer, map_blocks, map_uinvT, q, sm_count, st);
+                             const void* q, int n_pieces, bool pairs, cudaStream_t st) {
+  if (pairs)
+    return v.dtype == TWKV_BF16 ? launch_kscore_tc_t<true, true>(v, layer, map_blocks, map_uinvT, q, n_pieces, st)
+                                : launch_kscore_tc_t<false, true>(v, layer, map_blocks, map_uinvT, q, n_pieces, st);
+  return v.dtype == TWKV_BF16 ? launch_kscore_tc_t<true, false>(v, layer, map_blocks, map_uinvT, q, n_pieces, st)
+                              : launch_kscore_tc_t<false, false>(v, layer, map_blocks, map_uinvT, q, n_pieces, st);
 }
 
 }  // namespace twkv

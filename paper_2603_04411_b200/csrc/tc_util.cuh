@@ -109,6 +109,55 @@ __device__ __forceinline__ void mma_f16_ss(uint32_t d_tmem, uint64_t adesc, uint
 __device__ __forceinline__ uint32_t kmajor_sw128_desc_lo(uint32_t addr) { return ((addr >> 4) & 0x3fffu) | (1u << 16); }
 constexpr uint32_t KMAJOR_SW128_DESC_HI = 64u | (1u << 14) | (2u << 29);
 // Four MMAs over one 64-wide K panel (K steps of 16): D (+)= A[panel] * B[panel]^T, accumulate = 0 overwrites D first.
+// CG = 2: the CTA-pair form (M = 256 over the pair, each CTA supplies its own A rows and half of B's rows).
+#define TWKV_SS_PANEL_ASM(CGS)                                                                                          \
+  asm volatile(                                                                                                         \
+      "{\n\t.reg .pred p0, p1;\n\t.reg .b64 da, db;\n\t.reg .b32 al, bl;\n\t"                                          \
+      "setp.ne.b32 p0, %4, 0;\n\t"                                                                                      \
+      "setp.eq.b32 p1, %4, %4;\n\t"                                                                                     \
+      "mov.b64 da, {%1, %5};\n\tmov.b64 db, {%2, %5};\n\t"                                                             \
+      "tcgen05.mma.cta_group::" CGS ".kind::f16 [%0], da, db, %3, p0;\n\t"                                              \
+      "add.u32 al, %1, 2;\n\tadd.u32 bl, %2, 2;\n\tmov.b64 da, {al, %5};\n\tmov.b64 db, {bl, %5};\n\t"                \
+      "tcgen05.mma.cta_group::" CGS ".kind::f16 [%0], da, db, %3, p1;\n\t"                                              \
+      "add.u32 al, %1, 4;\n\tadd.u32 bl, %2, 4;\n\tmov.b64 da, {al, %5};\n\tmov.b64 db, {bl, %5};\n\t"                \
+      "tcgen05.mma.cta_group::" CGS ".kind::f16 [%0], da, db, %3, p1;\n\t"                                              \
+      "add.u32 al, %1, 6;\n\tadd.u32 bl, %2, 6;\n\tmov.b64 da, {al, %5};\n\tmov.b64 db, {bl, %5};\n\t"                \
+      "tcgen05.mma.cta_group::" CGS ".kind::f16 [%0], da, db, %3, p1;\n\t}"                                             \
+      ::"r"(d_tmem), "r"(a_lo), "r"(b_lo), "r"(idesc), "r"(accumulate), "r"(KMAJOR_SW128_DESC_HI) : "memory")
+template <int CG>
+__device__ __forceinline__ void mma_f16_ss_panel_cg(uint32_t d_tmem, uint32_t a_lo, uint32_t b_lo, uint32_t idesc, uint32_t accumulate) {
+  if constexpr (CG == 2) TWKV_SS_PANEL_ASM("2"); else TWKV_SS_PANEL_ASM("1");
+}
+#define TWKV_TS_K128_ASM(CGS)                                                                                           \
+  asm volatile(                                                                                                         \
+      "{\n\t.reg .pred p0, p1;\n\t.reg .b64 db;\n\t.reg .b32 bl, b2, ta;\n\t"                                          \
+      "setp.ne.b32 p0, %4, 0;\n\t"                                                                                      \
+      "setp.eq.b32 p1, %4, %4;\n\t"                                                                                     \
+      "add.u32 b2, %2, %6;\n\t"                                                                                         \
+      "mov.b64 db, {%2, %5};\n\t"                                                                                       \
+      "tcgen05.mma.cta_group::" CGS ".kind::f16 [%0], [%1], db, %3, p0;\n\t"                                            \
+      "add.u32 ta, %1, 8;\n\tadd.u32 bl, %2, 2;\n\tmov.b64 db, {bl, %5};\n\t"                                          \
+      "tcgen05.mma.cta_group::" CGS ".kind::f16 [%0], [ta], db, %3, p1;\n\t"                                            \
+      "add.u32 ta, %1, 16;\n\tadd.u32 bl, %2, 4;\n\tmov.b64 db, {bl, %5};\n\t"                                         \
+      "tcgen05.mma.cta_group::" CGS ".kind::f16 [%0], [ta], db, %3, p1;\n\t"                                            \
+      "add.u32 ta, %1, 24;\n\tadd.u32 bl, %2, 6;\n\tmov.b64 db, {bl, %5};\n\t"                                         \
+      "tcgen05.mma.cta_group::" CGS ".kind::f16 [%0], [ta], db, %3, p1;\n\t"                                            \
+      "add.u32 ta, %1, 32;\n\tmov.b64 db, {b2, %5};\n\t"                                                               \
+      "tcgen05.mma.cta_group::" CGS ".kind::f16 [%0], [ta], db, %3, p1;\n\t"                                            \
+      "add.u32 ta, %1, 40;\n\tadd.u32 bl, b2, 2;\n\tmov.b64 db, {bl, %5};\n\t"                                         \
+      "tcgen05.mma.cta_group::" CGS ".kind::f16 [%0], [ta], db, %3, p1;\n\t"                                            \
+      "add.u32 ta, %1, 48;\n\tadd.u32 bl, b2, 4;\n\tmov.b64 db, {bl, %5};\n\t"                                         \
+      "tcgen05.mma.cta_group::" CGS ".kind::f16 [%0], [ta], db, %3, p1;\n\t"                                            \
+      "add.u32 ta, %1, 56;\n\tadd.u32 bl, b2, 6;\n\tmov.b64 db, {bl, %5};\n\t"                                         \
+      "tcgen05.mma.cta_group::" CGS ".kind::f16 [%0], [ta], db, %3, p1;\n\t}"                                           \
+      ::"r"(d_tmem), "r"(a_tmem), "r"(b_lo), "r"(idesc), "r"(accumulate), "r"(KMAJOR_SW128_DESC_HI), "r"(panel_step) : "memory")
+// Eight MMAs over K = 128 with A in tensor memory (8 columns per K step) and B as two 64-wide K panels
+// `panel_step` (in 16-byte units) apart.
+template <int CG>
+__device__ __forceinline__ void mma_f16_ts_k128_cg(uint32_t d_tmem, uint32_t a_tmem, uint32_t b_lo, uint32_t panel_step, uint32_t idesc,
+                                                   uint32_t accumulate) {
+  if constexpr (CG == 2) TWKV_TS_K128_ASM("2"); else TWKV_TS_K128_ASM("1");
+}
 __device__ __forceinline__ void mma_f16_ss_panel(uint32_t d_tmem, uint32_t a_lo, uint32_t b_lo, uint32_t idesc, uint32_t accumulate) {
   asm volatile(
       "{\n\t.reg .pred p0, p1;\n\t.reg .b64 da, db;\n\t.reg .b32 al, bl;\n\t"
@@ -264,6 +313,10 @@ __device__ __forceinline__ void mma_f16_ss_pair(uint32_t d_tmem, uint64_t adesc,
       "setp.ne.b32 p, %4, 0;\n\t"
       "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t}"
       ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate) : "memory");
+}
+// arrives, once the pair's MMAs issued so far have retired, on one barrier (of the issuing CTA)
+__device__ __forceinline__ void mma_commit_pair(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
 }
 // arrives, once the pair's MMAs issued so far have retired, on the barrier at this offset in both CTAs
 __device__ __forceinline__ void mma_commit_pair_both(uint32_t bar) {

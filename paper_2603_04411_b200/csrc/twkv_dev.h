@@ -55,8 +55,9 @@ struct DevView {
   unsigned* seqmax;          // [S][Hq]  order-preserving encoding of the running max
   int* qslot;                // [S]   sequence id -> query index of the current decode call, -1
   int4* klist;               // [NT]  K tiles of the current decode call, widest class first: (tile, class | n_valid << 8, base block, query slot)
+  int4* kpairs;              // [NT + 64]  the same list as items of two tiles of one class (entries 2 i, 2 i + 1) for the CTA-pair kernel;
+                             //            a class with an odd number of tiles ends with a filler entry (.y bit 7 set)
   int* klist_count;          // [1]
-  unsigned* klist_cost;      // [NT]  exclusive prefix of the estimated cost of the listed tiles
   int* cta_start;            // [MAX_PLAN_CTAS + 1]  first list entry of every K-score CTA
   float* part_acc;           // [max_partials][Hq][d_kv]
   float* part_l;             // [max_partials][Hq]
@@ -131,7 +132,7 @@ cudaError_t launch_compress_pieces(const DevView& v, int layer, const void* K, c
                                   const int* positions, int n_tok, const unsigned short* levels, cudaStream_t st);
 struct TcMaps;   // tensor maps of the K-score kernel (api.cu)
 cudaError_t launch_decode(const DevView& v, int layer, const LayerParams& lp, const void* q, const int* seq_ids,
-                          int n_seq, void* out, int num_splits, int sm_count, const TcMaps* maps, cudaStream_t st);
+                          int n_seq, void* out, int num_splits, int sm_count, const TcMaps* maps, bool pairs, cudaStream_t st);
 struct GateMaps;   // tensor maps of the fused gate kernel (api.cu)
 cudaError_t launch_gate_ranks_tc(const DevView& v, const GateMaps& maps, const LayerParams& lp, int n_tok, unsigned short* levels,
                                  int sm_count, bool pairs, cudaStream_t st);
@@ -144,8 +145,7 @@ cudaError_t launch_project_tc(const ProjectMaps& maps, int n_tok, int d, int bf1
 int project_tc_max_pairs(int sm_count);
 cudaError_t launch_transpose16(const void* in, void* out, int n, cudaStream_t st);
 cudaError_t launch_uinv_panels(const void* in, void* out, int d, cudaStream_t st);
-size_t kscore_uinv_bytes(int d);
-size_t kscore_uinv_panel_rows(int d);
+int kscore_max_pairs(int sm_count);
 cudaError_t launch_gate_logits(const DevView& v, const LayerParams& lp, const void* K, const void* V, int n_tok,
                                float* logits, cudaStream_t st);
 cudaError_t launch_stats(const DevView& v, int layer, unsigned long long* out_dev, cudaStream_t st);
