@@ -23,11 +23,11 @@ namespace twkv {
 // is rewritten as items of two tiles of one class.  The list is then cut into n_cta contiguous pieces of
 // about equal estimated cost, so a CTA (pair) of the K-score kernel mostly stays inside one (class, sequence) run.
 __device__ __forceinline__ unsigned ktile_cost(int cls) {
-  // cycles per tile of the K-score kernel by rank class, measured on one-class workloads (8 KV heads): a fixed part
-  // (rotation factors, the per-slab epilogue and score products) plus a per-panel part; classes above 8 run as two
-  // passes.  Only the ratios matter.
-  constexpr unsigned kCost[TWKV_MAX_CLASSES] = {17100u, 17100u, 17900u, 19700u, 22700u, 25700u, 28600u, 31600u,
-                                                44000u, 46000u, 49000u, 52000u, 55000u, 58000u, 61000u, 63300u};
+  // cycles per tile of the K-score kernel by rank class, measured inside the kernel on the benchmark's mix of classes
+  // (8 KV heads, CTA pairs): a fixed part (rotation factors, the per-slab epilogue and score products) plus a per-panel
+  // part; classes above 8 run as two passes.  Only the ratios matter.
+  constexpr unsigned kCost[TWKV_MAX_CLASSES] = {16200u, 17900u, 19100u, 20300u, 22100u, 24200u, 26100u, 27600u,
+                                                42900u, 42900u, 43400u, 45300u, 47300u, 49500u, 51800u, 55300u};
   return kCost[min(max(cls, 1), TWKV_MAX_CLASSES) - 1];
 }
 
