@@ -15,6 +15,8 @@ patterns, exactly as the GPU receives them) are widened with `widen16`.
   reconstruct(xt, r, Uinv)         Eq. 3   xbar = x^[I] Uinv[I, :]
   rope(k, pos, n_heads, d_h, base) RoPE on reconstructed keys (after Eq. 3)
   decode_attn(...)                 Eq. 3 + reshape + RoPE + softmax attention, one sequence
+  prefill_attn(...)                the same for many causal queries of one sequence (a prompt chunk)
+  soft_gate(xt, z)                 Eq. 6, Eq. 7, Eq. 9's R: soft mask m, x~ (.) m, mean of m per token
   retain_rate(r, d)                Eq. 4   mean of r / d_kv
 """
 import ctypes
@@ -190,6 +192,36 @@ def decode_attn(xk, xv, rk, rv, pos, Uinv_k, Uinv_v, q, n_kv_heads: int,
     if rc != 0:
         raise MemoryError("oracle_decode_attn")
     return out
+
+
+def prefill_attn(xk, xv, rk, rv, pos, Uinv_k, Uinv_v, q, q_pos, n_kv_heads: int,
+                 rope_base: float, sm_scale: float) -> np.ndarray:
+    """Attention of a chunk of causal queries over one sequence's cached tokens.
+
+    The paper's long-context evaluation (Sec. 4.2) prefills prompts through the same compressed cache: every query
+    sees the reconstructed keys and values of Eq. 3 (keys rotated after reconstruction) of the tokens at or before
+    its own position.  This is that definition written out: query i attends to the cached tokens t with
+    pos[t] <= q_pos[i], each such set handed to decode_attn unchanged; a query that sees no token gets zeros.
+    xk/xv [T, d_kv], q [n_q, Hq, d_h], q_pos [n_q] -> out [n_q, Hq, d_h]."""
+    q = np.asarray(q, dtype=np.float64)
+    pos = np.asarray(pos)
+    out = np.zeros(q.shape, dtype=np.float64)
+    for i in range(q.shape[0]):
+        vis = np.nonzero(pos <= q_pos[i])[0]
+        if len(vis):
+            out[i] = decode_attn(np.asarray(xk)[vis], np.asarray(xv)[vis], np.asarray(rk)[vis], np.asarray(rv)[vis], pos[vis],
+                                 Uinv_k, Uinv_v, q[i], n_kv_heads, rope_base, sm_scale)
+    return out
+
+
+def soft_gate(xt, z):
+    """Soft gating of Eq. 6 and Eq. 7, and the per-token Retain Rate of the soft mask that Eq. 9 penalises.
+
+    m = Flip(cumsum(softmax(z))) (Eq. 6, the literal index reversal m_i = c_{d+1-i}); x^ = x~ (.) m (Eq. 7);
+    R = (1/d) sum_i m_i, Eq. 4 applied to the soft mask.  xt, z [n, d] -> (m [n, d], x^ [n, d], R [n])."""
+    xt = np.asarray(xt, dtype=np.float64)
+    _, _, m = gate_rank(z, 0.5, want_soft=True)
+    return m, xt * m, m.mean(axis=1)
 
 
 def retain_rate(r, d: int) -> float:

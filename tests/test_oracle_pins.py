@@ -484,3 +484,127 @@ def test_image_capacity_refusal_leaves_state_unchanged():
     ranks = np.full((200, 2), 128, np.int32)            # class 2: 2 tiles x 2 blocks x 2 sides = 8 blocks > 3
     assert not img.append(0, x, x, seq, pos, ranks)
     assert img.next_block == 0 and img.n_tiles.sum() == 0 and img.fill.sum() == 0
+
+
+# ---------------------------------------------------------------------------------------------
+# chunked-prefill attention: causal queries over the compressed cache
+def test_prefill_one_query_seeing_everything_is_decode():
+    rng = np.random.default_rng(21)
+    Hkv, Hq, dh, T = 2, 4, 8, 19
+    d = Hkv * dh
+    Uik, Uiv = rng.normal(size=(d, d)), rng.normal(size=(d, d))
+    xk, xv = rng.normal(size=(T, d)), rng.normal(size=(T, d))
+    rk = rng.integers(1, d + 1, T).astype(np.int32)
+    rv = rng.integers(1, d + 1, T).astype(np.int32)
+    pos = rng.permutation(50)[:T].astype(np.int32)
+    q = rng.normal(size=(1, Hq, dh))
+    got = oracle.prefill_attn(xk, xv, rk, rv, pos, Uik, Uiv, q, np.array([int(pos.max())]), Hkv, 1000.0, 0.3)
+    want = oracle.decode_attn(xk, xv, rk, rv, pos, Uik, Uiv, q[0], Hkv, 1000.0, 0.3)
+    np.testing.assert_allclose(got[0], want, rtol=0, atol=1e-13)
+
+
+def test_prefill_bruteforce_tiny_causal():
+    # literal Python sums with the causal mask written out, T = 7, mixed ranks, non-orthogonal U
+    rng = np.random.default_rng(22)
+    Hkv, Hq, dh, T = 2, 4, 4, 7
+    d = Hkv * dh
+    Uik, Uiv = rng.normal(size=(d, d)), rng.normal(size=(d, d))
+    xk, xv = rng.normal(size=(T, d)), rng.normal(size=(T, d))
+    rk = rng.integers(1, d + 1, T).astype(np.int32)
+    rv = rng.integers(1, d + 1, T).astype(np.int32)
+    pos = np.array([0, 2, 3, 5, 8, 9, 12], dtype=np.int32)
+    q_pos = np.array([3, 0, 12, 7])
+    q = rng.normal(size=(len(q_pos), Hq, dh))
+    base, scale = 50.0, 0.7
+    got = oracle.prefill_attn(xk, xv, rk, rv, pos, Uik, Uiv, q, q_pos, Hkv, base, scale)
+    for i, qp in enumerate(q_pos):
+        for h in range(Hq):
+            g = h // (Hq // Hkv)
+            num, den, smax, sc, vbars = [0.0] * dh, 0.0, -1e300, [], []
+            for t in range(T):
+                if pos[t] > qp:
+                    continue                                     # causal: the query does not see later tokens
+                kbar = [sum(xk[t][j] * Uik[j][g * dh + n] for j in range(rk[t])) for n in range(dh)]
+                vbars.append([sum(xv[t][j] * Uiv[j][g * dh + n] for j in range(rv[t])) for n in range(dh)])
+                rot = list(kbar)
+                for a in range(dh // 2):
+                    ang = pos[t] * base ** (-2.0 * a / dh)
+                    rot[a] = kbar[a] * math.cos(ang) - kbar[a + dh // 2] * math.sin(ang)
+                    rot[a + dh // 2] = kbar[a + dh // 2] * math.cos(ang) + kbar[a] * math.sin(ang)
+                sc.append(scale * sum(q[i][h][n] * rot[n] for n in range(dh)))
+            smax = max(sc)
+            w = [math.exp(x - smax) for x in sc]
+            den = sum(w)
+            for n in range(dh):
+                num[n] = sum(w[k] * vbars[k][n] for k in range(len(w))) / den
+            np.testing.assert_allclose(got[i][h], num, rtol=0, atol=1e-12)
+
+
+def test_prefill_full_rank_equals_exact_causal_attention_and_ignores_the_future():
+    rng = np.random.default_rng(23)
+    Hkv, Hq, dh, T = 2, 4, 16, 33
+    d = Hkv * dh
+    Uk, Uv = _rand_orth(rng, d), _rand_orth(rng, d)
+    xk, xv = rng.normal(size=(T, d)), rng.normal(size=(T, d))
+    pos = np.arange(T, dtype=np.int32)
+    full = np.full(T, d, np.int32)
+    q_pos = np.array([0, 5, 17, 32])
+    q = rng.normal(size=(len(q_pos), Hq, dh))
+    got = oracle.prefill_attn(xk @ Uk, xv @ Uv, full, full, pos, Uk.T, Uv.T, q, q_pos, Hkv, 10000.0, dh ** -0.5)
+    for i, qp in enumerate(q_pos):
+        want = _exact_attention_from_raw(xk[:qp + 1], xv[:qp + 1], pos[:qp + 1], q[i], Hkv, 10000.0, dh ** -0.5)
+        np.testing.assert_allclose(got[i], want, atol=1e-11)
+    # tokens after a query's position do not matter: replace them and compare
+    xk2, xv2 = xk.copy(), xv.copy()
+    xk2[18:] = rng.normal(size=(T - 18, d)); xv2[18:] = rng.normal(size=(T - 18, d))
+    got2 = oracle.prefill_attn(xk2 @ Uk, xv2 @ Uv, full, full, pos, Uk.T, Uv.T, q, q_pos, Hkv, 10000.0, dh ** -0.5)
+    np.testing.assert_array_equal(got[:3], got2[:3])
+    # a query before every cached token sees nothing
+    none = oracle.prefill_attn(xk @ Uk, xv @ Uv, full, full, pos + 5, Uk.T, Uv.T, q[:1], np.array([2]), Hkv, 10000.0, dh ** -0.5)
+    assert not none.any()
+
+
+# ---------------------------------------------------------------------------------------------
+# soft gating (Eq. 6, Eq. 7, the soft Retain Rate of Eq. 9)
+def test_soft_gate_closed_forms():
+    d = 16
+    # uniform logits: p_j = 1/d, c_n = n/d, m_i = c_{d+1-i} = (d+1-i)/d, mean = (d+1)/(2d)
+    z = np.zeros((1, d))
+    x = np.arange(1.0, d + 1)[None, :]
+    m, xh, R = oracle.soft_gate(x, z)
+    np.testing.assert_allclose(m[0], (d - np.arange(d)) / d, atol=1e-15)
+    np.testing.assert_allclose(xh[0], x[0] * (d - np.arange(d)) / d, atol=1e-13)
+    assert abs(R[0] - (d + 1) / (2 * d)) < 1e-15
+    # all mass on truncation index k (1-based): c_n = [n >= k], m_i = [i <= d+1-k]: keeps d+1-k leading components
+    for k in (1, 5, 16):
+        z = np.full((1, d), -800.0); z[0, k - 1] = 0.0
+        m, xh, R = oracle.soft_gate(x, z)
+        want = (np.arange(1, d + 1) <= d + 1 - k).astype(float)
+        np.testing.assert_array_equal(m[0], want)
+        np.testing.assert_array_equal(xh[0], x[0] * want)
+        assert R[0] == (d + 1 - k) / d
+    # two-point mass: p_a = 0.25, p_b = 0.75 (a < b): m = 1 up to d+1-b, 0.25 up to d+1-a, 0 after
+    a, b = 3, 11
+    z = np.full((1, d), -800.0); z[0, a - 1] = math.log(0.25); z[0, b - 1] = math.log(0.75)
+    m, _, R = oracle.soft_gate(x, z)
+    idx = np.arange(1, d + 1)
+    want = np.where(idx <= d + 1 - b, 1.0, np.where(idx <= d + 1 - a, 0.25, 0.0))
+    np.testing.assert_allclose(m[0], want, atol=1e-15)
+    assert abs(R[0] - want.mean()) < 1e-15
+
+
+def test_soft_gate_invariants_and_link_to_hard_mask():
+    rng = np.random.default_rng(31)
+    n, d = 40, 64
+    z = rng.normal(size=(n, d)) * 3
+    x = rng.normal(size=(n, d))
+    m, xh, R = oracle.soft_gate(x, z)
+    assert np.all(np.diff(m, axis=1) <= 1e-15) and np.allclose(m[:, 0], 1.0) and np.all(m >= 0)
+    np.testing.assert_allclose(xh, x * m, atol=0)
+    # the hard mask of Eq. 8 is the soft mask thresholded: r = #{i : m_i > tau}
+    for tau in (0.05, 0.1, 0.5):
+        r, _ = oracle.gate_rank(z, tau)
+        np.testing.assert_array_equal(r, (m > tau).sum(axis=1))
+    # adding a constant to a row's logits changes nothing
+    m2, _, _ = oracle.soft_gate(x, z + 7.0)
+    np.testing.assert_allclose(m2, m, atol=1e-14)
