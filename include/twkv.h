@@ -74,6 +74,7 @@ typedef enum {
 #define TWKV_BLOCK_BYTES 16384      /* one panel: 128 rows x 64 elements x 2 bytes                   */
 #define TWKV_PIECE_TOKENS 131072    /* a compress call is processed in pieces of this many tokens    */
 #define TWKV_MAX_CLASSES 16
+#define TWKV_PREFILL_MAX_QUERIES 16384   /* queries per twkv_prefill_attn call                          */
 
 typedef struct {
   int32_t n_layers;
@@ -167,12 +168,46 @@ twkv_status twkv_compress(twkv_cache* cache, int layer, const void* K, const voi
 twkv_status twkv_decode_attn(twkv_cache* cache, int layer, const void* q, const int32_t* seq_ids,
                              int n_seq, void* out, int num_splits, void* stream);
 
+/*
+ * Chunked-prefill attention: many causal queries per sequence over the same mixed-rank cache (the paper's
+ * long-context evaluation, Sec. 4.2, prefills prompts through the compressed cache; keys and values are the
+ * reconstructions of Eq. 3, keys rotated after reconstruction).  Query i attends to the tokens cached for
+ * sequence q_seq[i] in `layer` whose position is <= q_pos[i]; the usual order is twkv_compress of a prompt chunk,
+ * then this call with the chunk's queries, so that a query also sees its own token.  A query that sees no token
+ * gets zeros.
+ *   q, out   [n_q x n_q_heads x 128] dtype / out_dtype, device; q already rotated at its own position
+ *   q_seq    [n_q] int32, HOST memory: sequence id of every query (any order, repeats allowed)
+ *   q_pos    [n_q] int32, HOST memory: RoPE position of every query (>= 0)
+ *   n_q      at most TWKV_PREFILL_MAX_QUERIES
+ * The queries are served in waves of at most one query per sequence (the k-th query of every sequence together);
+ * each wave is one pass of the decode kernels with the causal limit applied to the scores.  The host arrays are
+ * read before the call returns.  Errors as for twkv_decode_attn; an id or position out of range returns
+ * TWKV_ERR_INVALID_ARG before anything is launched.
+ */
+twkv_status twkv_prefill_attn(twkv_cache* cache, int layer, const void* q, const int32_t* q_seq /*host*/,
+                              const int32_t* q_pos /*host*/, int n_q, void* out, int num_splits, void* stream);
+
 /* Synchronises `stream`, returns the sticky device status and clears it. */
 twkv_status twkv_cache_status(twkv_cache* cache, void* stream);
 /* Synchronises `stream`; layer = -1 sums all layers.  `out` is host memory. */
 twkv_status twkv_cache_stats(twkv_cache* cache, int layer, void* stream, twkv_stats* out /*host*/);
 /* Where the tables live inside the pool (host call, no device work). */
 twkv_status twkv_cache_layout(const twkv_cache* cache, twkv_layout* out /*host*/);
+/*
+ * Soft gating, the differentiable form of the gate the paper trains with, as an inference-time diagnostic:
+ *   m = Flip(cumsum(softmax(x~ W + b)))     Eq. 5, Eq. 6 (Flip = index reversal, m_1 = 1, m non-increasing)
+ *   x^ = x~ (.) m                           Eq. 7
+ *   R = (1/d_kv) sum_i m_i                  the Retain Rate of the soft mask, the R that Eq. 9 penalises
+ * for the K side and the V side of n_tok tokens, with the layer's gate parameters (W, b as in TWKV_GATE_COMPUTE).
+ * The hard mask of Eq. 8 is this m thresholded at tau.  Nothing is stored in the cache.
+ *   K, V          [n_tok x d_kv] spectral states, dtype, device
+ *   m_k, m_v      [n_tok x d_kv] fp32 soft masks (each may be NULL)
+ *   xh_k, xh_v    [n_tok x d_kv] fp32 gated states (each may be NULL)
+ *   retain        [n_tok x 2] fp32 (R_K, R_V) per token (may be NULL)
+ */
+twkv_status twkv_gate_soft(twkv_cache* cache, int layer, const void* K, const void* V, int n_tok, float* m_k, float* m_v,
+                           float* xh_k, float* xh_v, float* retain, void* stream);
+
 /*
  * Gate ranks without any caller-provided scratch (the paper has no counterpart; this is a
  * convenience of the library).  Computes, for n_tok tokens, the (r_K, r_V) of Eq. 5, 6, 8 as twkv_compress

@@ -18,11 +18,12 @@ TWKV_ERR_CUDA, TWKV_ERR_DEVICE_CHECK, TWKV_ERR_TIMEOUT = 4, 5, 6
 TWKV_F16, TWKV_BF16, TWKV_F32 = 0, 1, 2
 TWKV_GATE_FORCED, TWKV_GATE_LOGITS, TWKV_GATE_COMPUTE = 0, 1, 2
 TILE_TOKENS, PANEL_ELEMS, BLOCK_BYTES, PIECE_TOKENS, MAX_CLASSES = 128, 64, 16384, 131072, 16
+PREFILL_MAX_QUERIES = 16384
 
 EXPORTS = ["twkv_cache_required_bytes", "twkv_cache_create", "twkv_cache_destroy", "twkv_cache_reset",
-           "twkv_cache_set_layer_params", "twkv_compress", "twkv_decode_attn", "twkv_cache_status",
+           "twkv_cache_set_layer_params", "twkv_compress", "twkv_decode_attn", "twkv_prefill_attn", "twkv_cache_status",
            "twkv_cache_stats", "twkv_cache_layout", "twkv_launch_count", "twkv_status_string",
-           "twkv_profile_enable", "twkv_profile_read", "twkv_gate_ranks_static",
+           "twkv_profile_enable", "twkv_profile_read", "twkv_gate_ranks_static", "twkv_gate_soft",
            "twkv_projector_required_bytes", "twkv_projector_create", "twkv_projector_destroy", "twkv_project",
            "twkv_projector_status"]
 STATIC_GATE_MAX_ROWS = 1024
@@ -69,6 +70,9 @@ def _load():
     L.twkv_cache_set_layer_params.argtypes = [vp, i32, ctypes.POINTER(twkv_layer_params)]
     L.twkv_compress.argtypes = [vp, i32, vp, vp, vp, vp, i32, vp, vp, i32, vp]
     L.twkv_decode_attn.argtypes = [vp, i32, vp, vp, i32, vp, i32, vp]
+    L.twkv_prefill_attn.argtypes = [vp, i32, vp, ctypes.POINTER(ctypes.c_int32), ctypes.POINTER(ctypes.c_int32), i32, vp, i32, vp]
+    L.twkv_gate_soft.argtypes = [vp, i32, vp, vp, i32, vp, vp, vp, vp, vp, vp]
+    L.twkv_gate_soft.restype = i32
     L.twkv_cache_status.argtypes = [vp, vp]
     L.twkv_cache_stats.argtypes = [vp, i32, vp, ctypes.POINTER(twkv_stats)]
     L.twkv_cache_layout.argtypes = [vp, ctypes.POINTER(twkv_layout)]
@@ -91,7 +95,7 @@ def _load():
     L.twkv_status_string.argtypes = [i32]
     L.twkv_status_string.restype = ctypes.c_char_p
     for name in ["twkv_cache_create", "twkv_cache_destroy", "twkv_cache_reset", "twkv_cache_set_layer_params",
-                 "twkv_compress", "twkv_decode_attn", "twkv_cache_status", "twkv_cache_stats", "twkv_cache_layout",
+                 "twkv_compress", "twkv_decode_attn", "twkv_prefill_attn", "twkv_cache_status", "twkv_cache_stats", "twkv_cache_layout",
                  "twkv_profile_enable", "twkv_profile_read"]:
         getattr(L, name).restype = i32
     return L
@@ -168,6 +172,25 @@ def twkv_compress(cache, layer, K, V, seq_ids, positions, scores, levels, mode, 
 def twkv_decode_attn(cache, layer, q, seq_ids, out, num_splits=0, stream=None):
     _check(lib.twkv_decode_attn(cache, layer, _ptr(q), _ptr(seq_ids), seq_ids.numel(), _ptr(out), num_splits,
                                 _stream(stream)), "twkv_decode_attn")
+
+
+def twkv_prefill_attn(cache, layer, q, q_seq, q_pos, out, num_splits=0, stream=None):
+    """Causal attention of a chunk of queries over the cache.  q / out: [n_q, Hq, 128] CUDA tensors; q_seq / q_pos:
+    the queries' sequence ids and positions as HOST integers (lists, numpy arrays or CPU tensors)."""
+    seq = [int(x) for x in q_seq]
+    pos = [int(x) for x in q_pos]
+    n = len(seq)
+    assert len(pos) == n and q.shape[0] == n
+    arr = ctypes.c_int32 * max(n, 1)
+    _check(lib.twkv_prefill_attn(cache, layer, _ptr(q), arr(*seq), arr(*pos), n, _ptr(out), num_splits, _stream(stream)),
+           "twkv_prefill_attn")
+
+
+def twkv_gate_soft(cache, layer, K, V, m_k=None, m_v=None, xh_k=None, xh_v=None, retain=None, stream=None, n_tok=None):
+    """Soft mask m (Eq. 6), gated states x~ (.) m (Eq. 7) and the soft mask's Retain Rate per token, fp32 outputs."""
+    n = K.shape[0] if n_tok is None else n_tok
+    _check(lib.twkv_gate_soft(cache, layer, _ptr(K), _ptr(V), n, _ptr(m_k), _ptr(m_v), _ptr(xh_k), _ptr(xh_v), _ptr(retain),
+                              _stream(stream)), "twkv_gate_soft")
 
 
 def twkv_cache_status(cache, stream=None) -> int:

@@ -79,7 +79,7 @@ constexpr int GATE_TC_MIN_TOKENS = 1024;   // calls at least this large run the 
 struct Offsets {
   size_t status, pflags, rope_lo, rope_hi, n_tiles, tile_desc, tile_aux, tile_rank, fill, key_last, kclass_count,
       kclass_tiles, seq_vcount, seq_vtiles, seq_tokens, rank_sums, hist, key_cnt, key_old_fill, key_first_id,
-      key_first_base, key_old_last, scores, seqmax, qslot, klist, kpairs, klist_count, cta_start, part_acc, part_l, gate_scratch, gate_fix, stats_buf, tables_end, prep_uinvT, prep_wT,
+      key_first_base, key_old_last, scores, seqmax, qslot, klist, kpairs, klist_count, cta_start, wave_buf, part_acc, part_l, gate_scratch, gate_fix, stats_buf, tables_end, prep_uinvT, prep_wT,
       blocks, end_fixed;
 };
 
@@ -153,6 +153,7 @@ static Offsets layout_of(const twkv_config* c, const Dims& d) {
   o.klist_count = L.alloc(sizeof(int));
   o.kpairs = L.alloc((NT + 64) * sizeof(int4));
   o.cta_start = L.alloc((MAX_PLAN_CTAS + 1) * sizeof(int));
+  o.wave_buf = L.alloc((size_t)3 * TWKV_PREFILL_MAX_QUERIES * sizeof(int));
   o.part_acc = L.alloc((size_t)d.max_partials * Hq * d.d_kv * sizeof(float));
   o.part_l = L.alloc((size_t)d.max_partials * Hq * sizeof(float));
   {
@@ -248,6 +249,8 @@ static void fill_view(twkv_cache* c) {
   v.part_acc = (float*)(p + o.part_acc); v.part_l = (float*)(p + o.part_l);
   v.gate_scratch = (float*)(p + o.gate_scratch);
   v.gate_fix = (int4*)(p + o.gate_fix);
+  v.wave_buf = (int*)(p + o.wave_buf);
+  v.qmap = nullptr; v.qpos = nullptr;
 }
 
 twkv_status twkv_cache_reset(twkv_cache* c, void* stream) {
@@ -411,12 +414,11 @@ twkv_status twkv_compress(twkv_cache* c, int layer, const void* K, const void* V
   return TWKV_OK;
 }
 
-twkv_status twkv_decode_attn(twkv_cache* c, int layer, const void* q, const int32_t* seq_ids, int n_seq, void* out,
-                             int num_splits, void* stream) {
-  if (!c || layer < 0 || layer >= c->cfg.n_layers || n_seq < 0 || num_splits < 0) return TWKV_ERR_INVALID_ARG;
-  if (n_seq == 0) return TWKV_OK;
-  if (!q || !seq_ids || !out || n_seq > c->cfg.max_seqs) return TWKV_ERR_INVALID_ARG;
-  if (((uintptr_t)q | (uintptr_t)out) % 16) return TWKV_ERR_INVALID_ARG;
+// One pass of the decode kernels: one query per listed sequence.  qmap / qpos (device, per query slot) are set for a
+// prefill wave: the row of q / out a slot stands for, and the last position it may attend to.
+static twkv_status decode_pass(twkv_cache* c, int layer, const void* q, const int32_t* seq_ids, int n_seq, void* out,
+                               int num_splits, const int* qmap, const int* qpos, cudaStream_t stream) {
+  if (n_seq > c->cfg.max_seqs) return TWKV_ERR_INVALID_ARG;
   if (!c->params[layer].Uinv_k || !c->params[layer].Uinv_v) return TWKV_ERR_INVALID_ARG;
   const int head_groups = (c->cfg.n_q_heads + 31) / 32;
   if (num_splits == 0) {
@@ -440,8 +442,58 @@ twkv_status twkv_decode_attn(twkv_cache* c, int layer, const void* q, const int3
   TcMaps maps;
   maps.blocks = c->map_blocks;
   maps.uinvT_k = c->map_uinvT[layer];
-  if (launch_decode(c->view, layer, c->params[layer], q, seq_ids, n_seq, out, num_splits, c->sm_count, &maps, c->kscore_pairs,
+  DevView v = c->view;
+  v.qmap = qmap; v.qpos = qpos;
+  if (launch_decode(v, layer, c->params[layer], q, seq_ids, n_seq, out, num_splits, c->sm_count, &maps, c->kscore_pairs,
                     (cudaStream_t)stream) != cudaSuccess) return TWKV_ERR_CUDA;
+  return TWKV_OK;
+}
+
+twkv_status twkv_decode_attn(twkv_cache* c, int layer, const void* q, const int32_t* seq_ids, int n_seq, void* out,
+                             int num_splits, void* stream) {
+  if (!c || layer < 0 || layer >= c->cfg.n_layers || n_seq < 0 || num_splits < 0) return TWKV_ERR_INVALID_ARG;
+  if (n_seq == 0) return TWKV_OK;
+  if (!q || !seq_ids || !out || n_seq > c->cfg.max_seqs) return TWKV_ERR_INVALID_ARG;
+  if (((uintptr_t)q | (uintptr_t)out) % 16) return TWKV_ERR_INVALID_ARG;
+  return decode_pass(c, layer, q, seq_ids, n_seq, out, num_splits, nullptr, nullptr, (cudaStream_t)stream);
+}
+
+twkv_status twkv_prefill_attn(twkv_cache* c, int layer, const void* q, const int32_t* q_seq, const int32_t* q_pos, int n_q,
+                              void* out, int num_splits, void* stream) {
+  if (!c || layer < 0 || layer >= c->cfg.n_layers || n_q < 0 || num_splits < 0) return TWKV_ERR_INVALID_ARG;
+  if (n_q == 0) return TWKV_OK;
+  if (!q || !q_seq || !q_pos || !out || n_q > TWKV_PREFILL_MAX_QUERIES) return TWKV_ERR_INVALID_ARG;
+  if (((uintptr_t)q | (uintptr_t)out) % 16) return TWKV_ERR_INVALID_ARG;
+  const int S = c->cfg.max_seqs;
+  // wave k = the k-th query of every sequence, in order of appearance; inside a wave the sequences are distinct
+  std::vector<int> seen(S, 0), wave_of(n_q);
+  int n_waves = 0;
+  for (int i = 0; i < n_q; ++i) {
+    if (q_seq[i] < 0 || q_seq[i] >= S || q_pos[i] < 0) return TWKV_ERR_INVALID_ARG;
+    wave_of[i] = seen[q_seq[i]]++;
+    if (wave_of[i] + 1 > n_waves) n_waves = wave_of[i] + 1;
+  }
+  std::vector<int> wave_start(n_waves + 1, 0), fill(n_waves, 0);
+  for (int i = 0; i < n_q; ++i) ++wave_start[wave_of[i] + 1];
+  for (int w = 0; w < n_waves; ++w) wave_start[w + 1] += wave_start[w];
+  std::vector<int> host(3 * (size_t)TWKV_PREFILL_MAX_QUERIES);
+  for (int i = 0; i < n_q; ++i) {
+    const int at = wave_start[wave_of[i]] + fill[wave_of[i]]++;
+    host[at] = q_seq[i];
+    host[TWKV_PREFILL_MAX_QUERIES + at] = i;
+    host[2 * TWKV_PREFILL_MAX_QUERIES + at] = q_pos[i];
+  }
+  DeviceGuard g(c->device);
+  if (!g.ok) return TWKV_ERR_CUDA;
+  cudaStream_t st = (cudaStream_t)stream;
+  // the copy is staged from pageable memory before the call returns, so `host` may go out of scope afterwards
+  if (cudaMemcpyAsync(c->view.wave_buf, host.data(), host.size() * sizeof(int), cudaMemcpyHostToDevice, st) != cudaSuccess) return TWKV_ERR_CUDA;
+  for (int w = 0; w < n_waves; ++w) {
+    const int off = wave_start[w], n = wave_start[w + 1] - off;
+    twkv_status s = decode_pass(c, layer, q, c->view.wave_buf + off, n, out, num_splits, c->view.wave_buf + TWKV_PREFILL_MAX_QUERIES + off,
+                                c->view.wave_buf + 2 * TWKV_PREFILL_MAX_QUERIES + off, st);
+    if (s != TWKV_OK) return s;
+  }
   return TWKV_OK;
 }
 
@@ -458,6 +510,30 @@ twkv_status twkv_cache_status(twkv_cache* c, void* stream) {
     if (cudaStreamSynchronize(st) != cudaSuccess) return TWKV_ERR_CUDA;
   }
   return (twkv_status)code;
+}
+
+twkv_status twkv_gate_soft(twkv_cache* c, int layer, const void* K, const void* V, int n_tok, float* m_k, float* m_v, float* xh_k,
+                           float* xh_v, float* retain, void* stream) {
+  if (!c || layer < 0 || layer >= c->cfg.n_layers || n_tok < 0) return TWKV_ERR_INVALID_ARG;
+  if (n_tok == 0) return TWKV_OK;
+  if (!K || !V || ((uintptr_t)K | (uintptr_t)V) % 16) return TWKV_ERR_INVALID_ARG;
+  if (!c->params[layer].W_k || !c->params[layer].W_v) return TWKV_ERR_INVALID_ARG;
+  DeviceGuard g(c->device);
+  if (!g.ok) return TWKV_ERR_CUDA;
+  ProfBind pb(&c->prof);
+  cudaStream_t st = (cudaStream_t)stream;
+  const DevView& v = c->view;
+  const size_t row = (size_t)v.d_kv * 2, d = (size_t)v.d_kv;
+  for (int lo = 0; lo < n_tok; lo += GATE_PIECE) {               // the logits of a piece live in the gate scratch
+    const int n = n_tok - lo < GATE_PIECE ? n_tok - lo : GATE_PIECE;
+    const unsigned char* kp = (const unsigned char*)K + lo * row;
+    const unsigned char* vp = (const unsigned char*)V + lo * row;
+    if (launch_gate_logits(v, c->params[layer], kp, vp, n, v.gate_scratch, st) != cudaSuccess) return TWKV_ERR_CUDA;
+    if (launch_gate_soft(v, v.gate_scratch, kp, vp, m_k ? m_k + lo * d : nullptr, m_v ? m_v + lo * d : nullptr,
+                         xh_k ? xh_k + lo * d : nullptr, xh_v ? xh_v + lo * d : nullptr, retain ? retain + 2 * (size_t)lo : nullptr, n,
+                         st) != cudaSuccess) return TWKV_ERR_CUDA;
+  }
+  return TWKV_OK;
 }
 
 twkv_status twkv_cache_stats(twkv_cache* c, int layer, void* stream, twkv_stats* out) {

@@ -193,7 +193,11 @@ vacc_kernel(DevView v, int layer, const int* __restrict__ seq_ids, int n_splits)
   const int* aux = v.aux(layer, 1);
 
   for (int i = tid; i < P_BYTES / 4; i += NT) reinterpret_cast<unsigned*>(sP)[i] = 0u;
-  if (tid < 32) sM[tid] = tid < nh ? dec_ordered(v.seqmax[qs * Hq + h0 + tid]) : 0.f;
+  if (tid < 32) {
+    // a query that sees no token (chunked prefill, every cached position after its own) has no maximum: weights stay 0
+    const float m = tid < nh ? dec_ordered(v.seqmax[qs * Hq + h0 + tid]) : 0.f;
+    sM[tid] = m == -INFINITY ? 0.f : m;
+  }
   // Descriptors of this split's tiles (the k-th is list[split + k * n_splits]) are kept in a ring of 64 in
   // shared memory, refilled 16 at a time well ahead of both cursors, so neither the copy cursor nor the
   // consumer waits for the two dependent global reads list -> descriptor.
@@ -494,7 +498,8 @@ merge_kernel(DevView v, const unsigned short* __restrict__ Uinv_v, int n_splits,
 #pragma unroll
     for (int k = 0; k < MG_JGROUPS; ++k) val += red[k * REP * 128 + i];        // fixed order
     const int h = i >> 7, dc = i & 127;
-    const size_t oi = ((size_t)(qs0 + h / hp) * Hq + head0 + h % hp) * HEAD_DIM + dc;
+    const int oslot = qs0 + h / hp;
+    const size_t oi = ((size_t)(v.qmap ? v.qmap[oslot] : oslot) * Hq + head0 + h % hp) * HEAD_DIM + dc;
     if (v.out_dtype == TWKV_F32) reinterpret_cast<float*>(out)[oi] = val;
     else if (v.out_dtype == TWKV_BF16) reinterpret_cast<unsigned short*>(out)[oi] = from_f32<true>(val);
     else reinterpret_cast<unsigned short*>(out)[oi] = from_f32<false>(val);

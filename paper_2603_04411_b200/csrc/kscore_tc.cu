@@ -342,9 +342,10 @@ kscore_tc_kernel(const __grid_constant__ CUtensorMap map_blocks, const __grid_co
     // 8 hf + 2 c holds dimensions 32 hf + 8 c .. + 7, piece 8 hf + 2 c + 1 the dimensions 64 above them.
     // Only called when no score product that reads the rows can still be in flight.
     auto write_q = [&](int qs) {
+      const int qrow_of = v.qmap ? v.qmap[qs] : qs;                        // the row of q this query slot stands for
       for (int i = et; i < Hq * 16; i += KT_EPI) {
         const int head = i >> 4, ch = i & 15;                               // 8 dims per chunk
-        const uint4 raw = *reinterpret_cast<const uint4*>(q + ((size_t)qs * Hq + head) * HEAD_DIM + ch * 8);
+        const uint4 raw = *reinterpret_cast<const uint4*>(q + ((size_t)qrow_of * Hq + head) * HEAD_DIM + ch * 8);
         uint4 val = raw;
         if constexpr (BF16) {
           const unsigned short* e = reinterpret_cast<const unsigned short*>(&raw);
@@ -429,7 +430,8 @@ kscore_tc_kernel(const __grid_constant__ CUtensorMap map_blocks, const __grid_co
 
     KtPending p_old{nullptr, 0, 0u}, p_new{nullptr, 0, 0u};
     int4 e = w0 < total ? klist[KSTEP * w0] : kt_none;
-    if (w0 < total) { write_q(e.w); rope_setup(kpos[(size_t)e.x * TILE + row]); }
+    int pos_cur = w0 < total ? kpos[(size_t)e.x * TILE + row] : 0;              // this row's position in the current tile
+    if (w0 < total) { write_q(e.w); rope_setup(pos_cur); }
     for (int w = w0; w < total && ok; ++w) {
       const int4 nxt = w + 1 < total ? klist[KSTEP * (w + 1)] : kt_none;
       const int tile = e.x, cls = e.y & 0x7f, n_valid = e.y >> 8, qs = e.w;
@@ -437,7 +439,9 @@ kscore_tc_kernel(const __grid_constant__ CUtensorMap map_blocks, const __grid_co
       const int passes = (cls + KT_A_SLOTS - 1) / KT_A_SLOTS;
       const int pos_next = nxt.w >= 0 ? kpos[(size_t)nxt.x * TILE + row] : 0;      // fetched now, used after the tile's slabs
       float* const out_row = v.scores + ((size_t)tile * TILE + row) * Hq;
-      const uint32_t live_bit = row < n_valid ? KP_LIVE : 0u;
+      // a row counts if it holds a token and, for a causal (prefill) query, the token is not after the query
+      const int pos_limit = v.qpos ? v.qpos[qs] : 0x7fffffff;
+      const uint32_t live_bit = (row < n_valid && pos_cur <= pos_limit) ? KP_LIVE : 0u;
       for (int ps = 0; ps < passes && ok; ++ps) {
         const uint32_t mode = discard ? KP_DISCARD : passes == 1 ? KP_STORE_FINAL : (ps == 0 ? KP_STORE_PART : KP_ADD_FINAL);
         for (int sli = 0; sli < Hkv; ++sli) {
@@ -496,6 +500,7 @@ kscore_tc_kernel(const __grid_constant__ CUtensorMap map_blocks, const __grid_co
       }
       if (!ok) break;
       if (nxt.w >= 0) rope_setup(pos_next);
+      pos_cur = pos_next;
       if (nxt.w != qs) {
         // last tile of this query slot in the piece: the owed read-outs belong to it; the query operand may only change
         // once every score product that reads the old one has retired

@@ -54,6 +54,11 @@ struct DevView {
   float* scores;             // [NT*128][Hq]
   unsigned* seqmax;          // [S][Hq]  order-preserving encoding of the running max
   int* qslot;                // [S]   sequence id -> query index of the current decode call, -1
+  // chunked prefill (null for a decode call): per query slot, the row of q / out it stands for and the last position it
+  // may attend to
+  const int* qmap;
+  const int* qpos;
+  int* wave_buf;             // [3][TWKV_PREFILL_MAX_QUERIES]: sequence, row and position of a prefill call's queries, wave by wave
   int4* klist;               // [NT]  K tiles of the current decode call, widest class first: (tile, class | n_valid << 8, base block, query slot)
   int4* kpairs;              // [NT + 64]  the same list as items of two tiles of one class (entries 2 i, 2 i + 1) for the CTA-pair kernel;
                              //            a class with an odd number of tiles ends with a filler entry (.y bit 7 set)
@@ -148,6 +153,8 @@ cudaError_t launch_uinv_panels(const void* in, void* out, int d, cudaStream_t st
 int kscore_max_pairs(int sm_count);
 cudaError_t launch_gate_logits(const DevView& v, const LayerParams& lp, const void* K, const void* V, int n_tok,
                                float* logits, cudaStream_t st);
+cudaError_t launch_gate_soft(const DevView& v, const float* logits, const void* K, const void* V, float* mk, float* mv, float* xhk,
+                             float* xhv, float* retain, int n_tok, cudaStream_t st);
 cudaError_t launch_stats(const DevView& v, int layer, unsigned long long* out_dev, cudaStream_t st);
 
 }  // namespace twkv
