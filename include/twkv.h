@@ -187,6 +187,18 @@ twkv_status twkv_decode_attn(twkv_cache* cache, int layer, const void* q, const 
 twkv_status twkv_prefill_attn(twkv_cache* cache, int layer, const void* q, const int32_t* q_seq /*host*/,
                               const int32_t* q_pos /*host*/, int n_q, void* out, int num_splits, void* stream);
 
+/*
+ * Global token eviction with compaction (the paper's combination with token eviction, Sec. 5.2 "Implementation
+ * Details" and Table 5: the decomposition is joint across heads, so one token set is kept for all heads).  Of the
+ * tokens cached for `seq` in `layer`, exactly those whose position is listed survive, on the K and on the V side.
+ *   keep_positions  [n_keep] int32, device, any order; positions nothing is cached at are ignored; n_keep = 0 drops all
+ * Container rule: per (side, class) of the sequence the survivors move to the front of the tiles that key owns, in
+ * their stored order; vacated rows of the last tile still in use are zeroed; emptied tiles leave the tile lists and
+ * their blocks stay unused until twkv_cache_reset; V slots are relinked; later appends continue behind the
+ * survivors.  Decode and prefill attention afterwards see the survivors only.
+ */
+twkv_status twkv_evict(twkv_cache* cache, int layer, int seq, const int32_t* keep_positions, int n_keep, void* stream);
+
 /* Synchronises `stream`, returns the sticky device status and clears it. */
 twkv_status twkv_cache_status(twkv_cache* cache, void* stream);
 /* Synchronises `stream`; layer = -1 sums all layers.  `out` is host memory. */

@@ -27,6 +27,13 @@ Format
   the rank r.
 * K tiles are also listed per class (creation order); V tiles per sequence
   (creation order).
+* Eviction (the paper combines the method with token eviction, Sec. 5.2
+  "Implementation Details": one token set for all heads) keeps, of one
+  sequence in one layer, the tokens at the listed positions.  Per (side,
+  class) of the sequence the survivors move to the front of the key's tiles in
+  their stored order; the rows behind the last survivor in the last tile still
+  in use become zero; emptied tiles leave the lists (n_valid 0, blocks left as
+  they are and not reused); V slots are relinked to the K rows' new slots.
 """
 import numpy as np
 
@@ -149,6 +156,65 @@ class CacheImage:
             self.fill[layer, k] += cnt
         self.seq_tokens[layer] += add_tok
         return True
+
+    def evict(self, layer, seq, keep_positions):
+        """Keeps the tokens of `seq` whose position is listed; returns, per side, {old global slot: new global slot}."""
+        keep = set(int(p) for p in keep_positions)
+        moved = [{}, {}]
+        kept_tokens = 0
+        # who survives is decided on the tables as they are (a V slot finds its position through its K row)
+        survivors_of = {}
+        for side in range(2):
+            for c in range(1, self.NC + 1):
+                found = []
+                for tid in self.key_tiles[layer][self.key(side, seq, c)]:
+                    for slot in range(int(self.tile_desc[layer, side, tid, 2])):
+                        a = int(self.tile_aux[layer, side, tid, slot])
+                        pos = a if side == 0 else int(self.tile_aux[layer, 0, a // TILE, a % TILE])
+                        if pos in keep:
+                            found.append((tid, slot))
+                survivors_of[side, c] = found
+        for side in range(2):
+            for c in range(1, self.NC + 1):
+                k = self.key(side, seq, c)
+                tiles = self.key_tiles[layer][k]
+                survivors = survivors_of[side, c]
+                rows = []
+                for tid, slot in survivors:                      # everything is read before anything is written
+                    base = int(self.tile_desc[layer, side, tid, 3])
+                    rows.append(([self.blocks[base + j, slot * PANEL:(slot + 1) * PANEL].copy() for j in range(c)],
+                                 int(self.tile_aux[layer, side, tid, slot]), int(self.tile_rank[layer, side, tid, slot])))
+                for g, ((tid, slot), (row, a, r)) in enumerate(zip(survivors, rows)):
+                    dt, ds = tiles[g // TILE], g % TILE
+                    moved[side][tid * TILE + slot] = dt * TILE + ds
+                    base = int(self.tile_desc[layer, side, dt, 3])
+                    for j in range(c):
+                        self.blocks[base + j, ds * PANEL:(ds + 1) * PANEL] = row[j]
+                    self.tile_aux[layer, side, dt, ds] = a
+                    self.tile_rank[layer, side, dt, ds] = r
+                n = len(survivors)
+                n_kept = -(-n // TILE)
+                if n % TILE:
+                    base = int(self.tile_desc[layer, side, tiles[n_kept - 1], 3])
+                    for j in range(c):
+                        self.blocks[base + j, (n % TILE) * PANEL:] = 0
+                for ordinal, tid in enumerate(tiles):
+                    self.tile_desc[layer, side, tid, 2] = min(TILE, n - ordinal * TILE) if ordinal < n_kept else 0
+                gone = set(tiles[n_kept:])
+                self.key_tiles[layer][k] = tiles[:n_kept]
+                if side == 0:
+                    self.kclass_tiles[layer][c - 1] = [t for t in self.kclass_tiles[layer][c - 1] if t not in gone]
+                    kept_tokens += n
+                else:
+                    self.seq_vtiles[layer][seq] = [t for t in self.seq_vtiles[layer][seq] if t not in gone]
+                self.fill[layer, k] = n
+        # V slots follow their tokens' K rows
+        for c in range(1, self.NC + 1):
+            for tid in self.key_tiles[layer][self.key(1, seq, c)]:
+                for slot in range(int(self.tile_desc[layer, 1, tid, 2])):
+                    self.tile_aux[layer, 1, tid, slot] = moved[0][int(self.tile_aux[layer, 1, tid, slot])]
+        self.seq_tokens[layer, seq] = kept_tokens
+        return moved
 
     # ---- logical views used by the decode oracle ---------------------------------
     def stored_bytes(self, layer=None):

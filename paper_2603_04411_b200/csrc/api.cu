@@ -79,7 +79,7 @@ constexpr int GATE_TC_MIN_TOKENS = 1024;   // calls at least this large run the 
 struct Offsets {
   size_t status, pflags, rope_lo, rope_hi, n_tiles, tile_desc, tile_aux, tile_rank, fill, key_last, kclass_count,
       kclass_tiles, seq_vcount, seq_vtiles, seq_tokens, rank_sums, hist, key_cnt, key_old_fill, key_first_id,
-      key_first_base, key_old_last, scores, seqmax, qslot, klist, kpairs, klist_count, cta_start, wave_buf, part_acc, part_l, gate_scratch, gate_fix, stats_buf, tables_end, prep_uinvT, prep_wT,
+      key_first_base, key_old_last, scores, seqmax, qslot, klist, kpairs, klist_count, cta_start, wave_buf, evict_bitmap, evict_map, evict_fill, part_acc, part_l, gate_scratch, gate_fix, stats_buf, tables_end, prep_uinvT, prep_wT,
       blocks, end_fixed;
 };
 
@@ -154,6 +154,9 @@ static Offsets layout_of(const twkv_config* c, const Dims& d) {
   o.kpairs = L.alloc((NT + 64) * sizeof(int4));
   o.cta_start = L.alloc((MAX_PLAN_CTAS + 1) * sizeof(int));
   o.wave_buf = L.alloc((size_t)3 * TWKV_PREFILL_MAX_QUERIES * sizeof(int));
+  o.evict_bitmap = L.alloc((size_t)ROPE_LO * ROPE_HI / 8);
+  o.evict_map = L.alloc((size_t)2 * NT * TILE * sizeof(int));
+  o.evict_fill = L.alloc((size_t)2 * d.NC * sizeof(int));
   o.part_acc = L.alloc((size_t)d.max_partials * Hq * d.d_kv * sizeof(float));
   o.part_l = L.alloc((size_t)d.max_partials * Hq * sizeof(float));
   {
@@ -250,6 +253,7 @@ static void fill_view(twkv_cache* c) {
   v.gate_scratch = (float*)(p + o.gate_scratch);
   v.gate_fix = (int4*)(p + o.gate_fix);
   v.wave_buf = (int*)(p + o.wave_buf);
+  v.evict_bitmap = (unsigned*)(p + o.evict_bitmap); v.evict_map = (int*)(p + o.evict_map); v.evict_fill = (int*)(p + o.evict_fill);
   v.qmap = nullptr; v.qpos = nullptr;
 }
 
@@ -510,6 +514,16 @@ twkv_status twkv_cache_status(twkv_cache* c, void* stream) {
     if (cudaStreamSynchronize(st) != cudaSuccess) return TWKV_ERR_CUDA;
   }
   return (twkv_status)code;
+}
+
+twkv_status twkv_evict(twkv_cache* c, int layer, int seq, const int32_t* keep_positions, int n_keep, void* stream) {
+  if (!c || layer < 0 || layer >= c->cfg.n_layers || seq < 0 || seq >= c->cfg.max_seqs || n_keep < 0) return TWKV_ERR_INVALID_ARG;
+  if (n_keep > 0 && !keep_positions) return TWKV_ERR_INVALID_ARG;
+  DeviceGuard g(c->device);
+  if (!g.ok) return TWKV_ERR_CUDA;
+  ProfBind pb(&c->prof);
+  if (launch_evict(c->view, layer, seq, keep_positions, n_keep, (cudaStream_t)stream) != cudaSuccess) return TWKV_ERR_CUDA;
+  return TWKV_OK;
 }
 
 twkv_status twkv_gate_soft(twkv_cache* c, int layer, const void* K, const void* V, int n_tok, float* m_k, float* m_v, float* xh_k,

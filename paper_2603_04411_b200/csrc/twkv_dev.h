@@ -58,6 +58,10 @@ struct DevView {
   // may attend to
   const int* qmap;
   const int* qpos;
+  // scratch of twkv_evict
+  unsigned* evict_bitmap;    // one bit per position: the positions that stay
+  int* evict_map;            // [2][NT * 128]  new global slot of every K / V slot of the sequence, -1 = dropped
+  int* evict_fill;           // [2][NC]  survivors per key
   int* wave_buf;             // [3][TWKV_PREFILL_MAX_QUERIES]: sequence, row and position of a prefill call's queries, wave by wave
   int4* klist;               // [NT]  K tiles of the current decode call, widest class first: (tile, class | n_valid << 8, base block, query slot)
   int4* kpairs;              // [NT + 64]  the same list as items of two tiles of one class (entries 2 i, 2 i + 1) for the CTA-pair kernel;
@@ -155,6 +159,7 @@ cudaError_t launch_gate_logits(const DevView& v, const LayerParams& lp, const vo
                                float* logits, cudaStream_t st);
 cudaError_t launch_gate_soft(const DevView& v, const float* logits, const void* K, const void* V, float* mk, float* mv, float* xhk,
                              float* xhv, float* retain, int n_tok, cudaStream_t st);
+cudaError_t launch_evict(const DevView& v, int layer, int seq, const int* keep_positions, int n_keep, cudaStream_t st);
 cudaError_t launch_stats(const DevView& v, int layer, unsigned long long* out_dev, cudaStream_t st);
 
 }  // namespace twkv

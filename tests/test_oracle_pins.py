@@ -608,3 +608,57 @@ def test_soft_gate_invariants_and_link_to_hard_mask():
     # adding a constant to a row's logits changes nothing
     m2, _, _ = oracle.soft_gate(x, z + 7.0)
     np.testing.assert_allclose(m2, m, atol=1e-14)
+
+
+def test_image_eviction_keeps_exactly_the_listed_tokens_in_order():
+    # After an eviction the survivors of every (side, class) can be found again, in their arrival order, directly
+    # behind one another from the key's first tile on; their rows, ranks, positions and K <-> V links are intact, the
+    # rows behind the last one are zero, emptied tiles are off the lists, other sequences are untouched, and a later
+    # append lands behind the survivors.
+    rng = np.random.default_rng(41)
+    d, S, n = 256, 3, 900
+    ranks = rng.integers(1, d + 1, size=(n, 2)).astype(np.int32)
+    xk = rng.integers(1, 2 ** 16, size=(n, d)).astype(np.uint16)
+    xv = rng.integers(1, 2 ** 16, size=(n, d)).astype(np.uint16)
+    seq = rng.integers(0, S, n).astype(np.int32)
+    pos = rng.permutation(5000)[:n].astype(np.int32)
+    img = CacheImage(1, d, S, 1024, 4096)
+    assert img.append(0, xk[:700], xv[:700], seq[:700], pos[:700], ranks[:700])
+    ref = CacheImage(1, d, S, 1024, 4096)
+    assert ref.append(0, xk[:700], xv[:700], seq[:700], pos[:700], ranks[:700])
+    keep = rng.permutation(pos[:700][seq[:700] == 1])[:60]
+    img.evict(0, 1, np.concatenate([keep, [4999999]]))
+    alive = np.zeros(n, bool); alive[:700] = (seq[:700] != 1) | np.isin(pos[:700], keep)
+    assert img.append(0, xk[700:], xv[700:], seq[700:], pos[700:], ranks[700:])
+    alive[700:] = True
+    cls = -(-ranks // PANEL)
+    assert img.seq_tokens[0, 1] == int((alive & (seq == 1)).sum())
+    listed = [set(t for c in range(img.NC) for t in img.kclass_tiles[0][c]), set(t for s in range(S) for t in img.seq_vtiles[0][s])]
+    for side, x in ((0, xk), (1, xv)):
+        seen = {}
+        for i in np.nonzero(alive)[0]:
+            k = img.key(side, int(seq[i]), int(cls[i, side]))
+            g = seen.get(k, 0); seen[k] = g + 1
+            tid = img.key_tiles[0][k][g // TILE]; slot = g % TILE
+            s_, c_, nv, base = img.tile_desc[0, side, tid]
+            assert s_ == seq[i] and c_ == cls[i, side] and slot < nv and tid in listed[side]
+            row = np.concatenate([img.blocks[base + j, slot * PANEL:(slot + 1) * PANEL] for j in range(c_)])
+            r = ranks[i, side]
+            np.testing.assert_array_equal(row[:r], x[i, :r])
+            assert not row[r:].any() and img.tile_rank[0, side, tid, slot] == r
+            link = img.tile_aux[0, side, tid, slot]
+            assert (link if side == 0 else img.tile_aux[0, 0, link // TILE, link % TILE]) == pos[i]
+        for k, g in seen.items():
+            assert img.fill[0, k] == g and len(img.key_tiles[0][k]) == -(-g // TILE)
+            tid = img.key_tiles[0][k][-1]
+            base, c_ = img.tile_desc[0, side, tid, 3], img.tile_desc[0, side, tid, 1]
+            if g % TILE:
+                assert not any(img.blocks[base + j, (g % TILE) * PANEL:].any() for j in range(c_))
+        # every listed tile belongs to a key's current tile run; nothing of a dropped token is reachable
+        assert listed[side] == set(t for k in range(side * S * img.NC, (side + 1) * S * img.NC) for t in img.key_tiles[0][k])
+    # the other sequences' tiles did not change by the eviction itself
+    for side in range(2):
+        for tid in range(int(ref.n_tiles[0, side])):
+            if ref.tile_desc[0, side, tid, 0] != 1 and ref.tile_desc[0, side, tid, 2] == TILE:
+                base, c_ = ref.tile_desc[0, side, tid, 3], ref.tile_desc[0, side, tid, 1]
+                np.testing.assert_array_equal(img.blocks[base:base + c_], ref.blocks[base:base + c_])
