@@ -203,6 +203,23 @@ twkv_status twkv_evict(twkv_cache* cache, int layer, int seq, const int32_t* kee
 twkv_status twkv_cache_status(twkv_cache* cache, void* stream);
 /* Synchronises `stream`; layer = -1 sums all layers.  `out` is host memory. */
 twkv_status twkv_cache_stats(twkv_cache* cache, int layer, void* stream, twkv_stats* out /*host*/);
+/*
+ * Consistency check (a diagnostic of the library; the paper has no counterpart).  A kernel verifies the guard words
+ * written behind every region of the pool when the cache was created, and the tables of `layer` (-1 = all): tile
+ * descriptors inside their ranges, every stored rank inside its tile's class, every V slot linked to a live K slot of
+ * the same sequence, tile lists naming tiles of the right class / sequence.  Synchronises `stream`.  Returns TWKV_OK, or
+ * TWKV_ERR_DEVICE_CHECK with the number of violations in *violations (host, may be NULL); the sticky status is set too.
+ */
+twkv_status twkv_cache_check(twkv_cache* cache, int layer, void* stream, uint64_t* violations /*host*/);
+/*
+ * Self-test of the bounded device-side wait (diagnostic).  Every tensor-core kernel of the library waits on shared-
+ * memory barriers with an attempt limit; a wait that runs out raises its CTA's abort flag, all roles leave their loops
+ * and the kernel reports TWKV_ERR_TIMEOUT instead of hanging.  This call launches a one-CTA kernel whose barrier
+ * nobody ever completes, with the limit set to `attempts` (the production limit is 2^21), and synchronises `stream`.
+ * Returns TWKV_OK if the wait gave up and raised the flag; the sticky status is then TWKV_ERR_TIMEOUT, as after a
+ * production kernel's timeout, until twkv_cache_status reads it.  *elapsed_ns (host, may be NULL) = how long the wait took.
+ */
+twkv_status twkv_selftest_wait_timeout(twkv_cache* cache, uint32_t attempts, uint64_t* elapsed_ns /*host*/, void* stream);
 /* Where the tables live inside the pool (host call, no device work). */
 twkv_status twkv_cache_layout(const twkv_cache* cache, twkv_layout* out /*host*/);
 /*

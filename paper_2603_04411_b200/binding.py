@@ -21,7 +21,7 @@ TILE_TOKENS, PANEL_ELEMS, BLOCK_BYTES, PIECE_TOKENS, MAX_CLASSES = 128, 64, 1638
 PREFILL_MAX_QUERIES = 16384
 
 EXPORTS = ["twkv_cache_required_bytes", "twkv_cache_create", "twkv_cache_destroy", "twkv_cache_reset",
-           "twkv_cache_set_layer_params", "twkv_compress", "twkv_decode_attn", "twkv_prefill_attn", "twkv_evict", "twkv_cache_status",
+           "twkv_cache_set_layer_params", "twkv_compress", "twkv_decode_attn", "twkv_prefill_attn", "twkv_evict", "twkv_cache_check", "twkv_selftest_wait_timeout", "twkv_cache_status",
            "twkv_cache_stats", "twkv_cache_layout", "twkv_launch_count", "twkv_status_string",
            "twkv_profile_enable", "twkv_profile_read", "twkv_gate_ranks_static", "twkv_gate_soft",
            "twkv_projector_required_bytes", "twkv_projector_create", "twkv_projector_destroy", "twkv_project",
@@ -71,6 +71,10 @@ def _load():
     L.twkv_compress.argtypes = [vp, i32, vp, vp, vp, vp, i32, vp, vp, i32, vp]
     L.twkv_decode_attn.argtypes = [vp, i32, vp, vp, i32, vp, i32, vp]
     L.twkv_prefill_attn.argtypes = [vp, i32, vp, ctypes.POINTER(ctypes.c_int32), ctypes.POINTER(ctypes.c_int32), i32, vp, i32, vp]
+    L.twkv_cache_check.argtypes = [vp, i32, vp, ctypes.POINTER(ctypes.c_uint64)]
+    L.twkv_cache_check.restype = i32
+    L.twkv_selftest_wait_timeout.argtypes = [vp, ctypes.c_uint32, ctypes.POINTER(ctypes.c_uint64), vp]
+    L.twkv_selftest_wait_timeout.restype = i32
     L.twkv_evict.argtypes = [vp, i32, i32, vp, i32, vp]
     L.twkv_evict.restype = i32
     L.twkv_gate_soft.argtypes = [vp, i32, vp, vp, i32, vp, vp, vp, vp, vp, vp]
@@ -186,6 +190,20 @@ def twkv_prefill_attn(cache, layer, q, q_seq, q_pos, out, num_splits=0, stream=N
     arr = ctypes.c_int32 * max(n, 1)
     _check(lib.twkv_prefill_attn(cache, layer, _ptr(q), arr(*seq), arr(*pos), n, _ptr(out), num_splits, _stream(stream)),
            "twkv_prefill_attn")
+
+
+def twkv_cache_check(cache, layer=-1, stream=None):
+    """-> (status code, number of violations): guard words and table invariants, checked by a kernel."""
+    bad = ctypes.c_uint64(0)
+    code = int(lib.twkv_cache_check(cache, layer, _stream(stream), ctypes.byref(bad)))
+    return code, int(bad.value)
+
+
+def twkv_selftest_wait_timeout(cache, attempts, stream=None):
+    """-> (status code, elapsed ns) of a bounded wait that nobody ends; leaves TWKV_ERR_TIMEOUT as the sticky status."""
+    ns = ctypes.c_uint64(0)
+    code = int(lib.twkv_selftest_wait_timeout(cache, attempts, ctypes.byref(ns), _stream(stream)))
+    return code, int(ns.value)
 
 
 def twkv_evict(cache, layer, seq, keep_positions, stream=None):

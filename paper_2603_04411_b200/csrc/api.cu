@@ -63,12 +63,20 @@ bool make_tmap_2d(CUtensorMap* out, const void* base, uint64_t rows, uint64_t co
                 CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// Regions of the pool, each followed by one guard word (checked by twkv_cache_check).
 struct Layout {
   size_t total = 0;
+  std::vector<unsigned long long> guards;                  // byte offsets of the guard words
+  bool guard = true;                                       // off while the tables that a reset clears in one sweep are laid out
   size_t alloc(size_t bytes, size_t align = 256) {
     total = (total + align - 1) / align * align;
     const size_t off = total;
     total += bytes;
+    if (bytes && guard) {
+      total = (total + 7) / 8 * 8;
+      guards.push_back(total);
+      total += 8;
+    }
     return off;
   }
 };
@@ -79,7 +87,7 @@ constexpr int GATE_TC_MIN_TOKENS = 1024;   // calls at least this large run the 
 struct Offsets {
   size_t status, pflags, rope_lo, rope_hi, n_tiles, tile_desc, tile_aux, tile_rank, fill, key_last, kclass_count,
       kclass_tiles, seq_vcount, seq_vtiles, seq_tokens, rank_sums, hist, key_cnt, key_old_fill, key_first_id,
-      key_first_base, key_old_last, scores, seqmax, qslot, klist, kpairs, klist_count, cta_start, wave_buf, evict_bitmap, evict_map, evict_fill, part_acc, part_l, gate_scratch, gate_fix, stats_buf, tables_end, prep_uinvT, prep_wT,
+      key_first_base, key_old_last, scores, seqmax, qslot, klist, kpairs, klist_count, cta_start, wave_buf, evict_bitmap, evict_map, evict_fill, part_acc, part_l, gate_scratch, gate_fix, stats_buf, tables_end, prep_uinvT, prep_wT, guard_list,
       blocks, end_fixed;
 };
 
@@ -118,13 +126,14 @@ static Dims dims_of(const twkv_config* c) {
   return d;
 }
 
-static Offsets layout_of(const twkv_config* c, const Dims& d) {
+static Offsets layout_of(const twkv_config* c, const Dims& d, std::vector<unsigned long long>* guards = nullptr) {
   Layout L;
   Offsets o;
   const size_t Ls = c->n_layers, S = c->max_seqs, NT = d.NT, NK = d.NK, Hq = c->n_q_heads;
   o.status = L.alloc(8 * sizeof(int));
   o.rope_lo = L.alloc((size_t)ROPE_LO * 32 * sizeof(float4));
   o.rope_hi = L.alloc((size_t)ROPE_HI * 32 * sizeof(float4));
+  L.guard = false;
   o.n_tiles = L.alloc(Ls * 2 * sizeof(int));
   o.tile_desc = L.alloc(Ls * 2 * NT * sizeof(int4));
   o.tile_aux = L.alloc(Ls * 2 * NT * TILE * sizeof(int));
@@ -138,6 +147,8 @@ static Offsets layout_of(const twkv_config* c, const Dims& d) {
   o.seq_tokens = L.alloc(Ls * S * sizeof(int));
   o.rank_sums = L.alloc(Ls * 2 * sizeof(unsigned long long));
   o.tables_end = L.alloc(0);
+  L.guard = true;
+  L.alloc(8);                                              // one guard behind the tables
   const size_t PB = (size_t)d.batch;
   o.hist = L.alloc(PB * PIECE_CHUNKS * NK * sizeof(int));
   o.key_cnt = L.alloc(PB * NK * sizeof(int));
@@ -167,8 +178,10 @@ static Offsets layout_of(const twkv_config* c, const Dims& d) {
   o.stats_buf = L.alloc(64 * sizeof(unsigned long long));
   o.prep_uinvT = L.alloc(Ls * (size_t)d.d_kv * d.d_kv * 2, 1024);
   o.prep_wT = L.alloc(Ls * 2 * (size_t)d.d_kv * d.d_kv * 2, 1024);
+  o.guard_list = L.alloc(L.guards.size() * sizeof(unsigned long long) + 64);
   o.blocks = L.alloc(0, 1024);
   o.end_fixed = o.blocks;
+  if (guards) *guards = L.guards;
   return o;
 }
 
@@ -194,6 +207,7 @@ struct twkv_cache {
   std::vector<CUtensorMap> map_wT_half; // the same with 128-row boxes, for the CTA-pair kernel
   std::vector<char> prepared_w;        // per layer: those copies and maps are current
   bool kscore_pairs = false;           // the K-score kernel runs on CTA pairs (the device can co-schedule them)
+  std::vector<unsigned long long> guards;   // byte offsets (from the pool's start) of the guard words
 };
 
 
@@ -279,10 +293,12 @@ twkv_status twkv_cache_create(const twkv_config* cfg, void* pool, size_t pool_by
   if (cudaPointerGetAttributes(&attr, pool) != cudaSuccess) { cudaGetLastError(); return TWKV_ERR_CUDA; }
   if (attr.type != cudaMemoryTypeDevice && attr.type != cudaMemoryTypeManaged) return TWKV_ERR_INVALID_ARG;
   const Dims d = dims_of(cfg);
-  const Offsets o = layout_of(cfg, d);
+  std::vector<unsigned long long> guards;
+  const Offsets o = layout_of(cfg, d, &guards);
   if (pool_bytes < o.blocks + (size_t)BLOCK_BYTES) return TWKV_ERR_CAPACITY;
   twkv_cache* c = new (std::nothrow) twkv_cache();
   if (!c) return TWKV_ERR_INVALID_ARG;
+  c->guards = guards;
   c->cfg = *cfg; c->dims = d; c->off = o; c->pool = (unsigned char*)pool; c->pool_bytes = pool_bytes;
   c->device = attr.device;
   c->params.assign(cfg->n_layers, LayerParams{nullptr, nullptr, nullptr, nullptr, nullptr, nullptr});
@@ -296,12 +312,24 @@ twkv_status twkv_cache_create(const twkv_config* cfg, void* pool, size_t pool_by
     c->kscore_pairs = !(single && single[0] == '1') && kscore_max_pairs(c->sm_count) > 0;
   }
   fill_view(c);
+  {
+    const char* dbg = getenv("TWKV_DEBUG");
+    c->view.debug = (dbg && dbg[0] == '1') ? 1 : 0;
+  }
   c->map_uinvT.resize(cfg->n_layers);
   c->prepared.assign(cfg->n_layers, 0);
   c->map_wT.resize(2 * (size_t)cfg->n_layers);
   c->map_wT_half.resize(2 * (size_t)cfg->n_layers);
   c->prepared_w.assign(cfg->n_layers, 0);
   if (!make_tmap_2d(&c->map_blocks, c->view.blocks, (uint64_t)c->view.n_blocks * TILE, PANEL, PANEL * 2, TILE)) { delete c; return TWKV_ERR_CUDA; }
+  {
+    // guard words behind every region, and the list of their offsets for the check kernel
+    const unsigned long long word = TWKV_GUARD_WORD;
+    for (unsigned long long off : c->guards)
+      if (cudaMemcpyAsync(c->pool + off, &word, sizeof(word), cudaMemcpyHostToDevice, (cudaStream_t)stream) != cudaSuccess) { delete c; return TWKV_ERR_CUDA; }
+    if (cudaMemcpyAsync(c->pool + o.guard_list, c->guards.data(), c->guards.size() * sizeof(unsigned long long), cudaMemcpyHostToDevice,
+                        (cudaStream_t)stream) != cudaSuccess) { delete c; return TWKV_ERR_CUDA; }
+  }
   twkv_status s = twkv_cache_reset(c, stream);
   if (s != TWKV_OK) { delete c; return s; }
   if (launch_rope_tables(c->view, cfg->rope_base, (cudaStream_t)stream) != cudaSuccess) { delete c; return TWKV_ERR_CUDA; }
@@ -514,6 +542,36 @@ twkv_status twkv_cache_status(twkv_cache* c, void* stream) {
     if (cudaStreamSynchronize(st) != cudaSuccess) return TWKV_ERR_CUDA;
   }
   return (twkv_status)code;
+}
+
+twkv_status twkv_cache_check(twkv_cache* c, int layer, void* stream, uint64_t* violations) {
+  if (!c || layer < -1 || layer >= c->cfg.n_layers) return TWKV_ERR_INVALID_ARG;
+  DeviceGuard g(c->device);
+  if (!g.ok) return TWKV_ERR_CUDA;
+  cudaStream_t st = (cudaStream_t)stream;
+  unsigned long long* dev = (unsigned long long*)(c->pool + c->off.stats_buf);
+  // guard offsets are relative to the pool; the kernel addresses them from the status word, which sits at its start
+  if (launch_cache_check(c->view, layer, (const unsigned long long*)(c->pool + c->off.guard_list), (int)c->guards.size(), dev, st) != cudaSuccess)
+    return TWKV_ERR_CUDA;
+  unsigned long long bad = 0;
+  if (cudaMemcpyAsync(&bad, dev, sizeof(bad), cudaMemcpyDeviceToHost, st) != cudaSuccess) return TWKV_ERR_CUDA;
+  if (cudaStreamSynchronize(st) != cudaSuccess) return TWKV_ERR_CUDA;
+  if (violations) *violations = bad;
+  return bad ? TWKV_ERR_DEVICE_CHECK : TWKV_OK;
+}
+
+twkv_status twkv_selftest_wait_timeout(twkv_cache* c, uint32_t attempts, uint64_t* elapsed_ns, void* stream) {
+  if (!c || attempts == 0) return TWKV_ERR_INVALID_ARG;
+  DeviceGuard g(c->device);
+  if (!g.ok) return TWKV_ERR_CUDA;
+  cudaStream_t st = (cudaStream_t)stream;
+  unsigned long long* dev = (unsigned long long*)(c->pool + c->off.stats_buf);
+  if (launch_wait_timeout(c->view, attempts, dev, st) != cudaSuccess) return TWKV_ERR_CUDA;
+  unsigned long long h[3] = {0, 0, 0};
+  if (cudaMemcpyAsync(h, dev, sizeof(h), cudaMemcpyDeviceToHost, st) != cudaSuccess) return TWKV_ERR_CUDA;
+  if (cudaStreamSynchronize(st) != cudaSuccess) return TWKV_ERR_CUDA;
+  if (elapsed_ns) *elapsed_ns = h[0];
+  return (h[1] == 1 && h[2] == 1) ? TWKV_OK : TWKV_ERR_DEVICE_CHECK;     // the wait must have failed and raised the flag
 }
 
 twkv_status twkv_evict(twkv_cache* c, int layer, int seq, const int32_t* keep_positions, int n_keep, void* stream) {

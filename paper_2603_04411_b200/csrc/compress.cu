@@ -17,7 +17,7 @@ namespace twkv {
 // The comparison c_n <= tau is done as S_n <= tau * S_d on the unnormalised sums.
 // ------------------------------------------------------------------------------------------
 __global__ void __launch_bounds__(256) gate_rank_kernel(const float* __restrict__ logits, unsigned short* __restrict__ levels,
-                                                        int n_rows, int d, float tau) {
+                                                        int n_rows, int d, float tau, int* status) {
   const int warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
   const int lane = threadIdx.x & 31;
   if (warp >= n_rows) return;
@@ -58,14 +58,18 @@ __global__ void __launch_bounds__(256) gate_rank_kernel(const float* __restrict_
   for (int o = 16; o > 0; o >>= 1) below += __shfl_xor_sync(0xffffffffu, below, o);
   int r = d - below;
   if (r < 1) r = 1;                             // only reachable with tau >= 1 or NaN logits
-  if (lane == 0) levels[warp] = (unsigned short)r;
+  if (lane == 0) {
+    levels[warp] = (unsigned short)r;
+    // a row with a NaN or an infinite logit has no softmax: the rank above is a placeholder, the call reports it
+    if (status && !(total > 0.f && total < INFINITY)) atomicCAS(status, 0, TWKV_ERR_DEVICE_CHECK);
+  }
 }
 
 cudaError_t launch_gate_rank(const DevView& v, const float* logits, unsigned short* levels, int n_tok, cudaStream_t st) {
   const int rows = n_tok * 2;
   if (rows == 0) return cudaSuccess;
   const int blocks = (rows + 7) / 8;
-  { ProfScope ps(TWKV_K_GATE_RANK, st); gate_rank_kernel<<<blocks, 256, 0, st>>>(logits, levels, rows, v.d_kv, v.tau); }
+  { ProfScope ps(TWKV_K_GATE_RANK, st); gate_rank_kernel<<<blocks, 256, 0, st>>>(logits, levels, rows, v.d_kv, v.tau, v.status); }
   count_launch();
   return cudaGetLastError();
 }

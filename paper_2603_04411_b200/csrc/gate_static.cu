@@ -63,7 +63,7 @@ extern "C" twkv_status twkv_gate_ranks_static(const void* K, const void* V, cons
   if ((long long)n_tok * 2 * d_kv > (long long)STATIC_GATE_MAX_ELEMS) return TWKV_ERR_CAPACITY;   // beyond the fixed scratch
   float* scratch = nullptr;
   if (static_scratch(&scratch) != cudaSuccess) { cudaGetLastError(); return TWKV_ERR_CUDA; }
-  DevView v{};                    // only the shape fields the two launchers read
+  DevView v{};                    // only the shape fields the two launchers read (no status word: v.status stays null)
   v.d_kv = d_kv; v.dtype = dtype; v.tau = tau;
   LayerParams lp{nullptr, nullptr, W_k, W_v, b_k, b_v};
   cudaStream_t st = (cudaStream_t)stream;

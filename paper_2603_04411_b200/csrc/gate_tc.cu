@@ -165,7 +165,7 @@ __device__ __forceinline__ void gate_epilogue_role(uint32_t tmem_base, uint32_t 
                                                    const float* __restrict__ bias_k, const float* __restrict__ bias_v,
                                                    unsigned short* __restrict__ levels, int n_tok, int d, int NS, int n_slabs,
                                                    int ns_rot, int it0, int itstep, int n_items, float tau, uint32_t crank,
-                                                   const GateRaw raw, int bf16) {
+                                                   const GateRaw raw, int bf16, int* status) {
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int ew = warp - 2;                                   // 0..7
   const int quarter = warp & 3, chalf = ew >> 2;
@@ -241,6 +241,8 @@ __device__ __forceinline__ void gate_epilogue_role(uint32_t tmem_base, uint32_t 
       const float so = __shfl_xor_sync(0xffffffffu, s, 1);
       const float lo = hh ? so : s, hi = hh ? s : so;
       const float thr = tau * (lo + hi);                     // c_n <= tau  <=>  S_n <= tau * S_d
+      // a row with a NaN or an infinite logit has no softmax: its rank is a placeholder, the call reports it
+      if (hh == 0 && m0 + rr < n_tok && !(thr > 0.f && thr < INFINITY)) atomicCAS(status, 0, TWKV_ERR_DEVICE_CHECK);
       float run = hh ? lo : 0.f, base = 0.f;
       int bstar = -1;
       for (int b = b0; b < b0 + half; ++b) {
@@ -410,7 +412,7 @@ gate_tc_kernel(const __grid_constant__ CUtensorMap map_xk, const __grid_constant
     // ------------------------------------------------------------- epilogue + rank
     gate_epilogue_role<false>(tmem_base, acc_full, acc_empty, epi_bar, sBlk, abort_flag,
                               reinterpret_cast<unsigned short*>(stage_all) + (size_t)blockIdx.x * TILE * d, bias_k, bias_v, levels,
-                              n_tok, d, NS, n_slabs, ns_rot, it0, itstep, n_items, tau, 0u, raw, bf16);
+                              n_tok, d, NS, n_slabs, ns_rot, it0, itstep, n_items, tau, 0u, raw, bf16, status);
   }
 
   fence_before_sync();
@@ -542,7 +544,7 @@ gate_tc2_kernel(const __grid_constant__ CUtensorMap map_xk, const __grid_constan
     // ------------------------------------------------------------- epilogue + rank
     gate_epilogue_role<true>(tmem_base, acc_full, acc_empty, epi_bar, sBlk, abort_flag,
                               reinterpret_cast<unsigned short*>(stage_all) + (size_t)blockIdx.x * TILE * d, bias_k, bias_v, levels,
-                              n_tok, d, NS, n_slabs, ns_rot, it0, itstep, n_items, tau, crank, raw, bf16);
+                              n_tok, d, NS, n_slabs, ns_rot, it0, itstep, n_items, tau, crank, raw, bf16, status);
   }
 
   fence_before_sync();

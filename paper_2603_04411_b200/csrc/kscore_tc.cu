@@ -349,6 +349,11 @@ kscore_tc_kernel(const __grid_constant__ CUtensorMap map_blocks, const __grid_co
         uint4 val = raw;
         if constexpr (BF16) {
           const unsigned short* e = reinterpret_cast<const unsigned short*>(&raw);
+          // a bf16 query enters the score product as f16: one beyond the f16 range would be clamped, so it is reported
+          bool over = false;
+#pragma unroll
+          for (int k = 0; k < 8; ++k) over |= !(fabsf(kt_to_f32<true>(e[k])) <= 65504.f);
+          if (over) set_status(v, TWKV_ERR_DEVICE_CHECK);
           val.x = pack_f16x2_sat(kt_to_f32<true>(e[0]), kt_to_f32<true>(e[1]));
           val.y = pack_f16x2_sat(kt_to_f32<true>(e[2]), kt_to_f32<true>(e[3]));
           val.z = pack_f16x2_sat(kt_to_f32<true>(e[4]), kt_to_f32<true>(e[5]));
@@ -479,6 +484,14 @@ kscore_tc_kernel(const __grid_constant__ CUtensorMap map_blocks, const __grid_co
               oh[4 + u] = f2_to_f16x2_sat(bh);
               ol[u] = f2_to_f16x2_sat(f2_sub(a, ah));
               ol[4 + u] = f2_to_f16x2_sat(f2_sub(b, bh));
+            }
+            if (v.debug) {
+              // TWKV_DEBUG: a rotated key beyond the f16 range was clamped by the conversion above (its high part reads
+              // 0x7bff); without the flag that goes unreported
+              bool sat = false;
+#pragma unroll
+              for (int u = 0; u < 8; ++u) sat |= (oh[u] & 0x7fffu) == 0x7bffu || ((oh[u] >> 16) & 0x7fffu) == 0x7bffu;
+              if (sat && row < n_valid) set_status(v, TWKV_ERR_DEVICE_CHECK);
             }
             tmem_st8(sl_addr + 8 * c, oh);                                    // high parts: columns 0 .. 63 of the slab
             tmem_st8(sl_addr + 64 + 8 * c, ol);                               // low parts: columns 64 .. 127

@@ -11,7 +11,10 @@
 namespace twkv {
 namespace tc {
 
-constexpr uint32_t SPIN_LIMIT = 1u << 21;     // try_wait attempts (each suspends up to the HW time limit)
+// try_wait attempts of a bounded wait.  An attempt on a barrier that does not complete suspends the thread for about
+// 4 microseconds (measured: 16384 attempts take 66 ms), so a wait gives up after about one second; the longest
+// legitimate wait in any kernel of the library is a few milliseconds.
+constexpr uint32_t SPIN_LIMIT = 1u << 18;
 
 __device__ __forceinline__ uint32_t smem_addr(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
@@ -38,13 +41,16 @@ __device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity) {
   return ok != 0;
 }
 // Bounded wait.  Returns false if the wait ran out or another role already gave up.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
-  for (uint32_t i = 0; i < SPIN_LIMIT; ++i) {
+__device__ __forceinline__ bool mbar_wait_limited(uint32_t bar, uint32_t parity, volatile int* abort_flag, uint32_t limit) {
+  for (uint32_t i = 0; i < limit; ++i) {
     if (mbar_try(bar, parity)) return true;
     if ((i & 63u) == 63u && *abort_flag) return false;
   }
   *abort_flag = 1;
   return false;
+}
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+  return mbar_wait_limited(bar, parity, abort_flag, SPIN_LIMIT);
 }
 
 // The same wait for a role that runs on one thread and must spend few instructions: one attempt inline, the bounded

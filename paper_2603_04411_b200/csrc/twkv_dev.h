@@ -18,11 +18,13 @@ constexpr int ROPE_LO = 16;                 // pos = hi * 16 + lo
 constexpr int ROPE_HI = 32768;              // positions up to 16 * 32768 - 1
 constexpr int MAX_PARTIALS_EXTRA = 320;     // V-side partial slots beyond max_seqs
 constexpr int MAX_PLAN_CTAS = 1024;         // upper bound on the K-score kernel's grid
+constexpr unsigned long long TWKV_GUARD_WORD = 0x7477b2006b765f67ull;   // written behind every region of the pool
 
 // Device view of a cache: plain pointers into the caller's pool.  Passed to kernels by value.
 struct DevView {
   int L, Hq, Hkv, rep, d_kv, NC, S, tmax, NT, TPS, n_blocks, dtype, out_dtype, NK, max_partials;
   float tau, sm_scale;
+  int debug;                 // TWKV_DEBUG=1 at cache creation: extra device-side checks (rotated keys inside the f16 range)
   int* status;               // [8]: [0] sticky status, [1] next free block, [2] rows listed for the gate fix-up, [3] its finished CTAs
   int* pflags;               // [batch][2]: piece accepted, piece holds an invalid token (scratch of one compress call)
   int batch;                 // pieces of a compress call whose bookkeeping is launched together
@@ -160,6 +162,9 @@ cudaError_t launch_gate_logits(const DevView& v, const LayerParams& lp, const vo
 cudaError_t launch_gate_soft(const DevView& v, const float* logits, const void* K, const void* V, float* mk, float* mv, float* xhk,
                              float* xhv, float* retain, int n_tok, cudaStream_t st);
 cudaError_t launch_evict(const DevView& v, int layer, int seq, const int* keep_positions, int n_keep, cudaStream_t st);
+cudaError_t launch_wait_timeout(const DevView& v, unsigned attempts, unsigned long long* out_dev, cudaStream_t st);
+cudaError_t launch_cache_check(const DevView& v, int layer, const unsigned long long* guards_dev, int n_guards, unsigned long long* out_dev,
+                               cudaStream_t st);
 cudaError_t launch_stats(const DevView& v, int layer, unsigned long long* out_dev, cudaStream_t st);
 
 }  // namespace twkv
