@@ -8,6 +8,8 @@ compress tokens/s, HBM GB/s on the compressed bytes and the per-kernel times are
 beside it.  `--impl reference` times the fp64 CPU oracle on a bounded sample instead.
 
   python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+  python bench.py --config 1|3|4|5     the other synthetic workloads (tiny, high-batch serving with appends, long context
+                                       with a split-K sweep, 32-layer decode step): 20 warm + at least 100 timed iterations each
 """
 import argparse
 import json
@@ -238,6 +240,26 @@ def run_ours(args):
     total_ms, comp_ms, dec_ms = replicas.max_over_ranks([total_ms, comp_ms, dec_ms], dev)
     ms_per_step = total_ms / args.steps
 
+    # sustained leg: the same step back to back for at least two seconds with the clock sampler running, so that the
+    # burst figures above can be read beside what the board holds under its power cap
+    sustained = None
+    if not args.skip_sustained:
+        n_sus = max(args.steps, int(2200.0 / max(ms_per_step, 1e-3)))
+        sampler2 = ClockSampler(local) if rank == 0 else None
+        barrier()
+        s0, s1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        s0.record(stream)
+        for _ in range(n_sus):
+            step()
+        s1.record(stream)
+        barrier()
+        c2 = sampler2.stop() if sampler2 else None
+        sus_ms = replicas.max_over_ranks([s0.elapsed_time(s1) / n_sus], dev)[0]
+        if rank == 0:
+            sustained = {"steps": n_sus, "ms_per_step": sus_ms, "sm_mhz_median": c2["sm_mhz"], "reasons": c2["reasons"],
+                         "samples": c2["samples"], "power_w_max": c2.get("power_w_max"),
+                         "ms_x_mhz": sus_ms * c2["sm_mhz"] if c2["sm_mhz"] else None}
+
     # end to end: host buffers in, host result out, through the same C ABI calls
     e2e = None
     n_e2e = 0 if args.skip_e2e else min(args.steps, 3)
@@ -285,7 +307,9 @@ def run_ours(args):
         e2e_ms = replicas.max_over_ranks([g0.elapsed_time(g1) / n_e2e], dev)[0]
         h2d = sum(x.numel() * x.element_size() for x in (h_xk, h_xv, h_sid, h_pos, h_q))
         d2h = h_out.numel() * h_out.element_size()
-        e2e = {"value": replicas.whole_job_rate(n_tok, e2e_ms), "unit": "KV tokens/s through compress + decode, host buffers (state copies in pieces on a copy stream, each piece compressed when it has landed)",
+        e2e = {"value": replicas.whole_job_rate(n_tok, e2e_ms), "unit": UNIT,
+               "note": "compress + decode through the C ABI from pinned host buffers: state copies in pieces on a copy stream, each "
+                       "piece compressed when it has landed, the result copied back",
                "ms_per_step": e2e_ms, "steps": n_e2e, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h}
 
     if rank == 0:
@@ -388,30 +412,269 @@ def run_ours(args):
                            "head_dim": DH, "step": "cache reset + compress(COMPUTE gate) of B*T tokens + one decode-attention step",
                            "l2": "inputs_exceed_l2 (cache %.0f MB, states 2.1 GB)" % (st.bytes_stored / 1e6),
                            "sharding": "replica per GPU (independent sequences), no collective"},
-                "roofline": roofline, "roofline_decode_attn": roofline_decode, "cpu_baseline": cpu, "e2e": e2e, "gpu_launches": int(launches), "clocks": clocks}
+                "roofline": roofline, "roofline_decode_attn": roofline_decode, "cpu_baseline": cpu, "e2e": e2e, "gpu_launches": int(launches), "clocks": clocks,
+                "sustained": sustained}
         line.update(extra)
         print(json.dumps(line), flush=True)
     B.twkv_cache_destroy(cache)
     replicas.finish()
 
 
+# ------------------------------------------------------------------------------------------------------------------
+# The other four workloads (`--config 1|3|4|5`): one JSON line each, same objects as the headline line.
+def _median_min(xs):
+    xs = sorted(xs)
+    return {"median": xs[len(xs) // 2], "min": xs[0], "n": len(xs)}
+
+
+def _decode_flops(st, n_tok, hq):
+    """Algorithmic flops of one decode step over the cached tokens: K reconstruct 2 r_K d, RoPE 3 d, scores 2 Hq d_h,
+    absorbed PV 2 Hq r_V (per token), from the cache's rank sums."""
+    sum_rk, sum_rv = st.retain_rate_k * n_tok * D_KV, st.retain_rate_v * n_tok * D_KV
+    k_side = 2.0 * sum_rk * D_KV + n_tok * (3.0 * D_KV + 2.0 * hq * DH)
+    return k_side, k_side + 2.0 * hq * sum_rv
+
+
+def _decode_report(st, n_tok, hq, dec_ms, ks_ms, peaks):
+    k_flops, all_flops = _decode_flops(st, n_tok, hq)
+    gbs = st.bytes_stored / (dec_ms * 1e-3) / 1e9
+    bound_ms = max(st.bytes_stored / peaks["hbm_gbs"] / 1e6, all_flops / peaks["tflops"] / 1e9)
+    ach = k_flops / (ks_ms * 1e-3) / 1e12
+    return {"decode_kv_tokens_per_s": n_tok / (dec_ms * 1e-3), "decode_hbm_gbs_on_stored_bytes": gbs,
+            "decode_hbm_frac_of_8tbs": gbs / NOMINAL_HBM_GBS, "decode_hbm_frac_of_measured": gbs / peaks["hbm_gbs"],
+            "binding_bound_ms": bound_ms, "frac_of_binding_bound": bound_ms / dec_ms,
+            "roofline": {"kernel": "kscore_tc_kernel (tcgen05 on CTA pairs: K reconstruct + RoPE + q.K scores)", "bound": "tensor",
+                         "achieved": ach, "peak": peaks["tflops"], "unit": "TFLOP/s", "frac": ach / peaks["tflops"],
+                         "peak_source": f"{peaks['source']} bf16 burst", "traffic": None, "flops_per_launch": k_flops, "avg_launch_ms": ks_ms}}
+
+
+def _oracle_decode_baseline(li, ranks, seq, n_cap, dn, hq, label, full_tokens):
+    """The oracle's decode attention over (a prefix of) one sequence, timed; linear extrapolation to the whole workload."""
+    import numpy as np
+    import oracle
+    from tests.helpers import bits16
+    idx = (li.seq_ids == seq).nonzero().flatten()[:n_cap]
+    w = lambda t: oracle.widen16(bits16(t), dn)
+    xk, xv = w(li.xt_k[idx]), w(li.xt_v[idx])
+    r = ranks[idx].cpu().numpy().astype(np.int32)
+    pos = li.positions[idx].cpu().numpy()
+    Uk, Uv, q = w(li.Uinv_k), w(li.Uinv_v), w(li.q[seq])
+    t0 = time.perf_counter()
+    oracle.decode_attn(xk, xv, r[:, 0], r[:, 1], pos, Uk, Uv, q, HKV, 500000.0, DH ** -0.5)
+    dt = time.perf_counter() - t0
+    n = len(idx)
+    return {"value": n / dt, "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle",
+            "sample": f"{label}: decode attention over {n} tokens of sequence {seq}, all {hq} heads, {dt:.2f} s",
+            "extrapolated_s_per_step_whole_workload": full_tokens / (n / dt),
+            "extrapolation": "linear in the number of cached tokens (the oracle's cost per token does not depend on the context)"}
+
+
+def run_config(args):
+    import numpy as np
+    import torch
+    from paper_2603_04411_b200 import build as lib_build
+    lib_build.build()
+    from paper_2603_04411_b200 import binding as B, workloads
+    assert torch.cuda.is_available(), "bench.py needs a CUDA device; there is no CPU fallback"
+    torch.cuda.set_device(0)
+    dev = torch.device("cuda", 0)
+    peaks = measured_peaks()
+    ci = args.config
+    # at least 20 warm + 100 timed iterations; more where a step is short, so that the timed region spans ~0.4 s and the
+    # clock sampler (one nvidia-smi reading every 20 - 30 ms) sees it at least ten times
+    WARM, TIMED = 20, {1: 4000, 3: 600, 4: 1500, 5: 100}[ci]
+    shapes = {1: dict(S=1, ctx=1024, hq=8, dt=torch.float16, name="tiny_B1_ctx1024_mha8_fp16_uniform-levels"),
+              3: dict(S=64, ctx=8192, hq=32, dt=torch.float16, name="high-batch_B64_ctx8192_gqa4_fp16_mix10-20-40-30"),
+              4: dict(S=1, ctx=131072, hq=64, dt=torch.bfloat16, name="long-context_B1_ctx131072_gqa8_bf16_sink-recent"),
+              5: dict(S=32, ctx=16384, hq=32, dt=torch.float16, name="decode-step_32layers_B32_ctx16384_gqa4_fp16_dirichlet-mix")}[ci]
+    S, ctx, hq, dt = shapes["S"], shapes["ctx"], shapes["hq"], shapes["dt"]
+    dn = "f16" if dt == torch.float16 else "bf16"
+    layers = 32 if ci == 5 else 1
+    appends = ci in (3, 5)
+    n_app = (WARM + TIMED + 8) if appends else 0                    # appended tokens per sequence (FORCED steps + a few COMPUTE ones)
+    tot = ctx + n_app
+    if ci == 1:
+        li = workloads.config(1, device=dev)
+    elif ci == 3:
+        li = workloads.build_layer(2, n_seq=S, ctx=tot, n_q_heads=hq, dtype=dt, device=dev, outlier="pct:1", mode="forced",
+                                   level_probs=(0.10, 0.20, 0.40, 0.30), shuffle_positions=True)
+    elif ci == 4:
+        li = workloads.config(4, device=dev)
+    else:
+        li = workloads.build_layer(4, n_seq=S, ctx=tot, n_q_heads=hq, dtype=dt, device=dev, outlier="pct:1", mode="forced")
+    g = torch.Generator().manual_seed(4)
+    if ci == 5:                                                     # per-layer mix ~ Dirichlet(1, 1, 1, 1) over the four ranks
+        ranks = []
+        for _ in range(layers):
+            ex = -torch.log(torch.rand(4, generator=g))
+            ranks.append(workloads.forced_ranks(int(torch.randint(1 << 30, (1,), generator=g)), S * tot,
+                                                probs=tuple((ex / ex.sum()).tolist()), device=dev).to(torch.int16).contiguous())
+    else:
+        ranks = [li.ranks.to(torch.int16).contiguous()]
+    gate = workloads.gate_params(1, D_KV, dt, device=dev) if appends else None
+    cfg = B.make_config(n_layers=layers, n_q_heads=hq, n_kv_heads=HKV, dtype=dt, out_dtype=torch.float32 if dt == torch.bfloat16 else dt,
+                        max_seqs=S, max_tokens_per_seq=tot)
+    payload = sum(int((-(-r.long() // 64) * 128).sum().item()) for r in ranks) + (8 * S * layers * 4096 if appends else 0)
+    pool = torch.empty(B.twkv_cache_required_bytes(cfg, payload), dtype=torch.uint8, device=dev)
+    cache = B.twkv_cache_create(cfg, pool)
+    idx = torch.arange(S * tot, device=dev).reshape(S, tot)
+    pre = idx[:, :ctx].reshape(-1)
+    sel = lambda t, j: t[j].contiguous()
+    pk, pv, ps, pp = (sel(t, pre) for t in (li.xt_k, li.xt_v, li.seq_ids, li.positions))
+    ev = lambda: torch.cuda.Event(enable_timing=True)
+    pre_ms = []
+    for l in range(layers):
+        if gate:
+            B.twkv_cache_set_layer_params(cache, l, li.Uinv_k, li.Uinv_v, *gate)
+        else:
+            B.twkv_cache_set_layer_params(cache, l, li.Uinv_k, li.Uinv_v)
+        a, b = ev(), ev()
+        a.record()
+        B.twkv_compress(cache, l, pk, pv, ps, pp, None, sel(ranks[l], pre), B.TWKV_GATE_FORCED)
+        b.record()
+        torch.cuda.synchronize()
+        pre_ms.append(a.elapsed_time(b))
+    assert B.twkv_cache_status(cache) == B.TWKV_OK
+    st0 = B.twkv_cache_stats(cache, 0)
+    sid = torch.arange(S, dtype=torch.int32, device=dev)
+    out = torch.empty(S, hq, DH, dtype=torch.float32 if dt == torch.bfloat16 else dt, device=dev)
+    res = {"metric": METRIC, "unit": UNIT, "n_gpus": 1, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": dn,
+           "data": "synthetic", "warmup": WARM, "steps": TIMED,
+           "config": {"workload": shapes["name"], "batch": S, "context": ctx, "n_q_heads": hq, "n_kv_heads": HKV, "head_dim": DH, "layers": layers,
+                      "l2": "cache fits in L2: an L2-resident number, not an HBM one" if ci == 1 else "cache exceeds L2"},
+           "prefill_compress_forced_ms_per_layer": _median_min(pre_ms),
+           "prefill_compress_tokens_per_s": S * ctx / (sorted(pre_ms)[len(pre_ms) // 2] * 1e-3)}
+
+    def timed_loop(body, n_warm, n_timed):
+        for i in range(n_warm):
+            body(i)
+        torch.cuda.synchronize()
+        B.twkv_profile_enable(cache, True)
+        sampler = ClockSampler(0)
+        marks = [(ev(), ev()) for _ in range(n_timed)]
+        launches0 = B.twkv_launch_count()
+        for i in range(n_timed):
+            marks[i][0].record()
+            body(n_warm + i)
+            marks[i][1].record()
+        torch.cuda.synchronize()
+        clocks = sampler.stop()
+        prof = B.twkv_profile_read(cache)
+        B.twkv_profile_enable(cache, False)
+        return [a.elapsed_time(b) for a, b in marks], prof, clocks, B.twkv_launch_count() - launches0
+
+    if not appends:
+        sweep = None
+        if ci == 4:                                               # the split-K sweep of the long-context workload
+            sweep = {}
+            for splits in (1, 2, 4, 8, 16, 32, 64, 128, 256, 0):
+                ms, _, _, _ = timed_loop(lambda i: B.twkv_decode_attn(cache, 0, li.q, sid, out, splits), 3, 20)
+                sweep["auto" if splits == 0 else str(splits)] = _median_min(ms)
+        ms, prof, clocks, launches = timed_loop(lambda i: B.twkv_decode_attn(cache, 0, li.q, sid, out), WARM, TIMED)
+        st = st0
+        n_tok = S * ctx
+        dec = _median_min(ms)
+        res.update({"value": n_tok / (dec["median"] * 1e-3), "ms_per_step": dec["median"], "decode_ms": dec, "clocks": clocks,
+                    "gpu_launches": int(launches), "step": "one decode-attention call over the cache"})
+        res.update(_decode_report(st, n_tok, hq, dec["median"], prof["kscore"][0] / max(1, prof["kscore"][1]), peaks))
+        if sweep:
+            res["decode_ms_by_num_splits"] = sweep
+    else:
+        # the appended tokens of every step, gathered before anything is timed
+        app_x = [tuple(sel(t, idx[:, ctx + s_]) for t in (li.xt_k, li.xt_v, li.seq_ids, li.positions)) for s_ in range(n_app)]
+        app_r = [[sel(ranks[l], idx[:, ctx + s_]) for s_ in range(n_app)] for l in range(layers)]
+        app = lambda s_, l: app_x[s_] + (app_r[l][s_],)
+        dec_ms, app_ms = [], []
+
+        def body(i):
+            a, m, b = ev(), ev(), ev()
+            for l in range(layers):
+                xk, xv, sq, po, lv = app(i, l)
+                if l == 0: a.record()
+                B.twkv_compress(cache, l, xk, xv, sq, po, None, lv, B.TWKV_GATE_FORCED)
+                if l == 0: m.record()
+                B.twkv_decode_attn(cache, l, li.q, sid, out)
+                if l == 0: b.record()
+            body.marks.append((a, m, b))
+        body.marks = []
+        ms, prof, clocks, launches = timed_loop(body, WARM, TIMED)
+        for a, m, b in body.marks[WARM:]:
+            app_ms.append(a.elapsed_time(m)); dec_ms.append(m.elapsed_time(b))
+        assert B.twkv_cache_status(cache) == B.TWKV_OK
+        st = B.twkv_cache_stats(cache, 0)
+        n_tok = int(st.tokens)
+        step, dec, appf = _median_min(ms), _median_min(dec_ms), _median_min(app_ms)
+        res.update({"value": n_tok * layers / (step["median"] * 1e-3) if ci == 5 else n_tok / (dec["median"] * 1e-3),
+                    "ms_per_step": step["median"], "step_ms": step, "decode_ms_layer0": dec, "append_forced_ms_layer0": appf,
+                    "clocks": clocks, "gpu_launches": int(launches),
+                    "step": f"every layer ({layers}): append one token per sequence (FORCED ranks) + decode attention"})
+        if ci == 5:
+            res["attention_ms_per_generated_token"] = step["median"] / S
+            res["ms_per_layer"] = step["median"] / layers
+        ks_ms = prof["kscore"][0] / max(1, prof["kscore"][1])
+        res.update(_decode_report(st, n_tok, hq, dec["median"], ks_ms, peaks))
+        # the append with the gate computed by the library (small-call path: warp-MMA logits GEMM + rank kernel), bound by
+        # reading W_K and W_V (2 x 2 MiB) and the launch chain
+        cms = []
+        for j in range(8):
+            xk, xv, sq, po, _ = app(WARM + TIMED + j, 0)
+            lv = torch.zeros(S, 2, dtype=torch.int16, device=dev)
+            a, b = ev(), ev()
+            a.record()
+            B.twkv_compress(cache, 0, xk, xv, sq, po, None, lv, B.TWKV_GATE_COMPUTE)
+            b.record()
+            torch.cuda.synchronize()
+            cms.append(a.elapsed_time(b))
+        assert B.twkv_cache_status(cache) == B.TWKV_OK
+        cm = _median_min(cms[2:])
+        wbytes = 2.0 * D_KV * D_KV * 2 + 2.0 * S * D_KV * 2
+        res["append_compute_gate_ms_layer0"] = cm
+        res["append_compute_gate_roofline"] = {"kernel": "gate_gemm_kernel + gate_rank_kernel + alloc + pack (one call of %d tokens)" % S,
+                                               "bound": "hbm", "achieved": wbytes / (cm["median"] * 1e-3) / 1e9, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                                               "frac": wbytes / (cm["median"] * 1e-3) / 1e9 / peaks["hbm_gbs"],
+                                               "bytes": "W_K, W_V (2 x 2 MiB) + the call's states; a launch-latency-bound chain of four kernels"}
+    res["retain_rate_k"], res["retain_rate_v"] = st.retain_rate_k, st.retain_rate_v
+    res["bytes_stored_layer0"], res["bytes_algorithmic_layer0"] = st.bytes_stored, st.bytes_algorithmic
+    if not args.skip_cpu_baseline:
+        cap = {1: 1024, 3: 8192, 4: 16384, 5: 16384}[ci]
+        label = {1: "the whole workload", 3: "one sequence, one step", 4: "the first 16384 tokens of the sequence", 5: "one sequence, one layer, one step"}[ci]
+        rk = torch.stack([ranks[0][:, 0], ranks[0][:, 1]], dim=1)
+        res["cpu_baseline"] = _oracle_decode_baseline(li, rk, 0, cap, dn, hq, label, S * ctx * layers)
+    B.twkv_cache_destroy(cache)
+    print(json.dumps(res), flush=True)
+
+
 def main():
     global B_SEQ, CTX, WORKLOAD
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=40)
+    ap.add_argument("--steps", type=int, default=100)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--batch", type=int, default=B_SEQ, help="sequences (default: the benchmark workload's 16)")
     ap.add_argument("--ctx", type=int, default=CTX, help="context length (default: the benchmark workload's 32768)")
+    ap.add_argument("--config", type=int, default=2, choices=[1, 2, 3, 4, 5],
+                    help="which synthetic workload: 2 (default) is the headline 32k-context step, the others print their own line")
     ap.add_argument("--skip-e2e", action="store_true", help="profiling runs: leave the host-buffer leg out")
     ap.add_argument("--skip-cpu-baseline", action="store_true", help="profiling runs: leave the oracle leg out")
+    ap.add_argument("--skip-sustained", action="store_true", help="profiling runs: leave the two-second back-to-back leg out")
     args = ap.parse_args()
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ:
+        # started by hand with --gpus N: launch the N ranks (one per GPU) the way the driver does and hand over
+        import socket
+        with socket.socket() as sk:
+            sk.bind(("127.0.0.1", 0))
+            port = sk.getsockname()[1]
+        cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={args.gpus}", "--master-addr", "127.0.0.1",
+               "--master-port", str(port), os.path.abspath(__file__)] + sys.argv[1:]
+        sys.exit(subprocess.call(cmd))
     if (args.batch, args.ctx) != (B_SEQ, CTX):
         B_SEQ, CTX = args.batch, args.ctx
         WORKLOAD = f"reduced-for-profiling_B{B_SEQ}_ctx{CTX}_gqa4_fp16_gate-assigned-ranks"
     if args.impl == "reference":
         run_reference(args)
+    elif args.config != 2:
+        run_config(args)
     else:
         run_ours(args)
 

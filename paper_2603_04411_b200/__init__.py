@@ -4,9 +4,8 @@
   paper_2603_04411_b200.build      builds libtwkv.so in-tree with nvcc (sm_100a)
   paper_2603_04411_b200.workloads  seeded synthetic inputs
   paper_2603_04411_b200.replicas   barrier / max-over-ranks / whole-job rate for runs on several GPUs (replicas, no data-path collective)
-  paper_2603_04411_b200.config_bench  timings of the other benchmark shapes
 
 The CUDA library is the only implementation: importing `binding` without a built
 libtwkv.so raises.
 """
-__all__ = ["binding", "build", "workloads", "replicas", "config_bench"]
+__all__ = ["binding", "build", "workloads", "replicas"]

@@ -50,3 +50,21 @@ def test_single_rank_is_a_no_op(monkeypatch):
     assert replicas.max_over_ranks([1.5, 2.5]) == [1.5, 2.5]
     assert replicas.whole_job_rate(10.0, 5.0) == 10.0 / 5.0e-3
     replicas.finish()
+
+
+def test_bench_spawns_its_ranks_when_started_by_hand():
+    # `python bench.py --gpus 2` without a launcher's environment starts the two ranks itself; here through the
+    # reference arm (the CPU oracle), whose rank 0 prints the line and whose other ranks leave without work
+    import json
+    import subprocess
+    import sys
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    env = {k: v for k, v in os.environ.items() if k not in ("WORLD_SIZE", "RANK", "LOCAL_RANK", "MASTER_ADDR", "MASTER_PORT")}
+    r = subprocess.run([sys.executable, os.path.join(root, "bench.py"), "--gpus", "2", "--impl", "reference", "--steps", "1", "--warmup", "0"],
+                       capture_output=True, text=True, timeout=600, env=env, cwd=root)
+    assert r.returncode == 0, r.stderr[-2000:]
+    lines = [json.loads(l) for l in r.stdout.splitlines() if l.startswith("{")]
+    assert len(lines) == 1
+    line = lines[0]
+    assert line["impl"] == "reference" and line["n_gpus"] == 2 and line["metric"] == "decode_attn_kv_tokens_per_s"
+    assert line["unit"] == line["e2e"]["unit"] == "KV tokens/s" and line["value"] > 0
