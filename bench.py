@@ -336,8 +336,8 @@ def run_ours(args):
         # DRAM bytes per launch from the ncu captures summarised under profiles/ (reduced cases, scaled by tokens processed)
         scale = n_tok / (16 * 32768.0)
         rl_gate = tensor_roofline("gate_tc2_kernel (tcgen05 on CTA pairs: gate logits GEMM + softmax/prefix-sum/threshold rank)", flops_g, gg_avg_ms,
-                                  (146.2e6 + 68.4e6) * 16 * scale)
-        rl_ks = tensor_roofline("kscore_tc_kernel (tcgen05: K reconstruct + RoPE + q.K scores)", flops_k, ks_avg_ms, (82.9e6 + 4.1e6) * 4 * scale)
+                                  (572.4e6 + 361.3e6) * 4 * scale)
+        rl_ks = tensor_roofline("kscore_tc_kernel (tcgen05 on CTA pairs: K reconstruct + RoPE + q.K scores)", flops_k, ks_avg_ms, (83.9e6 + 4.1e6) * 4 * scale)
         roofline = rl_gate if gg_ms >= ks_ms else rl_ks
         roofline_decode = rl_ks
         va_ms, va_n = prof["vacc"]

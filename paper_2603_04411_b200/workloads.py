@@ -90,8 +90,11 @@ def pca_basis(x_calib: torch.Tensor) -> torch.Tensor:
     return v[:, order].contiguous()
 
 
-def project_states(x: torch.Tensor, U: torch.Tensor, dtype, chunk=65536) -> torch.Tensor:
-    """x~ = round16(x U): the spectral states handed to the library."""
+def synthetic_spectral_states(x: torch.Tensor, U: torch.Tensor, dtype, chunk=65536) -> torch.Tensor:
+    """Draws the spectral states the library's boundary takes: the raw draw expressed in the calibration basis and
+    rounded to the storage type.  This only gives the synthetic input its spectrum (energy concentrated in the leading
+    components, like states seen through a PCA basis); it is not the library's or the oracle's Eq. 1, which are
+    twkv_project and oracle.project + narrow16 and are tested against each other on raw states."""
     out = torch.empty(x.shape[0], U.shape[1], dtype=dtype, device=x.device)
     Ud = U.to(device=x.device, dtype=torch.float32)
     for lo in range(0, x.shape[0], chunk):
@@ -172,8 +175,8 @@ def build_layer(seed: int, *, n_seq: int, ctx: int, n_q_heads: int, n_kv_heads: 
     U_v = pca_basis(cv)
     del ck, cv
     xk, xv = raw_states(seed + 2, n_tok, d_kv, device=device, k_outliers=ch, heavy_tail=heavy)
-    xt_k = project_states(xk, U_k, dtype)
-    xt_v = project_states(xv, U_v, dtype)
+    xt_k = synthetic_spectral_states(xk, U_k, dtype)
+    xt_v = synthetic_spectral_states(xv, U_v, dtype)
     Uinv_k = U_k.T.contiguous().to(dtype).to(device)      # orthogonal basis: U^-1 = U^T
     Uinv_v = U_v.T.contiguous().to(dtype).to(device)
     g = _gen(seed + 3, "cpu")
