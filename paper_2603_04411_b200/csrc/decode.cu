@@ -26,8 +26,8 @@ __device__ __forceinline__ unsigned ktile_cost(int cls) {
   // cycles per tile of the K-score kernel by rank class, measured inside the kernel on the benchmark's mix of classes
   // (8 KV heads, CTA pairs): a fixed part (rotation factors, the per-slab epilogue and score products) plus a per-panel
   // part; classes above 8 run as two passes.  Only the ratios matter.
-  constexpr unsigned kCost[TWKV_MAX_CLASSES] = {16200u, 17900u, 19100u, 20300u, 22100u, 24200u, 26100u, 27600u,
-                                                42900u, 42900u, 43400u, 45300u, 47300u, 49500u, 51800u, 55300u};
+  constexpr unsigned kCost[TWKV_MAX_CLASSES] = {16300u, 17800u, 18900u, 19500u, 20900u, 21900u, 23900u, 24300u,
+                                                39800u, 39800u, 40700u, 41100u, 42400u, 42900u, 45000u, 46700u};
   return kCost[min(max(cls, 1), TWKV_MAX_CLASSES) - 1];
 }
 

@@ -92,13 +92,17 @@ constexpr int KE_DISCARD = 0x80;                               // list entry, .y
 // Barriers: a_full / b_full / kr_full / slab_empty / s_empty live in the even CTA (the odd CTA's copies complete on
 // them and its epilogue warps arrive on them through the cluster window); a_empty / b_empty / slab_full / s_full exist in
 // both and are signalled together by a multicast tcgen05.commit (a commit, not a load).
-template <bool BF16, int REP, bool PAIR>
+// DBG (caches created with TWKV_DEBUG=1): rotated keys that the f16 conversion clamps are reported.
+template <bool BF16, int REP, bool PAIR, bool DBG>
 __global__ void __launch_bounds__(KT_THREADS, 1)
 kscore_tc_kernel(const __grid_constant__ CUtensorMap map_blocks, const __grid_constant__ CUtensorMap map_uinvT,
                  DevView v, int layer, const unsigned short* __restrict__ q, int nb) {
   extern __shared__ __align__(1024) unsigned char smem_raw[];
   constexpr int CG = PAIR ? 2 : 1;
-  constexpr uint32_t B_STAGE_BYTES = PAIR ? PANEL_BYTES / 2 : PANEL_BYTES;
+  // a ring stage of U_K^-1 holds two consecutive panels of one KV head (their halves in a pair CTA): one barrier wait
+  // and one commit per eight MMAs keeps the issuing thread's own instructions below the tensor pipe's time
+  constexpr uint32_t B_PART_BYTES = PAIR ? PANEL_BYTES / 2 : PANEL_BYTES;
+  constexpr uint32_t B_STAGE_BYTES = 2 * B_PART_BYTES;
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int Hq = v.Hq, Hkv = v.Hkv;
   const uint32_t crank = PAIR ? cluster_cta_rank() : 0u;
@@ -202,14 +206,17 @@ kscore_tc_kernel(const __grid_constant__ CUtensorMap map_blocks, const __grid_co
           const int np = min(KT_A_SLOTS, cls - p0);
           for (int sl = 0; sl < Hkv && ok; ++sl) {
             const int g = sl + g_rot < Hkv ? sl + g_rot : sl + g_rot - Hkv;
-            for (int j = 0; j < np; ++j, ++bk) {
+            for (int j = 0; j < np; j += 2, ++bk) {
               const uint32_t st = bst, ph = bph;
               if (++bst == (uint32_t)nb) { bst = 0; bph ^= 1u; }
               if (!(ok = mbar_wait_thin(b_empty + 8 * st, ph ^ 1u, abort_flag))) break;
-              const int y = ((p0 + j) * Hkv + g) * HEAD_DIM + (PAIR ? (int)crank * (HEAD_DIM / 2) : 0);     // rows of the re-tiled copy
-              if (crank == 0) mbar_expect_tx(b_full + 8 * st, CG * B_STAGE_BYTES);
-              if constexpr (PAIR) tma_load_2d_pair(sB + st * B_STAGE_BYTES, &map_uinvT, b_full_own + 8 * st, 0, y);
-              else tma_load_2d(sB + st * B_STAGE_BYTES, &map_uinvT, b_full + 8 * st, 0, y);
+              const int npan = min(2, np - j);
+              if (crank == 0) mbar_expect_tx(b_full + 8 * st, CG * npan * B_PART_BYTES);
+              for (int k = 0; k < npan; ++k) {
+                const int y = ((p0 + j + k) * Hkv + g) * HEAD_DIM + (PAIR ? (int)crank * (HEAD_DIM / 2) : 0);     // rows of the re-tiled copy
+                if constexpr (PAIR) tma_load_2d_pair(sB + st * B_STAGE_BYTES + k * B_PART_BYTES, &map_uinvT, b_full_own + 8 * st, 0, y);
+                else tma_load_2d(sB + st * B_STAGE_BYTES + k * B_PART_BYTES, &map_uinvT, b_full + 8 * st, 0, y);
+              }
             }
           }
         }
@@ -245,17 +252,27 @@ kscore_tc_kernel(const __grid_constant__ CUtensorMap map_blocks, const __grid_co
             const uint32_t d = tmem_base + TM_SLAB + sbuf * 128;
             const bool first = sl == 0, last = sl == Hkv - 1;
             uint32_t an = ak;
-            for (int j = 0; j < np; ++j, ++an) {
-              const uint32_t slot = an & (KT_A_SLOTS - 1);
-              if (first && !(ok = mbar_wait_thin(a_full + 8 * slot, (an >> 3) & 1u, abort_flag))) break;
+            for (int j = 0; j < np; j += 2, an += 2) {
+              const bool two = j + 1 < np;
+              const uint32_t slot = an & (KT_A_SLOTS - 1), slot2 = (an + 1) & (KT_A_SLOTS - 1);
+              if (first) {
+                if (!(ok = mbar_wait_thin(a_full + 8 * slot, (an >> 3) & 1u, abort_flag))) break;
+                if (two && !(ok = mbar_wait_thin(a_full + 8 * slot2, ((an + 1) >> 3) & 1u, abort_flag))) break;
+              }
               const uint32_t st = bst;
               if (!(ok = mbar_wait_thin(b_full + 8 * st, bph, abort_flag))) break;
               if (++bst == (uint32_t)nb) { bst = 0; bph ^= 1u; }
               fence_after_sync();
               mma_f16_ss_panel_cg<CG>(d, a_lo0 + slot * (PANEL_BYTES >> 4), b_lo0 + st * (B_STAGE_BYTES >> 4), idesc_main, j > 0 ? 1u : 0u);
-              // ring stage reusable when these MMAs retire; after the last slab of the pass the X^_K panel is done too
-              if constexpr (PAIR) { mma_commit_pair_both(b_empty + 8 * st); if (last) mma_commit_pair_both(a_empty + 8 * slot); }
-              else { mma_commit(b_empty + 8 * st); if (last) mma_commit(a_empty + 8 * slot); }
+              if (two) mma_f16_ss_panel_cg<CG>(d, a_lo0 + slot2 * (PANEL_BYTES >> 4), b_lo0 + st * (B_STAGE_BYTES >> 4) + (B_PART_BYTES >> 4), idesc_main, 1u);
+              // ring stage reusable when these MMAs retire; after the last slab of the pass the X^_K panels are done too
+              if constexpr (PAIR) {
+                mma_commit_pair_both(b_empty + 8 * st);
+                if (last) { mma_commit_pair_both(a_empty + 8 * slot); if (two) mma_commit_pair_both(a_empty + 8 * slot2); }
+              } else {
+                mma_commit(b_empty + 8 * st);
+                if (last) { mma_commit(a_empty + 8 * slot); if (two) mma_commit(a_empty + 8 * slot2); }
+              }
             }
             if (!ok) break;
             if constexpr (PAIR) mma_commit_pair_both(slab_full + 8 * sbuf);     // slab accumulator complete
@@ -485,7 +502,7 @@ kscore_tc_kernel(const __grid_constant__ CUtensorMap map_blocks, const __grid_co
               ol[u] = f2_to_f16x2_sat(f2_sub(a, ah));
               ol[4 + u] = f2_to_f16x2_sat(f2_sub(b, bh));
             }
-            if (v.debug) {
+            if constexpr (DBG) {
               // TWKV_DEBUG: a rotated key beyond the f16 range was clamped by the conversion above (its high part reads
               // 0x7bff); without the flag that goes unreported
               bool sat = false;
@@ -590,12 +607,12 @@ size_t kscore_tc_smem_bytes(int nb, size_t stage_bytes) {
   return (size_t)KT_A_SLOTS * PANEL_BYTES + (size_t)nb * stage_bytes + 2 * KT_Q_PANEL_BYTES + KT_ROPE_STAGE_BYTES + 8 * (KT_N_BARS + 2 * nb) +
          2 * sizeof(int);
 }
-constexpr int KT_NB_SINGLE = 4, KT_NB_PAIR = 8;                // ring stages of U_K^-1 panels (16 KiB) / half panels (8 KiB)
+constexpr int KT_NB_SINGLE = 2, KT_NB_PAIR = 4;                // ring stages of two U_K^-1 panels (32 KiB) / two half panels (16 KiB)
 
 // CTA pairs of the pair kernel that can be resident at once on the current device (0: it cannot run).
 static int kscore_query_pairs(int sm_count) {
-  const size_t smem = kscore_tc_smem_bytes(KT_NB_PAIR, PANEL_BYTES / 2);
-  if (cudaFuncSetAttribute(kscore_tc_kernel<false, 4, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) { cudaGetLastError(); return 0; }
+  const size_t smem = kscore_tc_smem_bytes(KT_NB_PAIR, PANEL_BYTES);
+  if (cudaFuncSetAttribute(kscore_tc_kernel<false, 4, true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) { cudaGetLastError(); return 0; }
   cudaLaunchConfig_t cfg = {};
   cfg.blockDim = dim3(KT_THREADS);
   cfg.dynamicSmemBytes = smem;
@@ -606,7 +623,7 @@ static int kscore_query_pairs(int sm_count) {
   cfg.attrs = &pair_attr;
   cfg.numAttrs = 1;
   int n = 0;
-  if (cudaOccupancyMaxActiveClusters(&n, kscore_tc_kernel<false, 4, true>, &cfg) != cudaSuccess || n < 1) { cudaGetLastError(); n = 0; }
+  if (cudaOccupancyMaxActiveClusters(&n, kscore_tc_kernel<false, 4, true, false>, &cfg) != cudaSuccess || n < 1) { cudaGetLastError(); n = 0; }
   return n;
 }
 int kscore_max_pairs(int sm_count) {
@@ -614,11 +631,11 @@ int kscore_max_pairs(int sm_count) {
   return cached;
 }
 
-template <bool BF16, bool PAIR>
+template <bool BF16, bool PAIR, bool DBG>
 static cudaError_t launch_kscore_tc_t(const DevView& v, int layer, const CUtensorMap& map_blocks, const CUtensorMap& map_uinvT,
                                       const void* q, int n_pieces, cudaStream_t st) {
   const int nb = PAIR ? KT_NB_PAIR : KT_NB_SINGLE;
-  const size_t smem = kscore_tc_smem_bytes(nb, PAIR ? PANEL_BYTES / 2 : PANEL_BYTES);
+  const size_t smem = kscore_tc_smem_bytes(nb, PAIR ? PANEL_BYTES : 2 * PANEL_BYTES);
   const unsigned short* qq = reinterpret_cast<const unsigned short*>(q);
   cudaLaunchConfig_t cfg = {};
   cfg.blockDim = dim3(KT_THREADS);
@@ -634,9 +651,9 @@ static cudaError_t launch_kscore_tc_t(const DevView& v, int layer, const CUtenso
   cudaError_t e = cudaSuccess;
 #define TWKV_KT(REP)                                                                                                  \
   {                                                                                                                   \
-    e = cudaFuncSetAttribute(kscore_tc_kernel<BF16, REP, PAIR>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem); \
+    e = cudaFuncSetAttribute(kscore_tc_kernel<BF16, REP, PAIR, DBG>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem); \
     if (e != cudaSuccess) return e;                                                                                   \
-    e = cudaLaunchKernelEx(&cfg, kscore_tc_kernel<BF16, REP, PAIR>, map_blocks, map_uinvT, v, layer, qq, nb);        \
+    e = cudaLaunchKernelEx(&cfg, kscore_tc_kernel<BF16, REP, PAIR, DBG>, map_blocks, map_uinvT, v, layer, qq, nb);        \
   }
   switch (v.rep) {
     case 1: TWKV_KT(1) break;
@@ -652,11 +669,12 @@ static cudaError_t launch_kscore_tc_t(const DevView& v, int layer, const CUtenso
 // `pairs`: run on CTA pairs (n_pieces pairs, map_uinvT with 64-row boxes) instead of single CTAs (128-row boxes).
 cudaError_t launch_kscore_tc(const DevView& v, int layer, const CUtensorMap& map_blocks, const CUtensorMap& map_uinvT,
                              const void* q, int n_pieces, bool pairs, cudaStream_t st) {
-  if (pairs)
-    return v.dtype == TWKV_BF16 ? launch_kscore_tc_t<true, true>(v, layer, map_blocks, map_uinvT, q, n_pieces, st)
-                                : launch_kscore_tc_t<false, true>(v, layer, map_blocks, map_uinvT, q, n_pieces, st);
-  return v.dtype == TWKV_BF16 ? launch_kscore_tc_t<true, false>(v, layer, map_blocks, map_uinvT, q, n_pieces, st)
-                              : launch_kscore_tc_t<false, false>(v, layer, map_blocks, map_uinvT, q, n_pieces, st);
+#define TWKV_KS_LAUNCH(BF, PR)                                                                                  \
+  (v.debug ? launch_kscore_tc_t<BF, PR, true>(v, layer, map_blocks, map_uinvT, q, n_pieces, st)                 \
+           : launch_kscore_tc_t<BF, PR, false>(v, layer, map_blocks, map_uinvT, q, n_pieces, st))
+  if (pairs) return v.dtype == TWKV_BF16 ? TWKV_KS_LAUNCH(true, true) : TWKV_KS_LAUNCH(false, true);
+  return v.dtype == TWKV_BF16 ? TWKV_KS_LAUNCH(true, false) : TWKV_KS_LAUNCH(false, false);
+#undef TWKV_KS_LAUNCH
 }
 
 }  // namespace twkv
