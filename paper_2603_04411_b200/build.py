@@ -7,7 +7,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 INCLUDE = os.path.join(os.path.dirname(HERE), "include")
 LIB = os.path.join(HERE, "libtwkv.so")
-SOURCES = ["api.cu", "compress.cu", "gate_gemm.cu", "decode.cu", "kscore_tc.cu", "gate_tc.cu", "gate_static.cu", "gate_soft.cu", "evict.cu", "selfcheck.cu", "project_tc.cu", "project_api.cu"]
+SOURCES = ["api.cu", "compress.cu", "gate_gemm.cu", "decode.cu", "kscore_tc.cu", "vacc_tc.cu", "gate_tc.cu", "gate_static.cu", "gate_soft.cu", "evict.cu", "selfcheck.cu", "project_tc.cu", "project_api.cu"]
 
 
 def _stale() -> bool:

@@ -70,6 +70,7 @@ struct DevView {
                              //            a class with an odd number of tiles ends with a filler entry (.y bit 7 set)
   int* klist_count;          // [1]
   int* cta_start;            // [MAX_PLAN_CTAS + 1]  first list entry of every K-score CTA
+  int* vcut;                 // [query slots][n_splits + 1]  cut points of every sequence's V tile list into the splits of the V pass
   float* part_acc;           // [max_partials][Hq][d_kv]
   float* part_l;             // [max_partials][Hq]
   int4* gate_fix;            // rows the fused gate kernel hands to its fix-up kernel
@@ -111,6 +112,21 @@ __device__ inline float dec_ordered(unsigned u) {
 }
 
 __device__ inline void set_status(const DevView& v, int code) { atomicCAS(v.status, 0, code); }
+
+// The V pass walks a sequence's n V tiles in the order j -> (j * vtile_stride(n)) mod n: a stride near n / golden ratio,
+// coprime to n, so that any run of consecutive j is spread evenly over the list.  Tiles of one class sit together in the
+// list when a context was compressed in one call; a split that took a contiguous piece of the list itself would be all
+// narrow or all wide tiles, and the narrow ones cost more per byte.
+__device__ inline int vtile_stride(int n) {
+  if (n < 3) return 1;
+  int s = (int)(((long long)n * 618034ll) / 1000000ll);
+  if (s < 1) s = 1;
+  for (;; ++s) {
+    int a = s, b = n;
+    while (b) { const int t = a % b; a = b; b = t; }
+    if (a == 1) return s;
+  }
+}
 
 // Makes `dev` the current device for the scope of a host call.
 struct DeviceGuard {
