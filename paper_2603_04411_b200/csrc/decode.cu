@@ -23,11 +23,11 @@ namespace twkv {
 // is rewritten as items of two tiles of one class.  The list is then cut into n_cta contiguous pieces of
 // about equal estimated cost, so a CTA (pair) of the K-score kernel mostly stays inside one (class, sequence) run.
 __device__ __forceinline__ unsigned ktile_cost(int cls) {
-  // cycles per tile of the K-score kernel by rank class, measured inside the kernel on the benchmark's mix of classes
-  // (8 KV heads, CTA pairs): a fixed part (rotation factors, the per-slab epilogue and score products) plus a per-panel
-  // part; classes above 8 run as two passes.  Only the ratios matter.
-  constexpr unsigned kCost[TWKV_MAX_CLASSES] = {16300u, 17800u, 18900u, 19500u, 20900u, 21900u, 23900u, 24300u,
-                                                39800u, 39800u, 40700u, 41100u, 42400u, 42900u, 45000u, 46700u};
+  // cycles per tile of the K-score kernel by rank class: a least-squares fit of every CTA's busy time to its tile counts on
+  // the benchmark's mix of classes (8 KV heads, CTA pairs): a fixed part (rotation factors, the per-slab epilogue and
+  // score products) plus a per-panel part; classes above 8 run as two passes.  Only the ratios matter.
+  constexpr unsigned kCost[TWKV_MAX_CLASSES] = {14400u, 16200u, 18000u, 19700u, 21500u, 23300u, 25000u, 26800u,
+                                                37600u, 39400u, 41200u, 43000u, 44900u, 46700u, 48500u, 50300u};
   return kCost[min(max(cls, 1), TWKV_MAX_CLASSES) - 1];
 }
 

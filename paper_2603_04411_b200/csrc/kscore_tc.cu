@@ -13,18 +13,22 @@
 // fp32 columns become 32 columns of high parts and 32 of low parts), from where they are the A operands of the second
 // product (N = 16, the group's heads padded; one product per part).  The order of the 128 dimensions along the
 // contraction is whatever that in-place layout gives; the query operand is written in the same order.
-// Each slab's scores land in one of four 16-column accumulators and are read out by the epilogue warps two slabs
-// later (scaled, masked, stored, folded into the per-(sequence, head) maximum), so that a tile has no tail:
-// RoPE is the only per-element CUDA-core work.  Both products are linear in X^_K, so a class wider than 8 panels runs
-// as two passes over its panels; the second pass adds to the scores the first one stored.
+// Each slab's scores land in one of four 16-column accumulators and are read out by four warps of their own (scaled,
+// masked, stored, folded into the per-(sequence, head) maximum), so that the rotating warps never wait for a score
+// product and a tile has no tail: RoPE and the high / low split are the only per-element CUDA-core work.  Both products
+// are linear in X^_K, so a class wider than 8 panels runs as two passes over its panels; the second pass adds to the
+// scores the first one stored.
 //
 // Tensor memory (512 columns): slabs 3 x 128 | score accumulators 4 x 16.
-// Warp roles (384 threads, one persistent CTA per SM working through a contiguous, cost-balanced piece of the tile list):
+// Warp roles (512 threads, one persistent CTA per SM working through a contiguous, cost-balanced piece of the tile list;
+// the register file is re-divided by warpgroup with setmaxnreg: 56 registers per thread for the light roles, 184 for the
+// rotating warps, which then hold a slab's registers without spilling):
 //   warp 0      TMA producer of U_K^-1 panels (ring; one elected lane)
 //   warp 1      issuer of the main products (one elected lane; owns the TMEM allocation)
-//   warps 2-9   epilogue (thread = one token row x one half of the RoPE frequencies)
-//   warp 10     TMA producer of X^_K panels (ring of 8 slots; one elected lane, runs ahead into the next tiles)
-//   warp 11     issuer of the score products (one elected lane)
+//   warp 2      TMA producer of X^_K panels (ring of 8 slots; one elected lane, runs ahead into the next tiles)
+//   warp 3      issuer of the score products (one elected lane)
+//   warps 4-11  epilogue (thread = one token row x one half of the RoPE frequencies): rotation, high / low split
+//   warps 12-15 score read-out (thread = one token row)
 // A slab buffer goes round: main products (slab_full) -> epilogue (kr_full) -> score products (slab_empty).
 // All waits are bounded (tc_util.cuh); a wait that runs out ends the kernel with TWKV_ERR_TIMEOUT.
 //
@@ -37,8 +41,9 @@
 namespace twkv {
 using namespace tc;
 
-constexpr int KT_THREADS = 384;
+constexpr int KT_THREADS = 512;
 constexpr int KT_EPI = 256;
+constexpr int KT_REGS_LIGHT = 56, KT_REGS_EPI = 184;         // registers per thread after the roles re-divide the register file
 constexpr int KT_A_SLOTS = 8;                                  // power of two (slot = panel count & 7, phase = bit 3)
 constexpr int KT_SLABS = 3;                                    // slab buffers
 constexpr int KT_S_SLOTS = 4;                                  // score accumulators
@@ -68,19 +73,15 @@ __device__ __forceinline__ unsigned warp_max_u32(unsigned x) {
   return r;
 }
 
+__device__ __forceinline__ void regs_shrink() { asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(KT_REGS_LIGHT)); }
+__device__ __forceinline__ void regs_grow() { asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(KT_REGS_EPI)); }
+
 template <bool BF16> __device__ __forceinline__ float kt_to_f32(unsigned short bits) {
   if constexpr (BF16) return __uint_as_float((unsigned)bits << 16);
   else return __half2float(__ushort_as_half(bits));
 }
 
-// A score read-out that is still owed: which accumulator, where the scores go, how they combine.
-struct KtPending {
-  float* out;            // this thread's row of the score scratch, at the group's first head
-  int mxi;               // which of the reading thread's running maxima the scores fold into (slab index / 2)
-  uint32_t meta;         // bit 0 valid | bit 1 reader half | bits 2-3 mode | bits 4-5 accumulator | bit 6 its parity | bit 7 row is a token
-};
-constexpr uint32_t KP_VALID = 1u, KP_LIVE = 128u;
-constexpr uint32_t KP_STORE_PART = 0u, KP_STORE_FINAL = 1u, KP_ADD_FINAL = 2u, KP_DISCARD = 3u;      // modes
+constexpr uint32_t KP_STORE_PART = 0u, KP_STORE_FINAL = 1u, KP_ADD_FINAL = 2u, KP_DISCARD = 3u;      // what a read-out does with a slab's scores
 constexpr int KE_DISCARD = 0x80;                               // list entry, .y bit 7: a filler tile whose scores are not kept
 
 // PAIR: the kernel runs on CTA pairs (clusters of two, cta_group::2).  The two CTAs take two tiles of the same class
@@ -131,7 +132,7 @@ kscore_tc_kernel(const __grid_constant__ CUtensorMap map_blocks, const __grid_co
     for (int i = 0; i < KT_SLABS; ++i) {
       mbar_init(slab_full + 8 * i, 1); mbar_init(kr_full + 8 * i, CG * (KT_EPI / 32)); mbar_init(slab_empty + 8 * i, 1);
     }
-    for (int i = 0; i < KT_S_SLOTS; ++i) { mbar_init(s_full + 8 * i, 1); mbar_init(s_empty + 8 * i, CG * (KT_EPI / 64)); }
+    for (int i = 0; i < KT_S_SLOTS; ++i) { mbar_init(s_full + 8 * i, 1); mbar_init(s_empty + 8 * i, CG * 4); }
     *abort_flag = misaligned ? 1 : 0;
     mbar_init_fence();
   }
@@ -162,7 +163,9 @@ kscore_tc_kernel(const __grid_constant__ CUtensorMap map_blocks, const __grid_co
 
   if (misaligned) {
     // nothing was started; fall through to the common exit
-  } else if (warp == 10) {
+  } else if (warp < 4) {
+    regs_shrink();                                              // the register file is re-divided by role, whole warpgroups at a time
+    if (warp == 2) {
     // ------------------------------------------------------------- TMA producer: X^_K panels
     // One elected thread issues every copy, in ring order (slots free up in that order, so waiting for the oldest one
     // never holds back a copy that could go out), and runs ahead into the next tiles.  Only a thread picked by
@@ -285,7 +288,7 @@ kscore_tc_kernel(const __grid_constant__ CUtensorMap map_blocks, const __grid_co
       }
     }
     __syncwarp();
-  } else if (warp == 11) {
+  } else if (warp == 3) {
     // ------------------------------------------------------------- score-product issuer (one elected lane)
     // S (+)= Krot_g . Q_g^T as soon as the epilogue warps have stored a rotated slab; a thread of its own, so that
     // neither issue stream waits for the other's barriers
@@ -318,25 +321,19 @@ kscore_tc_kernel(const __grid_constant__ CUtensorMap map_blocks, const __grid_co
       }
     }
     __syncwarp();
-  } else if (warp >= 2 && warp <= 9) {
+    }
+  } else if (warp >= 4 && warp <= 11) {
+    regs_grow();                                                // the rotating warps take what the light roles gave up
     // ------------------------------------------------------------- epilogue
-    const int et = tid - 64;
-    const int quarter = warp & 3, hf = (warp - 2) >> 2;
+    const int et = tid - 128;
+    const int quarter = warp & 3, hf = (warp - 4) >> 2;
     const int row = quarter * 32 + lane;
     const uint32_t lane_addr = tmem_base + ((uint32_t)(quarter * 32) << 16);
-    const uint32_t s_col0 = TM_S + (PAIR ? 8u * crank : 0u);     // this CTA's columns of a score accumulator
-    const float sm_scale = v.sm_scale;
     const int* kpos = v.aux(layer, 0);
     const float4* __restrict__ rope_hi = v.rope_hi;
     uint32_t sbuf = 0, sph = 0, slot = 0, slph = 0;
     bool ok = true;
     uint64_t cs2[16], sn2[16];                                    // the tile's rotation factors, frequencies (2 t, 2 t + 1) packed
-    float tmax[4][REP];                                           // running maxima of the heads this thread reads out (slab index / 2)
-#pragma unroll
-    for (int a = 0; a < 4; ++a)
-#pragma unroll
-      for (int i = 0; i < REP; ++i) tmax[a][i] = -INFINITY;
-
     // cos / sin of (row, frequency): pos = hi * 16 + lo, the two table rows combine by the angle-addition formulas.
     // The lo row comes from shared memory (padded rows: lanes with different rows hit different banks), the hi row
     // from global memory (L2; neighbouring positions share it).
@@ -382,92 +379,18 @@ kscore_tc_kernel(const __grid_constant__ CUtensorMap map_blocks, const __grid_co
       }
       fence_proxy_async_smem();
     };
-    // Scores of one slab: REP columns of its accumulator, scaled, rows past the tile's last token masked; the reading
-    // half of the epilogue warps alternates from slab to slab.
-    auto read_out = [&](const KtPending& p) -> bool {
-      if (!(p.meta & KP_VALID) || (int)((p.meta >> 1) & 1u) != hf) return true;       // uniform over the warp
-      const uint32_t sl_ = (p.meta >> 4) & 3u, par = (p.meta >> 6) & 1u, mode = (p.meta >> 2) & 3u;
-      if (!__all_sync(0xffffffffu, mbar_wait(s_full + 8 * sl_, par, abort_flag))) return false;
-      fence_after_sync();
-      float sv[REP];
-      {
-        uint32_t* dst = reinterpret_cast<uint32_t*>(sv);
-        const uint32_t src = lane_addr + s_col0 + 16 * sl_;
-        if constexpr (REP == 1) tmem_ld1(src, dst);
-        else if constexpr (REP == 2) tmem_ld2(src, dst);
-        else if constexpr (REP == 4) tmem_ld4(src, dst);
-        else tmem_ld8(src, dst);
-      }
-      tmem_ld_wait();
-      fence_before_sync();
-      __syncwarp();
-      if (lane == 0) {
-        if constexpr (PAIR) mbar_arrive_cluster(s_empty_own + 8 * sl_);
-        else mbar_arrive(s_empty + 8 * sl_);
-      }
-      if (mode == KP_DISCARD) return true;
-      const bool live = (p.meta & KP_LIVE) != 0;
-      float* out = p.out;
-#pragma unroll
-      for (int i = 0; i < REP; ++i) {
-        float x = sv[i] * sm_scale;
-        if (mode == KP_ADD_FINAL) x += out[i];                                       // the first pass stored its part
-        sv[i] = live ? x : -INFINITY;
-      }
-      if constexpr (REP >= 4) {
-#pragma unroll
-        for (int i = 0; i < REP; i += 4) *reinterpret_cast<float4*>(out + i) = make_float4(sv[i], sv[i + 1], sv[i + 2], sv[i + 3]);
-      } else {
-#pragma unroll
-        for (int i = 0; i < REP; ++i) out[i] = sv[i];
-      }
-      if (mode != KP_STORE_PART) {
-        const int a_ = p.mxi;                                                        // slab index / 2: which maxima
-#pragma unroll
-        for (int a = 0; a < 4; ++a)
-#pragma unroll
-          for (int i = 0; i < REP; ++i) tmax[a][i] = a == a_ ? fmaxf(tmax[a][i], sv[i]) : tmax[a][i];
-      }
-      return true;
-    };
-    // Folds this thread's running maxima into the per-(sequence, head) maximum: over the warp's rows first, then one
-    // atomic per head (max is order-independent, so the result is deterministic).
-    auto flush_max = [&](int qs) {
-#pragma unroll
-      for (int a = 0; a < 4; ++a) {
-        const int sli = 2 * a + hf;
-        if (sli < Hkv) {
-          const int g = sli + g_rot < Hkv ? sli + g_rot : sli + g_rot - Hkv;
-          unsigned mine = 0u;
-#pragma unroll
-          for (int i = 0; i < REP; ++i) {
-            const unsigned m = warp_max_u32(enc_ordered(tmax[a][i]));
-            if (lane == i) mine = m;
-            tmax[a][i] = -INFINITY;
-          }
-          if (lane < REP) atomicMax(&v.seqmax[qs * Hq + g * REP + lane], mine);
-        }
-      }
-    };
-
-    KtPending p_old{nullptr, 0, 0u}, p_new{nullptr, 0, 0u};
+    uint32_t last_slot = 0, last_slph = 0;                          // score accumulator of the slab rotated last, and its phase
     int4 e = w0 < total ? klist[KSTEP * w0] : kt_none;
     int pos_cur = w0 < total ? kpos[(size_t)e.x * TILE + row] : 0;              // this row's position in the current tile
     if (w0 < total) { write_q(e.w); rope_setup(pos_cur); }
     for (int w = w0; w < total && ok; ++w) {
       const int4 nxt = w + 1 < total ? klist[KSTEP * (w + 1)] : kt_none;
-      const int tile = e.x, cls = e.y & 0x7f, n_valid = e.y >> 8, qs = e.w;
-      const bool discard = (e.y & KE_DISCARD) != 0;
+      const int cls = e.y & 0x7f, qs = e.w;
+      [[maybe_unused]] const int n_valid = e.y >> 8;
       const int passes = (cls + KT_A_SLOTS - 1) / KT_A_SLOTS;
       const int pos_next = nxt.w >= 0 ? kpos[(size_t)nxt.x * TILE + row] : 0;      // fetched now, used after the tile's slabs
-      float* const out_row = v.scores + ((size_t)tile * TILE + row) * Hq;
-      // a row counts if it holds a token and, for a causal (prefill) query, the token is not after the query
-      const int pos_limit = v.qpos ? v.qpos[qs] : 0x7fffffff;
-      const uint32_t live_bit = (row < n_valid && pos_cur <= pos_limit) ? KP_LIVE : 0u;
       for (int ps = 0; ps < passes && ok; ++ps) {
-        const uint32_t mode = discard ? KP_DISCARD : passes == 1 ? KP_STORE_FINAL : (ps == 0 ? KP_STORE_PART : KP_ADD_FINAL);
         for (int sli = 0; sli < Hkv; ++sli) {
-          const int g = sli + g_rot < Hkv ? sli + g_rot : sli + g_rot - Hkv;
           if (!(ok = __all_sync(0xffffffffu, mbar_wait(slab_full + 8 * sbuf, sph, abort_flag)))) break;
           fence_after_sync();
           const uint32_t sl_addr = lane_addr + TM_SLAB + sbuf * 128 + hf * 32;
@@ -476,7 +399,6 @@ kscore_tc_kernel(const __grid_constant__ CUtensorMap map_blocks, const __grid_co
           uint32_t va[16], vb[16];
           tmem_ld8(sl_addr, va);
           tmem_ld8(sl_addr + 64, va + 8);
-          if (!(ok = read_out(p_old))) break;                                // the scores of the slab before last
 #pragma unroll
           for (int c = 0; c < 4; ++c) {
             uint32_t* cur = (c & 1) ? vb : va;
@@ -520,10 +442,7 @@ kscore_tc_kernel(const __grid_constant__ CUtensorMap map_blocks, const __grid_co
             if constexpr (PAIR) mbar_arrive_cluster(kr_full_own + 8 * sbuf);
             else mbar_arrive(kr_full + 8 * sbuf);
           }
-          p_old = p_new;
-          p_new.out = out_row + g * REP;
-          p_new.mxi = sli >> 1;
-          p_new.meta = KP_VALID | ((uint32_t)(sli & 1) << 1) | (mode << 2) | (slot << 4) | (slph << 6) | live_bit;
+          last_slot = slot; last_slph = slph;
           if (++sbuf == (uint32_t)KT_SLABS) { sbuf = 0; sph ^= 1u; }
           if (++slot == (uint32_t)KT_S_SLOTS) { slot = 0; slph ^= 1u; }
         }
@@ -532,16 +451,92 @@ kscore_tc_kernel(const __grid_constant__ CUtensorMap map_blocks, const __grid_co
       if (nxt.w >= 0) rope_setup(pos_next);
       pos_cur = pos_next;
       if (nxt.w != qs) {
-        // last tile of this query slot in the piece: the owed read-outs belong to it; the query operand may only change
-        // once every score product that reads the old one has retired
-        if (!(ok = read_out(p_old))) break;
-        if (!(ok = __all_sync(0xffffffffu, mbar_wait(s_full + 8 * ((p_new.meta >> 4) & 3u), (p_new.meta >> 6) & 1u, abort_flag)))) break;
-        if (!(ok = read_out(p_new))) break;
-        p_old.meta = 0u;
-        p_new.meta = 0u;
-        flush_max(qs);
-        if (nxt.w >= 0) write_q(nxt.w);
+        // last tile of this query slot in the piece: the query operand may only change once every score product that
+        // reads the old one has retired; they retire in order, and the last pair completes the accumulator of the slab rotated last
+        if (nxt.w >= 0) {
+          if (!(ok = __all_sync(0xffffffffu, mbar_wait(s_full + 8 * last_slot, last_slph, abort_flag)))) break;
+          write_q(nxt.w);
+        }
       }
+      e = nxt;
+    }
+    tmem_ld_wait();                                                          // nothing of this thread is in flight when TMEM is freed
+  } else if (warp >= 12) {
+    regs_shrink();
+    // ------------------------------------------------------------- score read-out
+    // One warp per TMEM lane quarter (thread = token row) follows the score issuer: REP columns of a slab's accumulator
+    // as soon as its two products have retired, scaled, rows past the tile's last token (and, for a causal query, tokens
+    // after it) masked, stored, and folded into the per-(sequence, head) maximum (over the warp's rows first, then one
+    // atomic per head; max is order-independent, so the result is deterministic).  The rotating warps never wait for it.
+    const int quarter = warp & 3, row = quarter * 32 + lane;
+    const uint32_t lane_addr = tmem_base + ((uint32_t)(quarter * 32) << 16);
+    const uint32_t s_col0 = TM_S + (PAIR ? 8u * crank : 0u);     // this CTA's columns of a score accumulator
+    const float sm_scale = v.sm_scale;
+    const int* kpos = v.aux(layer, 0);
+    uint32_t slot = 0, slph = 0;
+    bool ok = true;
+    int4 e = w0 < total ? klist[KSTEP * w0] : kt_none;
+    int pos_cur = w0 < total ? kpos[(size_t)e.x * TILE + row] : 0;
+    for (int w = w0; w < total && ok; ++w) {
+      const int4 nxt = w + 1 < total ? klist[KSTEP * (w + 1)] : kt_none;
+      const int tile = e.x, cls = e.y & 0x7f, n_valid = e.y >> 8, qs = e.w;
+      const bool discard = (e.y & KE_DISCARD) != 0;
+      const int passes = (cls + KT_A_SLOTS - 1) / KT_A_SLOTS;
+      const int pos_next = nxt.w >= 0 ? kpos[(size_t)nxt.x * TILE + row] : 0;
+      float* const out_row = v.scores + ((size_t)tile * TILE + row) * Hq;
+      // a row counts if it holds a token and, for a causal (prefill) query, the token is not after the query
+      const int pos_limit = v.qpos ? v.qpos[qs] : 0x7fffffff;
+      const bool live = row < n_valid && pos_cur <= pos_limit;
+      for (int ps = 0; ps < passes && ok; ++ps) {
+        const uint32_t mode = discard ? KP_DISCARD : passes == 1 ? KP_STORE_FINAL : (ps == 0 ? KP_STORE_PART : KP_ADD_FINAL);
+        for (int sli = 0; sli < Hkv; ++sli) {
+          const int g = sli + g_rot < Hkv ? sli + g_rot : sli + g_rot - Hkv;
+          if (!(ok = __all_sync(0xffffffffu, mbar_wait(s_full + 8 * slot, slph, abort_flag)))) break;
+          fence_after_sync();
+          float sv[REP];
+          {
+            uint32_t* dst = reinterpret_cast<uint32_t*>(sv);
+            const uint32_t src = lane_addr + s_col0 + 16 * slot;
+            if constexpr (REP == 1) tmem_ld1(src, dst);
+            else if constexpr (REP == 2) tmem_ld2(src, dst);
+            else if constexpr (REP == 4) tmem_ld4(src, dst);
+            else tmem_ld8(src, dst);
+          }
+          tmem_ld_wait();
+          fence_before_sync();
+          __syncwarp();
+          if (lane == 0) {
+            if constexpr (PAIR) mbar_arrive_cluster(s_empty_own + 8 * slot);
+            else mbar_arrive(s_empty + 8 * slot);
+          }
+          if (++slot == (uint32_t)KT_S_SLOTS) { slot = 0; slph ^= 1u; }
+          if (mode == KP_DISCARD) continue;
+          float* out = out_row + g * REP;
+#pragma unroll
+          for (int i = 0; i < REP; ++i) {
+            float x = sv[i] * sm_scale;
+            if (mode == KP_ADD_FINAL) x += out[i];                                       // the first pass stored its part
+            sv[i] = live ? x : -INFINITY;
+          }
+          if constexpr (REP >= 4) {
+#pragma unroll
+            for (int i = 0; i < REP; i += 4) *reinterpret_cast<float4*>(out + i) = make_float4(sv[i], sv[i + 1], sv[i + 2], sv[i + 3]);
+          } else {
+#pragma unroll
+            for (int i = 0; i < REP; ++i) out[i] = sv[i];
+          }
+          if (mode != KP_STORE_PART) {
+            unsigned mine = 0u;
+#pragma unroll
+            for (int i = 0; i < REP; ++i) {
+              const unsigned m = warp_max_u32(enc_ordered(sv[i]));
+              if (lane == i) mine = m;
+            }
+            if (lane < REP) atomicMax(&v.seqmax[qs * Hq + g * REP + lane], mine);
+          }
+        }
+      }
+      pos_cur = pos_next;
       e = nxt;
     }
     tmem_ld_wait();                                                          // nothing of this thread is in flight when TMEM is freed
