@@ -20,12 +20,16 @@
  *     and the one `pool` buffer the cache lives in.  The library allocates no
  *     device memory; it allocates small host structures only.
  *   - Work is enqueued on `stream` (a cudaStream_t passed as void*; NULL = the
- *     default stream) and is asynchronous unless stated otherwise.
+ *     default stream) and is asynchronous unless stated otherwise.  All scratch
+ *     (scores, work lists, partial sums, gate staging) lives in the cache's one
+ *     pool and is shared by its layers: calls on one cache must be ordered, on
+ *     one stream or by events; calls that overlap on the GPU race.
  *   - Errors are return codes, never aborts.  Argument errors that the host can
  *     see are returned before anything is launched and leave the cache
  *     unchanged.  Errors only the device can see (pool exhausted, a rank or
  *     sequence id out of range) set a sticky status word; the offending piece
- *     of work is skipped as a whole and the code is returned by the next
+ *     of work is skipped as a whole (a decode query whose sequence id is out of
+ *     range gets zeros) and the code is returned by the next
  *     twkv_cache_status().
  *   - Supported shapes: head_dim = 128, 1..8 KV heads (d_kv = n_kv_heads * 128,
  *     at most 1024), n_q_heads / n_kv_heads in {1, 2, 4, 8}.
@@ -215,7 +219,7 @@ twkv_status twkv_cache_check(twkv_cache* cache, int layer, void* stream, uint64_
  * Self-test of the bounded device-side wait (diagnostic).  Every tensor-core kernel of the library waits on shared-
  * memory barriers with an attempt limit; a wait that runs out raises its CTA's abort flag, all roles leave their loops
  * and the kernel reports TWKV_ERR_TIMEOUT instead of hanging.  This call launches a one-CTA kernel whose barrier
- * nobody ever completes, with the limit set to `attempts` (the production limit is 2^21), and synchronises `stream`.
+ * nobody ever completes, with the limit set to `attempts` (the production limit is 2^18, about one second), and synchronises `stream`.
  * Returns TWKV_OK if the wait gave up and raised the flag; the sticky status is then TWKV_ERR_TIMEOUT, as after a
  * production kernel's timeout, until twkv_cache_status reads it.  *elapsed_ns (host, may be NULL) = how long the wait took.
  */

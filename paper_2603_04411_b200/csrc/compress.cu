@@ -1,6 +1,6 @@
 // Compress step: gate -> rank (Eq. 5, 6, 8), slot allocation, truncate + pack (Eq. 2).
 //
-// A compress piece (<= 65536 tokens) runs as: hist (per-chunk key counts) -> alloc (one CTA:
+// A compress piece (<= TWKV_PIECE_TOKENS = 131072 tokens) runs as: hist (per-chunk key counts) -> alloc (one CTA:
 // exclusive scans, capacity check, tile and block allocation in ascending key order) -> pack
 // (warp per token: 128-bit loads / stores of the retained prefix, +0 fill to the class width).
 // Slot assignment is a function of the token order only (no atomics decide placement), so the

@@ -244,43 +244,60 @@ merge_kernel(DevView v, const unsigned short* __restrict__ Uinv_v, int n_splits,
   const int Hq = v.Hq, d_kv = v.d_kv;
   const int REP = min(ns, n_seq - qs0) * hp;                    // rows
   const int head0 = g * v.rep + (blockIdx.y % parts) * hp;      // first query head of this CTA
-  if (tid < REP) {
-    const int qs = qs0 + tid / hp, head = head0 + tid % hp;
-    float l = 0.f;
-    for (int s = 0; s < n_splits; ++s) l += v.part_l[((size_t)qs * n_splits + s) * Hq + head];
-    sInvL[tid] = l > 0.f ? 1.f / l : 0.f;
-  }
-  __syncthreads();
-  // split sums in split order; four elements per thread at a time so that four reads per split are in flight
-  for (int i0 = tid; i0 < REP * d_kv; i0 += 4 * MG_THREADS) {
-    const float* p[4];
-    float a[4] = {0.f, 0.f, 0.f, 0.f};
-#pragma unroll
-    for (int u = 0; u < 4; ++u) {
-      const int i = min(i0 + u * MG_THREADS, REP * d_kv - 1), hh = i / d_kv, j = i - hh * d_kv;
-      p[u] = v.part_acc + (((size_t)(qs0 + hh / hp) * n_splits) * Hq + head0 + hh % hp) * d_kv + j;
-    }
-    for (int s = 0; s < n_splits; ++s) {
-#pragma unroll
-      for (int u = 0; u < 4; ++u) a[u] += __ldg(p[u] + (size_t)s * Hq * d_kv);
-    }
-#pragma unroll
-    for (int u = 0; u < 4; ++u) {
-      const int i = i0 + u * MG_THREADS;
-      if (i < REP * d_kv) sAcc[i] = a[u] * sInvL[i / d_kv];
-    }
-  }
-  __syncthreads();
+  // the first rows of U_V^-1 this thread needs do not depend on the sums below: their reads go out first
   const int dp = tid & 63, jg = tid >> 6;
   const int jn = d_kv / MG_JGROUPS, j0 = jg * jn;
+  const unsigned* ucol = reinterpret_cast<const unsigned*>(Uinv_v + g * HEAD_DIM) + dp;    // two 16-bit columns per load
+  unsigned u[16], un[16];
+#pragma unroll
+  for (int t = 0; t < 16; ++t) u[t] = __ldg(ucol + (size_t)(j0 + t) * (d_kv / 2));
+  // row sums over the splits: warp w takes row w, its lanes read the splits' parts together, lane 0 adds them in split order
+  if ((tid >> 5) < REP) {
+    const int r = tid >> 5, lane = tid & 31;
+    const int qs = qs0 + r / hp, head = head0 + r % hp;
+    float l = 0.f;
+    for (int s0 = 0; s0 < n_splits; s0 += 32) {
+      const float mine = s0 + lane < n_splits ? v.part_l[((size_t)qs * n_splits + s0 + lane) * Hq + head] : 0.f;
+      const int n = min(32, n_splits - s0);
+      for (int s = 0; s < n; ++s) l += __shfl_sync(0xffffffffu, mine, s);
+    }
+    if (lane == 0) sInvL[r] = l > 0.f ? 1.f / l : 0.f;
+  }
+  // split sums in split order: a thread owns four consecutive columns of one row (one 16-byte read per split) and has
+  // the reads of eight splits in flight before it adds them (a loop of dependent adds over one read at a time left
+  // this kernel waiting for memory latency)
+  for (int i0 = tid * 4; i0 < REP * d_kv; i0 += 4 * MG_THREADS) {
+    const int hh = i0 / d_kv, j = i0 - hh * d_kv;                     // d_kv is a multiple of 64: the four columns share a row
+    const float4* p = reinterpret_cast<const float4*>(
+        v.part_acc + (((size_t)(qs0 + hh / hp) * n_splits) * Hq + head0 + hh % hp) * d_kv + j);
+    const size_t stride = (size_t)Hq * d_kv / 4;
+    float4 a = make_float4(0.f, 0.f, 0.f, 0.f);
+    for (int s0 = 0; s0 < n_splits; s0 += 8) {
+      float4 t[8];
+#pragma unroll
+      for (int u = 0; u < 8; ++u) t[u] = s0 + u < n_splits ? __ldg(p + (size_t)(s0 + u) * stride) : make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+      for (int u = 0; u < 8; ++u)
+        if (s0 + u < n_splits) { a.x += t[u].x; a.y += t[u].y; a.z += t[u].z; a.w += t[u].w; }
+    }
+    *reinterpret_cast<float4*>(sAcc + i0) = a;
+  }
+  __syncthreads();
+  for (int i0 = tid * 4; i0 < REP * d_kv; i0 += 4 * MG_THREADS) {       // each thread scales what it wrote
+    const float il = sInvL[i0 / d_kv];
+    float4 a = *reinterpret_cast<float4*>(sAcc + i0);
+    a.x *= il; a.y *= il; a.z *= il; a.w *= il;
+    *reinterpret_cast<float4*>(sAcc + i0) = a;
+  }
+  __syncthreads();
   float o[8][2];
 #pragma unroll
   for (int h = 0; h < 8; ++h) { o[h][0] = 0.f; o[h][1] = 0.f; }
-  const unsigned* ucol = reinterpret_cast<const unsigned*>(Uinv_v + g * HEAD_DIM) + dp;    // two 16-bit columns per load
   for (int jb = 0; jb < jn; jb += 16) {                // jn is a multiple of 16 (d_kv a multiple of 128)
-    unsigned u[16];
+    if (jb + 16 < jn) {                                // the next sixteen rows are on their way while these are used
 #pragma unroll
-    for (int t = 0; t < 16; ++t) u[t] = __ldg(ucol + (size_t)(j0 + jb + t) * (d_kv / 2));
+      for (int t = 0; t < 16; ++t) un[t] = __ldg(ucol + (size_t)(j0 + jb + 16 + t) * (d_kv / 2));
+    }
 #pragma unroll
     for (int t = 0; t < 16; ++t) {
       const float u0 = to_f32<BF16>((unsigned short)(u[t] & 0xffffu)), u1 = to_f32<BF16>((unsigned short)(u[t] >> 16));
@@ -292,6 +309,8 @@ merge_kernel(DevView v, const unsigned short* __restrict__ Uinv_v, int n_splits,
           o[h][1] += a * u1;
         }
     }
+#pragma unroll
+    for (int t = 0; t < 16; ++t) u[t] = un[t];
   }
   __syncthreads();
   float* red = sAcc;                                 // reuse: [MG_JGROUPS][REP][128]

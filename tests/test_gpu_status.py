@@ -137,3 +137,23 @@ def test_non_finite_logits_and_out_of_range_values_are_reported():
         assert run(li.q) == B.TWKV_OK
     finally:
         del os.environ["TWKV_DEBUG"]
+
+
+def test_decode_query_with_a_sequence_id_outside_the_cache_gets_zeros():
+    """The header's promise for an id the host cannot check against anything (ids live in device memory): the code
+    is reported, that query's output is defined (zeros), the other query's output is what it is without the bad one."""
+    from paper_2603_04411_b200 import build
+    build.build()
+    from paper_2603_04411_b200 import binding as B
+    gc, li = _filled_cache(B)
+    good = _decode(B, gc, li)
+    assert B.twkv_cache_status(gc.h) == B.TWKV_OK
+    out = torch.full((2, 32, 128), 7.0, device="cuda")
+    B.twkv_decode_attn(gc.h, 0, li.q.cuda(), torch.tensor([0, 99], dtype=torch.int32, device="cuda"), out)
+    assert B.twkv_cache_status(gc.h) == B.TWKV_ERR_INVALID_ARG
+    assert torch.count_nonzero(out[1]).item() == 0
+    torch.testing.assert_close(out[0], good[0], rtol=0, atol=0)
+    again = _decode(B, gc, li)                                              # and the cache is as it was
+    assert B.twkv_cache_status(gc.h) == B.TWKV_OK
+    torch.testing.assert_close(again, good, rtol=0, atol=0)
+    gc.close()
