@@ -98,7 +98,7 @@ __global__ void __launch_bounds__(1024) plan_kernel(DevView v, int layer, const 
     vsplit_plan(v, layer, seq_ids, (int)blockIdx.x - 1, n_splits);
     return;
   }
-  __shared__ int s_cls_off[TWKV_MAX_CLASSES + 1];
+  __shared__ int s_cls_off[TWKV_MAX_CLASSES + 1], s_kcc[TWKV_MAX_CLASSES];
   __shared__ unsigned s_wsum[32];
   __shared__ unsigned s_base;                                     // entries kept so far
   __shared__ int s_keep[TWKV_MAX_CLASSES];                        // kept tiles per class run (run k = class NC - k)
@@ -107,10 +107,13 @@ __global__ void __launch_bounds__(1024) plan_kernel(DevView v, int layer, const 
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   for (int s = tid; s < v.S; s += blockDim.x) v.qslot[s] = -1;
   if (tid < TWKV_MAX_CLASSES) s_keep[tid] = 0;
+  // the class counts are read by sixteen threads at once: one thread reading them in a loop paid a memory round trip
+  // per class (8 of this kernel's 16 microseconds)
+  if (tid < v.NC) s_kcc[tid] = v.kcc(layer)[tid];
+  __syncthreads();
   if (tid == 0) {
-    const int* kcc = v.kcc(layer);
     int run = 0;
-    for (int c = v.NC; c >= 1; --c) { s_cls_off[v.NC - c] = run; run += kcc[c - 1]; }    // widest class first
+    for (int c = v.NC; c >= 1; --c) { s_cls_off[v.NC - c] = run; run += s_kcc[c - 1]; }    // widest class first
     s_cls_off[v.NC] = run;
     s_base = 0u;
   }
