@@ -329,7 +329,7 @@ gate_tc_kernel(const __grid_constant__ CUtensorMap map_xk, const __grid_constant
   volatile int* abort_flag = reinterpret_cast<int*>(s_tmem_base + 1);
 
   if (tid == 0) {
-    for (int i = 0; i < GT_STAGES; ++i) { mbar_init(full + 8 * i, 2); mbar_init(empty + 8 * i, 1); }   // two copies fill a stage
+    for (int i = 0; i < GT_STAGES; ++i) { mbar_init(full + 8 * i, 1); mbar_init(empty + 8 * i, 1); }   // the producer posts both copies' bytes
     for (int i = 0; i < 2; ++i) { mbar_init(acc_full + 8 * i, 1); mbar_init(acc_empty + 8 * i, GT_EPI / 32); }
     mbar_init(epi_bar, GT_EPI);
     *abort_flag = 0;
@@ -348,31 +348,24 @@ gate_tc_kernel(const __grid_constant__ CUtensorMap map_xk, const __grid_constant
   const int ns_rot = blockIdx.x % n_slabs;
 
   if (warp == 0) {
-    // ------------------------------------------------------------- TMA producer
-    if (lane < 2 * GT_STAGES) {
-      const bool is_x = lane >= GT_STAGES;
-      const uint32_t my = is_x ? lane - GT_STAGES : lane;      // the ring stage this lane serves
-      if (lane == 0) { tma_prefetch_desc(&map_wk); tma_prefetch_desc(&map_wv); }
-      if (lane == GT_STAGES) { tma_prefetch_desc(&map_xk); tma_prefetch_desc(&map_xv); }
+    // ------------------------------------------------------------- TMA producer (one elected thread, ring order)
+    if (elect_one()) {
+      tma_prefetch_desc(&map_wk); tma_prefetch_desc(&map_wv);
+      tma_prefetch_desc(&map_xk); tma_prefetch_desc(&map_xv);
       bool ok = true;
       uint32_t st = 0, ph = 0;
       for (int it = it0; it < n_items && ok; it += itstep) {
         const int m0 = (it >> 1) * TILE;
-        const CUtensorMap* map = is_x ? ((it & 1) ? &map_xv : &map_xk) : ((it & 1) ? &map_wv : &map_wk);
+        const CUtensorMap* map_x = (it & 1) ? &map_xv : &map_xk;
+        const CUtensorMap* map_w = (it & 1) ? &map_wv : &map_wk;
         for (int sl = 0; sl < n_slabs && ok; ++sl) {
           const int ns = sl + ns_rot < n_slabs ? sl + ns_rot : sl + ns_rot - n_slabs;
           for (int p = 0; p < KP; ++p) {
-            const uint32_t cst = st, cph = ph;
+            if (!(ok = mbar_wait_thin(empty + 8 * st, ph ^ 1u, abort_flag))) break;
+            mbar_expect_tx(full + 8 * st, GT_PANEL_BYTES + b_stage_bytes);
+            tma_load_2d(sA + st * stage_bytes, map_x, full + 8 * st, p * PANEL, m0);
+            tma_load_2d(sA + st * stage_bytes + GT_PANEL_BYTES, map_w, full + 8 * st, p * PANEL, ns * NS);
             if (++st == GT_STAGES) { st = 0; ph ^= 1u; }
-            if (cst != my) continue;
-            if (!(ok = mbar_wait(empty + 8 * cst, cph ^ 1u, abort_flag))) break;
-            if (is_x) {
-              mbar_expect_tx(full + 8 * cst, GT_PANEL_BYTES);
-              tma_load_2d(sA + cst * stage_bytes, map, full + 8 * cst, p * PANEL, m0);
-            } else {
-              mbar_expect_tx(full + 8 * cst, b_stage_bytes);
-              tma_load_2d(sA + cst * stage_bytes + GT_PANEL_BYTES, map, full + 8 * cst, p * PANEL, ns * NS);
-            }
           }
         }
       }
@@ -460,7 +453,7 @@ gate_tc2_kernel(const __grid_constant__ CUtensorMap map_xk, const __grid_constan
   volatile int* abort_flag = reinterpret_cast<int*>(s_tmem_base + 1);
 
   if (tid == 0) {
-    for (int i = 0; i < GT2_STAGES; ++i) { mbar_init(full + 8 * i, 2); mbar_init(empty + 8 * i, 1); }   // even CTA: its two lanes post both CTAs' bytes
+    for (int i = 0; i < GT2_STAGES; ++i) { mbar_init(full + 8 * i, 1); mbar_init(empty + 8 * i, 1); }   // even CTA: its producer posts both CTAs' bytes
     for (int i = 0; i < 2; ++i) { mbar_init(acc_full + 8 * i, 1); mbar_init(acc_empty + 8 * i, 2 * (GT_EPI / 32)); }
     mbar_init(epi_bar, GT_EPI);
     *abort_flag = misaligned ? 1 : 0;
@@ -483,27 +476,27 @@ gate_tc2_kernel(const __grid_constant__ CUtensorMap map_xk, const __grid_constan
     // nothing was started; fall through to the common exit
   } else if (warp == 0) {
     // ------------------------------------------------------------- TMA producer
-    if (lane < 2 * GT2_STAGES) {
-      const bool is_x = lane >= GT2_STAGES;
-      const uint32_t my = is_x ? lane - GT2_STAGES : lane;     // the ring stage this lane serves
-      if (lane == 0) { tma_prefetch_desc(&map_wk); tma_prefetch_desc(&map_wv); }
-      if (lane == GT2_STAGES) { tma_prefetch_desc(&map_xk); tma_prefetch_desc(&map_xv); }
-      const uint32_t full_even = cluster_map(full + 8 * my, 0);            // the even CTA's barrier of this lane's stage
+    // One elected thread issues every copy in ring order (stages free up in that order): a copy instruction issued
+    // from a lane picked by its index costs that warp hundreds of cycles, and lanes of one warp that wait on different
+    // barriers wait one after the other.
+    if (elect_one()) {
+      tma_prefetch_desc(&map_wk); tma_prefetch_desc(&map_wv);
+      tma_prefetch_desc(&map_xk); tma_prefetch_desc(&map_xv);
       bool ok = true;
       uint32_t st = 0, ph = 0;
       for (int it = it0; it < n_items && ok; it += itstep) {
         const int m0 = (it >> 1) * (2 * TILE) + (int)crank * TILE;
-        const CUtensorMap* map = is_x ? ((it & 1) ? &map_xv : &map_xk) : ((it & 1) ? &map_wv : &map_wk);
+        const CUtensorMap* map_x = (it & 1) ? &map_xv : &map_xk;
+        const CUtensorMap* map_w = (it & 1) ? &map_wv : &map_wk;
         for (int sl = 0; sl < n_slabs && ok; ++sl) {
           const int ns = sl + ns_rot < n_slabs ? sl + ns_rot : sl + ns_rot - n_slabs;
           for (int p = 0; p < KP; ++p) {
-            const uint32_t cst = st, cph = ph;
+            if (!(ok = mbar_wait_thin(empty + 8 * st, ph ^ 1u, abort_flag))) break;
+            const uint32_t full_even = cluster_map(full + 8 * st, 0);          // the even CTA's barrier of this stage
+            if (crank == 0) mbar_expect_tx(full + 8 * st, 4 * GT_PANEL_BYTES);   // both CTAs' two copies
+            tma_load_2d_pair(sA + st * stage_bytes, map_x, full_even, p * PANEL, m0);
+            tma_load_2d_pair(sA + st * stage_bytes + GT_PANEL_BYTES, map_w, full_even, p * PANEL, ns * NS + (int)crank * TILE);
             if (++st == GT2_STAGES) { st = 0; ph ^= 1u; }
-            if (cst != my) continue;
-            if (!(ok = mbar_wait(empty + 8 * cst, cph ^ 1u, abort_flag))) break;
-            if (crank == 0) mbar_expect_tx(full + 8 * cst, 2 * GT_PANEL_BYTES);      // this lane's copy and the partner's
-            if (is_x) tma_load_2d_pair(sA + cst * stage_bytes, map, full_even, p * PANEL, m0);
-            else tma_load_2d_pair(sA + cst * stage_bytes + GT_PANEL_BYTES, map, full_even, p * PANEL, ns * NS + (int)crank * TILE);
           }
         }
       }

@@ -87,7 +87,7 @@ project_tc_kernel(const __grid_constant__ CUtensorMap map_xk, const __grid_const
   volatile int* abort_flag = reinterpret_cast<int*>(s_tmem_base + 1);
 
   if (tid == 0) {
-    for (int i = 0; i < PJ_STAGES; ++i) { mbar_init(full + 8 * i, 2); mbar_init(empty + 8 * i, 1); }
+    for (int i = 0; i < PJ_STAGES; ++i) { mbar_init(full + 8 * i, 1); mbar_init(empty + 8 * i, 1); }
     for (int i = 0; i < 2; ++i) { mbar_init(acc_full + 8 * i, 1); mbar_init(acc_empty + 8 * i, PJ_EPI / 32); }
     *abort_flag = 0;
     mbar_init_fence();
@@ -105,29 +105,24 @@ project_tc_kernel(const __grid_constant__ CUtensorMap map_xk, const __grid_const
 
   if (warp == 0) {
     // ------------------------------------------------------------- TMA producer
-    if (lane < 2 * PJ_STAGES) {
-      const bool is_x = lane >= PJ_STAGES;
-      const uint32_t my = is_x ? lane - PJ_STAGES : lane;
-      if (lane == 0) { tma_prefetch_desc(&map_uk); tma_prefetch_desc(&map_uv); }
-      if (lane == PJ_STAGES) { tma_prefetch_desc(&map_xk); tma_prefetch_desc(&map_xv); }
+    // one elected thread issues every copy in ring order: a copy issued from a lane picked by its index costs the warp
+    // hundreds of cycles, and lanes of one warp that wait on different barriers wait one after the other
+    if (elect_one()) {
+      tma_prefetch_desc(&map_uk); tma_prefetch_desc(&map_uv);
+      tma_prefetch_desc(&map_xk); tma_prefetch_desc(&map_xv);
       bool ok = true;
       uint32_t st = 0, ph = 0;
       for (int it = it0; it < n_items && ok; it += itstep) {
         const int rem = it % per_tile, m0 = (it / per_tile) * TILE;
         const int side = side0 + rem / n_slabs, ns = rem % n_slabs;
-        const CUtensorMap* map = is_x ? (side ? &map_xv : &map_xk) : (side ? &map_uv : &map_uk);
+        const CUtensorMap* map_x = side ? &map_xv : &map_xk;
+        const CUtensorMap* map_u = side ? &map_uv : &map_uk;
         for (int p = 0; p < KP; ++p) {
-          const uint32_t cst = st, cph = ph;
+          if (!(ok = mbar_wait_thin(empty + 8 * st, ph ^ 1u, abort_flag))) break;
+          mbar_expect_tx(full + 8 * st, PJ_PANEL_BYTES + b_stage_bytes);
+          tma_load_2d(sA + st * stage_bytes, map_x, full + 8 * st, p * PANEL, m0);
+          tma_load_2d(sA + st * stage_bytes + PJ_PANEL_BYTES, map_u, full + 8 * st, p * PANEL, ns * NS);
           if (++st == PJ_STAGES) { st = 0; ph ^= 1u; }
-          if (cst != my) continue;
-          if (!(ok = mbar_wait(empty + 8 * cst, cph ^ 1u, abort_flag))) break;
-          if (is_x) {
-            mbar_expect_tx(full + 8 * cst, PJ_PANEL_BYTES);
-            tma_load_2d(sA + cst * stage_bytes, map, full + 8 * cst, p * PANEL, m0);
-          } else {
-            mbar_expect_tx(full + 8 * cst, b_stage_bytes);
-            tma_load_2d(sA + cst * stage_bytes + PJ_PANEL_BYTES, map, full + 8 * cst, p * PANEL, ns * NS);
-          }
         }
       }
     }
@@ -257,7 +252,7 @@ project_tc2_kernel(const __grid_constant__ CUtensorMap map_xk, const __grid_cons
   volatile int* abort_flag = reinterpret_cast<int*>(s_tmem_base + 1);
 
   if (tid == 0) {
-    for (int i = 0; i < PJ2_STAGES; ++i) { mbar_init(full + 8 * i, 2); mbar_init(empty + 8 * i, 1); }
+    for (int i = 0; i < PJ2_STAGES; ++i) { mbar_init(full + 8 * i, 1); mbar_init(empty + 8 * i, 1); }
     for (int i = 0; i < 2; ++i) { mbar_init(acc_full + 8 * i, 1); mbar_init(acc_empty + 8 * i, 2 * (PJ_EPI / 32)); }
     *abort_flag = misaligned ? 1 : 0;
     mbar_init_fence();
@@ -277,27 +272,24 @@ project_tc2_kernel(const __grid_constant__ CUtensorMap map_xk, const __grid_cons
   if (misaligned) {
     // nothing was started; fall through to the common exit
   } else if (warp == 0) {
-    // ------------------------------------------------------------- TMA producer (both CTAs)
-    if (lane < 2 * PJ2_STAGES) {
-      const bool is_x = lane >= PJ2_STAGES;
-      const uint32_t my = is_x ? lane - PJ2_STAGES : lane;
-      if (lane == 0) { tma_prefetch_desc(&map_uk); tma_prefetch_desc(&map_uv); }
-      if (lane == PJ2_STAGES) { tma_prefetch_desc(&map_xk); tma_prefetch_desc(&map_xv); }
-      const uint32_t full_even = cluster_map(full + 8 * my, 0);            // the even CTA's barrier of this lane's stage
+    // ------------------------------------------------------------- TMA producer (both CTAs; one elected thread, ring order)
+    if (elect_one()) {
+      tma_prefetch_desc(&map_uk); tma_prefetch_desc(&map_uv);
+      tma_prefetch_desc(&map_xk); tma_prefetch_desc(&map_xv);
       bool ok = true;
       uint32_t st = 0, ph = 0;
       for (int it = it0; it < n_items && ok; it += itstep) {
         const int rem = it % per_tile, m0 = (it / per_tile) * (2 * TILE) + (int)crank * TILE;
         const int side = side0 + rem / n_slabs, ns = rem % n_slabs;
-        const CUtensorMap* map = is_x ? (side ? &map_xv : &map_xk) : (side ? &map_uv : &map_uk);
+        const CUtensorMap* map_x = side ? &map_xv : &map_xk;
+        const CUtensorMap* map_u = side ? &map_uv : &map_uk;
         for (int p = 0; p < KP; ++p) {
-          const uint32_t cst = st, cph = ph;
+          if (!(ok = mbar_wait_thin(empty + 8 * st, ph ^ 1u, abort_flag))) break;
+          const uint32_t full_even = cluster_map(full + 8 * st, 0);            // the even CTA's barrier of this stage
+          if (crank == 0) mbar_expect_tx(full + 8 * st, 4 * PJ_PANEL_BYTES);     // both CTAs' two copies
+          tma_load_2d_pair(sA + st * PJ2_STAGE_BYTES, map_x, full_even, p * PANEL, m0);
+          tma_load_2d_pair(sA + st * PJ2_STAGE_BYTES + PJ_PANEL_BYTES, map_u, full_even, p * PANEL, ns * 256 + (int)crank * TILE);
           if (++st == PJ2_STAGES) { st = 0; ph ^= 1u; }
-          if (cst != my) continue;
-          if (!(ok = mbar_wait(empty + 8 * cst, cph ^ 1u, abort_flag))) break;
-          if (crank == 0) mbar_expect_tx(full + 8 * cst, 2 * PJ_PANEL_BYTES);      // this lane's copy and the partner's
-          if (is_x) tma_load_2d_pair(sA + cst * PJ2_STAGE_BYTES, map, full_even, p * PANEL, m0);
-          else tma_load_2d_pair(sA + cst * PJ2_STAGE_BYTES + PJ_PANEL_BYTES, map, full_even, p * PANEL, ns * 256 + (int)crank * TILE);
         }
       }
     }
