@@ -161,7 +161,7 @@ project_tc_kernel(const __grid_constant__ CUtensorMap map_xk, const __grid_const
     const int quarter = warp & 3, chalf = ew >> 2;
     const int row = quarter * 32 + lane;
     const uint32_t lane_addr = tmem_base + ((uint32_t)(quarter * 32) << 16);
-    const bool leader = (ew & 3) == 0 && lane == 0;            // issues this half's stores
+    const bool lead_warp = (ew & 3) == 0;                      // one elected lane of this warp issues this half's stores
     unsigned char* my_panel = out_stage + chalf * PJ_PANEL_BYTES;
     const uint32_t my_panel_addr = smem_addr(my_panel);
     const int bar_id = 1 + chalf;
@@ -192,7 +192,7 @@ project_tc_kernel(const __grid_constant__ CUtensorMap map_xk, const __grid_const
           pk[u] = bf16 ? pack_bf16x2_rn(a[2 * u], a[2 * u + 1]) : pack_f16x2_rn(a[2 * u], a[2 * u + 1]);
           pk[16 + u] = bf16 ? pack_bf16x2_rn(b[2 * u], b[2 * u + 1]) : pack_f16x2_rn(b[2 * u], b[2 * u + 1]);
         }
-        if (leader) bulk_wait_read_all();                      // the previous store has left the staging panel
+        if (lead_warp && elect_one()) bulk_wait_read_all();                      // the previous store has left the staging panel
         named_bar_sync(bar_id, 128);
 #pragma unroll
         for (int c8 = 0; c8 < 8; ++c8)                         // 16-byte chunk c8 of the row sits at chunk c8 ^ (row % 8)
@@ -200,13 +200,13 @@ project_tc_kernel(const __grid_constant__ CUtensorMap map_xk, const __grid_const
               make_uint4(pk[4 * c8], pk[4 * c8 + 1], pk[4 * c8 + 2], pk[4 * c8 + 3]);
         fence_proxy_async_smem();
         named_bar_sync(bar_id, 128);
-        if (leader) {
+        if (lead_warp && elect_one()) {
           tma_store_2d(omap, my_panel_addr, ns * NS + col, m0);
           bulk_commit();
         }
       }
     }
-    if (leader) bulk_wait_all();
+    if (lead_warp && elect_one()) bulk_wait_all();
   }
 
   fence_before_sync();
@@ -329,7 +329,7 @@ project_tc2_kernel(const __grid_constant__ CUtensorMap map_xk, const __grid_cons
     const int quarter = warp & 3, chalf = ew >> 2;
     const int row = quarter * 32 + lane;
     const uint32_t lane_addr = tmem_base + ((uint32_t)(quarter * 32) << 16);
-    const bool leader = (ew & 3) == 0 && lane == 0;
+    const bool lead_warp = (ew & 3) == 0;                      // one elected lane of this warp issues this half's stores
     unsigned char* my_panel = out_stage + chalf * PJ_PANEL_BYTES;
     const uint32_t my_panel_addr = smem_addr(my_panel);
     const int bar_id = 1 + chalf;
@@ -360,7 +360,7 @@ project_tc2_kernel(const __grid_constant__ CUtensorMap map_xk, const __grid_cons
           pk[u] = bf16 ? pack_bf16x2_rn(a[2 * u], a[2 * u + 1]) : pack_f16x2_rn(a[2 * u], a[2 * u + 1]);
           pk[16 + u] = bf16 ? pack_bf16x2_rn(b[2 * u], b[2 * u + 1]) : pack_f16x2_rn(b[2 * u], b[2 * u + 1]);
         }
-        if (leader) bulk_wait_read_all();
+        if (lead_warp && elect_one()) bulk_wait_read_all();
         named_bar_sync(bar_id, 128);
 #pragma unroll
         for (int c8 = 0; c8 < 8; ++c8)
@@ -368,13 +368,13 @@ project_tc2_kernel(const __grid_constant__ CUtensorMap map_xk, const __grid_cons
               make_uint4(pk[4 * c8], pk[4 * c8 + 1], pk[4 * c8 + 2], pk[4 * c8 + 3]);
         fence_proxy_async_smem();
         named_bar_sync(bar_id, 128);
-        if (leader && m0 < n_tok) {                            // the pair's second tile may lie past the last token
+        if (lead_warp && m0 < n_tok && elect_one()) {                            // the pair's second tile may lie past the last token
           tma_store_2d(omap, my_panel_addr, ns * 256 + col, m0);
           bulk_commit();
         }
       }
     }
-    if (leader) bulk_wait_all();
+    if (lead_warp && elect_one()) bulk_wait_all();
   }
 
   fence_before_sync();
