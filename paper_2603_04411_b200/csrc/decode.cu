@@ -23,11 +23,12 @@ namespace twkv {
 // is rewritten as items of two tiles of one class.  The list is then cut into n_cta contiguous pieces of
 // about equal estimated cost, so a CTA (pair) of the K-score kernel mostly stays inside one (class, sequence) run.
 __device__ __forceinline__ unsigned ktile_cost(int cls) {
-  // cycles per tile of the K-score kernel by rank class: a least-squares fit of every CTA's busy time to its tile counts on
-  // the benchmark's mix of classes (8 KV heads, CTA pairs): a fixed part (rotation factors, the per-slab epilogue and
-  // score products) plus a per-panel part; classes above 8 run as two passes.  Only the ratios matter.
-  constexpr unsigned kCost[TWKV_MAX_CLASSES] = {14400u, 16200u, 18000u, 19700u, 21500u, 23300u, 25000u, 26800u,
-                                                37600u, 39400u, 41200u, 43000u, 44900u, 46700u, 48500u, 50300u};
+  // cycles per tile of the K-score kernel by rank class: a least-squares fit, one coefficient per class, of every CTA's busy
+  // time to its tile counts on the benchmark's mix of classes (8 KV heads, CTA pairs; residual 1.3 us rms of 330): a fixed
+  // part (rotation factors, the per-slab epilogue and score products) plus a per-panel part, an odd panel count costing a
+  // little more than the even one above it saves; classes above 8 run as two passes.  Only the ratios matter.
+  constexpr unsigned kCost[TWKV_MAX_CLASSES] = {14300u, 16600u, 18600u, 19500u, 22100u, 23000u, 25400u, 26200u,
+                                                38800u, 38700u, 42000u, 42800u, 45600u, 45800u, 49300u, 50700u};
   return kCost[min(max(cls, 1), TWKV_MAX_CLASSES) - 1];
 }
 
