@@ -308,7 +308,7 @@ gate_tc_kernel(const __grid_constant__ CUtensorMap map_xk, const __grid_constant
                const float* __restrict__ bias_k, const float* __restrict__ bias_v, int n_tok, int d, int bf16, float tau,
                float* __restrict__ stage_all, unsigned short* __restrict__ levels, int* status, const GateRaw raw) {
   extern __shared__ __align__(1024) unsigned char smem_raw[];
-  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int tid = threadIdx.x, warp = tid >> 5;
   const int KP = d / PANEL;                                   // K panels of the token tile
   const int NS = (d % 256 == 0) ? 256 : 128;                  // logits per slab
   const int n_slabs = d / NS;
@@ -346,60 +346,30 @@ gate_tc_kernel(const __grid_constant__ CUtensorMap map_xk, const __grid_constant
   const int it0 = blockIdx.x, itstep = gridDim.x;
 
   const int ns_rot = blockIdx.x % n_slabs;
+  // accumulators this CTA produces: its items x the slabs of an item
+  const uint32_t n_acc = it0 < n_items ? (uint32_t)((n_items - it0 + itstep - 1) / itstep) * (uint32_t)n_slabs : 0u;
 
   if (warp == 0) {
     // ------------------------------------------------------------- TMA producer (one elected thread, ring order)
     if (elect_one()) {
       tma_prefetch_desc(&map_wk); tma_prefetch_desc(&map_wv);
       tma_prefetch_desc(&map_xk); tma_prefetch_desc(&map_xv);
-      bool ok = true;
-      uint32_t st = 0, ph = 0;
-      for (int it = it0; it < n_items && ok; it += itstep) {
-        const int m0 = (it >> 1) * TILE;
-        const CUtensorMap* map_x = (it & 1) ? &map_xv : &map_xk;
-        const CUtensorMap* map_w = (it & 1) ? &map_wv : &map_wk;
-        for (int sl = 0; sl < n_slabs && ok; ++sl) {
-          const int ns = sl + ns_rot < n_slabs ? sl + ns_rot : sl + ns_rot - n_slabs;
-          for (int p = 0; p < KP; ++p) {
-            if (!(ok = mbar_wait_thin(empty + 8 * st, ph ^ 1u, abort_flag))) break;
-            mbar_expect_tx(full + 8 * st, GT_PANEL_BYTES + b_stage_bytes);
-            tma_load_2d(sA + st * stage_bytes, map_x, full + 8 * st, p * PANEL, m0);
-            tma_load_2d(sA + st * stage_bytes + GT_PANEL_BYTES, map_w, full + 8 * st, p * PANEL, ns * NS);
-            if (++st == GT_STAGES) { st = 0; ph ^= 1u; }
-          }
-        }
-      }
+      ring_gemm_produce<1>(n_acc, KP, GT_STAGES, sA, stage_bytes, GT_PANEL_BYTES, GT_PANEL_BYTES + b_stage_bytes, full, empty, 0u, abort_flag,
+                           [&](uint32_t a, const CUtensorMap*& mx, const CUtensorMap*& mw, int& m0, int& n0) {
+                             const int it = it0 + (int)(a / (uint32_t)n_slabs) * itstep, sl = (int)(a % (uint32_t)n_slabs);
+                             const int ns = sl + ns_rot < n_slabs ? sl + ns_rot : sl + ns_rot - n_slabs;
+                             mx = (it & 1) ? &map_xv : &map_xk;
+                             mw = (it & 1) ? &map_wv : &map_wk;
+                             m0 = (it >> 1) * TILE;
+                             n0 = ns * NS;
+                           });
     }
     __syncwarp();
   } else if (warp == 1) {
     // ------------------------------------------------------------- MMA issuer
-    if (elect_one()) {
-      const uint32_t idesc = idesc_f16(bf16 ? 1 : 0, 128, NS);
-      const uint64_t adesc0 = kmajor_sw128_desc(sA), bdesc0 = kmajor_sw128_desc(sA + GT_PANEL_BYTES);
-      bool ok = true;
-      uint32_t st = 0, ph = 0, ac = 0;
-      for (int it = it0; it < n_items && ok; it += itstep) {
-        for (int sl = 0; sl < n_slabs && ok; ++sl, ++ac) {
-          const uint32_t buf = ac & 1u;
-          if (!(ok = mbar_wait(acc_empty + 8 * buf, ((ac >> 1) & 1u) ^ 1u, abort_flag))) break;
-          const uint32_t dcol = tmem_base + buf * 256;
-          for (int p = 0; p < KP; ++p) {
-            const uint32_t cst = st, cph = ph;
-            if (++st == GT_STAGES) { st = 0; ph ^= 1u; }
-            if (!(ok = mbar_wait(full + 8 * cst, cph, abort_flag))) break;
-            fence_after_sync();
-            const uint64_t adesc = adesc0 + (uint64_t)(cst * (stage_bytes >> 4));
-            const uint64_t bdesc = bdesc0 + (uint64_t)(cst * (stage_bytes >> 4));
-            mma_f16_ss(dcol, adesc, bdesc, idesc, p > 0 ? 1u : 0u);
-#pragma unroll
-            for (int ks = 1; ks < 4; ++ks) mma_f16_ss(dcol, adesc + 2 * ks, bdesc + 2 * ks, idesc, 1u);
-            mma_commit(empty + 8 * cst);
-          }
-          if (!ok) break;
-          mma_commit(acc_full + 8 * buf);
-        }
-      }
-    }
+    if (elect_one())
+      ring_gemm_issue<1>(n_acc, KP, GT_STAGES, sA, stage_bytes, GT_PANEL_BYTES, idesc_f16(bf16 ? 1 : 0, 128, NS), tmem_base, full, empty,
+                         acc_full, acc_empty, abort_flag);
     __syncwarp();
   } else {
     // ------------------------------------------------------------- epilogue + rank
@@ -435,7 +405,7 @@ gate_tc2_kernel(const __grid_constant__ CUtensorMap map_xk, const __grid_constan
                const float* __restrict__ bias_k, const float* __restrict__ bias_v, int n_tok, int d, int bf16, float tau,
                float* __restrict__ stage_all, unsigned short* __restrict__ levels, int* status, const GateRaw raw) {
   extern __shared__ __align__(1024) unsigned char smem_raw[];
-  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int tid = threadIdx.x, warp = tid >> 5;
   const uint32_t crank = cluster_cta_rank();                  // 0 = even CTA: issues the MMAs, owns full / acc_empty
   const int KP = d / PANEL;                                   // K panels of the token tile
   constexpr int NS = 256;                                     // logits per slab (d is a multiple of 256 here)
@@ -471,6 +441,8 @@ gate_tc2_kernel(const __grid_constant__ CUtensorMap map_xk, const __grid_constan
   const int it0 = blockIdx.x >> 1, itstep = gridDim.x >> 1;
 
   const int ns_rot = (blockIdx.x >> 1) % n_slabs;
+  // accumulators this pair produces: its items x the slabs of an item
+  const uint32_t n_acc = it0 < n_items ? (uint32_t)((n_items - it0 + itstep - 1) / itstep) * (uint32_t)n_slabs : 0u;
 
   if (misaligned) {
     // nothing was started; fall through to the common exit
@@ -482,56 +454,22 @@ gate_tc2_kernel(const __grid_constant__ CUtensorMap map_xk, const __grid_constan
     if (elect_one()) {
       tma_prefetch_desc(&map_wk); tma_prefetch_desc(&map_wv);
       tma_prefetch_desc(&map_xk); tma_prefetch_desc(&map_xv);
-      bool ok = true;
-      uint32_t st = 0, ph = 0;
-      for (int it = it0; it < n_items && ok; it += itstep) {
-        const int m0 = (it >> 1) * (2 * TILE) + (int)crank * TILE;
-        const CUtensorMap* map_x = (it & 1) ? &map_xv : &map_xk;
-        const CUtensorMap* map_w = (it & 1) ? &map_wv : &map_wk;
-        for (int sl = 0; sl < n_slabs && ok; ++sl) {
-          const int ns = sl + ns_rot < n_slabs ? sl + ns_rot : sl + ns_rot - n_slabs;
-          for (int p = 0; p < KP; ++p) {
-            if (!(ok = mbar_wait_thin(empty + 8 * st, ph ^ 1u, abort_flag))) break;
-            const uint32_t full_even = cluster_map(full + 8 * st, 0);          // the even CTA's barrier of this stage
-            if (crank == 0) mbar_expect_tx(full + 8 * st, 4 * GT_PANEL_BYTES);   // both CTAs' two copies
-            tma_load_2d_pair(sA + st * stage_bytes, map_x, full_even, p * PANEL, m0);
-            tma_load_2d_pair(sA + st * stage_bytes + GT_PANEL_BYTES, map_w, full_even, p * PANEL, ns * NS + (int)crank * TILE);
-            if (++st == GT2_STAGES) { st = 0; ph ^= 1u; }
-          }
-        }
-      }
+      ring_gemm_produce<2>(n_acc, KP, GT2_STAGES, sA, stage_bytes, GT_PANEL_BYTES, 4 * GT_PANEL_BYTES, full, empty, crank, abort_flag,
+                           [&](uint32_t a, const CUtensorMap*& mx, const CUtensorMap*& mw, int& m0, int& n0) {
+                             const int it = it0 + (int)(a / (uint32_t)n_slabs) * itstep, sl = (int)(a % (uint32_t)n_slabs);
+                             const int ns = sl + ns_rot < n_slabs ? sl + ns_rot : sl + ns_rot - n_slabs;
+                             mx = (it & 1) ? &map_xv : &map_xk;
+                             mw = (it & 1) ? &map_wv : &map_wk;
+                             m0 = (it >> 1) * (2 * TILE) + (int)crank * TILE;
+                             n0 = ns * NS + (int)crank * TILE;
+                           });
     }
     __syncwarp();
   } else if (warp == 1) {
-    // ------------------------------------------------------------- MMA issuer
-    if (crank == 0 && elect_one()) {
-      const uint32_t idesc = idesc_f16(bf16 ? 1 : 0, 256, NS);
-      const uint64_t adesc0 = kmajor_sw128_desc(sA), bdesc0 = kmajor_sw128_desc(sA + GT_PANEL_BYTES);
-      bool ok = true;
-      uint32_t st = 0, ph = 0, ac = 0;
-      for (int it = it0; it < n_items && ok; it += itstep) {
-        for (int sl = 0; sl < n_slabs && ok; ++sl, ++ac) {
-          const uint32_t buf = ac & 1u;
-          if (!(ok = mbar_wait(acc_empty + 8 * buf, ((ac >> 1) & 1u) ^ 1u, abort_flag))) break;
-          fence_after_sync();
-          const uint32_t dcol = tmem_base + buf * 256;
-          for (int p = 0; p < KP; ++p) {
-            const uint32_t cst = st, cph = ph;
-            if (++st == GT2_STAGES) { st = 0; ph ^= 1u; }
-            if (!(ok = mbar_wait(full + 8 * cst, cph, abort_flag))) break;
-            fence_after_sync();
-            const uint64_t adesc = adesc0 + (uint64_t)(cst * (stage_bytes >> 4));
-            const uint64_t bdesc = bdesc0 + (uint64_t)(cst * (stage_bytes >> 4));
-            mma_f16_ss_pair(dcol, adesc, bdesc, idesc, p > 0 ? 1u : 0u);
-#pragma unroll
-            for (int ks = 1; ks < 4; ++ks) mma_f16_ss_pair(dcol, adesc + 2 * ks, bdesc + 2 * ks, idesc, 1u);
-            mma_commit_pair_both(empty + 8 * cst);
-          }
-          if (!ok) break;
-          mma_commit_pair_both(acc_full + 8 * buf);
-        }
-      }
-    }
+    // ------------------------------------------------------------- MMA issuer (even CTA only)
+    if (crank == 0 && elect_one())
+      ring_gemm_issue<2>(n_acc, KP, GT2_STAGES, sA, stage_bytes, GT_PANEL_BYTES, idesc_f16(bf16 ? 1 : 0, 256, NS), tmem_base, full, empty,
+                         acc_full, acc_empty, abort_flag);
     __syncwarp();
   } else {
     // ------------------------------------------------------------- epilogue + rank

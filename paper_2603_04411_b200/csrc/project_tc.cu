@@ -102,6 +102,7 @@ project_tc_kernel(const __grid_constant__ CUtensorMap map_xk, const __grid_const
   const int per_tile = n_sides * n_slabs;
   const int n_items = per_tile * ((n_tok + TILE - 1) / TILE);
   const int it0 = blockIdx.x, itstep = gridDim.x;
+  const uint32_t n_acc = it0 < n_items ? (uint32_t)((n_items - it0 + itstep - 1) / itstep) : 0u;      // one accumulator per item
 
   if (warp == 0) {
     // ------------------------------------------------------------- TMA producer
@@ -110,50 +111,22 @@ project_tc_kernel(const __grid_constant__ CUtensorMap map_xk, const __grid_const
     if (elect_one()) {
       tma_prefetch_desc(&map_uk); tma_prefetch_desc(&map_uv);
       tma_prefetch_desc(&map_xk); tma_prefetch_desc(&map_xv);
-      bool ok = true;
-      uint32_t st = 0, ph = 0;
-      for (int it = it0; it < n_items && ok; it += itstep) {
-        const int rem = it % per_tile, m0 = (it / per_tile) * TILE;
-        const int side = side0 + rem / n_slabs, ns = rem % n_slabs;
-        const CUtensorMap* map_x = side ? &map_xv : &map_xk;
-        const CUtensorMap* map_u = side ? &map_uv : &map_uk;
-        for (int p = 0; p < KP; ++p) {
-          if (!(ok = mbar_wait_thin(empty + 8 * st, ph ^ 1u, abort_flag))) break;
-          mbar_expect_tx(full + 8 * st, PJ_PANEL_BYTES + b_stage_bytes);
-          tma_load_2d(sA + st * stage_bytes, map_x, full + 8 * st, p * PANEL, m0);
-          tma_load_2d(sA + st * stage_bytes + PJ_PANEL_BYTES, map_u, full + 8 * st, p * PANEL, ns * NS);
-          if (++st == PJ_STAGES) { st = 0; ph ^= 1u; }
-        }
-      }
+      ring_gemm_produce<1>(n_acc, KP, PJ_STAGES, sA, stage_bytes, PJ_PANEL_BYTES, PJ_PANEL_BYTES + b_stage_bytes, full, empty, 0u, abort_flag,
+                           [&](uint32_t a, const CUtensorMap*& mx, const CUtensorMap*& mu, int& m0, int& n0) {
+                             const int it = it0 + (int)a * itstep, rem = it % per_tile;
+                             const int side = side0 + rem / n_slabs;
+                             mx = side ? &map_xv : &map_xk;
+                             mu = side ? &map_uv : &map_uk;
+                             m0 = (it / per_tile) * TILE;
+                             n0 = (rem % n_slabs) * NS;
+                           });
     }
     __syncwarp();
   } else if (warp == 1) {
     // ------------------------------------------------------------- MMA issuer
-    if (elect_one()) {
-      const uint32_t idesc = idesc_f16(bf16 ? 1 : 0, 128, NS);
-      const uint64_t adesc0 = kmajor_sw128_desc(sA), bdesc0 = kmajor_sw128_desc(sA + PJ_PANEL_BYTES);
-      bool ok = true;
-      uint32_t st = 0, ph = 0, ac = 0;
-      for (int it = it0; it < n_items && ok; it += itstep, ++ac) {
-        const uint32_t buf = ac & 1u;
-        if (!(ok = mbar_wait(acc_empty + 8 * buf, ((ac >> 1) & 1u) ^ 1u, abort_flag))) break;
-        const uint32_t dcol = tmem_base + buf * 256;
-        for (int p = 0; p < KP; ++p) {
-          const uint32_t cst = st, cph = ph;
-          if (++st == PJ_STAGES) { st = 0; ph ^= 1u; }
-          if (!(ok = mbar_wait(full + 8 * cst, cph, abort_flag))) break;
-          fence_after_sync();
-          const uint64_t adesc = adesc0 + (uint64_t)(cst * (stage_bytes >> 4));
-          const uint64_t bdesc = bdesc0 + (uint64_t)(cst * (stage_bytes >> 4));
-          mma_f16_ss(dcol, adesc, bdesc, idesc, p > 0 ? 1u : 0u);
-#pragma unroll
-          for (int ks = 1; ks < 4; ++ks) mma_f16_ss(dcol, adesc + 2 * ks, bdesc + 2 * ks, idesc, 1u);
-          mma_commit(empty + 8 * cst);
-        }
-        if (!ok) break;
-        mma_commit(acc_full + 8 * buf);
-      }
-    }
+    if (elect_one())
+      ring_gemm_issue<1>(n_acc, KP, PJ_STAGES, sA, stage_bytes, PJ_PANEL_BYTES, idesc_f16(bf16 ? 1 : 0, 128, NS), tmem_base, full, empty,
+                         acc_full, acc_empty, abort_flag);
     __syncwarp();
   } else {
     // ------------------------------------------------------------- epilogue
@@ -268,6 +241,7 @@ project_tc2_kernel(const __grid_constant__ CUtensorMap map_xk, const __grid_cons
   const int per_tile = n_sides * n_slabs;
   const int n_items = per_tile * ((n_tok + 2 * TILE - 1) / (2 * TILE));
   const int it0 = blockIdx.x >> 1, itstep = gridDim.x >> 1;
+  const uint32_t n_acc = it0 < n_items ? (uint32_t)((n_items - it0 + itstep - 1) / itstep) : 0u;      // one accumulator per item
 
   if (misaligned) {
     // nothing was started; fall through to the common exit
@@ -276,52 +250,22 @@ project_tc2_kernel(const __grid_constant__ CUtensorMap map_xk, const __grid_cons
     if (elect_one()) {
       tma_prefetch_desc(&map_uk); tma_prefetch_desc(&map_uv);
       tma_prefetch_desc(&map_xk); tma_prefetch_desc(&map_xv);
-      bool ok = true;
-      uint32_t st = 0, ph = 0;
-      for (int it = it0; it < n_items && ok; it += itstep) {
-        const int rem = it % per_tile, m0 = (it / per_tile) * (2 * TILE) + (int)crank * TILE;
-        const int side = side0 + rem / n_slabs, ns = rem % n_slabs;
-        const CUtensorMap* map_x = side ? &map_xv : &map_xk;
-        const CUtensorMap* map_u = side ? &map_uv : &map_uk;
-        for (int p = 0; p < KP; ++p) {
-          if (!(ok = mbar_wait_thin(empty + 8 * st, ph ^ 1u, abort_flag))) break;
-          const uint32_t full_even = cluster_map(full + 8 * st, 0);            // the even CTA's barrier of this stage
-          if (crank == 0) mbar_expect_tx(full + 8 * st, 4 * PJ_PANEL_BYTES);     // both CTAs' two copies
-          tma_load_2d_pair(sA + st * PJ2_STAGE_BYTES, map_x, full_even, p * PANEL, m0);
-          tma_load_2d_pair(sA + st * PJ2_STAGE_BYTES + PJ_PANEL_BYTES, map_u, full_even, p * PANEL, ns * 256 + (int)crank * TILE);
-          if (++st == PJ2_STAGES) { st = 0; ph ^= 1u; }
-        }
-      }
+      ring_gemm_produce<2>(n_acc, KP, PJ2_STAGES, sA, PJ2_STAGE_BYTES, PJ_PANEL_BYTES, 4 * PJ_PANEL_BYTES, full, empty, crank, abort_flag,
+                           [&](uint32_t a, const CUtensorMap*& mx, const CUtensorMap*& mu, int& m0, int& n0) {
+                             const int it = it0 + (int)a * itstep, rem = it % per_tile;
+                             const int side = side0 + rem / n_slabs;
+                             mx = side ? &map_xv : &map_xk;
+                             mu = side ? &map_uv : &map_uk;
+                             m0 = (it / per_tile) * (2 * TILE) + (int)crank * TILE;
+                             n0 = (rem % n_slabs) * 256 + (int)crank * TILE;
+                           });
     }
     __syncwarp();
   } else if (warp == 1) {
     // ------------------------------------------------------------- MMA issuer (even CTA only)
-    if (crank == 0 && elect_one()) {
-      const uint32_t idesc = idesc_f16(bf16 ? 1 : 0, 256, 256);
-      const uint64_t adesc0 = kmajor_sw128_desc(sA), bdesc0 = kmajor_sw128_desc(sA + PJ_PANEL_BYTES);
-      bool ok = true;
-      uint32_t st = 0, ph = 0, ac = 0;
-      for (int it = it0; it < n_items && ok; it += itstep, ++ac) {
-        const uint32_t buf = ac & 1u;
-        if (!(ok = mbar_wait(acc_empty + 8 * buf, ((ac >> 1) & 1u) ^ 1u, abort_flag))) break;
-        fence_after_sync();
-        const uint32_t dcol = tmem_base + buf * 256;
-        for (int p = 0; p < KP; ++p) {
-          const uint32_t cst = st, cph = ph;
-          if (++st == PJ2_STAGES) { st = 0; ph ^= 1u; }
-          if (!(ok = mbar_wait(full + 8 * cst, cph, abort_flag))) break;
-          fence_after_sync();
-          const uint64_t adesc = adesc0 + (uint64_t)(cst * (PJ2_STAGE_BYTES >> 4));
-          const uint64_t bdesc = bdesc0 + (uint64_t)(cst * (PJ2_STAGE_BYTES >> 4));
-          mma_f16_ss_pair(dcol, adesc, bdesc, idesc, p > 0 ? 1u : 0u);
-#pragma unroll
-          for (int ks = 1; ks < 4; ++ks) mma_f16_ss_pair(dcol, adesc + 2 * ks, bdesc + 2 * ks, idesc, 1u);
-          mma_commit_pair_both(empty + 8 * cst);
-        }
-        if (!ok) break;
-        mma_commit_pair_both(acc_full + 8 * buf);
-      }
-    }
+    if (crank == 0 && elect_one())
+      ring_gemm_issue<2>(n_acc, KP, PJ2_STAGES, sA, PJ2_STAGE_BYTES, PJ_PANEL_BYTES, idesc_f16(bf16 ? 1 : 0, 256, 256), tmem_base, full, empty,
+                         acc_full, acc_empty, abort_flag);
     __syncwarp();
   } else {
     // ------------------------------------------------------------- epilogue (both CTAs, own 128 rows)

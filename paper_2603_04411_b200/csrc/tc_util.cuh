@@ -330,6 +330,68 @@ __device__ __forceinline__ void mma_commit_pair_both(uint32_t bar) {
                ::"r"(bar), "h"((unsigned short)3) : "memory");
 }
 
+// ---- the main loop shared by the dense kernels whose operands stream through a ring (gate logits, projection) ----
+// A ring stage holds one K = 64 panel of the row operand (`x_bytes` at offset 0: 128 rows of this CTA) and one of the
+// column operand (at `b_off`: N rows, or this CTA's half of them in a pair).  An accumulator is KP stages; accumulators
+// alternate between two 256-column TMEM buffers.  CG = 2: the CTA-pair form (both CTAs produce, the even CTA issues;
+// `full` and `acc_empty` live in the even CTA, `empty` and `acc_full` are signalled in both by a multicast commit).
+//
+// Producer: one elected thread issues every copy in ring order.  coord(a, map_x, map_w, m0, n0) names the tensor maps
+// and the first rows of accumulator a's operands.
+template <int CG, class Coord>
+__device__ __forceinline__ void ring_gemm_produce(uint32_t n_acc, int KP, uint32_t stages, uint32_t sA, uint32_t stage_bytes, uint32_t b_off,
+                                                  uint32_t tx_bytes, uint32_t full, uint32_t empty, uint32_t crank,
+                                                  volatile int* abort_flag, Coord coord) {
+  uint32_t st = 0, ph = 0;
+  for (uint32_t a = 0; a < n_acc; ++a) {
+    const CUtensorMap *map_x, *map_w;
+    int m0, n0;
+    coord(a, map_x, map_w, m0, n0);
+    for (int p = 0; p < KP; ++p) {
+      if (!mbar_wait_thin(empty + 8 * st, ph ^ 1u, abort_flag)) return;
+      if constexpr (CG == 2) {
+        const uint32_t full_even = cluster_map(full + 8 * st, 0);              // the even CTA's barrier of this stage
+        if (crank == 0) mbar_expect_tx(full + 8 * st, tx_bytes);                // both CTAs' two copies
+        tma_load_2d_pair(sA + st * stage_bytes, map_x, full_even, p * TWKV_PANEL_ELEMS, m0);
+        tma_load_2d_pair(sA + st * stage_bytes + b_off, map_w, full_even, p * TWKV_PANEL_ELEMS, n0);
+      } else {
+        mbar_expect_tx(full + 8 * st, tx_bytes);
+        tma_load_2d(sA + st * stage_bytes, map_x, full + 8 * st, p * TWKV_PANEL_ELEMS, m0);
+        tma_load_2d(sA + st * stage_bytes + b_off, map_w, full + 8 * st, p * TWKV_PANEL_ELEMS, n0);
+      }
+      if (++st == stages) { st = 0; ph ^= 1u; }
+    }
+  }
+}
+// Issuer: one elected thread (of the even CTA in a pair); four MMAs per stage, the stage handed back when they retire.
+template <int CG>
+__device__ __forceinline__ void ring_gemm_issue(uint32_t n_acc, int KP, uint32_t stages, uint32_t sA, uint32_t stage_bytes, uint32_t b_off,
+                                                uint32_t idesc, uint32_t tmem_base, uint32_t full, uint32_t empty, uint32_t acc_full,
+                                                uint32_t acc_empty, volatile int* abort_flag) {
+  const uint64_t adesc0 = kmajor_sw128_desc(sA), bdesc0 = kmajor_sw128_desc(sA + b_off);
+  uint32_t st = 0, ph = 0;
+  for (uint32_t ac = 0; ac < n_acc; ++ac) {
+    const uint32_t buf = ac & 1u;
+    if (!mbar_wait(acc_empty + 8 * buf, ((ac >> 1) & 1u) ^ 1u, abort_flag)) return;
+    fence_after_sync();
+    const uint32_t dcol = tmem_base + buf * 256;
+    for (int p = 0; p < KP; ++p) {
+      if (!mbar_wait(full + 8 * st, ph, abort_flag)) return;
+      fence_after_sync();
+      const uint64_t adesc = adesc0 + (uint64_t)(st * (stage_bytes >> 4));
+      const uint64_t bdesc = bdesc0 + (uint64_t)(st * (stage_bytes >> 4));
+#pragma unroll
+      for (int ks = 0; ks < 4; ++ks) {
+        if constexpr (CG == 2) mma_f16_ss_pair(dcol, adesc + 2 * ks, bdesc + 2 * ks, idesc, (p > 0 || ks > 0) ? 1u : 0u);
+        else mma_f16_ss(dcol, adesc + 2 * ks, bdesc + 2 * ks, idesc, (p > 0 || ks > 0) ? 1u : 0u);
+      }
+      if constexpr (CG == 2) mma_commit_pair_both(empty + 8 * st); else mma_commit(empty + 8 * st);
+      if (++st == stages) { st = 0; ph ^= 1u; }
+    }
+    if constexpr (CG == 2) mma_commit_pair_both(acc_full + 8 * buf); else mma_commit(acc_full + 8 * buf);
+  }
+}
+
 }  // namespace tc
 
 // Tensor maps the decode path needs: the block pool as rows of 64 elements, and the layer's transposed U_K^-1.
