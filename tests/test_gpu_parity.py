@@ -225,6 +225,19 @@ def test_rank_one_and_full_rank(B):
     assert max_abs < MAX_ABS and rel_l2 < REL_L2, (max_abs, rel_l2)
 
 
+def test_one_split_over_more_tiles_than_the_v_pass_stages_at_once(B):
+    # One sequence of 36 000 tokens (about 290 V tiles over four classes) decoded with a single split: the V pass stages
+    # the tile descriptors of a split in shared memory 256 at a time, so this split crosses a refill; and with the
+    # default split count (many short splits, some of them a single tile) the answer is the same within the bars.
+    li = to_cuda(workloads.build_layer(47, n_seq=1, ctx=36000, n_q_heads=8, mode="forced", n_calib=2048))
+    ranks = li.ranks.cpu().numpy().astype(np.int64)
+    (max_abs, rel_l2), got1, want = run_case(B, li, ranks, mode=B.TWKV_GATE_FORCED, num_splits=1, check_image=False)
+    assert max_abs < MAX_ABS and rel_l2 < REL_L2, (max_abs, rel_l2)
+    (max_abs, rel_l2), got0, _ = run_case(B, li, ranks, mode=B.TWKV_GATE_FORCED, num_splits=0, check_image=False)
+    assert max_abs < MAX_ABS and rel_l2 < REL_L2, (max_abs, rel_l2)
+    assert np.abs(got1 - got0).max() < MAX_ABS
+
+
 def test_subset_decode_empty_sequence_and_determinism(B):
     li = to_cuda(workloads.build_layer(41, n_seq=3, ctx=150, n_q_heads=32, mode="forced"))
     ranks = li.ranks.cpu().numpy().astype(np.int64)
