@@ -158,15 +158,23 @@ def twkv_cache_create(cfg: twkv_config, pool: torch.Tensor, stream=None):
 
 def twkv_cache_destroy(cache):
     _check(lib.twkv_cache_destroy(cache), "twkv_cache_destroy")
+    _borrowed.pop(cache.value, None)
 
 
 def twkv_cache_reset(cache, stream=None):
     _check(lib.twkv_cache_reset(cache, _stream(stream)), "twkv_cache_reset")
 
 
+# The library borrows a layer's parameter tensors until the cache is destroyed or the parameters are replaced.  The
+# binding keeps a reference to them for that long, so that a caller who passes temporaries (x.cuda()) does not leave the
+# cache with pointers into memory the allocator has taken back.
+_borrowed = {}
+
+
 def twkv_cache_set_layer_params(cache, layer, Uinv_k, Uinv_v, W_k=None, W_v=None, b_k=None, b_v=None):
     p = twkv_layer_params(_ptr(Uinv_k), _ptr(Uinv_v), _ptr(W_k), _ptr(W_v), _ptr(b_k), _ptr(b_v))
     _check(lib.twkv_cache_set_layer_params(cache, layer, ctypes.byref(p)), "twkv_cache_set_layer_params")
+    _borrowed.setdefault(cache.value, {})[layer] = (Uinv_k, Uinv_v, W_k, W_v, b_k, b_v)
 
 
 def twkv_compress(cache, layer, K, V, seq_ids, positions, scores, levels, mode, stream=None, n_tok=None):

@@ -19,7 +19,8 @@ def _filled_cache(B):
     ranks = li.ranks.numpy().astype(np.int64)
     gc = GpuCache(B, n_layers=1, n_q_heads=32, n_kv_heads=8, dtype=torch.float16, out_dtype=torch.float32, max_seqs=2,
                   max_tokens_per_seq=300, payload_bytes=int((-(-ranks // 64) * 128).sum()))
-    B.twkv_cache_set_layer_params(gc.h, 0, li.Uinv_k.cuda(), li.Uinv_v.cuda())
+    gc.layer_params = (li.Uinv_k.cuda(), li.Uinv_v.cuda())              # borrowed by the cache: they must outlive it
+    B.twkv_cache_set_layer_params(gc.h, 0, *gc.layer_params)
     B.twkv_compress(gc.h, 0, li.xt_k.cuda(), li.xt_v.cuda(), li.seq_ids.cuda(), li.positions.cuda(), None,
                     torch.from_numpy(ranks.astype(np.int16)).cuda(), B.TWKV_GATE_FORCED)
     return gc, li
@@ -156,4 +157,32 @@ def test_decode_query_with_a_sequence_id_outside_the_cache_gets_zeros():
     again = _decode(B, gc, li)                                              # and the cache is as it was
     assert B.twkv_cache_status(gc.h) == B.TWKV_OK
     torch.testing.assert_close(again, good, rtol=0, atol=0)
+    gc.close()
+
+
+def test_decode_call_replays_from_a_cuda_graph():
+    """A decode call enqueues kernels only (no allocation, no synchronisation, no host-side reads of device state), so a
+    captured call can be replayed: the replay's output equals the eager call's bit for bit."""
+    from paper_2603_04411_b200 import build
+    build.build()
+    from paper_2603_04411_b200 import binding as B
+    gc, li = _filled_cache(B)
+    eager = _decode(B, gc, li)                                              # also the first call's one-time set-up
+    assert B.twkv_cache_status(gc.h) == B.TWKV_OK
+    q = li.q.cuda()
+    sid = torch.tensor([0, 1], dtype=torch.int32, device="cuda")
+    out = torch.zeros(2, 32, 128, device="cuda")
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.stream(side):
+        with torch.cuda.graph(graph, stream=side):
+            B.twkv_decode_attn(gc.h, 0, q, sid, out)
+    torch.cuda.current_stream().wait_stream(side)
+    for _ in range(2):
+        out.zero_()
+        graph.replay()
+        torch.cuda.synchronize()
+        torch.testing.assert_close(out, eager, rtol=0, atol=0)
+    assert B.twkv_cache_status(gc.h) == B.TWKV_OK
     gc.close()
