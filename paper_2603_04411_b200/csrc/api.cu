@@ -87,7 +87,7 @@ constexpr int GATE_TC_MIN_TOKENS = 1024;   // calls at least this large run the 
 struct Offsets {
   size_t status, pflags, rope_lo, rope_hi, n_tiles, tile_desc, tile_aux, tile_rank, fill, key_last, kclass_count,
       kclass_tiles, seq_vcount, seq_vtiles, seq_tokens, rank_sums, hist, key_cnt, key_old_fill, key_first_id,
-      key_first_base, key_old_last, scores, seqmax, qslot, klist, kpairs, klist_count, cta_start, vcut, wave_buf, evict_bitmap, evict_map, evict_fill, part_acc, part_l, gate_scratch, gate_fix, stats_buf, tables_end, prep_uinvT, prep_wT, guard_list,
+      key_first_base, key_old_last, scores, seqmax, qslot, klist, kpairs, klist_count, cta_start, vcut, kv_link, wave_buf, evict_bitmap, evict_map, evict_fill, part_acc, part_l, gate_scratch, gate_fix, stats_buf, tables_end, prep_uinvT, prep_wT, guard_list,
       blocks, end_fixed;
 };
 
@@ -165,6 +165,7 @@ static Offsets layout_of(const twkv_config* c, const Dims& d, std::vector<unsign
   o.kpairs = L.alloc((NT + 64) * sizeof(int4));
   o.cta_start = L.alloc((MAX_PLAN_CTAS + 1) * sizeof(int));
   o.vcut = L.alloc((size_t)(d.max_partials + S + 1) * sizeof(int));
+  o.kv_link = L.alloc((size_t)NT * TILE * sizeof(int));
   o.wave_buf = L.alloc((size_t)3 * TWKV_PREFILL_MAX_QUERIES * sizeof(int));
   o.evict_bitmap = L.alloc((size_t)ROPE_LO * ROPE_HI / 8);
   o.evict_map = L.alloc((size_t)2 * NT * TILE * sizeof(int));
@@ -263,7 +264,7 @@ static void fill_view(twkv_cache* c) {
   v.key_old_last = (int*)(p + o.key_old_last);
   v.scores = (float*)(p + o.scores); v.seqmax = (unsigned*)(p + o.seqmax); v.qslot = (int*)(p + o.qslot);
   v.klist = (int4*)(p + o.klist); v.klist_count = (int*)(p + o.klist_count);
-  v.kpairs = (int4*)(p + o.kpairs); v.cta_start = (int*)(p + o.cta_start); v.vcut = (int*)(p + o.vcut);
+  v.kpairs = (int4*)(p + o.kpairs); v.cta_start = (int*)(p + o.cta_start); v.vcut = (int*)(p + o.vcut); v.kv_link = (int*)(p + o.kv_link);
   v.part_acc = (float*)(p + o.part_acc); v.part_l = (float*)(p + o.part_l);
   v.gate_scratch = (float*)(p + o.gate_scratch);
   v.gate_fix = (int4*)(p + o.gate_fix);

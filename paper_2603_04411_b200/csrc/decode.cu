@@ -1,7 +1,7 @@
 // Decode attention over the mixed-rank cache (Eq. 3, reshape to heads, RoPE, softmax attention).
 //
 //   plan_kernel    sequence id -> query slot map, running-max reset, K-tile work list; cut points of every
-//                  sequence's V tiles into the splits of the V pass
+//                  sequence's V tiles into the splits of the V pass; K slot -> V slot links of the sequences' tokens
 //   kscore_tc_kernel (kscore_tc.cu)  per K tile: Kbar = X^_K U_K^-1, RoPE by stored position,
 //                  s = q . Kbar * scale for the GQA group, scores to scratch, per-sequence max
 //   vacc_tc_kernel (vacc_tc.cu)  per (sequence, split): p = exp(s - max), acc += p^T X^_V in spectral
@@ -93,8 +93,30 @@ __device__ void vsplit_plan(const DevView& v, int layer, const int* __restrict__
   if (tid == 0) cut[n_splits] = n;
 }
 
+// K slot -> V slot of every token of one sequence (the V slots carry the opposite link): the K-score kernel stores a
+// token's scores at its V slot, so that the V pass finds a tile's score rows next to each other.  CTA j of the vj CTAs of
+// a sequence takes the V tiles j * 8 .. j * 8 + 7, then vj * 8 further on, eight tiles (1024 slots) at a time.
+__device__ void vlink_plan(const DevView& v, int layer, const int* __restrict__ seq_ids, int qs, int j, int vj) {
+  const int seq = seq_ids[qs];
+  if (seq < 0 || seq >= v.S) return;
+  const int n = v.svc(layer)[seq];
+  const int* list = v.svt(layer) + (size_t)seq * v.TPS;
+  const int4* desc = v.desc(layer, 1);
+  const int* aux = v.aux(layer, 1);
+  const int sub = threadIdx.x >> 7, slot = threadIdx.x & (TILE - 1);
+  for (int t = j * 8 + sub; t < n; t += vj * 8) {
+    const int vt = list[t];
+    if (slot < desc[vt].z) v.kv_link[aux[(size_t)vt * TILE + slot]] = vt * TILE + slot;
+  }
+}
+
 __global__ void __launch_bounds__(1024) plan_kernel(DevView v, int layer, const int* __restrict__ seq_ids, int n_seq, int n_cta, int pairs,
-                                                    int n_splits) {
+                                                    int n_splits, int vj) {
+  if ((int)blockIdx.x > n_seq) {                                  // the last n_seq * vj CTAs: K slot -> V slot links
+    const int idx = (int)blockIdx.x - 1 - n_seq;
+    vlink_plan(v, layer, seq_ids, idx / vj, idx % vj, vj);
+    return;
+  }
   if (blockIdx.x > 0) {                                           // CTAs 1 .. n_seq: the V pass's split plan, one sequence each
     vsplit_plan(v, layer, seq_ids, (int)blockIdx.x - 1, n_splits);
     return;
@@ -346,7 +368,9 @@ static cudaError_t launch_decode_t(const DevView& v, int layer, const LayerParam
                                    int n_seq, void* out, int n_splits, int sm_count, const TcMaps* maps, bool pairs, cudaStream_t st) {
   // the K-score kernel's work is cut into one piece per persistent CTA, or per CTA pair
   const int n_pieces = pairs ? kscore_max_pairs(sm_count) : sm_count;
-  { ProfScope ps(TWKV_K_PLAN, st); plan_kernel<<<1 + n_seq, 1024, 0, st>>>(v, layer, seq_ids, n_seq, n_pieces, pairs ? 1 : 0, n_splits); }
+  // CTAs per sequence that invert the V -> K links: enough of them that they finish inside the K work list's time
+  const int vj = n_seq >= 256 ? 1 : (256 / n_seq > 64 ? 64 : 256 / n_seq);
+  { ProfScope ps(TWKV_K_PLAN, st); plan_kernel<<<1 + n_seq + n_seq * vj, 1024, 0, st>>>(v, layer, seq_ids, n_seq, n_pieces, pairs ? 1 : 0, n_splits, vj); }
   {
     cudaError_t e = launch_kscore_tc(v, layer, maps->blocks, maps->uinvT_k, q, n_pieces, pairs, st);
     if (e != cudaSuccess) return e;

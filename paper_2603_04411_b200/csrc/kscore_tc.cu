@@ -477,13 +477,17 @@ kscore_tc_kernel(const __grid_constant__ CUtensorMap map_blocks, const __grid_co
     bool ok = true;
     int4 e = w0 < total ? klist[KSTEP * w0] : kt_none;
     int pos_cur = w0 < total ? kpos[(size_t)e.x * TILE + row] : 0;
+    // the row of the score scratch this token's scores go to: its V slot (rows past the tile's last token have none)
+    int vrow_cur = w0 < total && row < (e.y >> 8) ? v.kv_link[(size_t)e.x * TILE + row] : 0;
     for (int w = w0; w < total && ok; ++w) {
       const int4 nxt = w + 1 < total ? klist[KSTEP * (w + 1)] : kt_none;
-      const int tile = e.x, cls = e.y & 0x7f, n_valid = e.y >> 8, qs = e.w;
+      const int cls = e.y & 0x7f, n_valid = e.y >> 8, qs = e.w;
       const bool discard = (e.y & KE_DISCARD) != 0;
       const int passes = (cls + KT_A_SLOTS - 1) / KT_A_SLOTS;
       const int pos_next = nxt.w >= 0 ? kpos[(size_t)nxt.x * TILE + row] : 0;
-      float* const out_row = v.scores + ((size_t)tile * TILE + row) * Hq;
+      const int vrow_next = nxt.w >= 0 && row < (nxt.y >> 8) ? v.kv_link[(size_t)nxt.x * TILE + row] : 0;
+      const bool has_row = row < n_valid;
+      float* const out_row = v.scores + (size_t)vrow_cur * Hq;
       // a row counts if it holds a token and, for a causal (prefill) query, the token is not after the query
       const int pos_limit = v.qpos ? v.qpos[qs] : 0x7fffffff;
       const bool live = row < n_valid && pos_cur <= pos_limit;
@@ -515,15 +519,17 @@ kscore_tc_kernel(const __grid_constant__ CUtensorMap map_blocks, const __grid_co
 #pragma unroll
           for (int i = 0; i < REP; ++i) {
             float x = sv[i] * sm_scale;
-            if (mode == KP_ADD_FINAL) x += out[i];                                       // the first pass stored its part
+            if (mode == KP_ADD_FINAL && has_row) x += out[i];                            // the first pass stored its part
             sv[i] = live ? x : -INFINITY;
           }
-          if constexpr (REP >= 4) {
+          if (has_row) {
+            if constexpr (REP >= 4) {
 #pragma unroll
-            for (int i = 0; i < REP; i += 4) *reinterpret_cast<float4*>(out + i) = make_float4(sv[i], sv[i + 1], sv[i + 2], sv[i + 3]);
-          } else {
+              for (int i = 0; i < REP; i += 4) *reinterpret_cast<float4*>(out + i) = make_float4(sv[i], sv[i + 1], sv[i + 2], sv[i + 3]);
+            } else {
 #pragma unroll
-            for (int i = 0; i < REP; ++i) out[i] = sv[i];
+              for (int i = 0; i < REP; ++i) out[i] = sv[i];
+            }
           }
           if (mode != KP_STORE_PART) {
             unsigned mine = 0u;
@@ -537,6 +543,7 @@ kscore_tc_kernel(const __grid_constant__ CUtensorMap map_blocks, const __grid_co
         }
       }
       pos_cur = pos_next;
+      vrow_cur = vrow_next;
       e = nxt;
     }
     tmem_ld_wait();                                                          // nothing of this thread is in flight when TMEM is freed

@@ -53,7 +53,7 @@ struct DevView {
   int* key_first_id;         // [NK]  id of the key's first new tile
   int* key_first_base;       // [NK]  base block of the key's first new tile
   int* key_old_last;         // [NK]  the key's newest tile before the piece
-  float* scores;             // [NT*128][Hq]
+  float* scores;             // [NT*128][Hq]  row = V slot of the token (the V pass reads a tile's rows together)
   unsigned* seqmax;          // [S][Hq]  order-preserving encoding of the running max
   int* qslot;                // [S]   sequence id -> query index of the current decode call, -1
   // chunked prefill (null for a decode call): per query slot, the row of q / out it stands for and the last position it
@@ -70,6 +70,7 @@ struct DevView {
                              //            a class with an odd number of tiles ends with a filler entry (.y bit 7 set)
   int* klist_count;          // [1]
   int* cta_start;            // [MAX_PLAN_CTAS + 1]  first list entry of every K-score CTA
+  int* kv_link;              // [NT * 128]  K slot -> V slot of the same token, for the sequences of the current decode pass (rebuilt by every pass)
   int* vcut;                 // [query slots][n_splits + 1]  cut points of every sequence's V tile list into the splits of the V pass
   float* part_acc;           // [max_partials][Hq][d_kv]
   float* part_l;             // [max_partials][Hq]

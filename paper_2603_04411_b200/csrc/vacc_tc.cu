@@ -13,11 +13,11 @@
 // points the second atom at a small zero block instead (the leading byte offset is free per instruction), so the pair's
 // upper accumulator half adds zeros.
 // The probabilities are the B operand (K-major: [head][token], two 64-token halves), written by 8 warps: thread =
-// (head, 8 consecutive tokens), one 16-byte swizzled store per 8 weights.  Score rows arrive through the V slot's link
-// to its K score row: each warp copies the rows of its own token groups with cp.async into a ring of four tiles in
-// shared memory, and the links themselves the same way four tiles further ahead, so that four tiles of scores are in
-// flight per SM and no thread waits for a load it has just issued; a narrow tile reads as many bytes of scores as of
-// values, and with one tile in flight their latency bound the kernel.
+// (head, 8 consecutive tokens), one 16-byte swizzled store per 8 weights.  The K-score kernel stores a token's scores at
+// its V slot, so a tile's 128 score rows lie next to each other: each warp copies the rows of its own token groups with
+// cp.async into a ring of four tiles in shared memory, so that four tiles of scores are in flight per SM and no thread
+// waits for a load it has just issued; a narrow tile reads as many bytes of scores as of values, and with one tile in
+// flight their latency bound the kernel.
 // bf16 weights go in as two bf16 parts (see below), two chains per pair.
 //
 // Warp roles (320 threads, one CTA per SM):
@@ -41,7 +41,6 @@ constexpr uint32_t VT_STAGE_BYTES = 2 * VT_PANEL_BYTES;
 constexpr uint32_t VT_ZERO_BYTES = 2048;                       // 16 token rows of zeros: the missing partner of a lone panel
 constexpr uint32_t VT_SMEM_MAX = 232448;
 constexpr int VT_SC = 4;                                       // tiles of scores in flight
-constexpr int VT_LK = 8;                                       // ring of link rows: a tile's links land VT_SC iterations before its scores are asked for
 
 template <bool BF16, int N>
 struct VtCfg {
@@ -49,7 +48,7 @@ struct VtCfg {
   static constexpr uint32_t P_HALF_BYTES = N * 128;            // [N heads][64 tokens]
   static constexpr uint32_t P_PART_BYTES = 2 * P_HALF_BYTES;
   static constexpr uint32_t P_BUF_BYTES = PARTS * P_PART_BYTES;
-  static constexpr uint32_t TAIL_BYTES = VT_META * 16 + VT_LK * 512 + VT_PTHREADS * 4 + 256;      // descriptors, links, row sums, barriers
+  static constexpr uint32_t TAIL_BYTES = VT_META * 16 + VT_PTHREADS * 4 + 256;      // descriptors, row sums, barriers
   static constexpr uint32_t SC_STAGE_BYTES = 128 * N * 4;      // [128 tokens][N heads] fp32
   static constexpr uint32_t FIXED_BYTES = VT_ZERO_BYTES + 2 * P_BUF_BYTES + VT_SC * SC_STAGE_BYTES + TAIL_BYTES + 1024;   // + alignment slack
   static constexpr int STAGES_FIT = (int)((VT_SMEM_MAX - FIXED_BYTES) / VT_STAGE_BYTES);
@@ -96,7 +95,6 @@ vacc_tc_kernel(const __grid_constant__ CUtensorMap map_blocks, DevView v, int la
   const long long t_stride = vtile_stride(n_tiles);
   const int* list = v.svt(layer) + (size_t)(seq_ok ? seq : 0) * v.TPS;
   const int4* desc = v.desc(layer, 1);
-  const int* aux = v.aux(layer, 1);
 
   // shared memory: ring | zero block | probabilities [2 buffers][PARTS][2 halves][N][128 B] | score ring | descriptors | row sums | barriers
   const uint32_t s0 = smem_addr(smem_raw);
@@ -109,8 +107,7 @@ vacc_tc_kernel(const __grid_constant__ CUtensorMap map_blocks, DevView v, int la
   unsigned char* sS_ptr = sP_ptr + 2 * C::P_BUF_BYTES;                                // score ring
   const uint32_t sS = sP + 2 * C::P_BUF_BYTES;
   int4* s_meta = reinterpret_cast<int4*>(sS_ptr + VT_SC * C::SC_STAGE_BYTES);          // (tile, class, tokens, first block)
-  int* s_link = reinterpret_cast<int*>(s_meta + VT_META);                              // [VT_LK][128]
-  float* s_l = reinterpret_cast<float*>(s_link + VT_LK * TILE);
+  float* s_l = reinterpret_cast<float*>(s_meta + VT_META);
   unsigned char* tail = reinterpret_cast<unsigned char*>(s_l + VT_PTHREADS);
   const uint32_t bars = smem_addr(tail);
   const uint32_t full = bars, empty = full + 8 * S, p_full = empty + 8 * S, p_empty = p_full + 16, acc_done = p_empty + 16;
@@ -232,46 +229,28 @@ vacc_tc_kernel(const __grid_constant__ CUtensorMap map_blocks, DevView v, int la
       __syncwarp();
     } else {
       // ------------------------------------------------------------- probabilities
-      // Copies go out in one cp.async group per iteration: the score rows of tile i + VT_SC - 1 and the links of tile
-      // i + VT_LK - 1.  Waiting for all but the newest VT_SC - 1 groups then guarantees tile i's scores, and (one iteration
-      // later) the links the next score copies need.  A warp copies and reads only the rows of its own token groups.
+      // One cp.async group per iteration: the score rows of tile i + VT_SC - 1.  Waiting for all but the newest
+      // VT_SC - 1 groups then guarantees tile i's scores.  A warp copies and reads only the rows of its own token groups.
       constexpr int GL = N == 16 ? 16 : 32;                     // lanes that share an item
       const int gl = lane & (GL - 1);
       const bool al16 = (Hq & 3) == 0;                          // score rows start on 16-byte boundaries
-      const uint32_t s_link_a = smem_addr(s_link);
-      auto issue_links = [&](int i) {                           // tile i of the chunk: 8 links per item, 16 bytes per lane
-        if (i < cn && gl < 2) {
-          const int tile = s_meta[i].x;
-#pragma unroll
-          for (int it = 0; it < ITEMS; ++it) {
-            const int t = ((it * VT_PTHREADS + pt) / N) * 8 + gl * 4;
-            cp_async16(s_link_a + (uint32_t)((((c0 + i) % VT_LK) * TILE + t) * 4), aux + (size_t)tile * TILE + t);
-          }
-        }
-      };
-      // Starts the copies of tile i's score rows (named by its links, landed by now) into its stage of the score ring.  Every row of the
-      // stage is written: rows past the tile's last token, and heads past the CTA's last, get -inf (weight 0).
+      // Starts the copies of tile i's score rows into its stage of the score ring.  Every row of the stage is written:
+      // rows past the tile's last token, and heads past the CTA's last, get -inf (weight 0).
       auto issue_scores = [&](int i) {
         if (i < cn) {
           const uint32_t stage = (uint32_t)((c0 + i) % VT_SC) * C::SC_STAGE_BYTES;
-          const int* lk = s_link + ((c0 + i) % VT_LK) * TILE;
-          const int n_valid = s_meta[i].z;
-          // all of this thread's links first, then the copies: a branch per copy would put the shared-memory round trips
-          // of the link reads one behind the other
+          const int4 m = s_meta[i];
+          const int n_valid = m.z;
+          const float* rows = v.scores + (size_t)m.x * TILE * Hq + h0;            // the tile's first score row, at this CTA's heads
           if (al16) {
             constexpr int CPR = N / 4, R = 8 * CPR / GL;        // 16-byte pieces per row; pieces per lane and item
-            int l[ITEMS][R];
-#pragma unroll
-            for (int it = 0; it < ITEMS; ++it)
-#pragma unroll
-              for (int r = 0; r < R; ++r) l[it][r] = lk[((it * VT_PTHREADS + pt) / N) * 8 + (r * GL + gl) / CPR];
 #pragma unroll
             for (int it = 0; it < ITEMS; ++it)
 #pragma unroll
               for (int r = 0; r < R; ++r) {
                 const int row = ((it * VT_PTHREADS + pt) / N) * 8 + (r * GL + gl) / CPR, ch = (r * GL + gl) % CPR;
                 const uint32_t off = stage + (uint32_t)((row * N + 4 * ch) * 4);
-                if (row < n_valid && 4 * ch < nh) cp_async16(sS + off, v.scores + (size_t)l[it][r] * Hq + h0 + 4 * ch);
+                if (row < n_valid && 4 * ch < nh) cp_async16(sS + off, rows + (size_t)row * Hq + 4 * ch);
                 else *reinterpret_cast<float4*>(sS_ptr + off) = make_float4(-INFINITY, -INFINITY, -INFINITY, -INFINITY);
               }
           } else {
@@ -282,25 +261,18 @@ vacc_tc_kernel(const __grid_constant__ CUtensorMap map_blocks, DevView v, int la
               for (int r = 0; r < R; ++r) {
                 const int row = ((it * VT_PTHREADS + pt) / N) * 8 + (r * GL + gl) / N, hh = (r * GL + gl) % N;
                 const uint32_t off = stage + (uint32_t)((row * N + hh) * 4);
-                if (row < n_valid && hh < nh) cp_async4(sS + off, v.scores + (size_t)lk[row] * Hq + h0 + hh);
+                if (row < n_valid && hh < nh) cp_async4(sS + off, rows + (size_t)row * Hq + hh);
                 else *reinterpret_cast<float*>(sS_ptr + off) = -INFINITY;
               }
           }
         }
       };
-      // prologue: the links of the first tiles, then (once they have landed) the first score rows with the next links
 #pragma unroll 1
-      for (int d = 0; d < VT_SC; ++d) issue_links(d);
-      cp_async_commit();
-      cp_async_wait<0>();
-      __syncwarp();
-#pragma unroll 1
-      for (int d = 0; d < VT_SC - 1; ++d) { issue_scores(d); issue_links(VT_SC + d); cp_async_commit(); }
+      for (int d = 0; d < VT_SC - 1; ++d) { issue_scores(d); cp_async_commit(); }
       for (int i = 0; i < cn && ok; ++i) {
         const int k = c0 + i;
         max_cls = max(max_cls, s_meta[i].y);
         issue_scores(i + VT_SC - 1);
-        issue_links(i + VT_LK - 1);
         cp_async_commit();
         cp_async_wait<VT_SC - 1>();                             // this thread's copies of tile i have landed
         __syncwarp();                                           // ... and the other lanes'
