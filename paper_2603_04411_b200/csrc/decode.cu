@@ -130,8 +130,8 @@ __global__ void __launch_bounds__(1024) plan_kernel(DevView v, int layer, const 
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   for (int s = tid; s < v.S; s += blockDim.x) v.qslot[s] = -1;
   if (tid < TWKV_MAX_CLASSES) s_keep[tid] = 0;
-  // the class counts are read by sixteen threads at once: one thread reading them in a loop paid a memory round trip
-  // per class (8 of this kernel's 16 microseconds)
+  // the class counts are read by sixteen threads at once (one thread reading them in a loop pays a memory round trip
+  // per class)
   if (tid < v.NC) s_kcc[tid] = v.kcc(layer)[tid];
   __syncthreads();
   if (tid == 0) {
