@@ -145,7 +145,8 @@ def run_reference(args):
                                device="cpu", outlier="pct:1", mode="forced")
     gate = workloads.gate_params(1, D_KV, torch.float16)
     s = oracle_sample_inputs(li, gate, n_max)
-    n = sized_oracle_sample(s, 4.0, n_max)
+    # the sample per step shrinks with the number of steps, so that the whole run stays within about two minutes
+    n = sized_oracle_sample(s, min(4.0, 120.0 / max(args.steps, 1)), n_max)
     for _ in range(args.warmup):
         oracle_step(s, min(n, 512))
     t_dec = []
