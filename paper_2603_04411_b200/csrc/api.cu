@@ -63,6 +63,23 @@ bool make_tmap_2d(CUtensorMap* out, const void* base, uint64_t rows, uint64_t co
                 CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// 2-D tensor map over a row-major fp32 matrix [rows][cols], box [box_rows][box_cols], no swizzle.
+static bool make_tmap_2d_f32(CUtensorMap* out, const void* base, uint64_t rows, uint64_t cols, uint32_t box_rows, uint32_t box_cols) {
+  void* fn = nullptr;
+  cudaDriverEntryPointQueryResult qres;
+  if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) != cudaSuccess || !fn) {
+    cudaGetLastError();
+    return false;
+  }
+  const cuuint64_t dims[2] = {cols, rows};
+  const cuuint64_t strides[1] = {cols * sizeof(float)};
+  const cuuint32_t box[2] = {box_cols, box_rows};
+  const cuuint32_t estr[2] = {1, 1};
+  return reinterpret_cast<PFN_cuTensorMapEncodeTiled_v12000>(fn)(out, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, const_cast<void*>(base), dims, strides,
+                                                                  box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE,
+                                                                  CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
 // Regions of the pool, each followed by one guard word (checked by twkv_cache_check).
 struct Layout {
   size_t total = 0;
@@ -203,6 +220,8 @@ struct twkv_cache {
   std::vector<LayerParams> params;
   Prof prof;
   CUtensorMap map_blocks;
+  CUtensorMap map_scores;              // the score scratch as [V slot][Hq] fp32, boxes of one tile's rows x one V-pass CTA's heads
+  bool scores_tma = false;             // the head count allows that map (rows must start on 16-byte boundaries)
   std::vector<CUtensorMap> map_uinvT;  // per layer, over the transposed copy of U_K^-1 inside the pool
   std::vector<char> prepared;          // per layer: transposed copy and its map are current
   std::vector<CUtensorMap> map_wT;     // per layer x side, over the transposed copies of the gate weights (box = one slab)
@@ -324,6 +343,11 @@ twkv_status twkv_cache_create(const twkv_config* cfg, void* pool, size_t pool_by
   c->map_wT_half.resize(2 * (size_t)cfg->n_layers);
   c->prepared_w.assign(cfg->n_layers, 0);
   if (!make_tmap_2d(&c->map_blocks, c->view.blocks, (uint64_t)c->view.n_blocks * TILE, PANEL, PANEL * 2, TILE)) { delete c; return TWKV_ERR_CUDA; }
+  if (c->cfg.n_q_heads % 4 == 0) {
+    const int hq = c->cfg.n_q_heads, nb = hq < 16 ? hq : (hq <= 16 ? 16 : 32);
+    if (!make_tmap_2d_f32(&c->map_scores, c->view.scores, (uint64_t)c->dims.NT * TILE, (uint64_t)hq, TILE, (uint32_t)(nb < hq ? nb : hq))) { delete c; return TWKV_ERR_CUDA; }
+    c->scores_tma = true;
+  }
   {
     // guard words behind every region, and the list of their offsets for the check kernel
     const unsigned long long word = TWKV_GUARD_WORD;
@@ -475,6 +499,7 @@ static twkv_status decode_pass(twkv_cache* c, int layer, const void* q, const in
   }
   TcMaps maps;
   maps.blocks = c->map_blocks;
+  maps.scores = c->scores_tma ? &c->map_scores : nullptr;
   maps.uinvT_k = c->map_uinvT[layer];
   DevView v = c->view;
   v.qmap = qmap; v.qpos = qpos;

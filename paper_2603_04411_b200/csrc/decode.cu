@@ -360,8 +360,8 @@ merge_kernel(DevView v, const unsigned short* __restrict__ Uinv_v, int n_splits,
 // ------------------------------------------------------------------------- host side
 cudaError_t launch_kscore_tc(const DevView& v, int layer, const CUtensorMap& map_blocks, const CUtensorMap& map_uinvT,
                              const void* q, int n_pieces, bool pairs, cudaStream_t st);
-cudaError_t launch_vacc_tc(const DevView& v, int layer, const CUtensorMap& map_blocks, const int* seq_ids, int n_seq, int n_splits,
-                           cudaStream_t st);
+cudaError_t launch_vacc_tc(const DevView& v, int layer, const CUtensorMap& map_blocks, const CUtensorMap* map_scores, const int* seq_ids,
+                           int n_seq, int n_splits, cudaStream_t st);
 
 template <bool BF16>
 static cudaError_t launch_decode_t(const DevView& v, int layer, const LayerParams& lp, const void* q, const int* seq_ids,
@@ -377,7 +377,7 @@ static cudaError_t launch_decode_t(const DevView& v, int layer, const LayerParam
   }
   {
     ProfScope ps(TWKV_K_VACC, st);
-    cudaError_t e = launch_vacc_tc(v, layer, maps->blocks, seq_ids, n_seq, n_splits, st);
+    cudaError_t e = launch_vacc_tc(v, layer, maps->blocks, maps->scores, seq_ids, n_seq, n_splits, st);
     if (e != cudaSuccess) return e;
   }
   // query heads per merge CTA: the whole group when the batch fills the device, fewer (a divisor) for small batches;

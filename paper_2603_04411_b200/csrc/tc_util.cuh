@@ -395,7 +395,8 @@ __device__ __forceinline__ void ring_gemm_issue(uint32_t n_acc, int KP, uint32_t
 }  // namespace tc
 
 // Tensor maps the decode path needs: the block pool as rows of 64 elements, and the layer's transposed U_K^-1.
-struct TcMaps { CUtensorMap blocks, uinvT_k; };
+// `scores`: the score scratch for the V pass's TMA copies, or null when the head count does not allow them.
+struct TcMaps { CUtensorMap blocks, uinvT_k; const CUtensorMap* scores; };
 // Tensor maps of the fused gate kernel: the call's K and V states, and the layer's transposed gate weights.
 // `raw`: the same four operands as plain pointers (states row-major, weights transposed), for the rows the kernel
 // decides again in fp32.

@@ -14,10 +14,11 @@
 // upper accumulator half adds zeros.
 // The probabilities are the B operand (K-major: [head][token], two 64-token halves), written by 8 warps: thread =
 // (head, 8 consecutive tokens), one 16-byte swizzled store per 8 weights.  The K-score kernel stores a token's scores at
-// its V slot, so a tile's 128 score rows lie next to each other: each warp copies the rows of its own token groups with
-// cp.async into a ring of four tiles in shared memory, so that four tiles of scores are in flight per SM and no thread
-// waits for a load it has just issued; a narrow tile reads as many bytes of scores as of values, and with one tile in
-// flight their latency bound the kernel.
+// its V slot, so a tile's 128 score rows lie next to each other: one TMA box [128 rows x the CTA's heads] per tile,
+// issued by the producer thread two tiles ahead into a ring of four tiles in shared memory (TS = true).  A narrow tile
+// reads as many bytes of scores as of values, and with one tile in flight their latency bound the kernel.  Where the
+// head count is not a multiple of four (rows not 16-byte aligned: no tensor map) each warp copies the rows of its own
+// token groups with cp.async instead (TS = false).
 // bf16 weights go in as two bf16 parts (see below), two chains per pair.
 //
 // Warp roles (320 threads, one CTA per SM):
@@ -75,9 +76,10 @@ template <bool BF16> __device__ __forceinline__ uint32_t vt_pack2(float a, float
 // Instruction descriptor: kind::f16, fp32 accumulate, A MN-major (bit 15), B K-major, M = 128.
 __host__ __device__ constexpr uint32_t vt_idesc(int fmt, int n) { return idesc_f16(fmt, 128, n) | (1u << 15); }
 
-template <bool BF16, int N>
+template <bool BF16, int N, bool TS>
 __global__ void __launch_bounds__(VT_THREADS, 1)
-vacc_tc_kernel(const __grid_constant__ CUtensorMap map_blocks, DevView v, int layer, const int* __restrict__ seq_ids, int n_splits) {
+vacc_tc_kernel(const __grid_constant__ CUtensorMap map_blocks, const __grid_constant__ CUtensorMap map_scores, DevView v, int layer,
+               const int* __restrict__ seq_ids, int n_splits) {
   using C = VtCfg<BF16, N>;
   constexpr int S = C::STAGES, PARTS = C::PARTS, ITEMS = C::ITEMS;
   extern __shared__ __align__(1024) unsigned char smem_raw[];
@@ -85,6 +87,7 @@ vacc_tc_kernel(const __grid_constant__ CUtensorMap map_blocks, DevView v, int la
   const int Hq = v.Hq, d_kv = v.d_kv;
   const int qs = blockIdx.x / n_splits, split = blockIdx.x - qs * n_splits;
   const int h0 = blockIdx.y * N, nh = min(N, Hq - h0);
+  const int NB = min(N, Hq);                                    // heads per score row in shared memory (TS: the box's width)
   const int seq = seq_ids[qs];
   const bool seq_ok = seq >= 0 && seq < v.S;
   // this split's range of the sequence's V tile list in stride order, cut by plan_kernel to equal cost; an id outside
@@ -111,7 +114,8 @@ vacc_tc_kernel(const __grid_constant__ CUtensorMap map_blocks, DevView v, int la
   unsigned char* tail = reinterpret_cast<unsigned char*>(s_l + VT_PTHREADS);
   const uint32_t bars = smem_addr(tail);
   const uint32_t full = bars, empty = full + 8 * S, p_full = empty + 8 * S, p_empty = p_full + 16, acc_done = p_empty + 16;
-  uint32_t* s_tmem_base = reinterpret_cast<uint32_t*>(tail + 8 * (2 * S + 5));
+  const uint32_t sc_full = acc_done + 8, sc_empty = sc_full + 8 * VT_SC;
+  uint32_t* s_tmem_base = reinterpret_cast<uint32_t*>(tail + 8 * (2 * S + 5 + 2 * VT_SC));
   volatile int* abort_flag = reinterpret_cast<int*>(s_tmem_base + 1);
 
   const int n_pairs = (v.NC + 1) >> 1;
@@ -122,6 +126,7 @@ vacc_tc_kernel(const __grid_constant__ CUtensorMap map_blocks, DevView v, int la
     for (int i = 0; i < S; ++i) { mbar_init(full + 8 * i, 1); mbar_init(empty + 8 * i, 1); }
     for (int i = 0; i < 2; ++i) { mbar_init(p_full + 8 * i, VT_PWARPS); mbar_init(p_empty + 8 * i, 1); }
     mbar_init(acc_done, 1);
+    for (int i = 0; i < VT_SC; ++i) { mbar_init(sc_full + 8 * i, 1); mbar_init(sc_empty + 8 * i, VT_PWARPS); }
     *abort_flag = 0;
     mbar_init_fence();
   }
@@ -137,6 +142,7 @@ vacc_tc_kernel(const __grid_constant__ CUtensorMap map_blocks, DevView v, int la
   // role state that survives the descriptor chunks
   uint32_t st = 0, st_ph = 0;                                   // producer / issuer: ring stage and its phase
   uint32_t n_loaded = 0;                                        // producer: stages filled so far
+  uint32_t n_boxes = 0;                                         // producer: score boxes requested so far
   uint32_t touched = 0;                                         // issuer: panel pairs whose accumulator holds a value
   bool ok = true;
   int max_cls = 0;                                              // probability warps: widest class seen (which accumulators to read)
@@ -165,9 +171,24 @@ vacc_tc_kernel(const __grid_constant__ CUtensorMap map_blocks, DevView v, int la
     if (warp == 0) {
       // ------------------------------------------------------------- TMA producer
       if (elect_one()) {
-        if (c0 == 0) tma_prefetch_desc(&map_blocks);
+        if (c0 == 0) { tma_prefetch_desc(&map_blocks); if constexpr (TS) tma_prefetch_desc(&map_scores); }
+        // the score rows of tile i of the chunk: one box [128 rows x NB heads] into stage (c0 + i) % VT_SC
+        auto score_box = [&](int i) -> bool {
+          const uint32_t k = (uint32_t)(c0 + i), stg = k % VT_SC;
+          if (!mbar_wait_thin(sc_empty + 8 * stg, ((k / VT_SC) & 1u) ^ 1u, abort_flag)) return false;
+          mbar_expect_tx(sc_full + 8 * stg, (uint32_t)(TILE * NB * 4));
+          tma_load_2d(sS + stg * C::SC_STAGE_BYTES, &map_scores, sc_full + 8 * stg, h0, s_meta[i].x * TILE);
+          n_boxes = k + 1;
+          return true;
+        };
+        if constexpr (TS) {
+          for (int i = 0; i < 2 && i < cn && ok; ++i) ok = score_box(i);
+        }
         for (int i = 0; i < cn && ok; ++i) {
           const int4 m = s_meta[i];
+          if constexpr (TS) {
+            if (i + 2 < cn && !(ok = score_box(i + 2))) break;
+          }
           for (int j = 0; j < m.y; j += 2) {
             if (!(ok = mbar_wait_thin(empty + 8 * st, st_ph ^ 1u, abort_flag))) break;
             const bool two = j + 1 < m.y;
@@ -182,6 +203,10 @@ vacc_tc_kernel(const __grid_constant__ CUtensorMap map_blocks, DevView v, int la
           for (uint32_t i = 0; i < (uint32_t)S && i < n_loaded; ++i) {
             const uint32_t n = n_loaded - 1 - i;
             mbar_wait_drain(full + 8 * (n % S), (n / S) & 1u);
+          }
+          for (uint32_t i = 0; i < (uint32_t)VT_SC && i < n_boxes; ++i) {
+            const uint32_t n = n_boxes - 1 - i;
+            mbar_wait_drain(sc_full + 8 * (n % VT_SC), (n / VT_SC) & 1u);
           }
         }
       }
@@ -267,19 +292,29 @@ vacc_tc_kernel(const __grid_constant__ CUtensorMap map_blocks, DevView v, int la
           }
         }
       };
+      if constexpr (!TS) {
 #pragma unroll 1
-      for (int d = 0; d < VT_SC - 1; ++d) { issue_scores(d); cp_async_commit(); }
+        for (int d = 0; d < VT_SC - 1; ++d) { issue_scores(d); cp_async_commit(); }
+      }
       for (int i = 0; i < cn && ok; ++i) {
         const int k = c0 + i;
         max_cls = max(max_cls, s_meta[i].y);
-        issue_scores(i + VT_SC - 1);
-        cp_async_commit();
-        cp_async_wait<VT_SC - 1>();                             // this thread's copies of tile i have landed
-        __syncwarp();                                           // ... and the other lanes'
+        const int n_valid_i = s_meta[i].z;
+        if constexpr (TS) {
+          if (!(ok = __all_sync(0xffffffffu, mbar_wait(sc_full + 8 * ((uint32_t)k % VT_SC), ((uint32_t)k / VT_SC) & 1u, abort_flag)))) break;
+        } else {
+          issue_scores(i + VT_SC - 1);
+          cp_async_commit();
+          cp_async_wait<VT_SC - 1>();                           // this thread's copies of tile i have landed
+          __syncwarp();                                         // ... and the other lanes'
+        }
         const uint32_t buf = (uint32_t)k & 1u;
         if (!(ok = __all_sync(0xffffffffu, mbar_wait(p_empty + 8 * buf, (((uint32_t)k >> 1) & 1u) ^ 1u, abort_flag)))) break;
         unsigned char* pb = sP_ptr + buf * C::P_BUF_BYTES;
         const float* srow = reinterpret_cast<const float*>(sS_ptr + (uint32_t)(k % VT_SC) * C::SC_STAGE_BYTES) + ph_;
+        const int rs = TS ? NB : N;                             // floats per score row in the stage
+        // a box holds whatever the scratch holds in rows past the tile's last token and has no columns past the last head
+        const bool head_ok = !TS || ph_ < nh;
 #pragma unroll
         for (int it = 0; it < ITEMS; ++it) {
           const int tg = (it * VT_PTHREADS + pt) / N;
@@ -287,7 +322,11 @@ vacc_tc_kernel(const __grid_constant__ CUtensorMap map_blocks, DevView v, int la
           [[maybe_unused]] uint32_t lo[4];
 #pragma unroll
           for (int u = 0; u < 8; u += 2) {
-            const float p0 = __expf(srow[(tg * 8 + u) * N] - m_h), p1 = __expf(srow[(tg * 8 + u + 1) * N] - m_h);
+            float p0 = __expf(srow[(tg * 8 + u) * rs] - m_h), p1 = __expf(srow[(tg * 8 + u + 1) * rs] - m_h);
+            if constexpr (TS) {
+              p0 = (head_ok && tg * 8 + u < n_valid_i) ? p0 : 0.f;
+              p1 = (head_ok && tg * 8 + u + 1 < n_valid_i) ? p1 : 0.f;
+            }
             // two weights per conversion instruction (single conversions run at a quarter of the rate and bound this loop)
             float r0, r1;
             hi[u >> 1] = vt_pack2<BF16>(p0, p1, r0, r1);
@@ -306,9 +345,12 @@ vacc_tc_kernel(const __grid_constant__ CUtensorMap map_blocks, DevView v, int la
         }
         fence_proxy_async_smem();
         __syncwarp();                                           // also: the stage is read before the next copies into it start
-        if (lane == 0) mbar_arrive(p_full + 8 * buf);
+        if (lane == 0) {
+          mbar_arrive(p_full + 8 * buf);
+          if constexpr (TS) mbar_arrive(sc_empty + 8 * ((uint32_t)k % VT_SC));
+        }
       }
-      cp_async_wait<0>();
+      if constexpr (!TS) cp_async_wait<0>();
     }
     __syncthreads();                                            // the descriptors may be replaced
     ok = ok && !*abort_flag;
@@ -361,26 +403,29 @@ vacc_tc_kernel(const __grid_constant__ CUtensorMap map_blocks, DevView v, int la
   if (tid == 0 && *abort_flag) set_status(v, TWKV_ERR_TIMEOUT);
 }
 
-template <bool BF16, int N>
-static cudaError_t launch_vacc_tc_n(const DevView& v, int layer, const CUtensorMap& map_blocks, const int* seq_ids, int n_seq,
-                                    int n_splits, cudaStream_t st) {
+template <bool BF16, int N, bool TS>
+static cudaError_t launch_vacc_tc_n(const DevView& v, int layer, const CUtensorMap& map_blocks, const CUtensorMap& map_scores,
+                                    const int* seq_ids, int n_seq, int n_splits, cudaStream_t st) {
   using C = VtCfg<BF16, N>;
   static_assert(C::STAGES >= 3, "the ring needs a few stages");
-  cudaError_t e = cudaFuncSetAttribute(vacc_tc_kernel<BF16, N>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)C::SMEM_BYTES);
+  cudaError_t e = cudaFuncSetAttribute(vacc_tc_kernel<BF16, N, TS>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)C::SMEM_BYTES);
   if (e != cudaSuccess) return e;
   const dim3 grid(n_seq * n_splits, (v.Hq + N - 1) / N);
-  vacc_tc_kernel<BF16, N><<<grid, VT_THREADS, C::SMEM_BYTES, st>>>(map_blocks, v, layer, seq_ids, n_splits);
+  vacc_tc_kernel<BF16, N, TS><<<grid, VT_THREADS, C::SMEM_BYTES, st>>>(map_blocks, map_scores, v, layer, seq_ids, n_splits);
   return cudaGetLastError();
 }
 
-cudaError_t launch_vacc_tc(const DevView& v, int layer, const CUtensorMap& map_blocks, const int* seq_ids, int n_seq, int n_splits,
-                           cudaStream_t st) {
+// map_scores: the score scratch as a tensor map (boxes of 128 rows x min(N, Hq) heads), or null: rows copied with cp.async.
+cudaError_t launch_vacc_tc(const DevView& v, int layer, const CUtensorMap& map_blocks, const CUtensorMap* map_scores, const int* seq_ids,
+                           int n_seq, int n_splits, cudaStream_t st) {
   const bool bf16 = v.dtype == TWKV_BF16;
   // up to 32 heads per CTA; more heads run as further CTAs that read the same panels (through L2)
-  if (v.Hq <= 16) return bf16 ? launch_vacc_tc_n<true, 16>(v, layer, map_blocks, seq_ids, n_seq, n_splits, st)
-                              : launch_vacc_tc_n<false, 16>(v, layer, map_blocks, seq_ids, n_seq, n_splits, st);
-  return bf16 ? launch_vacc_tc_n<true, 32>(v, layer, map_blocks, seq_ids, n_seq, n_splits, st)
-              : launch_vacc_tc_n<false, 32>(v, layer, map_blocks, seq_ids, n_seq, n_splits, st);
+#define TWKV_VT(BF, NN)                                                                                                   \
+  (map_scores ? launch_vacc_tc_n<BF, NN, true>(v, layer, map_blocks, *map_scores, seq_ids, n_seq, n_splits, st)           \
+              : launch_vacc_tc_n<BF, NN, false>(v, layer, map_blocks, map_blocks, seq_ids, n_seq, n_splits, st))
+  if (v.Hq <= 16) return bf16 ? TWKV_VT(true, 16) : TWKV_VT(false, 16);
+  return bf16 ? TWKV_VT(true, 32) : TWKV_VT(false, 32);
+#undef TWKV_VT
 }
 
 }  // namespace twkv
