@@ -337,8 +337,8 @@ def run_ours(args):
         # DRAM bytes per launch from the ncu captures summarised under profiles/ (reduced cases, scaled by tokens processed)
         scale = n_tok / (16 * 32768.0)
         rl_gate = tensor_roofline("gate_tc2_kernel (tcgen05 on CTA pairs: gate logits GEMM + softmax/prefix-sum/threshold rank)", flops_g, gg_avg_ms,
-                                  (570.4e6 + 360.0e6) * 4 * scale)
-        rl_ks = tensor_roofline("kscore_tc_kernel (tcgen05 on CTA pairs: K reconstruct + RoPE + q.K scores)", flops_k, ks_avg_ms, (83.9e6 + 4.3e6) * 4 * scale)
+                                  (577.4e6 + 364.0e6) * 4 * scale)
+        rl_ks = tensor_roofline("kscore_tc_kernel (tcgen05 on CTA pairs: K reconstruct + RoPE + q.K scores)", flops_k, ks_avg_ms, (84.4e6 + 4.4e6) * 4 * scale)
         roofline = rl_gate if gg_ms >= ks_ms else rl_ks
         roofline_decode = rl_ks
         va_ms, va_n = prof["vacc"]
@@ -368,7 +368,7 @@ def run_ours(args):
             extra["roofline_vacc"] = {"kernel": "vacc_tc_kernel (softmax weights + absorbed V accumulate)", "bound": "hbm", "achieved": extra["vacc_gbs"],
                                       "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": extra["vacc_gbs"] / peaks["hbm_gbs"],
                                       "bytes": "stored V rows + 4 Hq bytes of scores per token",
-                                      "traffic": (97.2e6 + 3.5e6) * 4 * scale}
+                                      "traffic": (97.2e6 + 3.7e6) * 4 * scale}
         if extra["pack_gbs"]:
             extra["roofline_pack"] = {"kernel": "pack_kernel (truncate + pack)", "bound": "hbm", "achieved": extra["pack_gbs"],
                                       "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": extra["pack_gbs"] / peaks["hbm_gbs"],
